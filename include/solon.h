@@ -1,0 +1,195 @@
+/*
+ * solon.h - C interface of libsolon: the encode step and the robust decode step of Solon
+ * (arXiv 2110.01595, Section 3), for all P simulated compute nodes on one sm_100a GPU.
+ *
+ * Notation (paper -> this header): compression ratio r_c -> m; coded length d_c = ceil(d / m);
+ * redundancy ratio r = group size; s = Byzantine nodes tolerated; P nodes = P partition
+ * gradients (the paper takes B = P); q groups ("blocks" of the linear block code).
+ *
+ * Conventions for every call
+ *   - Returns 0 (SOLON_OK) or a negative solon_status.  Nothing is printed, thrown or aborted.
+ *   - "device" pointers are CUDA device memory owned by the caller, float32, contiguous,
+ *     row-major, and 16-byte aligned at their base; the library never frees or resizes them and
+ *     never writes its inputs.  "host" pointers are ordinary host memory.
+ *   - Work is enqueued on the plan's stream (default: the legacy default stream) and the call
+ *     returns without synchronising, unless stated otherwise.
+ *   - A plan is not thread-safe; use one plan per host thread / stream.
+ *   - There is no CPU fallback: without a CUDA device every call that needs one fails with
+ *     SOLON_ERR_CUDA.
+ */
+#ifndef SOLON_H_
+#define SOLON_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum solon_status {
+  SOLON_OK = 0,
+  SOLON_ERR_INVALID_ARG = -1, /* null pointer, misaligned pointer, value out of range          */
+  SOLON_ERR_INFEASIBLE = -2,  /* 2 s + m > P: no mechanism exists (corollary of Theorem 2)     */
+  SOLON_ERR_CUDA = -3,        /* a CUDA runtime call failed or no device is present            */
+  SOLON_ERR_UNDECODABLE = -4, /* some group has no consistent set of <= s corrupt nodes        */
+  SOLON_ERR_INTERNAL = -5,    /* a bounded device-side wait expired (should not happen)        */
+  SOLON_ERR_NOMEM = -6        /* host or device allocation failed                              */
+} solon_status;
+
+/* Limits of this implementation. */
+#define SOLON_MAX_NODES 1024      /* P; also P * m <= 16384 (recovery table in shared memory) */
+#define SOLON_MAX_GROUP 128       /* largest group size the locator handles                   */
+#define SOLON_MAX_M 32            /* compression ratio (the paper reports trouble above 14)   */
+#define SOLON_MAX_S 16            /* adversaries per group                                    */
+#define SOLON_MAX_PROJECTIONS 4   /* random projections K                                     */
+
+typedef struct solon_plan solon_plan;
+
+/* ------------------------------------------------------------------------------------------
+ * Plan-free host helpers (no device needed).
+ * ---------------------------------------------------------------------------------------- */
+
+/* Feasibility of a mechanism (Theorem 2: r >= 2 s + m; its corollary: 2 s + m <= P; r <= P).
+ * Returns SOLON_OK, SOLON_ERR_INFEASIBLE (2 s + m > P) or SOLON_ERR_INVALID_ARG (anything else,
+ * including the limits above). */
+int solon_check_params(int P, int s, int m, int r, int64_t d);
+
+/* Group layout of the linear block code (Section 3.4, A = I_q (x) 1_{r x r}): q = floor(P / r)
+ * groups of consecutive nodes; when r does not divide P the P - q r left-over nodes are dealt
+ * one at a time to the first groups, so every group has at least r members.
+ * starts: host array of q + 1 ints (capacity given by starts_capacity), group g owns nodes
+ * [starts[g], starts[g+1]).  *q_out receives q. */
+int solon_group_layout(int P, int r, int* starts, int starts_capacity, int* q_out);
+
+/* The "distinct nonzero scalars w_1..w_P" of Section 3.4.  Each group of size r_g uses the first
+ * r_g of the n' Chebyshev points cos((2k-1) pi / (2 n')), k = 1..n', n' = r_g rounded up to even.
+ * w: host array of P doubles. */
+int solon_node_scalars(int P, int r, double* w);
+
+/* Host mirror of the device locator (the same source compiled for the CPU), for one group:
+ * the floating-point reading of the locator phi of Section 3.4 and of the block decoder's
+ * inverse (psi).
+ *   rho   host, K x n row-major: projected values f_kappa . R_k of the group's n nodes
+ *   nu    host, n: row energies sum_p R_k[p]^2
+ *   w_g   host, n: the group's node scalars
+ *   tau   relative tolerance of the "!=" test (see solon_plan_set_tolerance)
+ * Outputs (host): mask[n] (1 = located as corrupt); *t_out the accepted error count;
+ * rec_rows[n] / *n_rec the nodes (indices inside the group) whose rows the recovery reads;
+ * coeff[n_rec * m], coeff[j*m + l] = weight of row rec_rows[j] in coordinate l of a chunk.
+ * Returns SOLON_OK or SOLON_ERR_UNDECODABLE (outputs then hold the best guess). */
+int solon_locate_host(int n, int m, int s, int K, const double* rho, const double* nu,
+                      const double* w_g, double tau, uint8_t* mask, int* t_out, int* rec_rows,
+                      int* n_rec, double* coeff);
+
+const char* solon_strerror(int status);
+
+/* ------------------------------------------------------------------------------------------
+ * Plan.
+ * ---------------------------------------------------------------------------------------- */
+
+/* Build the mechanism (A, E, D) of Section 3.4 for P nodes, s adversaries per group,
+ * compression ratio m, minimum group size r (>= 2 s + m) and gradient length d: group layout,
+ * node scalars, K = 2 projection vectors f_kappa[p] = 1 + N(0,1) drawn on the device from
+ * `seed` (f ~ N(1, I) in Section 3.4), and all device workspace.  Uses the current CUDA device.
+ * Synchronises the device once.  *out receives the plan, to be released by solon_plan_destroy. */
+int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solon_plan** out);
+int solon_plan_destroy(solon_plan* plan);
+
+/* Stream on which later calls enqueue (a cudaStream_t passed as void*). */
+int solon_plan_set_stream(solon_plan* plan, void* cuda_stream);
+
+/* Number of random projections K in 1..SOLON_MAX_PROJECTIONS (default 2; 1 is the paper's
+ * single f).  All projections share one error-locator polynomial.  Redraws f; synchronises. */
+int solon_plan_set_num_projections(solon_plan* plan, int K);
+
+/* Redraw the projection vectors from a new seed (the paper draws a fresh f for every decode).
+ * Enqueued on the plan's stream. */
+int solon_plan_reseed(solon_plan* plan, uint64_t seed);
+
+/* tau of the floating-point "!=" test of the locator: node k is inconsistent with a fitted
+ * polynomial Q when |rho_k - Q(w_k)| > tau * sqrt(2 * median_k nu_k).  Default 1e-5, about
+ * thirty times the rounding noise of float32 coded vectors. */
+int solon_plan_set_tolerance(solon_plan* plan, double tau);
+
+/* Rows per partition for solon_lsq_grads (default 256). */
+int solon_plan_set_lsq_rows(solon_plan* plan, int rows_per_partition);
+
+/* Queries (host, no synchronisation unless stated). */
+int64_t solon_plan_dc(const solon_plan* plan);          /* d_c = ceil(d / m)                    */
+int solon_plan_num_groups(const solon_plan* plan);      /* q                                    */
+int solon_plan_group_of(const solon_plan* plan, int node);
+int solon_plan_group_start(const solon_plan* plan, int group);
+int solon_plan_group_size(const solon_plan* plan, int group);
+int solon_plan_num_projections(const solon_plan* plan);
+int solon_plan_get_node_scalars(const solon_plan* plan, double* w /* host, P */);
+/* Copies f (K x d_c, row-major) to the host; synchronises the plan's stream. */
+int solon_plan_get_projection_vectors(solon_plan* plan, float* f /* host, K * d_c */);
+
+/* ------------------------------------------------------------------------------------------
+ * The hot path.
+ * ---------------------------------------------------------------------------------------- */
+
+/* Encode (Section 3.4, z_j = W_j Y_j 1_P with W_j = I_{d_c} (x) [1, w_j, ..., w_j^{m-1}]).
+ *   partition_grads  device, P x d: row i is partition gradient g_i
+ *   coded            device, P x d_c: row k receives node k's coded vector,
+ *                    coded[k][p] = sum_{l<m} w_k^l * ybar_g[p m + l], where ybar_g is the sum of
+ *                    the gradients of k's group, zero-padded to m d_c entries.
+ * The group sum and the mix are evaluated in float64 and rounded once to float32. */
+int solon_encode(solon_plan* plan, const float* partition_grads, float* coded);
+
+/* Robust decode (Algorithm 1 with the locator phi and block decoder psi of Section 3.4).
+ *   received  device, P x d_c: what the P nodes sent (coded vectors, up to s rows per group
+ *             replaced by arbitrary values, non-finite values included); may alias `coded`
+ *   agg_grad  device, d: receives u = sum over groups of the recovered group sums = G 1_P
+ *   byz_mask  device, P bytes: 1 for every node located as Byzantine, else 0
+ * Three kernels: projections rho = f R and row energies (one pass over `received`), the locator
+ * (tiny, on device), the recovery (one pass over the trusted rows it needs).  If some group has
+ * no consistent set of at most s corrupt nodes the outputs hold a best guess and
+ * solon_decode_status reports SOLON_ERR_UNDECODABLE. */
+int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask);
+
+/* Status of the most recent solon_decode: synchronises the plan's stream, then returns SOLON_OK,
+ * SOLON_ERR_UNDECODABLE, SOLON_ERR_INTERNAL or SOLON_ERR_CUDA. */
+int solon_decode_status(solon_plan* plan);
+
+/* Least-squares partition gradients g_i = X_i^T (X_i w - y_i) (the paper accepts any method that
+ * needs a sum of per-partition functions, Section 1; this one feeds the encode step).
+ *   X      device, (P * rows) x d; partition i owns rows [i rows, (i+1) rows)
+ *   y      device, P * rows
+ *   w      device, d
+ *   grads  device, P x d (output) */
+int solon_lsq_grads(solon_plan* plan, const float* X, const float* y, const float* w, float* grads);
+
+/* One whole step with HOST buffers: copies the gradients to the device, encodes, overwrites the
+ * rows of the n_byz listed nodes with the given vectors (the adversary sits between encode and
+ * decode), decodes, copies the aggregate and the mask back, and synchronises.
+ *   grads_host     host, P x d          byz_nodes      host, n_byz node indices (may be NULL if 0)
+ *   byz_rows_host  host, n_byz x d_c    agg_host       host, d (output)
+ *   mask_host      host, P bytes (output)
+ * Device staging buffers are owned by the plan and allocated on the first call.  Returns the
+ * decode status.  Pinned host memory makes the copies asynchronous to each other but the call
+ * still returns only when everything is done. */
+int solon_step_host(solon_plan* plan, const float* grads_host, int n_byz, const int* byz_nodes,
+                    const float* byz_rows_host, float* agg_host, uint8_t* mask_host);
+
+/* ------------------------------------------------------------------------------------------
+ * Introspection of the last decode (for parity tests and diagnostics; each synchronises).
+ * ---------------------------------------------------------------------------------------- */
+
+/* rho (K x P, row-major) and nu (P) computed by the projection kernel. */
+int solon_plan_get_projections(solon_plan* plan, double* rho /* host, K * P */, double* nu /* host, P */);
+
+/* Recovery table chosen by the locator: n_rec[g] rows for group g, their node indices in
+ * rec_rows (concatenated over groups), coefficients coeff (concatenated, n_rec[g] * m each,
+ * coeff[j*m + l]), and the accepted error count t[g] (-1 if the group was undecodable).
+ * Capacities: n_rec and t hold q ints, rec_rows P ints, coeff P * m doubles. */
+int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows, double* coeff);
+
+/* Number of kernels the library launched on behalf of this plan since creation. */
+int64_t solon_plan_kernel_launches(const solon_plan* plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOLON_H_ */

@@ -1,0 +1,53 @@
+// solon_decode (Algorithm 1: locate, then decode every group from its trusted nodes, then sum) and the
+// host-buffer convenience call solon_step_host.
+#include "solon_internal.h"
+
+using namespace solon;
+
+extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask) {
+  if (!plan || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
+  if (((uintptr_t)received & 3) || ((uintptr_t)agg_grad & 15)) return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), plan->stream));
+  int rc;
+  if (plan->s > 0 && (rc = launch_project(plan, received))) return rc;   // s = 0: nothing to locate
+  if ((rc = launch_locate(plan, byz_mask))) return rc;
+  return launch_recover(plan, received, agg_grad);
+}
+
+template <typename T>
+static int stage_alloc(T** ptr, size_t count) {
+  if (*ptr) return SOLON_OK;
+  cudaError_t err = cudaMalloc((void**)ptr, count * sizeof(T));
+  if (err != cudaSuccess) {
+    (void)cudaGetLastError();
+    *ptr = nullptr;
+    return err == cudaErrorMemoryAllocation ? SOLON_ERR_NOMEM : SOLON_ERR_CUDA;
+  }
+  return SOLON_OK;
+}
+
+extern "C" int solon_step_host(solon_plan* plan, const float* grads_host, int n_byz, const int* byz_nodes,
+                               const float* byz_rows_host, float* agg_host, uint8_t* mask_host) {
+  if (!plan || !grads_host || !agg_host || !mask_host || n_byz < 0) return SOLON_ERR_INVALID_ARG;
+  if (n_byz > 0 && (!byz_nodes || !byz_rows_host)) return SOLON_ERR_INVALID_ARG;
+  for (int i = 0; i < n_byz; ++i)
+    if (byz_nodes[i] < 0 || byz_nodes[i] >= plan->P) return SOLON_ERR_INVALID_ARG;
+  int rc;
+  const size_t n_grad = (size_t)plan->P * plan->d, n_coded = (size_t)plan->P * plan->d_c;
+  if ((rc = stage_alloc(&plan->d_stage_grads, n_grad))) return rc;
+  if ((rc = stage_alloc(&plan->d_stage_coded, n_coded))) return rc;
+  if ((rc = stage_alloc(&plan->d_stage_agg, (size_t)plan->d))) return rc;
+  if ((rc = stage_alloc(&plan->d_stage_mask, (size_t)plan->P))) return rc;
+  cudaStream_t st = plan->stream;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_stage_grads, grads_host, n_grad * sizeof(float), cudaMemcpyHostToDevice, st));
+  if ((rc = solon_encode(plan, plan->d_stage_grads, plan->d_stage_coded))) return rc;
+  for (int i = 0; i < n_byz; ++i) {
+    SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_stage_coded + (size_t)byz_nodes[i] * plan->d_c,
+                                   byz_rows_host + (size_t)i * plan->d_c, (size_t)plan->d_c * sizeof(float),
+                                   cudaMemcpyHostToDevice, st));
+  }
+  if ((rc = solon_decode(plan, plan->d_stage_coded, plan->d_stage_agg, plan->d_stage_mask))) return rc;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(agg_host, plan->d_stage_agg, (size_t)plan->d * sizeof(float), cudaMemcpyDeviceToHost, st));
+  SOLON_CUDA_TRY(cudaMemcpyAsync(mask_host, plan->d_stage_mask, (size_t)plan->P, cudaMemcpyDeviceToHost, st));
+  return solon_decode_status(plan);
+}

@@ -1,0 +1,277 @@
+// Encode kernel (Section 3.4): z_k = W_k (Y_k 1_P), W_k = I_{d_c} (x) [1, w_k, ..., w_k^{m-1}].
+//
+// One pass over the P x d gradient matrix.  A tile is (group g, a run of chunks); the r_g rows of the
+// group are streamed through shared memory in batches by a producer warp that issues one bulk
+// asynchronous copy (cp.async.bulk, completion on an mbarrier) per row segment, so every gradient
+// byte is read from HBM exactly once and many kilobytes per SM are in flight without occupying
+// registers.  Consumer warps add the rows into the group sum ybar (float64, shared memory), then
+// each thread evaluates, for its chunks, the r_g polynomials sum_l w_k^l ybar[p m + l] by Horner's rule
+// in float64 and stores one float32 per node (coalesced along the chunk axis).
+//
+// Row segments start at arbitrary 4-byte offsets (d need not be a multiple of 4): the copy starts at
+// the enclosing 16-byte boundary and consumers index from the remainder; the last few floats of the
+// whole matrix, where rounding the end up would leave the buffer, are fetched with ordinary loads.
+#include "solon_internal.h"
+#include "stream_pipe.cuh"
+
+namespace solon {
+
+constexpr int kEncConsumers = 256;                 // consumer threads per CTA
+constexpr int kEncThreads = kEncConsumers + 32;    // + one producer warp
+constexpr int kEncMaxBatch = 32;                   // rows per pipeline stage (one per producer lane)
+
+struct EncodeParams {
+  const float* grads;
+  float* coded;
+  const int* group_start;
+  const double* w;
+  int q, m;
+  int64_t d, d_c;
+  int64_t total_floats;   // P * d
+  int chunks_per_thread;  // tile = kEncConsumers * chunks_per_thread chunks
+  int row_batch;          // rows per stage
+  int stages;
+  int slot_floats;        // shared-memory floats per row slot (multiple of 4)
+  int64_t tiles_per_group;
+  int* status;            // device status words: [1] collects wait-expiry bits
+};
+
+// Horner evaluation for all nodes of the group with the chunk held in registers.
+template <int M>
+__device__ __forceinline__ void mix_chunk(const double* __restrict__ y, const double* __restrict__ w_g, int r_g,
+                                          float* __restrict__ out, int64_t out_stride) {
+  double c[M];
+#pragma unroll
+  for (int l = 0; l < M; ++l) c[l] = y[l];
+  for (int k = 0; k < r_g; ++k) {
+    double wk = w_g[k];
+    double acc = c[M - 1];
+#pragma unroll
+    for (int l = M - 2; l >= 0; --l) acc = fma(acc, wk, c[l]);
+    out[(int64_t)k * out_stride] = (float)acc;
+  }
+}
+
+__device__ __forceinline__ void mix_chunk_generic(const double* __restrict__ y, int m, const double* __restrict__ w_g,
+                                                  int r_g, float* __restrict__ out, int64_t out_stride) {
+  for (int k = 0; k < r_g; ++k) {
+    double wk = w_g[k];
+    double acc = y[m - 1];
+    for (int l = m - 2; l >= 0; --l) acc = fma(acc, wk, y[l]);
+    out[(int64_t)k * out_stride] = (float)acc;
+  }
+}
+
+template <int M>
+__global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(EncodeParams prm) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x;
+  const int m = (M > 0) ? M : prm.m;
+  const int tile_chunks = kEncConsumers * prm.chunks_per_thread;
+  const int tile_floats = tile_chunks * m;
+
+  // shared memory: [barriers][w_g x 2][ybar x 2][stages x row_batch x slot]; w_g and ybar are double
+  // buffered by tile parity so that one consumer barrier per tile suffices
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
+  uint64_t* empty_bar = full_bar + prm.stages;
+  int* abort_flag = reinterpret_cast<int*>(empty_bar + prm.stages);
+  double* w_s = reinterpret_cast<double*>(smem_raw + 256);
+  double* ybar = w_s + 2 * SOLON_MAX_GROUP;
+  float* ring = reinterpret_cast<float*>(ybar + 2 * (size_t)tile_floats);
+  const size_t stage_floats = (size_t)prm.row_batch * prm.slot_floats;
+
+  if (tid == 0) {
+    for (int s = 0; s < prm.stages; ++s) {
+      pipe::mbar_init(&full_bar[s], 32);                     // every producer lane arrives
+      pipe::mbar_init(&empty_bar[s], kEncConsumers / 32);    // one arrival per consumer warp
+    }
+    *abort_flag = 0;
+    pipe::fence_barrier_init();
+  }
+  __syncthreads();
+
+  const int64_t total_tiles = prm.tiles_per_group * prm.q;
+  const bool is_producer = tid >= kEncConsumers;
+
+  if (is_producer) {
+    const int lane = tid - kEncConsumers;
+    uint32_t it = 0;   // running stage counter
+    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int g = (int)(tile / prm.tiles_per_group);
+      const int64_t ct = tile - (int64_t)g * prm.tiles_per_group;
+      const int row0 = prm.group_start[g], r_g = prm.group_start[g + 1] - row0;
+      const int64_t e0 = ct * tile_floats;
+      int64_t e1 = e0 + tile_floats;
+      if (e1 > prm.d) e1 = prm.d;
+      for (int b0 = 0; b0 < r_g; b0 += prm.row_batch, ++it) {
+        const int stage = it % prm.stages;
+        const uint32_t phase = (it / prm.stages) & 1;
+        if (it >= (uint32_t)prm.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, prm.status + 1);
+        const int nb = min(prm.row_batch, r_g - b0);
+        if (lane < nb && e1 > e0) {
+          const int64_t first = (int64_t)(row0 + b0 + lane) * prm.d + e0;    // float index of the segment
+          const int64_t last = first + (e1 - e0);
+          const int64_t a0 = first & ~(int64_t)3;                            // enclosing 16-byte boundary
+          int64_t a1 = (last + 3) & ~(int64_t)3;
+          const int64_t safe_end = prm.total_floats & ~(int64_t)3;           // bulk copies stay inside the matrix
+          if (a1 > safe_end) a1 = safe_end;
+          float* slot = ring + stage * stage_floats + (size_t)lane * prm.slot_floats;
+          uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
+          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.grads[e];   // <= 3 floats
+          if (bytes) {
+            pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
+            pipe::bulk_load(slot, prm.grads + a0, bytes, &full_bar[stage]);
+          } else {
+            pipe::mbar_arrive(&full_bar[stage]);
+          }
+        } else {
+          pipe::mbar_arrive(&full_bar[stage]);
+        }
+      }
+    }
+    // Every copy issued above is awaited by the consumers before they finish, unless a wait expired;
+    // in that case drain here so no copy is in flight into shared memory when the CTA exits.
+    if (*(volatile int*)abort_flag) pipe::drain_delay();
+  } else {
+    uint32_t it = 0;
+    int parity = 0;   // ybar double buffer
+    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, parity ^= 1) {
+      const int g = (int)(tile / prm.tiles_per_group);
+      const int64_t ct = tile - (int64_t)g * prm.tiles_per_group;
+      const int row0 = prm.group_start[g], r_g = prm.group_start[g + 1] - row0;
+      const int64_t e0 = ct * tile_floats;
+      int64_t e1 = e0 + tile_floats;
+      if (e1 > prm.d) e1 = prm.d;
+      const int valid = (int)(e1 > e0 ? e1 - e0 : 0);
+      double* y = ybar + (size_t)parity * tile_floats;
+      double* w_g = w_s + (size_t)parity * SOLON_MAX_GROUP;
+      for (int k = tid; k < r_g; k += kEncConsumers) w_g[k] = prm.w[row0 + k];
+      const int d_mod4 = (int)(prm.d & 3), e0_mod4 = (int)(e0 & 3);
+
+      for (int b0 = 0; b0 < r_g; b0 += prm.row_batch, ++it) {
+        const int stage = it % prm.stages;
+        const uint32_t phase = (it / prm.stages) & 1;
+        pipe::mbar_wait(&full_bar[stage], phase, abort_flag, prm.status + 1);
+        const int nb = min(prm.row_batch, r_g - b0);
+        const float* base = ring + stage * stage_floats;
+        // each thread owns elements tid + i * 256 of the tile, four at a time
+        for (int eb = tid; eb < tile_floats; eb += 4 * kEncConsumers) {
+          double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
+          const bool v0 = eb < valid, v1 = eb + kEncConsumers < valid, v2 = eb + 2 * kEncConsumers < valid,
+                     v3 = eb + 3 * kEncConsumers < valid;
+          for (int j = 0; j < nb; ++j) {
+            const int shift = ((((row0 + b0 + j) & 3) * d_mod4) + e0_mod4) & 3;   // (row * d + e0) mod 4
+            const float* src = base + (size_t)j * prm.slot_floats + shift + eb;
+            if (v0) acc0 += (double)src[0];
+            if (v1) acc1 += (double)src[kEncConsumers];
+            if (v2) acc2 += (double)src[2 * kEncConsumers];
+            if (v3) acc3 += (double)src[3 * kEncConsumers];
+          }
+          if (b0 == 0) {
+            y[eb] = acc0;
+            if (eb + kEncConsumers < tile_floats) y[eb + kEncConsumers] = acc1;
+            if (eb + 2 * kEncConsumers < tile_floats) y[eb + 2 * kEncConsumers] = acc2;
+            if (eb + 3 * kEncConsumers < tile_floats) y[eb + 3 * kEncConsumers] = acc3;
+          } else {
+            y[eb] += acc0;
+            if (eb + kEncConsumers < tile_floats) y[eb + kEncConsumers] += acc1;
+            if (eb + 2 * kEncConsumers < tile_floats) y[eb + 2 * kEncConsumers] += acc2;
+            if (eb + 3 * kEncConsumers < tile_floats) y[eb + 3 * kEncConsumers] += acc3;
+          }
+        }
+        __syncwarp();
+        if ((tid & 31) == 0) pipe::mbar_arrive(&empty_bar[stage]);
+      }
+      pipe::named_barrier_sync(1, kEncConsumers);   // ybar (and w_s) complete
+
+      const int64_t c0 = ct * tile_chunks;
+      for (int i = 0; i < prm.chunks_per_thread; ++i) {
+        const int p = tid + i * kEncConsumers;
+        if (c0 + p < prm.d_c) {
+          float* out = prm.coded + (int64_t)row0 * prm.d_c + c0 + p;
+          if (M > 0) mix_chunk<(M > 0 ? M : 1)>(y + (size_t)p * m, w_g, r_g, out, prm.d_c);
+          else mix_chunk_generic(y + (size_t)p * m, m, w_g, r_g, out, prm.d_c);
+        }
+      }
+    }
+  }
+}
+
+static size_t encode_smem_bytes(int m, int cpt, int row_batch, int stages, int slot_floats) {
+  size_t tile_floats = (size_t)kEncConsumers * cpt * m;
+  return 256 + 2 * SOLON_MAX_GROUP * sizeof(double) + 2 * tile_floats * sizeof(double) +
+         (size_t)stages * row_batch * slot_floats * sizeof(float);
+}
+
+template <int M>
+static int launch_encode_m(solon_plan* plan, EncodeParams& prm, size_t smem, int grid) {
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(encode_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  encode_kernel<M><<<grid, kEncThreads, smem, plan->stream>>>(prm);
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
+int launch_encode(solon_plan* plan, const float* grads, float* coded) {
+  EncodeParams prm;
+  prm.grads = grads;
+  prm.coded = coded;
+  prm.group_start = plan->d_group_start;
+  prm.w = plan->d_w;
+  prm.q = plan->q;
+  prm.m = plan->m;
+  prm.d = plan->d;
+  prm.d_c = plan->d_c;
+  prm.total_floats = (int64_t)plan->P * plan->d;
+  prm.status = plan->d_status;
+  // tile: about 1024..2048 floats per row for small m, one chunk per thread otherwise
+  int cpt = 1;
+  while (cpt < 8 && kEncConsumers * cpt * plan->m < 1024) cpt *= 2;
+  prm.chunks_per_thread = cpt;
+  int tile_floats = kEncConsumers * cpt * plan->m;
+  prm.slot_floats = ((tile_floats + 3) / 4) * 4 + 8;
+  size_t slot_bytes = (size_t)prm.slot_floats * 4;
+  int row_batch = (int)((size_t)24 * 1024 / slot_bytes);
+  if (row_batch < 1) row_batch = 1;
+  if (row_batch > kEncMaxBatch) row_batch = kEncMaxBatch;
+  if (row_batch > plan->max_group) row_batch = plan->max_group;
+  // prefer batches that divide the group evenly (fewer ragged stages)
+  {
+    int nb = (plan->max_group + row_batch - 1) / row_batch;
+    row_batch = (plan->max_group + nb - 1) / nb;
+  }
+  prm.row_batch = row_batch;
+  const size_t budget = 200 * 1024;
+  int stages = 4;
+  while (stages > 2 && encode_smem_bytes(plan->m, cpt, row_batch, stages, prm.slot_floats) > budget) --stages;
+  while (prm.row_batch > 1 && encode_smem_bytes(plan->m, cpt, prm.row_batch, stages, prm.slot_floats) > budget) --prm.row_batch;
+  if (encode_smem_bytes(plan->m, cpt, prm.row_batch, stages, prm.slot_floats) > budget) return SOLON_ERR_INVALID_ARG;
+  prm.stages = stages;
+  size_t smem = encode_smem_bytes(plan->m, cpt, prm.row_batch, stages, prm.slot_floats);
+  prm.tiles_per_group = (plan->d_c + (int64_t)kEncConsumers * cpt - 1) / ((int64_t)kEncConsumers * cpt);
+  int64_t total_tiles = prm.tiles_per_group * plan->q;
+  int per_sm = (int)((size_t)220 * 1024 / (smem + 1024));
+  if (per_sm > 2) per_sm = 2;
+  if (per_sm < 1) per_sm = 1;
+  int64_t resident = (int64_t)plan->num_sms * per_sm;
+  int grid = (int)(total_tiles < resident ? total_tiles : resident);
+  plan->launches += 1;
+  switch (plan->m) {
+    case 1: return launch_encode_m<1>(plan, prm, smem, grid);
+    case 2: return launch_encode_m<2>(plan, prm, smem, grid);
+    case 3: return launch_encode_m<3>(plan, prm, smem, grid);
+    case 4: return launch_encode_m<4>(plan, prm, smem, grid);
+    case 5: return launch_encode_m<5>(plan, prm, smem, grid);
+    case 6: return launch_encode_m<6>(plan, prm, smem, grid);
+    case 8: return launch_encode_m<8>(plan, prm, smem, grid);
+    case 10: return launch_encode_m<10>(plan, prm, smem, grid);
+    default: return launch_encode_m<0>(plan, prm, smem, grid);
+  }
+}
+
+}  // namespace solon
+
+extern "C" int solon_encode(solon_plan* plan, const float* partition_grads, float* coded) {
+  if (!plan || !partition_grads || !coded) return SOLON_ERR_INVALID_ARG;
+  if (((uintptr_t)partition_grads & 15) || ((uintptr_t)coded & 3)) return SOLON_ERR_INVALID_ARG;
+  return solon::launch_encode(plan, partition_grads, coded);
+}

@@ -1,0 +1,206 @@
+// Locator kernel (phi of Section 3.4) and recovery table (the inverse inside psi), on the device, plus
+// the host mirror solon_locate_host built from the same source (locate_core.cuh).
+//
+// Grid (s + 1, q): CTA (t, g) is one warp that assumes exactly t corrupt nodes in group g.  All error
+// counts are tried concurrently; the last CTA of a group to finish (atomic ticket, nobody waits) picks
+// the smallest accepted count, writes the group's part of the mask and builds the recovery table.
+#include <vector>
+
+#include "locate_core.cuh"
+#include "solon_internal.h"
+
+namespace solon {
+
+struct LocateParams {
+  const int* group_start;
+  const double* w;
+  const double* rho;     // K x P
+  const double* nu;      // P
+  int P, m, s, K;
+  double tau;
+  TaskRecord* records;   // q x (s + 1)
+  uint8_t* task_flags;   // (s + 1) x P
+  unsigned int* group_ticket;   // q
+  double* ws_global;     // q x (s + 1) x ws_stride, used when shared memory is too small
+  size_t ws_stride;
+  int use_smem;
+  uint8_t* mask;         // P (caller's buffer)
+  int* t_acc;            // q
+  int* n_rec;            // q
+  int* rec_rows;         // P
+  double* coeff;         // P x m
+  int* status;
+};
+
+// Workspace carving shared by the device kernel and the host mirror.
+struct GroupScratch {
+  int* idx;          // n
+  uint8_t* cand;     // n
+  uint8_t* bad;      // n
+  uint8_t* trusted;  // n
+  double* rho_n;     // K x n
+  double* w_c;       // n
+  double* scratch;   // n
+  double* task_ws;   // rest
+};
+
+SOLON_HD static inline size_t group_scratch_doubles(int n, int K) {
+  // ints and bytes are carved out of double-sized cells to keep everything 8-byte aligned
+  return (size_t)(n + 1) / 2 + 1 + 3 * ((size_t)n / 8 + 1) + (size_t)(K + 2) * n;
+}
+
+SOLON_HD static inline GroupScratch carve(double* ws, int n, int K) {
+  GroupScratch sc;
+  double* p = ws;
+  sc.idx = reinterpret_cast<int*>(p);            p += (n + 1) / 2 + 1;
+  sc.cand = reinterpret_cast<uint8_t*>(p);       p += n / 8 + 1;
+  sc.bad = reinterpret_cast<uint8_t*>(p);        p += n / 8 + 1;
+  sc.trusted = reinterpret_cast<uint8_t*>(p);    p += n / 8 + 1;
+  sc.rho_n = p;                                  p += (size_t)K * n;
+  sc.w_c = p;                                    p += n;
+  sc.scratch = p;                                p += n;
+  sc.task_ws = p;
+  return sc;
+}
+
+__global__ void __launch_bounds__(32) locate_kernel(LocateParams prm) {
+  extern __shared__ __align__(16) double smem_ws[];
+  const int t = blockIdx.x, g = blockIdx.y;
+  const int row0 = prm.group_start[g];
+  const int n = prm.group_start[g + 1] - row0;
+  double* ws = prm.use_smem ? smem_ws : prm.ws_global + ((size_t)g * (prm.s + 1) + t) * prm.ws_stride;
+  GroupScratch sc = carve(ws, n, prm.K);
+  __shared__ unsigned int s_ticket;
+
+  TaskRecord* recs = prm.records + (size_t)g * (prm.s + 1);
+  uint8_t* flags = prm.task_flags + (size_t)t * prm.P + row0;
+  double tau_eff = 0.0;
+  int n_eff = n;
+  if (prm.s == 0) {
+    // pure compression code: nothing to locate, every node is trusted
+    for (int k = threadIdx.x; k < n; k += 32) {
+      sc.idx[k] = k;
+      flags[k] = 0;
+    }
+    if (threadIdx.x == 0) {
+      recs[0].accept = 1;
+      recs[0].n_flagged = 0;
+      recs[0].max_fit = 0.0;
+    }
+    __syncwarp();
+  } else {
+    n_eff = locate_prepare(n, prm.K, prm.rho + row0, prm.P, prm.nu + row0, prm.w + row0, prm.tau, sc.idx, sc.rho_n,
+                           sc.w_c, &tau_eff, sc.scratch);
+  }
+  const int s_eff = prm.s - (n - n_eff);
+  if (prm.s == 0) {
+  } else if (t <= s_eff && n_eff >= prm.m + 2 * t) {
+    locate_task(n_eff, prm.m, prm.K, t, sc.rho_n, sc.w_c, tau_eff, flags, sc.cand, sc.bad, sc.task_ws, &recs[t]);
+  } else if (threadIdx.x == 0) {
+    recs[t].accept = 0;
+    recs[t].n_flagged = 0;
+    recs[t].max_fit = INFINITY;
+  }
+  __threadfence();
+  __syncwarp();
+  if (threadIdx.x == 0) s_ticket = atomicAdd(&prm.group_ticket[g], 1u);
+  __syncwarp();
+  if (s_ticket != (unsigned int)prm.s) return;
+  __threadfence();
+  // Group epilogue.  Records and flags written by the other CTAs are read through L2.
+  TaskRecord* recs_l = reinterpret_cast<TaskRecord*>(sc.task_ws);                  // s + 1 records
+  uint8_t* flags_l = reinterpret_cast<uint8_t*>(recs_l + (prm.s + 1));             // (s + 1) x n
+  double* ep_ws = sc.task_ws + ((size_t)(prm.s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1;
+  for (int i = threadIdx.x; i <= prm.s; i += 32) {
+    recs_l[i].accept = __ldcg(&recs[i].accept);
+    recs_l[i].n_flagged = __ldcg(&recs[i].n_flagged);
+    recs_l[i].max_fit = __ldcg(&recs[i].max_fit);
+  }
+  for (int i = threadIdx.x; i < (prm.s + 1) * n; i += 32) {
+    int tt = i / n, k = i - tt * n;
+    flags_l[i] = __ldcg(prm.task_flags + (size_t)tt * prm.P + row0 + k);
+  }
+  __syncwarp();
+  int* rec_rows_g = prm.rec_rows + row0;
+  const int ok = locate_epilogue(n, prm.m, s_eff, n_eff, sc.idx, prm.w + row0, recs_l, flags_l, n, prm.mask + row0,
+                                 &prm.t_acc[g], rec_rows_g, &prm.n_rec[g], prm.coeff + (size_t)row0 * prm.m,
+                                 sc.trusted, ep_ws);
+  // recovery rows as global node indices
+  const int n_rec = prm.n_rec[g];
+  for (int j = threadIdx.x; j < n_rec; j += 32) rec_rows_g[j] += row0;
+  if (threadIdx.x == 0) {
+    if (!ok) atomicOr(prm.status, kStatusUndecodable);
+    prm.group_ticket[g] = 0u;   // ready for the next decode
+  }
+}
+
+size_t locate_ws_doubles(int n, int m, int K, int s) {
+  size_t task = locate_task_ws_doubles(n, m, K, s);
+  size_t epi = ((size_t)(s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1 + locate_epilogue_ws_doubles(n, m);
+  return group_scratch_doubles(n, K) + (task > epi ? task : epi) + 8;
+}
+
+int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
+  LocateParams prm;
+  prm.group_start = plan->d_group_start;
+  prm.w = plan->d_w;
+  prm.rho = plan->d_rho;
+  prm.nu = plan->d_nu;
+  prm.P = plan->P; prm.m = plan->m; prm.s = plan->s; prm.K = plan->K;
+  prm.tau = plan->tau;
+  prm.records = reinterpret_cast<TaskRecord*>(plan->d_task_records);
+  prm.task_flags = plan->d_task_flags;
+  prm.group_ticket = plan->d_group_ticket;
+  prm.ws_global = plan->d_locate_ws;
+  prm.ws_stride = plan->locate_ws_stride;
+  prm.mask = byz_mask;
+  prm.t_acc = plan->d_t_acc;
+  prm.n_rec = plan->d_n_rec;
+  prm.rec_rows = plan->d_rec_rows;
+  prm.coeff = plan->d_coeff;
+  prm.status = plan->d_status;
+  size_t need = locate_ws_doubles(plan->max_group, plan->m, plan->K, plan->s) * sizeof(double);
+  if (need > plan->locate_ws_stride * sizeof(double)) return SOLON_ERR_INTERNAL;
+  prm.use_smem = need <= 96 * 1024 ? 1 : 0;
+  size_t smem = prm.use_smem ? need : 0;
+  if (prm.use_smem && smem > 48 * 1024)
+    SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid(plan->s + 1, plan->q);
+  locate_kernel<<<grid, 32, smem, plan->stream>>>(prm);
+  plan->launches += 1;
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
+}  // namespace solon
+
+using namespace solon;
+
+extern "C" int solon_locate_host(int n, int m, int s, int K, const double* rho, const double* nu, const double* w_g,
+                                 double tau, uint8_t* mask, int* t_out, int* rec_rows, int* n_rec, double* coeff) {
+  if (!rho || !nu || !w_g || !mask || !t_out || !rec_rows || !n_rec || !coeff) return SOLON_ERR_INVALID_ARG;
+  if (n < 1 || n > SOLON_MAX_GROUP || m < 1 || m > SOLON_MAX_M || s < 0 || s > SOLON_MAX_S || K < 1 ||
+      K > SOLON_MAX_PROJECTIONS || n < 2 * s + m)
+    return SOLON_ERR_INVALID_ARG;
+  std::vector<double> ws(group_scratch_doubles(n, K) + locate_task_ws_doubles(n, m, K, s) +
+                         locate_epilogue_ws_doubles(n, m) + 64);
+  GroupScratch sc = carve(ws.data(), n, K);
+  std::vector<TaskRecord> recs(s + 1);
+  std::vector<uint8_t> flags((size_t)(s + 1) * n, 0);
+  double tau_eff = 0.0;
+  const int n_eff = locate_prepare(n, K, rho, n, nu, w_g, tau, sc.idx, sc.rho_n, sc.w_c, &tau_eff, sc.scratch);
+  const int s_eff = s - (n - n_eff);
+  for (int t = 0; t <= s; ++t) {
+    if (t <= s_eff && n_eff >= m + 2 * t) {
+      locate_task(n_eff, m, K, t, sc.rho_n, sc.w_c, tau_eff, flags.data() + (size_t)t * n, sc.cand, sc.bad, sc.task_ws,
+                  &recs[t]);
+    } else {
+      recs[t].accept = 0;
+      recs[t].n_flagged = 0;
+      recs[t].max_fit = INFINITY;
+    }
+  }
+  const int ok = locate_epilogue(n, m, s_eff, n_eff, sc.idx, w_g, recs.data(), flags.data(), n, mask, t_out, rec_rows,
+                                 n_rec, coeff, sc.trusted, sc.task_ws);
+  return ok ? SOLON_OK : SOLON_ERR_UNDECODABLE;
+}

@@ -1,0 +1,364 @@
+// Plan construction (Section 3.4: allocation, node scalars, projection vectors), queries, and the
+// plan-free host helpers of the C interface.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "locate_core.cuh"
+#include "solon_internal.h"
+
+namespace solon {
+
+int check_params(int P, int s, int m, int r, int64_t d) {
+  if (P < 1 || s < 0 || m < 1 || d < 1 || r < 1) return SOLON_ERR_INVALID_ARG;
+  if (P > SOLON_MAX_NODES || m > SOLON_MAX_M || s > SOLON_MAX_S) return SOLON_ERR_INVALID_ARG;
+  if ((int64_t)2 * s + m > P) return SOLON_ERR_INFEASIBLE;   // corollary of Theorem 2
+  if (r < 2 * s + m) return SOLON_ERR_INVALID_ARG;            // Theorem 2
+  if (r > P) return SOLON_ERR_INVALID_ARG;
+  return SOLON_OK;
+}
+
+// q = floor(P / r) groups of consecutive nodes; left-over nodes dealt to the first groups.
+void group_layout(int P, int r, std::vector<int>* start) {
+  int q = P / r;
+  int extra = P - q * r;
+  start->assign(q + 1, 0);
+  for (int g = 0; g < q; ++g) {
+    int size = r + extra / q + (g < extra % q ? 1 : 0);
+    (*start)[g + 1] = (*start)[g] + size;
+  }
+}
+
+// Chebyshev points of the first kind, n' = group size rounded up to even (so none is zero).
+void node_scalars(const std::vector<int>& start, std::vector<double>* w) {
+  const double pi = 3.14159265358979323846;
+  int q = (int)start.size() - 1;
+  w->assign(start[q], 0.0);
+  for (int g = 0; g < q; ++g) {
+    int size = start[g + 1] - start[g];
+    int n_prime = size + (size & 1);
+    for (int k = 1; k <= size; ++k) (*w)[start[g] + k - 1] = cos((2 * k - 1) * pi / (2.0 * n_prime));
+  }
+}
+
+// ---- projection vectors: f[kappa][p] = 1 + N(0,1), Philox4x32-10 counters + Box-Muller -------------
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t out[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0;
+    k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+__global__ void fill_projection_kernel(float* __restrict__ f, int64_t d_c, int64_t pitch, int K, uint64_t seed) {
+  int64_t quads = (d_c + 3) / 4;
+  int64_t total = quads * K;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int kappa = (int)(i / quads);
+    int64_t quad = i - (int64_t)kappa * quads;
+    uint32_t x[4];
+    philox4x32_10((uint32_t)quad, (uint32_t)(quad >> 32), (uint32_t)kappa, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+    float v[4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float u1 = ((float)x[2 * h] + 0.5f) * 2.3283064365386963e-10f;       // (0, 1]
+      float u2 = ((float)x[2 * h + 1] + 0.5f) * 2.3283064365386963e-10f;
+      u1 = fminf(fmaxf(u1, 1.0e-12f), 1.0f);
+      float rad = sqrtf(-2.0f * logf(u1));
+      float sn, cs;
+      sincospif(2.0f * u2, &sn, &cs);
+      v[2 * h] = 1.0f + rad * cs;
+      v[2 * h + 1] = 1.0f + rad * sn;
+    }
+    float* row = f + (int64_t)kappa * pitch + quad * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) row[e] = (quad * 4 + e < d_c) ? v[e] : 0.0f;   // pitch is a multiple of 4
+  }
+}
+
+int launch_fill_projection(solon_plan* plan) {
+  int64_t total = ((plan->d_c + 3) / 4) * plan->K;
+  int threads = 256;
+  int64_t want = (total + threads - 1) / threads;
+  int blocks = (int)(want < (int64_t)plan->num_sms * 8 ? (want < 1 ? 1 : want) : (int64_t)plan->num_sms * 8);
+  fill_projection_kernel<<<blocks, threads, 0, plan->stream>>>(plan->d_f, plan->d_c, plan->f_pitch, plan->K, plan->seed);
+  plan->launches += 1;
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
+template <typename T>
+static int dev_alloc(T** ptr, size_t count) {
+  *ptr = nullptr;
+  if (count == 0) count = 1;
+  cudaError_t err = cudaMalloc((void**)ptr, count * sizeof(T));
+  if (err != cudaSuccess) {
+    (void)cudaGetLastError();
+    return err == cudaErrorMemoryAllocation ? SOLON_ERR_NOMEM : SOLON_ERR_CUDA;
+  }
+  return SOLON_OK;
+}
+
+static void free_device(solon_plan* p) {
+  cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f);
+  cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
+  cudaFree(p->d_task_records); cudaFree(p->d_task_flags); cudaFree(p->d_group_ticket); cudaFree(p->d_locate_ws);
+  cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status);
+  cudaFree(p->d_resid);
+  cudaFree(p->d_stage_grads); cudaFree(p->d_stage_coded); cudaFree(p->d_stage_agg); cudaFree(p->d_stage_mask);
+  (void)cudaGetLastError();
+}
+
+static int alloc_projection(solon_plan* p) {
+  int rc;
+  cudaFree(p->d_f); cudaFree(p->d_partials); cudaFree(p->d_rho);
+  cudaFree(p->d_locate_ws);
+  (void)cudaGetLastError();
+  p->d_f = nullptr; p->d_partials = nullptr; p->d_rho = nullptr; p->d_locate_ws = nullptr;
+  if ((rc = dev_alloc(&p->d_f, (size_t)p->K * p->f_pitch))) return rc;
+  if ((rc = dev_alloc(&p->d_partials, (size_t)p->proj_grid * (p->K + 1) * p->P))) return rc;
+  if ((rc = dev_alloc(&p->d_rho, (size_t)p->K * p->P))) return rc;
+  p->locate_ws_stride = locate_ws_doubles(p->max_group, p->m, p->K, p->s);
+  if ((rc = dev_alloc(&p->d_locate_ws, (size_t)p->q * (p->s + 1) * p->locate_ws_stride))) return rc;
+  return SOLON_OK;
+}
+
+}  // namespace solon
+
+using namespace solon;
+
+extern "C" {
+
+int solon_check_params(int P, int s, int m, int r, int64_t d) { return check_params(P, s, m, r, d); }
+
+int solon_group_layout(int P, int r, int* starts, int starts_capacity, int* q_out) {
+  if (!starts || !q_out || P < 1 || r < 1 || r > P) return SOLON_ERR_INVALID_ARG;
+  std::vector<int> start;
+  group_layout(P, r, &start);
+  if ((int)start.size() > starts_capacity) return SOLON_ERR_INVALID_ARG;
+  memcpy(starts, start.data(), start.size() * sizeof(int));
+  *q_out = (int)start.size() - 1;
+  return SOLON_OK;
+}
+
+int solon_node_scalars(int P, int r, double* w) {
+  if (!w || P < 1 || r < 1 || r > P) return SOLON_ERR_INVALID_ARG;
+  std::vector<int> start;
+  std::vector<double> ws;
+  group_layout(P, r, &start);
+  node_scalars(start, &ws);
+  memcpy(w, ws.data(), ws.size() * sizeof(double));
+  return SOLON_OK;
+}
+
+const char* solon_strerror(int status) {
+  switch (status) {
+    case SOLON_OK: return "ok";
+    case SOLON_ERR_INVALID_ARG: return "invalid argument";
+    case SOLON_ERR_INFEASIBLE: return "infeasible: 2 s + m > P";
+    case SOLON_ERR_CUDA: return "CUDA error or no CUDA device";
+    case SOLON_ERR_UNDECODABLE: return "undecodable: more than s inconsistent nodes in a group";
+    case SOLON_ERR_INTERNAL: return "internal error: bounded device wait expired";
+    case SOLON_ERR_NOMEM: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solon_plan** out) {
+  if (!out) return SOLON_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_params(P, s, m, r, d);
+  if (rc) return rc;
+  std::vector<int> start;
+  group_layout(P, r, &start);
+  int q = (int)start.size() - 1;
+  int max_group = 0;
+  for (int g = 0; g < q; ++g) max_group = start[g + 1] - start[g] > max_group ? start[g + 1] - start[g] : max_group;
+  if (max_group > SOLON_MAX_GROUP) return SOLON_ERR_INVALID_ARG;
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1) {
+    (void)cudaGetLastError();
+    return SOLON_ERR_CUDA;
+  }
+  solon_plan* p = new (std::nothrow) solon_plan();
+  if (!p) return SOLON_ERR_NOMEM;
+  p->P = P; p->s = s; p->m = m; p->r = r; p->K = 2; p->d = d; p->d_c = (d + m - 1) / m;
+  p->seed = seed; p->tau = 1e-5; p->lsq_rows = 256; p->stream = 0; p->launches = 0;
+  p->group_start = start; p->q = q; p->max_group = max_group;
+  p->group_of.assign(P, 0);
+  for (int g = 0; g < q; ++g)
+    for (int k = start[g]; k < start[g + 1]; ++k) p->group_of[k] = g;
+  node_scalars(start, &p->w);
+  p->f_pitch = (p->d_c + 3) / 4 * 4;
+
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&p->device) != cudaSuccess || cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) {
+    (void)cudaGetLastError();
+    delete p;
+    return SOLON_ERR_CUDA;
+  }
+  p->num_sms = prop.multiProcessorCount;
+  p->proj_grid = p->num_sms * 2;
+
+  rc = SOLON_OK;
+  do {
+    if ((rc = dev_alloc(&p->d_group_start, q + 1))) break;
+    if ((rc = dev_alloc(&p->d_group_of, P))) break;
+    if ((rc = dev_alloc(&p->d_w, P))) break;
+    if ((rc = alloc_projection(p))) break;
+    if ((rc = dev_alloc(&p->d_nu, P))) break;
+    if ((rc = dev_alloc(&p->d_proj_ticket, 1))) break;
+    TaskRecord* recs = nullptr;
+    if ((rc = dev_alloc(&recs, (size_t)q * (s + 1)))) break;
+    p->d_task_records = recs;
+    if ((rc = dev_alloc(&p->d_task_flags, (size_t)(s + 1) * P))) break;
+    if ((rc = dev_alloc(&p->d_group_ticket, q))) break;
+    if ((rc = dev_alloc(&p->d_t_acc, q))) break;
+    if ((rc = dev_alloc(&p->d_n_rec, q))) break;
+    if ((rc = dev_alloc(&p->d_rec_rows, P))) break;
+    if ((rc = dev_alloc(&p->d_coeff, (size_t)P * m))) break;
+    if ((rc = dev_alloc(&p->d_status, 2))) break;
+    cudaError_t e = cudaSuccess;
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_group_start, start.data(), (q + 1) * sizeof(int), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_group_of, p->group_of.data(), P * sizeof(int), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_w, p->w.data(), P * sizeof(double), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_group_ticket, 0, q * sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 2 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_n_rec, 0, q * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_t_acc, 0, q * sizeof(int));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); rc = SOLON_ERR_CUDA; break; }
+    if ((rc = launch_fill_projection(p))) break;
+    if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); rc = SOLON_ERR_CUDA; break; }
+  } while (0);
+  if (rc) {
+    free_device(p);
+    delete p;
+    return rc;
+  }
+  *out = p;
+  return SOLON_OK;
+}
+
+int solon_plan_destroy(solon_plan* plan) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  cudaStreamSynchronize(plan->stream);
+  free_device(plan);
+  delete plan;
+  return SOLON_OK;
+}
+
+int solon_plan_set_stream(solon_plan* plan, void* cuda_stream) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  plan->stream = (cudaStream_t)cuda_stream;
+  return SOLON_OK;
+}
+
+int solon_plan_set_num_projections(solon_plan* plan, int K) {
+  if (!plan || K < 1 || K > SOLON_MAX_PROJECTIONS) return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  plan->K = K;
+  int rc = alloc_projection(plan);
+  if (rc) return rc;
+  if ((rc = launch_fill_projection(plan))) return rc;
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  return SOLON_OK;
+}
+
+int solon_plan_reseed(solon_plan* plan, uint64_t seed) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  plan->seed = seed;
+  return launch_fill_projection(plan);
+}
+
+int solon_plan_set_tolerance(solon_plan* plan, double tau) {
+  if (!plan || !(tau >= 0.0)) return SOLON_ERR_INVALID_ARG;
+  plan->tau = tau;
+  return SOLON_OK;
+}
+
+int solon_plan_set_lsq_rows(solon_plan* plan, int rows) {
+  if (!plan || rows < 1) return SOLON_ERR_INVALID_ARG;
+  plan->lsq_rows = rows;
+  return SOLON_OK;
+}
+
+int64_t solon_plan_dc(const solon_plan* plan) { return plan ? plan->d_c : SOLON_ERR_INVALID_ARG; }
+int solon_plan_num_groups(const solon_plan* plan) { return plan ? plan->q : SOLON_ERR_INVALID_ARG; }
+int solon_plan_num_projections(const solon_plan* plan) { return plan ? plan->K : SOLON_ERR_INVALID_ARG; }
+int solon_plan_group_of(const solon_plan* plan, int node) {
+  if (!plan || node < 0 || node >= plan->P) return SOLON_ERR_INVALID_ARG;
+  return plan->group_of[node];
+}
+int solon_plan_group_start(const solon_plan* plan, int group) {
+  if (!plan || group < 0 || group >= plan->q) return SOLON_ERR_INVALID_ARG;
+  return plan->group_start[group];
+}
+int solon_plan_group_size(const solon_plan* plan, int group) {
+  if (!plan || group < 0 || group >= plan->q) return SOLON_ERR_INVALID_ARG;
+  return plan->group_start[group + 1] - plan->group_start[group];
+}
+int solon_plan_get_node_scalars(const solon_plan* plan, double* w) {
+  if (!plan || !w) return SOLON_ERR_INVALID_ARG;
+  memcpy(w, plan->w.data(), plan->P * sizeof(double));
+  return SOLON_OK;
+}
+int solon_plan_get_projection_vectors(solon_plan* plan, float* f) {
+  if (!plan || !f) return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaMemcpy2DAsync(f, plan->d_c * sizeof(float), plan->d_f, plan->f_pitch * sizeof(float),
+                                   plan->d_c * sizeof(float), plan->K, cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  return SOLON_OK;
+}
+
+int solon_plan_get_projections(solon_plan* plan, double* rho, double* nu) {
+  if (!plan || !rho || !nu) return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(rho, plan->d_rho, (size_t)plan->K * plan->P * sizeof(double), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaMemcpyAsync(nu, plan->d_nu, (size_t)plan->P * sizeof(double), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  return SOLON_OK;
+}
+
+int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows, double* coeff) {
+  if (!plan || !n_rec || !t || !rec_rows || !coeff) return SOLON_ERR_INVALID_ARG;
+  std::vector<int> rows(plan->P);
+  std::vector<double> cf((size_t)plan->P * plan->m);
+  SOLON_CUDA_TRY(cudaMemcpyAsync(n_rec, plan->d_n_rec, plan->q * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaMemcpyAsync(t, plan->d_t_acc, plan->q * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaMemcpyAsync(rows.data(), plan->d_rec_rows, plan->P * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaMemcpyAsync(cf.data(), plan->d_coeff, cf.size() * sizeof(double), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  size_t out = 0;
+  for (int g = 0; g < plan->q; ++g) {
+    int base = plan->group_start[g];
+    for (int j = 0; j < n_rec[g]; ++j, ++out) {
+      rec_rows[out] = rows[base + j];
+      memcpy(coeff + out * plan->m, cf.data() + (size_t)(base + j) * plan->m, plan->m * sizeof(double));
+    }
+  }
+  return SOLON_OK;
+}
+
+int64_t solon_plan_kernel_launches(const solon_plan* plan) { return plan ? plan->launches : SOLON_ERR_INVALID_ARG; }
+
+int solon_decode_status(solon_plan* plan) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  int word[2] = {0, 0};
+  SOLON_CUDA_TRY(cudaMemcpyAsync(word, plan->d_status, 2 * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  if ((word[0] | word[1]) & kStatusWaitExpired) return SOLON_ERR_INTERNAL;
+  if (word[0] & kStatusUndecodable) return SOLON_ERR_UNDECODABLE;
+  return SOLON_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,171 @@
+// Detection projections (Section 3.4): rho[kappa][k] = f_kappa . R_k for the K random vectors f_kappa
+// and all P received rows, plus the row energies nu[k] = ||R_k||^2 that scale the locator's tolerance.
+//
+// One pass over the P x d_c received matrix.  Every CTA owns one contiguous range of the chunk axis,
+// walks it in tiles, keeps the tile of f in shared memory as float64 and lets each warp stream its own
+// rows (two at a time) against it, so each received byte is read once and f is read once per CTA.
+// Products are exact in float64 and accumulated in float64; nu is accumulated in float32 per lane and
+// in float64 across lanes and tiles.  Per-CTA partial sums go to global memory; the last CTA to
+// finish (atomic ticket, no waiting) adds them in a fixed order, so results are bit-reproducible.
+#include "solon_internal.h"
+
+namespace solon {
+
+constexpr int kProjThreads = 256;
+constexpr int kProjWarps = kProjThreads / 32;
+
+template <int K>
+struct ProjAcc {
+  double rho[K];
+  float nu;
+};
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+template <int K>
+__global__ void __launch_bounds__(kProjThreads) project_kernel(const float* __restrict__ R, const float* __restrict__ f,
+                                                               int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
+                                                               int tile_cols, double* __restrict__ partials,
+                                                               double* __restrict__ rho_out, double* __restrict__ nu_out,
+                                                               unsigned int* ticket) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* fs = reinterpret_cast<double*>(smem_raw);            // K x tile_cols
+  double* sacc = fs + (size_t)K * tile_cols;                  // P x (K + 1)
+  __shared__ unsigned int s_ticket;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_acc = (K + 1) * P;
+  for (int i = tid; i < n_acc; i += kProjThreads) sacc[i] = 0.0;
+
+  const int64_t c_begin = (int64_t)blockIdx.x * range_len;
+  int64_t c_end = c_begin + range_len;
+  if (c_end > d_c) c_end = d_c;
+
+  for (int64_t c0 = c_begin; c0 < c_end; c0 += tile_cols) {
+    const int cols = (int)((c_end - c0) < tile_cols ? (c_end - c0) : tile_cols);
+    __syncthreads();   // previous tile fully consumed (also orders the zeroing of sacc)
+    // f tile -> float64 shared memory; c0 is a multiple of 4 and f rows are 16-byte aligned
+    for (int i = tid * 4; i < cols; i += kProjThreads * 4) {
+#pragma unroll
+      for (int kappa = 0; kappa < K; ++kappa) {
+        const float* src = f + (int64_t)kappa * f_pitch + c0 + i;
+        float4 v = *reinterpret_cast<const float4*>(src);     // pitch padding keeps this in bounds
+        double* dst = fs + (size_t)kappa * tile_cols + i;
+        dst[0] = (double)v.x;
+        if (i + 1 < cols) dst[1] = (double)v.y;
+        if (i + 2 < cols) dst[2] = (double)v.z;
+        if (i + 3 < cols) dst[3] = (double)v.w;
+      }
+    }
+    __syncthreads();
+    // rows in batches of two; batch b belongs to warp b mod kProjWarps
+    for (int row = warp * 2; row < P; row += kProjWarps * 2) {
+      const bool two = row + 1 < P;
+      const float* ra = R + (int64_t)row * d_c + c0;
+      const float* rb = two ? ra + d_c : ra;
+      double a_rho[K], b_rho[K];
+      float a_nu = 0.f, b_nu = 0.f;
+#pragma unroll
+      for (int kappa = 0; kappa < K; ++kappa) a_rho[kappa] = b_rho[kappa] = 0.0;
+      int c = lane;
+      for (; c + 7 * 32 < cols; c += 8 * 32) {
+        float va[8], vb[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          va[u] = __ldcs(ra + c + u * 32);
+          vb[u] = __ldcs(rb + c + u * 32);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const double da = (double)va[u], db = (double)vb[u];
+#pragma unroll
+          for (int kappa = 0; kappa < K; ++kappa) {
+            const double fv = fs[(size_t)kappa * tile_cols + c + u * 32];
+            a_rho[kappa] = fma(fv, da, a_rho[kappa]);
+            b_rho[kappa] = fma(fv, db, b_rho[kappa]);
+          }
+          a_nu = fmaf(va[u], va[u], a_nu);
+          b_nu = fmaf(vb[u], vb[u], b_nu);
+        }
+      }
+      for (; c < cols; c += 32) {
+        const float va = __ldcs(ra + c), vb = __ldcs(rb + c);
+        const double da = (double)va, db = (double)vb;
+#pragma unroll
+        for (int kappa = 0; kappa < K; ++kappa) {
+          const double fv = fs[(size_t)kappa * tile_cols + c];
+          a_rho[kappa] = fma(fv, da, a_rho[kappa]);
+          b_rho[kappa] = fma(fv, db, b_rho[kappa]);
+        }
+        a_nu = fmaf(va, va, a_nu);
+        b_nu = fmaf(vb, vb, b_nu);
+      }
+#pragma unroll
+      for (int kappa = 0; kappa < K; ++kappa) {
+        const double sa = warp_sum(a_rho[kappa]);
+        const double sb = warp_sum(b_rho[kappa]);
+        if (lane == 0) {
+          sacc[(size_t)kappa * P + row] += sa;
+          if (two) sacc[(size_t)kappa * P + row + 1] += sb;
+        }
+      }
+      const double na = warp_sum((double)a_nu), nb = warp_sum((double)b_nu);
+      if (lane == 0) {
+        sacc[(size_t)K * P + row] += na;
+        if (two) sacc[(size_t)K * P + row + 1] += nb;
+      }
+    }
+  }
+  __syncthreads();
+  double* mine = partials + (size_t)blockIdx.x * n_acc;
+  for (int i = tid; i < n_acc; i += kProjThreads) mine[i] = sacc[i];
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_ticket = atomicAdd(ticket, 1u);
+  __syncthreads();
+  if (s_ticket != gridDim.x - 1) return;
+  // last CTA: add the per-CTA partial sums in a fixed order (lane-strided, then a fixed shuffle tree)
+  __threadfence();
+  for (int i = warp; i < n_acc; i += kProjWarps) {
+    double acc = 0.0;
+    for (unsigned int b = lane; b < gridDim.x; b += 32) acc += __ldcg(partials + (size_t)b * n_acc + i);
+    acc = warp_sum(acc);
+    if (lane == 0) {
+      if (i < K * P) rho_out[i] = acc;
+      else nu_out[i - K * P] = acc;
+    }
+  }
+  if (tid == 0) *ticket = 0u;   // ready for the next decode
+}
+
+template <int K>
+static int launch_project_k(solon_plan* plan, const float* received) {
+  int tile_cols = K <= 2 ? 4096 : 2048;
+  int64_t range_len = (plan->d_c + plan->proj_grid - 1) / plan->proj_grid;
+  range_len = (range_len + 3) / 4 * 4;
+  if (range_len < tile_cols) tile_cols = (int)range_len;
+  size_t smem = (size_t)K * tile_cols * sizeof(double) + (size_t)(K + 1) * plan->P * sizeof(double);
+  if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(project_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  project_kernel<K><<<plan->proj_grid, kProjThreads, smem, plan->stream>>>(
+      received, plan->d_f, plan->f_pitch, plan->P, plan->d_c, range_len, tile_cols, plan->d_partials, plan->d_rho,
+      plan->d_nu, plan->d_proj_ticket);
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
+int launch_project(solon_plan* plan, const float* received) {
+  plan->launches += 1;
+  switch (plan->K) {
+    case 1: return launch_project_k<1>(plan, received);
+    case 2: return launch_project_k<2>(plan, received);
+    case 3: return launch_project_k<3>(plan, received);
+    case 4: return launch_project_k<4>(plan, received);
+    default: return SOLON_ERR_INVALID_ARG;
+  }
+}
+
+}  // namespace solon

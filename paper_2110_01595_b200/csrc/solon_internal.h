@@ -1,0 +1,111 @@
+// Internal definitions shared by the translation units of libsolon (not part of the C interface).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/solon.h"
+
+#define SOLON_CUDA_TRY(expr)                   \
+  do {                                         \
+    cudaError_t solon_err__ = (expr);          \
+    if (solon_err__ != cudaSuccess) {          \
+      (void)cudaGetLastError();                \
+      return SOLON_ERR_CUDA;                   \
+    }                                          \
+  } while (0)
+
+namespace solon {
+
+// Device-side view of the group layout, passed by value to kernels.
+struct GroupTable {
+  const int* start;   // q + 1 entries, device
+  const double* w;    // P node scalars, device
+  int q;
+  int P;
+};
+
+// Bit positions of the device status word.
+enum : int {
+  kStatusUndecodable = 1,  // some group had no consistent set of <= s corrupt nodes
+  kStatusWaitExpired = 2,  // a bounded wait on a shared-memory barrier ran out
+};
+
+}  // namespace solon
+
+struct solon_plan {
+  int P, s, m, r, K;
+  int64_t d, d_c;
+  uint64_t seed;
+  double tau;
+  int lsq_rows;
+  cudaStream_t stream;
+  int device;
+  int num_sms;
+  int64_t launches;
+
+  // host copies
+  std::vector<int> group_start;   // q + 1
+  std::vector<int> group_of;      // P
+  std::vector<double> w;          // P
+  int q;
+  int max_group;
+
+  // device tables
+  int* d_group_start;      // q + 1
+  int* d_group_of;         // P
+  double* d_w;             // P (float64 node scalars)
+  float* d_f;              // K x f_pitch projection vectors
+  int64_t f_pitch;         // row pitch of d_f in floats (multiple of 4)
+
+  // projection workspace
+  int proj_grid;           // CTAs of the projection kernel = number of partial sums
+  double* d_partials;      // proj_grid x (K + 1) x P
+  double* d_rho;           // K x P
+  double* d_nu;            // P
+  unsigned int* d_proj_ticket;   // 1
+
+  // locator workspace / outputs
+  void* d_task_records;    // q x (s + 1) TaskRecord
+  uint8_t* d_task_flags;   // (s + 1) x P
+  unsigned int* d_group_ticket;  // q
+  double* d_locate_ws;     // q x (s + 1) x locate_ws_stride doubles (global fallback workspace)
+  size_t locate_ws_stride;
+  int* d_t_acc;            // q
+  int* d_n_rec;            // q
+  int* d_rec_rows;         // P   (global node index of the j-th recovery row of group g at start[g] + j)
+  double* d_coeff;         // P x m
+  int* d_status;           // [0] status bits of the last decode, [1] sticky bits (expired waits)
+
+  // lsq workspace
+  float* d_resid;          // P * lsq_rows
+  int64_t resid_capacity;
+
+  // host-step staging (allocated on first use)
+  float* d_stage_grads;
+  float* d_stage_coded;
+  float* d_stage_agg;
+  uint8_t* d_stage_mask;
+};
+
+namespace solon {
+
+// Kernel launchers (each enqueues on plan->stream and returns a solon_status).
+int launch_fill_projection(solon_plan* plan);
+int launch_encode(solon_plan* plan, const float* grads, float* coded);
+int launch_project(solon_plan* plan, const float* received);
+int launch_locate(solon_plan* plan, uint8_t* byz_mask);
+int launch_recover(solon_plan* plan, const float* received, float* agg);
+int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w, float* grads);
+
+// Doubles of workspace one locator CTA needs for a group of n nodes.
+size_t locate_ws_doubles(int n, int m, int K, int s);
+
+// Host-side layout rules (also used by the plan-free helpers).
+int check_params(int P, int s, int m, int r, int64_t d);
+void group_layout(int P, int r, std::vector<int>* start);
+void node_scalars(const std::vector<int>& start, std::vector<double>* w);
+
+}  // namespace solon

@@ -1,0 +1,91 @@
+// Shared-memory pipeline primitives for sm_100a: mbarrier objects, bulk asynchronous copies
+// (cp.async.bulk, global -> shared, completion counted in bytes on an mbarrier) and named barriers.
+// Every wait is bounded in time: when it expires the waiter raises the CTA's abort flag and a bit in
+// a global status word, and all later waits of that CTA return at once, so the kernel always ends.
+#pragma once
+
+#include <stdint.h>
+
+namespace solon {
+namespace pipe {
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per CTA before giving up
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_addr(bar)),
+               "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Wait for the phase with the given parity to complete.  Bounded: after kWaitLimitNs the abort flag
+// (shared) and bit 1 of *status (global) are set and the call returns as if the wait had succeeded.
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* abort_flag, int* status) {
+  if (mbar_try_wait(bar, parity)) return;
+  if (*(volatile int*)abort_flag) return;
+  const unsigned long long t0 = global_timer_ns();
+  uint32_t polls = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++polls & 63u) == 0) {
+      if (*(volatile int*)abort_flag) return;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *(volatile int*)abort_flag = 1;
+        atomicOr(status, 2);
+        return;
+      }
+    }
+  }
+}
+
+// After an expired wait: give copies that may still be in flight a bounded time (1 ms) to land.
+__device__ __forceinline__ void drain_delay() {
+  const unsigned long long t0 = global_timer_ns();
+  while (global_timer_ns() - t0 < 1000000ull) __nanosleep(1000);
+}
+
+// 1-D bulk copy global -> shared; src, dst 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_addr(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+}  // namespace pipe
+}  // namespace solon

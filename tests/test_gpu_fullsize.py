@@ -1,0 +1,66 @@
+"""GPU parity at the full sizes of the ResNet-18-sized and VGG-13-sized configurations, in the launch
+configuration the benchmark times: inputs are generated on the device, and the oracle checks sampled
+outputs one by one (coded chunks, aggregate coordinates) plus the mask, which is known exactly."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import solon_oracle as so
+from paper_2110_01595_b200 import binding, build, synth
+
+pytestmark = pytest.mark.gpu
+
+AGG_TOL = 1e-4
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def _sample_chunks(d_c, n, seed):
+    rng = np.random.default_rng(seed)
+    picks = rng.integers(0, d_c, size=n)
+    edges = np.array([0, 1, 255, 256, 257, d_c // 2, d_c - 257, d_c - 256, d_c - 2, d_c - 1])
+    return np.unique(np.clip(np.concatenate([picks, edges]), 0, d_c - 1))
+
+
+@pytest.mark.parametrize("name", ["resnet18", "vgg13", "vgg13_clean"])
+def test_full_size(name):
+    wl = synth.WORKLOADS[name]
+    sizes = so.group_sizes(wl.P, wl.r)
+    w = so.node_scalars(sizes)
+    G = synth.make_grads(wl, "cuda")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.cpu().numpy().nonzero()[0].tolist() == nodes                  # bit-exact mask
+        chunks = _sample_chunks(plan.d_c, 4000, wl.seed)
+        # coded vectors of the sampled chunks: oracle encode of the matching gradient slices
+        cols = (chunks[:, None] * wl.m + np.arange(wl.m)[None, :]).reshape(-1)
+        in_range = cols < wl.d
+        G_s = np.zeros((wl.P, cols.size), dtype=np.float32)
+        G_s[:, in_range] = G[:, torch.from_numpy(cols[in_range]).cuda()].cpu().numpy()
+        Z_s = so.encode(G_s, wl.m, sizes, w)                                       # P x len(chunks)
+        got_Z = coded[:, torch.from_numpy(chunks).cuda()].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got_Z - Z_s) <= 2.0 ** -24 * 1.0001 * np.abs(Z_s) + 1e-13 * np.abs(G_s).max() * wl.P)
+        # aggregate at the sampled coordinates against the plain float64 sum
+        want_s = so.plain_sum(G_s)[in_range]
+        got_s = agg[torch.from_numpy(cols[in_range]).cuda()].cpu().numpy().astype(np.float64)
+        scale = float(G.sum(dim=0, dtype=torch.float64).abs().max())              # ||sum||_inf over all of d
+        assert np.abs(got_s - want_s).max() <= AGG_TOL * scale
+        # a property that holds at any size: the whole aggregate against a float64 device-side sum
+        ref = G.sum(dim=0, dtype=torch.float64)
+        assert float((agg.double() - ref).abs().max()) <= AGG_TOL * scale
+        if name == "resnet18":
+            # projections of the full received matrix against the oracle's matrix product
+            f = plan.projection_vectors()
+            R = received.cpu().numpy()
+            rho, nu = plan.projections()
+            o_rho, o_nu = so.project(R, f), so.row_energy(R)
+            lim = np.sqrt((f.astype(np.float64) ** 2).sum(1))[:, None] * np.sqrt(o_nu)[None, :]
+            assert np.all(np.abs(rho - o_rho) <= 1e-11 * lim)
+            assert np.allclose(nu, o_nu, rtol=1e-4)

@@ -1,0 +1,292 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the float64 oracle on the same
+seeded inputs.  Bars: Byzantine mask bit-exact; aggregate within 1e-4 of ||sum||_inf; coded vectors within
+one float32 rounding of the oracle's float64 values; projections to float64 accuracy."""
+
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import solon_oracle as so
+from paper_2110_01595_b200 import binding, build, synth
+
+pytestmark = pytest.mark.gpu
+
+AGG_TOL = 1e-4          # max |agg_gpu - agg*| / ||agg*||_inf
+TAU = 1e-5              # the library's default detection tolerance, also given to the oracle
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _oracle_plan(wl):
+    sizes = so.group_sizes(wl.P, wl.r)
+    return sizes, so.node_scalars(sizes)
+
+
+def _check_encode(plan, G_cpu, coded_gpu, m, sizes, w):
+    Z = so.encode(G_cpu.numpy(), m, sizes, w)
+    got = coded_gpu.cpu().numpy().astype(np.float64)
+    # float64 evaluation rounded once to float32: half an ulp of the value, plus float64 reordering noise
+    absG = np.abs(G_cpu.numpy()).astype(np.float64)
+    bound = np.zeros_like(Z)
+    for start, size in zip(so.group_starts(sizes), sizes):
+        s_abs = so.group_sum(absG, start, size, m).reshape(-1, m)
+        for k in range(start, start + size):
+            bound[k] = s_abs @ np.abs(w[k]) ** np.arange(m)
+    err = np.abs(got - Z)
+    assert np.all(err <= 2.0 ** -24 * np.abs(Z) * 1.0001 + 1e-14 * bound + 1e-45), float((err / (np.abs(Z) + 1e-30)).max())
+    return Z
+
+
+def _run_case(wl, n_byz=None, check_intermediates=True):
+    """Encode on the GPU, attack, decode on the GPU; compare everything with the oracle."""
+    if n_byz is not None:
+        wl = dataclasses.replace(wl, n_byz=n_byz, fixed_byz=(), attack=wl.attack if n_byz else "none")
+    sizes, w = _oracle_plan(wl)
+    G_cpu = synth.make_grads(wl, "cpu")
+    G = G_cpu.cuda()
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        assert plan.group_sizes() == sizes
+        assert np.allclose(plan.node_scalars(), w, rtol=0, atol=1e-15)
+        coded = plan.encode(G)
+        torch.cuda.synchronize()
+        if check_intermediates:
+            _check_encode(plan, G_cpu, coded, wl.m, sizes, w)
+        received, nodes = synth.apply_attack(wl, coded)
+        agg, mask = plan.decode(received)
+        status = plan.decode_status()
+        assert status == 0, binding.strerror(status)
+        R = received.cpu().numpy()
+        want_mask = so.true_mask(R, coded.cpu().numpy())
+        assert want_mask.nonzero()[0].tolist() == nodes
+        assert np.array_equal(mask.cpu().numpy(), want_mask)                       # bit-exact
+        want = so.plain_sum(G_cpu.numpy())
+        scale = np.abs(want).max()
+        got = agg.cpu().numpy().astype(np.float64)
+        assert np.abs(got - want).max() <= AGG_TOL * scale, np.abs(got - want).max() / scale
+        # the oracle's own decode of the very same received matrix (Algorithm 1 in float64)
+        f = plan.projection_vectors()
+        u, o_mask, o_status = so.decode(R, wl.d, wl.m, wl.s, sizes, w, f, tau=TAU)
+        assert o_status == 0 and np.array_equal(o_mask, want_mask)
+        assert np.abs(got - u).max() <= AGG_TOL * scale
+        if check_intermediates and wl.s > 0:
+            rho, nu = plan.projections()
+            o_rho = so.project(R, f)
+            o_nu = so.row_energy(R)
+            f64 = f.astype(np.float64)
+            lim = np.sqrt((f64 ** 2).sum(1))[:, None] * np.sqrt(o_nu)[None, :]
+            assert np.all(np.abs(rho - o_rho) <= 1e-12 * lim + 1e-300)
+            assert np.allclose(nu, o_nu, rtol=1e-4)
+            n_rec, t_acc, rows, coeff = plan.recovery()
+            starts = so.group_starts(sizes)
+            off = 0
+            for g, (start, size) in enumerate(zip(starts, sizes)):
+                in_group = [k for k in nodes if start <= k < start + size]
+                assert t_acc[g] == len(in_group)
+                rg = rows[off:off + n_rec[g]]
+                assert n_rec[g] == (wl.m if wl.m <= 6 else size - len(in_group))
+                assert all(start <= k < start + size and k not in nodes for k in rg)
+                Wm = so.w_hat(w[start:start + size], wl.m - 1)[rg - start]
+                assert np.allclose(coeff[off:off + n_rec[g]].T @ Wm, np.eye(wl.m), atol=1e-8)
+                off += n_rec[g]
+        return np.abs(got - want).max() / scale
+
+
+# ---------------------------------------------------------------- the five configurations, small
+
+
+def test_config_tiny():
+    _run_case(synth.WORKLOADS["tiny"])
+
+
+def test_config_resnet18_shape_small():
+    # same plan, layered sigma profile and attack; spans many encode tiles and a ragged tail (d % m != 0)
+    _run_case(synth.small_variant(synth.WORKLOADS["resnet18"], 1_117_397))
+
+
+def test_config_vgg13_shape_small():
+    _run_case(synth.small_variant(synth.WORKLOADS["vgg13"], 283_321))
+    _run_case(synth.small_variant(synth.WORKLOADS["vgg13_clean"], 283_321))
+
+
+@pytest.mark.parametrize("P,s,m", [(15, 1, 1), (15, 1, 2), (15, 1, 5), (15, 1, 10), (15, 3, 5), (15, 5, 2), (15, 5, 5),
+                                   (45, 1, 10), (45, 3, 1), (45, 3, 10), (45, 5, 5), (45, 5, 10), (105, 1, 1),
+                                   (105, 3, 5), (105, 5, 10), (105, 5, 2)])
+def test_config_sweep_small(P, s, m):
+    wl = synth.Workload(f"sweep_P{P}_s{s}_m{m}", P, s, m, 100_003, "normal", 1.0, "gaussian", s, 5000 + P + 10 * s + m)
+    _run_case(wl)
+
+
+def test_config_lsq_small():
+    wl = dataclasses.replace(synth.WORKLOADS["lsq"], d=5_003, lsq_rows=64)
+    sizes, w = _oracle_plan(wl)
+    X, y, wvec = synth.make_lsq_problem(wl, "cpu")
+    want_G = so.lsq_grads(X.numpy(), y.numpy(), wvec.numpy(), wl.lsq_rows)
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        G = plan.lsq_grads(X.cuda(), y.cuda(), wvec.cuda(), rows=wl.lsq_rows)
+        got_G = G.cpu().numpy().astype(np.float64)
+        Xa = np.abs(X.numpy()).astype(np.float64)
+        e = np.abs(X.numpy().astype(np.float64) @ wvec.numpy().astype(np.float64) - y.numpy())
+        for i in range(wl.P):
+            rows = slice(i * wl.lsq_rows, (i + 1) * wl.lsq_rows)
+            bound = Xa[rows].T @ e[rows]                      # sum of |terms|
+            assert np.all(np.abs(got_G[i] - want_G[i]) <= 3e-7 * bound + 1e-30)
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.cpu().numpy().nonzero()[0].tolist() == nodes and len(nodes) == 1
+        want = want_G.sum(0)                                   # the oracle's own float64 gradients
+        assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+
+
+# ---------------------------------------------------------------- edge cases
+
+
+@pytest.mark.parametrize("P,s,m,r,d", [
+    (4, 1, 2, 4, 2),          # the introduction's example: d_c = 1
+    (5, 1, 3, 5, 1),          # d < m: one padded chunk
+    (5, 0, 5, 5, 23),         # s = 0: pure compression code, no locator
+    (9, 2, 1, 5, 1000),       # m = 1: repetition code
+    (7, 3, 1, 7, 255),        # maximal s for P
+    (16, 2, 4, 8, 4096),      # r divides P (the paper's layout), m = 4
+    (11, 1, 7, 9, 1234),      # m without a specialised kernel
+    (23, 1, 3, 23, 777),      # r = P, one odd-sized group
+    (40, 2, 12, 20, 3000),    # m = 12 (generic kernels), two groups of 20
+    (128, 1, 2, 128, 513),    # largest group the locator handles
+])
+def test_edge_shapes(P, s, m, r, d):
+    wl = synth.Workload("edge", P, s, m, d, "normal", 1.0, "gaussian", s, 99)
+    wl_r = dataclasses.replace(wl)
+    sizes = so.group_sizes(P, r)
+    w = so.node_scalars(sizes)
+    G_cpu = synth.make_grads(wl, "cpu")
+    with binding.Plan(P, s, m, r, d, seed=7) as plan:
+        assert plan.group_sizes() == sizes
+        coded = plan.encode(G_cpu.cuda())
+        _check_encode(plan, G_cpu, coded, m, sizes, w)
+        received, nodes = synth.apply_attack(wl_r, coded)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.cpu().numpy().nonzero()[0].tolist() == nodes
+        want = so.plain_sum(G_cpu.numpy())
+        tol = AGG_TOL if m <= 10 else 1e-2      # m = 12 is past the float32 budget (the paper warns above 14)
+        assert np.abs(agg.cpu().numpy() - want).max() <= tol * max(np.abs(want).max(), 1e-30)
+
+
+def test_all_attackers_in_one_group_and_every_count():
+    base = synth.Workload("placement", 45, 3, 5, 50_001, "normal", 1.0, "alie", 3, 321)
+    sizes, w = _oracle_plan(base)
+    G_cpu = synth.make_grads(base, "cpu")
+    want = so.plain_sum(G_cpu.numpy())
+    with binding.Plan(base.P, base.s, base.m, base.r, base.d, seed=1) as plan:
+        coded = plan.encode(G_cpu.cuda())
+        for nodes in ([], [0], [44], [12, 13], [33, 34, 35], [12, 22, 23], [0, 11, 44], [1, 5, 9, 13, 20, 25, 34, 40, 44]):
+            wl = dataclasses.replace(base, n_byz=len(nodes), fixed_byz=tuple(nodes), attack="alie" if nodes else "none")
+            received, _ = synth.apply_attack(wl, coded)
+            agg, mask = plan.decode(received)
+            assert plan.decode_status() == 0      # up to s = 3 per group, nine in total in the last case
+            assert mask.cpu().numpy().nonzero()[0].tolist() == nodes
+            assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+
+
+def test_non_finite_rows_are_located():
+    wl = synth.Workload("nan", 15, 2, 5, 20_000, "normal", 1.0, "none", 0, 11)
+    G_cpu = synth.make_grads(wl, "cpu")
+    want = so.plain_sum(G_cpu.numpy())
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
+        coded = plan.encode(G_cpu.cuda())
+        received = coded.clone()
+        received[4] = float("nan")
+        received[9, 17] = float("inf")
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.cpu().numpy().nonzero()[0].tolist() == [4, 9]
+        assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+
+
+def test_more_than_s_attackers_reports_undecodable():
+    wl = synth.Workload("over", 9, 2, 5, 10_000, "normal", 1.0, "gaussian", 3, 5, fixed_byz=(1, 4, 7))
+    G_cpu = synth.make_grads(wl, "cpu")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
+        coded = plan.encode(G_cpu.cuda())
+        received, _ = synth.apply_attack(wl, coded)
+        plan.decode(received)
+        assert plan.decode_status() == binding.ERR_UNDECODABLE
+        # the plan stays usable: a clean decode afterwards succeeds
+        agg, mask = plan.decode(coded)
+        assert plan.decode_status() == 0 and int(mask.sum()) == 0
+
+
+def test_decode_is_bit_reproducible_and_reusable():
+    wl = synth.small_variant(synth.WORKLOADS["vgg13"], 200_000)
+    G = synth.make_grads(wl, "cuda")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        a1, m1 = plan.decode(received)
+        r1 = plan.projections()
+        a2, m2 = plan.decode(received)
+        r2 = plan.projections()
+        assert torch.equal(a1, a2) and torch.equal(m1, m2)
+        assert np.array_equal(r1[0], r2[0]) and np.array_equal(r1[1], r2[1])
+        c2 = plan.encode(G)
+        assert torch.equal(coded, c2)
+
+
+def test_projection_settings():
+    wl = synth.small_variant(synth.WORKLOADS["resnet18"], 60_000)
+    G = synth.make_grads(wl, "cuda")
+    want = so.plain_sum(G.cpu().numpy())
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=3) as plan:
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        f2 = plan.projection_vectors()
+        assert abs(f2.mean() - 1.0) < 0.02 and abs(f2.std() - 1.0) < 0.02     # f ~ N(1, I)
+        for K in (1, 3, 4, 2):
+            plan.set_num_projections(K)
+            assert plan.projection_vectors().shape == (K, plan.d_c)
+            agg, mask = plan.decode(received)
+            assert plan.decode_status() == 0 and mask.cpu().numpy().nonzero()[0].tolist() == nodes
+            assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+        plan.reseed(12345)
+        f_new = plan.projection_vectors()
+        assert not np.array_equal(f_new, f2)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0 and mask.cpu().numpy().nonzero()[0].tolist() == nodes
+
+
+def test_step_host_matches_device_path():
+    wl = synth.small_variant(synth.WORKLOADS["resnet18"], 300_007)
+    G_cpu = synth.make_grads(wl, "cpu").pin_memory()
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
+        coded = plan.encode(G_cpu.cuda())
+        nodes = synth.byzantine_nodes(wl)
+        rows = synth.byzantine_rows(wl, coded, nodes).cpu().pin_memory()
+        agg_h = torch.empty(wl.d, dtype=torch.float32).pin_memory()
+        mask_h = torch.empty(wl.P, dtype=torch.uint8).pin_memory()
+        status = plan.step_host(G_cpu, nodes, rows, agg_h, mask_h)
+        assert status == 0
+        assert mask_h.numpy().nonzero()[0].tolist() == nodes
+        want = so.plain_sum(G_cpu.numpy())
+        assert np.abs(agg_h.numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+
+
+def test_argument_checks():
+    with binding.Plan(8, 1, 2, 4, 64) as plan:
+        lib = binding.lib()
+        assert lib.solon_encode(plan._h, None, None) == binding.ERR_INVALID_ARG
+        assert lib.solon_decode(plan._h, None, None, None) == binding.ERR_INVALID_ARG
+        buf = torch.zeros(8 * 64 + 4, dtype=torch.float32, device="cuda")
+        out = torch.zeros(8 * 32, dtype=torch.float32, device="cuda")
+        import ctypes
+        misaligned = ctypes.c_void_p(buf.data_ptr() + 4)
+        assert lib.solon_encode(plan._h, misaligned, ctypes.c_void_p(out.data_ptr())) == binding.ERR_INVALID_ARG
+    for args in ((15, 5, 10, 15, 100), (8, 1, 2, 3, 64), (8, 1, 2, 9, 64), (0, 0, 1, 1, 1), (300, 1, 2, 200, 64)):
+        with pytest.raises(binding.SolonError):
+            binding.Plan(*args)
