@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the Solon encode + robust-decode path on synthetic gradients.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vgg13] [--impl ours|reference]
+
+One step = encode all P partition gradients, let the Byzantine nodes overwrite their coded rows, decode
+(projections, locator, recovery + sum).  Prints ONE JSON line (rank 0).  With N > 1 (under torchrun) every
+rank runs its own independent problem on its own GPU: the path has no collective, scaling is weak.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2110_01595_b200 import dist_util, synth
+
+METRIC = "encode+decode gradient GB/s"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+
+
+def algorithmic_bytes(wl, n_rec_rows: int):
+    """Bytes each kernel must move (float32): encode 4 P d + 4 P d_c; projections 4 P d_c + 4 K d_c;
+    recovery 4 n_rows d_c + 4 d with n_rows the trusted rows the locator selected."""
+    d_c = wl.d_c
+    enc = 4 * wl.P * wl.d + 4 * wl.P * d_c
+    proj = 4 * wl.P * d_c + 4 * 2 * d_c
+    rec = 4 * n_rec_rows * d_c + 4 * wl.d
+    return enc, proj, rec
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines: list[str] = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_step_seconds(wl, G_host: np.ndarray, nodes, byz_rows_host, f_host: np.ndarray):
+    """One pass of the float64 oracle (encode, attack, decode) over the given gradient slice; returns seconds."""
+    from oracle import solon_oracle as so
+
+    sizes = so.group_sizes(wl.P, wl.r)
+    w = so.node_scalars(sizes)
+    t0 = time.perf_counter()
+    Z = so.encode(G_host, wl.m, sizes, w).astype(np.float32)
+    if len(nodes):
+        Z[nodes] = byz_rows_host
+    u, mask, status = so.decode(Z, G_host.shape[1], wl.m, wl.s, sizes, w, f_host, tau=1e-5)
+    dt = time.perf_counter() - t0
+    if status != 0 or mask.nonzero()[0].tolist() != sorted(nodes):
+        raise RuntimeError("oracle failed to decode its sample")
+    return dt
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+
+        counts = [info.get("num_threads", 1) for info in threadpool_info()]
+        return max(counts) if counts else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(wl, d_sample: int, device):
+    """A bounded sample of the workload for the CPU oracle: its first d_sample coordinates."""
+    import dataclasses
+
+    d_sample = min(d_sample, wl.d)
+    d_sample -= d_sample % wl.m
+    small = dataclasses.replace(wl, d=d_sample)
+    G = synth.make_grads(small, device)
+    G_host = G.cpu().numpy()
+    nodes = synth.byzantine_nodes(small)
+    from oracle import solon_oracle as so
+
+    sizes = so.group_sizes(wl.P, wl.r)
+    Z = torch.from_numpy(so.encode(G_host, wl.m, sizes, so.node_scalars(sizes)).astype(np.float32))
+    rows = synth.byzantine_rows(small, Z, nodes).numpy()
+    rng = np.random.default_rng(wl.seed)
+    f = (1.0 + rng.normal(size=(2, small.d_c))).astype(np.float32)
+    return small, G_host, nodes, rows, f
+
+
+# ----------------------------------------------------------------------------- arms
+
+
+def run_reference(args, wl):
+    """The oracle as it stands, timed on the host cores, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    small, G_host, nodes, rows, f = oracle_sample(wl, args.oracle_d, "cpu")
+    for _ in range(min(args.warmup, 1)):
+        oracle_step_seconds(small, G_host, nodes, rows, f)
+    times = [oracle_step_seconds(small, G_host, nodes, rows, f) for _ in range(args.steps)]
+    total = float(sum(times))
+    value = small.P * small.d * 4 * args.steps / total / 1e9
+    cores = blas_threads()
+    sample = f"first {small.d} of {wl.d} coordinates of every partition gradient, all {wl.P} nodes"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "sample_d": small.d},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, wl):
+    from paper_2110_01595_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist_util.init("nccl", device_id=local_rank)
+    build.build()
+
+    import dataclasses
+
+    wl_rank = dataclasses.replace(wl, seed=wl.seed + 17 * rank)      # every rank its own problem
+    G = synth.make_grads(wl_rank, "cuda")
+    plan = binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl_rank.seed)
+    coded = plan.encode(G)
+    nodes = synth.byzantine_nodes(wl_rank)
+    byz_rows = synth.byzantine_rows(wl_rank, coded, nodes)
+    agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+    mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
+
+    def step(events=None):
+        if events is not None:
+            events[0].record()
+        plan.encode(G, coded)
+        if events is not None:
+            events[1].record()
+        for i, k in enumerate(nodes):
+            coded[k].copy_(byz_rows[i])                       # the adversary: plain device-to-device copies
+        if events is not None:
+            events[2].record()
+        plan.decode(coded, agg, mask)
+        if events is not None:
+            events[3].record()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    status = plan.decode_status()
+    if status != 0 or mask.nonzero().flatten().tolist() != nodes:
+        raise RuntimeError(f"warm-up decode failed: status {status}")
+    n_rec, _, _, _ = plan.recovery()
+    enc_b, proj_b, rec_b = algorithmic_bytes(wl, int(n_rec.sum()))
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    launches0 = plan.kernel_launches()
+    dist_util.barrier()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(args.steps):
+        step(evs[i])
+    stop.record()
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    launches = plan.kernel_launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    status = plan.decode_status()
+    if status != 0 or mask.nonzero().flatten().tolist() != nodes:
+        raise RuntimeError(f"timed decode failed: status {status}")
+
+    enc_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    dec_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    units = wl.P * wl.d * 4 * args.steps                       # gradient bytes this rank processed
+    max_ms, total_units = dist_util.combine(elapsed_ms, units)
+
+    # end to end through the host-buffer entry point: pinned host memory in, host results out
+    e2e = None
+    if not args.no_e2e:
+        G_host = torch.empty((wl.P, wl.d), dtype=torch.float32).pin_memory()
+        G_host.copy_(G)
+        rows_host = byz_rows.cpu().pin_memory() if nodes else torch.empty((0, wl.d_c))
+        agg_host = torch.empty(wl.d, dtype=torch.float32).pin_memory()
+        mask_host = torch.empty(wl.P, dtype=torch.uint8).pin_memory()
+        plan.step_host(G_host, nodes, rows_host, agg_host, mask_host)             # allocates staging, warms up
+        dist_util.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            st = plan.step_host(G_host, nodes, rows_host, agg_host, mask_host)
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3
+        if st != 0 or mask_host.nonzero().flatten().tolist() != nodes:
+            raise RuntimeError("host-buffer step failed")
+        e2e_max_ms, e2e_units = dist_util.combine(e2e_ms, wl.P * wl.d * 4 * args.e2e_steps)
+        e2e = {"value": e2e_units / (e2e_max_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": wl.P * wl.d * 4 + len(nodes) * wl.d_c * 4, "d2h_bytes_per_step": wl.d * 4 + wl.P,
+               "steps": args.e2e_steps}
+        del G_host, agg_host
+
+    if rank != 0:
+        dist_util.shutdown()
+        return
+
+    peak, peak_kind = measured_peak()
+    enc_gbs = enc_b / (enc_ms * 1e-3) / 1e9
+    total_b = enc_b + proj_b + rec_b
+    path_gbs = total_b / ((enc_ms + dec_ms) * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": total_units / (max_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 in/out, f64 arithmetic", "data": "synthetic",
+        "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "n_byz": len(nodes),
+                   "attack": wl.attack, "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * wl.d * 4 / 1e9),
+                   "parallelism": "independent problems per GPU, no collective"},
+        "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(wl.name),
+                     "algorithmic_bytes": enc_b, "ms": enc_ms},
+        "path": {"encode_ms": enc_ms, "decode_ms": dec_ms, "decodes_per_s": 1e3 / dec_ms, "algorithmic_bytes": total_b,
+                 "hbm_gbs": path_gbs, "frac_of_peak": path_gbs / peak, "frac_of_8TBs": path_gbs / 8000.0},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        small, G_s, nodes_s, rows_s, f_s = oracle_sample(wl, args.oracle_d, "cpu")
+        dt = oracle_step_seconds(small, G_s, nodes_s, rows_s, f_s)
+        line["cpu_baseline"] = {"value": small.P * small.d * 4 / dt / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"first {small.d} of {wl.d} coordinates of every partition gradient, all {wl.P} nodes, one step ({dt:.1f} s)"}
+    print(json.dumps(line), flush=True)
+    dist_util.shutdown()
+
+
+# DRAM bytes (read + write) per encode launch from an ncu capture, by workload; None = not captured for this build.
+TRAFFIC: dict = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vgg13")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    XX
+    args = ap.parse_args()
+    if args.workload in synth.WORKLOADS:
+        wl = synth.WORKLOADS[args.workload]
+    else:
+        match = [p for p in synth.sweep_points() if p.name == args.workload]
+        if not match:
+            raise SystemExit(f"unknown workload {args.workload}")
+        wl = match[0]
+    if wl.grads == "lsq":
+        raise SystemExit("the lsq configuration is a parity case, not a bench workload")
+    if args.oracle_d is None:
+        args.oracle_d = 2_000_000 if args.impl == "reference" else 16_000_000
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
