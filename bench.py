@@ -325,7 +325,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    XX
+    ap.add_argument("--oracle-d", type=int, default=None,
+                    help="coordinates per gradient in the oracle's sample (default: 16M for the cpu_baseline leg, "
+                         "2M per step for --impl reference)")
     args = ap.parse_args()
     if args.workload in synth.WORKLOADS:
         wl = synth.WORKLOADS[args.workload]
@@ -336,6 +338,8 @@ def main():
         wl = match[0]
     if wl.grads == "lsq":
         raise SystemExit("the lsq configuration is a parity case, not a bench workload")
+    if args.oracle_d is None:
+        args.oracle_d = 2_000_000 if args.impl == "reference" else 16_000_000
     if args.oracle_d is None:
         args.oracle_d = 2_000_000 if args.impl == "reference" else 16_000_000
     if args.impl == "reference":
