@@ -4,9 +4,12 @@
 // group are streamed through shared memory in batches by a producer warp that issues one bulk
 // asynchronous copy (cp.async.bulk, completion on an mbarrier) per row segment, so every gradient
 // byte is read from HBM exactly once and many kilobytes per SM are in flight without occupying
-// registers.  Consumer warps add the rows into the group sum ybar (float64, shared memory), then
-// each thread evaluates, for its chunks, the r_g polynomials sum_l w_k^l ybar[p m + l] by Horner's rule
-// in float64 and stores one float32 per node (coalesced along the chunk axis).
+// registers.  In the specialised kernels (m = 1, 2, 3, 5, 6, 10) each consumer thread owns whole chunks:
+// it adds the r_g rows of its chunks into registers straight from the staged rows, then evaluates the
+// r_g polynomials sum_l w_k^l ybar[p m + l] by Horner's rule and stores one float32 per node (coalesced
+// along the chunk axis); no CTA-wide barrier is needed.  Arithmetic is float32 for m <= 6 and float64
+// (rounded once) for larger m, where the decoder's noise amplification leaves no room for the encoder's
+// rounding.  The generic kernel (any m) sums into a float64 ybar in shared memory first.
 //
 // Row segments start at arbitrary 4-byte offsets (d need not be a multiple of 4): the copy starts at
 // the enclosing 16-byte boundary and consumers index from the remainder; the last few floats of the
@@ -25,7 +28,7 @@ struct EncodeParams {
   float* coded;
   const int* group_start;
   const double* w;
-  int q, m;
+  int q, m, P;
   int64_t d, d_c;
   int64_t total_floats;   // P * d
   int chunks_per_thread;  // tile = kEncConsumers * chunks_per_thread chunks
@@ -197,6 +200,150 @@ __global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(EncodeParams prm
   }
 }
 
+
+// ---- specialised kernels: a thread owns CPT whole chunks of M coordinates ---------------------------
+
+template <typename Acc>
+__device__ __forceinline__ Acc acc_fma(Acc a, Acc b, Acc c);
+template <>
+__device__ __forceinline__ float acc_fma<float>(float a, float b, float c) { return fmaf(a, b, c); }
+template <>
+__device__ __forceinline__ double acc_fma<double>(double a, double b, double c) { return fma(a, b, c); }
+
+template <int M, int CPT, typename Acc, int kMinBlocks>
+__global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(EncodeParams prm) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x;
+  constexpr int kTileChunks = kEncConsumers * CPT;
+  constexpr int kTileFloats = kTileChunks * M;
+
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
+  uint64_t* empty_bar = full_bar + prm.stages;
+  int* abort_flag = reinterpret_cast<int*>(empty_bar + prm.stages);
+  Acc* w_s = reinterpret_cast<Acc*>(smem_raw + 256);                       // all P node scalars
+  float* ring = reinterpret_cast<float*>(smem_raw + 256 + (((size_t)prm.P * sizeof(Acc) + 15) & ~(size_t)15));
+  const size_t stage_floats = (size_t)prm.row_batch * prm.slot_floats;
+
+  if (tid == 0) {
+    for (int s = 0; s < prm.stages; ++s) {
+      pipe::mbar_init(&full_bar[s], 32);
+      pipe::mbar_init(&empty_bar[s], kEncConsumers / 32);
+    }
+    *abort_flag = 0;
+    pipe::fence_barrier_init();
+  }
+  for (int k = tid; k < prm.P; k += kEncThreads) w_s[k] = (Acc)prm.w[k];
+  __syncthreads();
+
+  const int64_t total_tiles = prm.tiles_per_group * prm.q;
+
+  if (tid >= kEncConsumers) {
+    const int lane = tid - kEncConsumers;
+    uint32_t it = 0;
+    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int g = (int)(tile / prm.tiles_per_group);
+      const int64_t ct = tile - (int64_t)g * prm.tiles_per_group;
+      const int row0 = prm.group_start[g], r_g = prm.group_start[g + 1] - row0;
+      const int64_t e0 = ct * kTileFloats;
+      int64_t e1 = e0 + kTileFloats;
+      if (e1 > prm.d) e1 = prm.d;
+      for (int b0 = 0; b0 < r_g; b0 += prm.row_batch, ++it) {
+        const int stage = it % prm.stages;
+        const uint32_t phase = (it / prm.stages) & 1;
+        if (it >= (uint32_t)prm.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, prm.status + 1);
+        const int nb = min(prm.row_batch, r_g - b0);
+        if (lane < nb) {
+          const int64_t first = (int64_t)(row0 + b0 + lane) * prm.d + e0;
+          const int64_t last = first + (e1 - e0);
+          const int64_t a0 = first & ~(int64_t)3;
+          int64_t a1 = (last + 3) & ~(int64_t)3;
+          const int64_t safe_end = prm.total_floats & ~(int64_t)3;
+          if (a1 > safe_end) a1 = safe_end;
+          float* slot = ring + stage * stage_floats + (size_t)lane * prm.slot_floats;
+          const uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
+          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.grads[e];   // <= 3 floats
+          if (bytes) {
+            pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
+            pipe::bulk_load(slot, prm.grads + a0, bytes, &full_bar[stage]);
+          } else {
+            pipe::mbar_arrive(&full_bar[stage]);
+          }
+        } else {
+          pipe::mbar_arrive(&full_bar[stage]);
+        }
+      }
+    }
+    if (*(volatile int*)abort_flag) pipe::drain_delay();
+    return;
+  }
+
+  uint32_t it = 0;
+  const int d_mod4 = (int)(prm.d & 3);
+  for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    const int g = (int)(tile / prm.tiles_per_group);
+    const int64_t ct = tile - (int64_t)g * prm.tiles_per_group;
+    const int row0 = prm.group_start[g], r_g = prm.group_start[g + 1] - row0;
+    const int64_t e0 = ct * kTileFloats;
+    const int valid = (int)((prm.d - e0) < kTileFloats ? (prm.d - e0) : kTileFloats);
+    const bool full_tile = valid == kTileFloats;
+    Acc acc[CPT][M];
+#pragma unroll
+    for (int i = 0; i < CPT; ++i)
+#pragma unroll
+      for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
+
+    for (int b0 = 0; b0 < r_g; b0 += prm.row_batch, ++it) {
+      const int stage = it % prm.stages;
+      const uint32_t phase = (it / prm.stages) & 1;
+      pipe::mbar_wait(&full_bar[stage], phase, abort_flag, prm.status + 1);
+      const int nb = min(prm.row_batch, r_g - b0);
+      const float* slot = ring + stage * stage_floats + tid * M;
+      int shift = ((((row0 + b0) & 3) * d_mod4) + (int)(e0 & 3)) & 3;        // (row * d + e0) mod 4
+      if (full_tile) {
+        for (int j = 0; j < nb; ++j) {
+          const float* src = slot + shift;
+#pragma unroll
+          for (int i = 0; i < CPT; ++i)
+#pragma unroll
+            for (int l = 0; l < M; ++l) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
+          slot += prm.slot_floats;
+          shift = (shift + d_mod4) & 3;
+        }
+      } else {
+        for (int j = 0; j < nb; ++j) {
+          const float* src = slot + shift;
+#pragma unroll
+          for (int i = 0; i < CPT; ++i)
+#pragma unroll
+            for (int l = 0; l < M; ++l)
+              if ((tid + i * kEncConsumers) * M + l < valid) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
+          slot += prm.slot_floats;
+          shift = (shift + d_mod4) & 3;
+        }
+      }
+      __syncwarp();
+      if ((tid & 31) == 0) pipe::mbar_arrive(&empty_bar[stage]);
+    }
+
+    const int64_t c0 = ct * kTileChunks;
+    float* out = prm.coded + (int64_t)row0 * prm.d_c + c0 + tid;
+    bool ok[CPT];
+#pragma unroll
+    for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kEncConsumers < prm.d_c;
+    for (int k = 0; k < r_g; ++k) {
+      const Acc wk = w_s[row0 + k];
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) {
+        Acc z = acc[i][M - 1];
+#pragma unroll
+        for (int l = M - 2; l >= 0; --l) z = acc_fma<Acc>(z, wk, acc[i][l]);
+        if (ok[i]) out[i * kEncConsumers] = (float)z;
+      }
+      out += prm.d_c;
+    }
+  }
+}
+
 static size_t encode_smem_bytes(int m, int cpt, int row_batch, int stages, int slot_floats) {
   size_t tile_floats = (size_t)kEncConsumers * cpt * m;
   return 256 + 2 * SOLON_MAX_GROUP * sizeof(double) + 2 * tile_floats * sizeof(double) +
@@ -204,25 +351,7 @@ static size_t encode_smem_bytes(int m, int cpt, int row_batch, int stages, int s
 }
 
 template <int M>
-static int launch_encode_m(solon_plan* plan, EncodeParams& prm, size_t smem, int grid) {
-  SOLON_CUDA_TRY(cudaFuncSetAttribute(encode_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  encode_kernel<M><<<grid, kEncThreads, smem, plan->stream>>>(prm);
-  SOLON_CUDA_TRY(cudaGetLastError());
-  return SOLON_OK;
-}
-
-int launch_encode(solon_plan* plan, const float* grads, float* coded) {
-  EncodeParams prm;
-  prm.grads = grads;
-  prm.coded = coded;
-  prm.group_start = plan->d_group_start;
-  prm.w = plan->d_w;
-  prm.q = plan->q;
-  prm.m = plan->m;
-  prm.d = plan->d;
-  prm.d_c = plan->d_c;
-  prm.total_floats = (int64_t)plan->P * plan->d;
-  prm.status = plan->d_status;
+static int launch_encode_generic(solon_plan* plan, EncodeParams& prm) {
   // tile: about 1024..2048 floats per row for small m, one chunk per thread otherwise
   int cpt = 1;
   while (cpt < 8 && kEncConsumers * cpt * plan->m < 1024) cpt *= 2;
@@ -234,9 +363,8 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   if (row_batch < 1) row_batch = 1;
   if (row_batch > kEncMaxBatch) row_batch = kEncMaxBatch;
   if (row_batch > plan->max_group) row_batch = plan->max_group;
-  // prefer batches that divide the group evenly (fewer ragged stages)
   {
-    int nb = (plan->max_group + row_batch - 1) / row_batch;
+    int nb = (plan->max_group + row_batch - 1) / row_batch;   // batches that divide the group evenly
     row_batch = (plan->max_group + nb - 1) / nb;
   }
   prm.row_batch = row_batch;
@@ -254,17 +382,72 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   if (per_sm < 1) per_sm = 1;
   int64_t resident = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(total_tiles < resident ? total_tiles : resident);
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(encode_kernel<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  encode_kernel<M><<<grid, kEncThreads, smem, plan->stream>>>(prm);
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
+template <int M, int CPT, typename Acc, int kMinBlocks>
+static int launch_encode_direct(solon_plan* plan, EncodeParams& prm) {
+  constexpr int kTileFloats = kEncConsumers * CPT * M;
+  prm.chunks_per_thread = CPT;
+  prm.slot_floats = ((kTileFloats + 3) / 4) * 4 + 8;
+  const size_t slot_bytes = (size_t)prm.slot_floats * 4;
+  const size_t fixed = 256 + (((size_t)plan->P * sizeof(Acc) + 15) & ~(size_t)15);
+  const size_t per_cta = (size_t)227 * 1024 / kMinBlocks - 1024;      // shared memory one CTA may take
+  // rows per stage: about 20 KB per stage, an even split of the largest group
+  int row_batch = (int)((size_t)20 * 1024 / slot_bytes);
+  if (row_batch < 1) row_batch = 1;
+  if (row_batch > kEncMaxBatch) row_batch = kEncMaxBatch;
+  if (row_batch > plan->max_group) row_batch = plan->max_group;
+  {
+    int nb = (plan->max_group + row_batch - 1) / row_batch;
+    row_batch = (plan->max_group + nb - 1) / nb;
+  }
+  int stages = 4;
+  while (stages > 2 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --stages;
+  while (row_batch > 1 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --row_batch;
+  const size_t smem = fixed + (size_t)stages * row_batch * slot_bytes;
+  if (smem > (size_t)226 * 1024) return SOLON_ERR_INVALID_ARG;
+  prm.row_batch = row_batch;
+  prm.stages = stages;
+  prm.tiles_per_group = (plan->d_c + (int64_t)kEncConsumers * CPT - 1) / ((int64_t)kEncConsumers * CPT);
+  const int64_t total_tiles = prm.tiles_per_group * plan->q;
+  int per_sm = (int)((size_t)227 * 1024 / (smem + 1024));
+  if (per_sm > kMinBlocks) per_sm = kMinBlocks;
+  if (per_sm < 1) per_sm = 1;
+  const int64_t resident = (int64_t)plan->num_sms * per_sm;
+  const int grid = (int)(total_tiles < resident ? total_tiles : resident);
+  auto kernel = encode_direct_kernel<M, CPT, Acc, kMinBlocks>;
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kernel<<<grid, kEncThreads, smem, plan->stream>>>(prm);
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
+int launch_encode(solon_plan* plan, const float* grads, float* coded) {
+  EncodeParams prm;
+  prm.grads = grads;
+  prm.coded = coded;
+  prm.group_start = plan->d_group_start;
+  prm.w = plan->d_w;
+  prm.q = plan->q;
+  prm.m = plan->m;
+  prm.P = plan->P;
+  prm.d = plan->d;
+  prm.d_c = plan->d_c;
+  prm.total_floats = (int64_t)plan->P * plan->d;
+  prm.status = plan->d_status;
   plan->launches += 1;
   switch (plan->m) {
-    case 1: return launch_encode_m<1>(plan, prm, smem, grid);
-    case 2: return launch_encode_m<2>(plan, prm, smem, grid);
-    case 3: return launch_encode_m<3>(plan, prm, smem, grid);
-    case 4: return launch_encode_m<4>(plan, prm, smem, grid);
-    case 5: return launch_encode_m<5>(plan, prm, smem, grid);
-    case 6: return launch_encode_m<6>(plan, prm, smem, grid);
-    case 8: return launch_encode_m<8>(plan, prm, smem, grid);
-    case 10: return launch_encode_m<10>(plan, prm, smem, grid);
-    default: return launch_encode_m<0>(plan, prm, smem, grid);
+    case 1: return launch_encode_direct<1, 4, float, 3>(plan, prm);
+    case 2: return launch_encode_direct<2, 2, float, 3>(plan, prm);
+    case 3: return launch_encode_direct<3, 2, float, 3>(plan, prm);
+    case 5: return launch_encode_direct<5, 1, float, 3>(plan, prm);
+    case 6: return launch_encode_direct<6, 1, float, 3>(plan, prm);
+    case 10: return launch_encode_direct<10, 1, double, 2>(plan, prm);
+    default: return launch_encode_generic<0>(plan, prm);
   }
 }
 

@@ -1,7 +1,7 @@
 // Locator kernel (phi of Section 3.4) and recovery table (the inverse inside psi), on the device, plus
 // the host mirror solon_locate_host built from the same source (locate_core.cuh).
 //
-// Grid (s + 1, q): CTA (t, g) is one warp that assumes exactly t corrupt nodes in group g.  All error
+// Grid (s + 1, q): CTA (t, g) assumes exactly t corrupt nodes in group g.  All error
 // counts are tried concurrently; the last CTA of a group to finish (atomic ticket, nobody waits) picks
 // the smallest accepted count, writes the group's part of the mask and builds the recovery table.
 #include <vector>
@@ -63,9 +63,12 @@ SOLON_HD static inline GroupScratch carve(double* ws, int n, int K) {
   return sc;
 }
 
-__global__ void __launch_bounds__(32) locate_kernel(LocateParams prm) {
+constexpr int kLocThreads = 256;
+
+__global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
   extern __shared__ __align__(16) double smem_ws[];
   const int t = blockIdx.x, g = blockIdx.y;
+  const int tid = threadIdx.x;
   const int row0 = prm.group_start[g];
   const int n = prm.group_start[g + 1] - row0;
   double* ws = prm.use_smem ? smem_ws : prm.ws_global + ((size_t)g * (prm.s + 1) + t) * prm.ws_stride;
@@ -78,16 +81,16 @@ __global__ void __launch_bounds__(32) locate_kernel(LocateParams prm) {
   int n_eff = n;
   if (prm.s == 0) {
     // pure compression code: nothing to locate, every node is trusted
-    for (int k = threadIdx.x; k < n; k += 32) {
+    for (int k = tid; k < n; k += kLocThreads) {
       sc.idx[k] = k;
       flags[k] = 0;
     }
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
       recs[0].accept = 1;
       recs[0].n_flagged = 0;
       recs[0].max_fit = 0.0;
     }
-    __syncwarp();
+    __syncthreads();
   } else {
     n_eff = locate_prepare(n, prm.K, prm.rho + row0, prm.P, prm.nu + row0, prm.w + row0, prm.tau, sc.idx, sc.rho_n,
                            sc.w_c, &tau_eff, sc.scratch);
@@ -96,39 +99,39 @@ __global__ void __launch_bounds__(32) locate_kernel(LocateParams prm) {
   if (prm.s == 0) {
   } else if (t <= s_eff && n_eff >= prm.m + 2 * t) {
     locate_task(n_eff, prm.m, prm.K, t, sc.rho_n, sc.w_c, tau_eff, flags, sc.cand, sc.bad, sc.task_ws, &recs[t]);
-  } else if (threadIdx.x == 0) {
+  } else if (tid == 0) {
     recs[t].accept = 0;
     recs[t].n_flagged = 0;
     recs[t].max_fit = INFINITY;
   }
   __threadfence();
-  __syncwarp();
-  if (threadIdx.x == 0) s_ticket = atomicAdd(&prm.group_ticket[g], 1u);
-  __syncwarp();
+  __syncthreads();
+  if (tid == 0) s_ticket = atomicAdd(&prm.group_ticket[g], 1u);
+  __syncthreads();
   if (s_ticket != (unsigned int)prm.s) return;
   __threadfence();
   // Group epilogue.  Records and flags written by the other CTAs are read through L2.
   TaskRecord* recs_l = reinterpret_cast<TaskRecord*>(sc.task_ws);                  // s + 1 records
   uint8_t* flags_l = reinterpret_cast<uint8_t*>(recs_l + (prm.s + 1));             // (s + 1) x n
   double* ep_ws = sc.task_ws + ((size_t)(prm.s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1;
-  for (int i = threadIdx.x; i <= prm.s; i += 32) {
+  for (int i = tid; i <= prm.s; i += kLocThreads) {
     recs_l[i].accept = __ldcg(&recs[i].accept);
     recs_l[i].n_flagged = __ldcg(&recs[i].n_flagged);
     recs_l[i].max_fit = __ldcg(&recs[i].max_fit);
   }
-  for (int i = threadIdx.x; i < (prm.s + 1) * n; i += 32) {
+  for (int i = tid; i < (prm.s + 1) * n; i += kLocThreads) {
     int tt = i / n, k = i - tt * n;
     flags_l[i] = __ldcg(prm.task_flags + (size_t)tt * prm.P + row0 + k);
   }
-  __syncwarp();
+  __syncthreads();
   int* rec_rows_g = prm.rec_rows + row0;
   const int ok = locate_epilogue(n, prm.m, s_eff, n_eff, sc.idx, prm.w + row0, recs_l, flags_l, n, prm.mask + row0,
                                  &prm.t_acc[g], rec_rows_g, &prm.n_rec[g], prm.coeff + (size_t)row0 * prm.m,
                                  sc.trusted, ep_ws);
   // recovery rows as global node indices
   const int n_rec = prm.n_rec[g];
-  for (int j = threadIdx.x; j < n_rec; j += 32) rec_rows_g[j] += row0;
-  if (threadIdx.x == 0) {
+  for (int j = tid; j < n_rec; j += kLocThreads) rec_rows_g[j] += row0;
+  if (tid == 0) {
     if (!ok) atomicOr(prm.status, kStatusUndecodable);
     prm.group_ticket[g] = 0u;   // ready for the next decode
   }
@@ -166,7 +169,7 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
   if (prm.use_smem && smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(plan->s + 1, plan->q);
-  locate_kernel<<<grid, 32, smem, plan->stream>>>(prm);
+  locate_kernel<<<grid, kLocThreads, smem, plan->stream>>>(prm);
   plan->launches += 1;
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;

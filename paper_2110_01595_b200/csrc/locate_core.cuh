@@ -1,8 +1,10 @@
 // Locator (phi) and recovery-table (psi) arithmetic of Solon's decoder, Section 3.4, in float64.
 //
-// One source, two builds: on the device every function is executed by one warp (lanes share the
-// loops marked SOLON_PAR_FOR and meet at SOLON_SYNC); on the host the same code runs serially
-// (one "lane"), which is what solon_locate_host exposes for CPU tests.
+// One source, two builds.  On the device every function is executed by one CTA: matrices live in
+// shared memory column by column, a warp owns columns (SOLON_FOR_WARPS), its lanes own rows
+// (SOLON_FOR_LANES, partial sums combined by lane_sum), element-wise work is spread over all threads
+// (SOLON_FOR_THREADS) and SOLON_SYNC is the CTA barrier.  On the host the same code runs serially
+// (one warp of one lane), which is what solon_locate_host exposes for CPU tests.
 //
 // Reading of the paper's exact-arithmetic locator used here:
 //   * the error count is tried incrementally, t = 0..s; for each t the rational-interpolation
@@ -20,15 +22,25 @@
 #include <stdint.h>
 
 #if defined(__CUDA_ARCH__)
+#define SOLON_TID ((int)threadIdx.x)
+#define SOLON_NTHREADS ((int)blockDim.x)
 #define SOLON_LANE ((int)(threadIdx.x & 31))
 #define SOLON_NLANES 32
-#define SOLON_SYNC() __syncwarp()
+#define SOLON_WARP ((int)(threadIdx.x >> 5))
+#define SOLON_NWARPS ((int)(blockDim.x >> 5))
+#define SOLON_SYNC() __syncthreads()
 #else
+#define SOLON_TID 0
+#define SOLON_NTHREADS 1
 #define SOLON_LANE 0
 #define SOLON_NLANES 1
+#define SOLON_WARP 0
+#define SOLON_NWARPS 1
 #define SOLON_SYNC() ((void)0)
 #endif
-#define SOLON_PAR_FOR(i, n) for (int i = SOLON_LANE; i < (n); i += SOLON_NLANES)
+#define SOLON_FOR_THREADS(i, n) for (int i = SOLON_TID; i < (n); i += SOLON_NTHREADS)
+#define SOLON_FOR_WARPS(i, n) for (int i = SOLON_WARP; i < (n); i += SOLON_NWARPS)
+#define SOLON_FOR_LANES(i, n) for (int i = SOLON_LANE; i < (n); i += SOLON_NLANES)
 
 #if defined(__CUDACC__)
 #define SOLON_HD __host__ __device__
@@ -40,6 +52,15 @@
 #define SOLON_THETA_MAX 16   /* largest error count per group (SOLON_MAX_S) */
 
 namespace solon {
+
+// Sum of x over the lanes of the calling warp, returned to every lane (the value itself on the host).
+SOLON_HD inline double lane_sum(double x) {
+#if defined(__CUDA_ARCH__)
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+#endif
+  return x;
+}
 
 // One (group, t) record written by locate_task and read by the group's epilogue.
 struct TaskRecord {
@@ -54,13 +75,13 @@ SOLON_HD inline size_t locate_task_ws_doubles(int n, int m, int K, int t) {
   size_t ncol = (size_t)K * (m + t) + t;
   size_t rows = (size_t)K * n;
   size_t solve = rows * (ncol + 1) + (ncol + 1) + (size_t)t * (t + 1) + ncol + n;
-  size_t fit = (size_t)n * (m + K) + (m + K) + (size_t)m * (m + K) + m + (size_t)K * m + n;
+  size_t fit = (size_t)n * (m + K) + (m + K) + (size_t)m * (m + K) + m + (size_t)K * m + n + (size_t)n / 2 + 2;
   return (size_t)n * ncheb + (solve > fit ? solve : fit) + 8;
 }
 
 // Doubles of workspace the epilogue needs.
 SOLON_HD inline size_t locate_epilogue_ws_doubles(int n, int m) {
-  return (size_t)n * m + (size_t)m * m + m + 64;
+  return (size_t)n * m + (size_t)m * m + 2 * (size_t)m + 64;
 }
 
 // T_i(x) for i = 0..count-1 into out[0..count).
@@ -74,52 +95,48 @@ SOLON_HD inline void chebyshev_row(double x, int count, double* out) {
   }
 }
 
-// Modified Gram-Schmidt on the first `nq` columns of the row-major matrix A (rows x ld), applied
-// to all `ncols` columns (the trailing ones are right-hand sides).  Columns stay un-normalised.
+// norm0[c] = squared norm of column c of the column-major matrix A (rows x ncols, column stride ldc).
+SOLON_HD inline void column_norms(const double* A, int rows, int ldc, int ncols, double* norm0) {
+  SOLON_FOR_WARPS(c, ncols) {
+    double acc = 0.0;
+    SOLON_FOR_LANES(i, rows) acc = fma(A[(size_t)c * ldc + i], A[(size_t)c * ldc + i], acc);
+    acc = lane_sum(acc);
+    if (SOLON_LANE == 0) norm0[c] = acc;
+  }
+  SOLON_SYNC();
+}
+
+// Modified Gram-Schmidt on the first `nq` columns of the column-major matrix A, applied to all
+// `ncols` columns (the trailing ones are right-hand sides).  Columns stay un-normalised.
 // R (row-major, leading dimension ldr) receives the rows j >= r_first of the triangular factor,
 // right-hand-side columns included, with entry (j, c) stored at R[(j - r_first) * ldr + c - r_first];
 // diag[j] = ||q_j|| (0 for a numerically dependent column).
-SOLON_HD inline void mgs_factor(double* A, int rows, int ld, int nq, int ncols, const double* norm0,
+SOLON_HD inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols, const double* norm0,
                                 double* R, int ldr, int r_first, double* diag) {
   for (int j = 0; j < nq; ++j) {
-    double s0 = 0.0, s1 = 0.0;
-    int i = 0;
-    for (; i + 1 < rows; i += 2) {
-      double a0 = A[(size_t)i * ld + j], a1 = A[(size_t)(i + 1) * ld + j];
-      s0 = fma(a0, a0, s0);
-      s1 = fma(a1, a1, s1);
-    }
-    if (i < rows) {
-      double a0 = A[(size_t)i * ld + j];
-      s0 = fma(a0, a0, s0);
-    }
-    double nrm2 = s0 + s1;
-    bool dead = !(nrm2 > norm0[j] * 1e-26) || !(nrm2 > 0.0);
-    double nrm = dead ? 0.0 : sqrt(nrm2);
-    double inv2 = dead ? 0.0 : 1.0 / nrm2;
-    if (SOLON_LANE == 0) {
+    const double* qj = A + (size_t)j * ldc;
+    double acc = 0.0;
+    SOLON_FOR_LANES(i, rows) acc = fma(qj[i], qj[i], acc);
+    const double nrm2 = lane_sum(acc);               // every warp computes the same value
+    const bool dead = !(nrm2 > norm0[j] * 1e-26) || !(nrm2 > 0.0);
+    const double nrm = dead ? 0.0 : sqrt(nrm2);
+    const double inv2 = dead ? 0.0 : 1.0 / nrm2;
+    if (SOLON_TID == 0) {
       diag[j] = nrm;
       if (j >= r_first) R[(size_t)(j - r_first) * ldr + (j - r_first)] = nrm;
     }
-    if (!dead) {
-      int todo = ncols - (j + 1);
-      SOLON_PAR_FOR(cc, todo) {
-        int c = j + 1 + cc;
-        double d0 = 0.0, d1 = 0.0;
-        int k = 0;
-        for (; k + 1 < rows; k += 2) {
-          d0 = fma(A[(size_t)k * ld + j], A[(size_t)k * ld + c], d0);
-          d1 = fma(A[(size_t)(k + 1) * ld + j], A[(size_t)(k + 1) * ld + c], d1);
-        }
-        if (k < rows) d0 = fma(A[(size_t)k * ld + j], A[(size_t)k * ld + c], d0);
-        double dot = d0 + d1;
-        double coef = dot * inv2;
-        for (k = 0; k < rows; ++k) A[(size_t)k * ld + c] = fma(-coef, A[(size_t)k * ld + j], A[(size_t)k * ld + c]);
-        if (j >= r_first) R[(size_t)(j - r_first) * ldr + (c - r_first)] = dot / nrm;
+    const int todo = ncols - (j + 1);
+    SOLON_FOR_WARPS(cc, todo) {
+      const int c = j + 1 + cc;
+      double* ac = A + (size_t)c * ldc;
+      double dot = 0.0;
+      if (!dead) {
+        SOLON_FOR_LANES(i, rows) dot = fma(qj[i], ac[i], dot);
+        dot = lane_sum(dot);
+        const double coef = dot * inv2;
+        SOLON_FOR_LANES(i, rows) ac[i] = fma(-coef, qj[i], ac[i]);
       }
-    } else if (j >= r_first) {
-      int todo = ncols - (j + 1);
-      SOLON_PAR_FOR(cc, todo) R[(size_t)(j - r_first) * ldr + (j + 1 + cc - r_first)] = 0.0;
+      if (j >= r_first && SOLON_LANE == 0) R[(size_t)(j - r_first) * ldr + (c - r_first)] = dead ? 0.0 : dot / nrm;
     }
     SOLON_SYNC();
   }
@@ -127,36 +144,36 @@ SOLON_HD inline void mgs_factor(double* A, int rows, int ld, int nq, int ncols, 
 
 // Verification: fit a degree-(m-1) polynomial to every projection on the non-candidates and test
 // all nodes.  cheb: n x ncheb table of T_i(w_k); rho_n: K x n projected values divided by the
-// scale; cand[k] != 0 marks candidates.  bad[k] receives 1 where some projection is off by more
-// than tau (or is not a number).  Returns through rec.
+// scale; cand[k] != 0 marks the n_cand candidates.  bad[k] receives 1 where some projection is off by
+// more than tau (or is not a number).  Returns through rec.
 SOLON_HD inline void locate_verify(int n, int m, int K, const double* cheb, int ncheb, const double* rho_n,
-                                   double tau, const uint8_t* cand, uint8_t* bad, double* ws, TaskRecord* rec) {
-  const int ld = m + K;
-  double* B = ws;                       // n_U x ld
-  double* norm0 = B + (size_t)n * ld;   // ld
-  double* Rf = norm0 + ld;              // m x ld
-  double* diag = Rf + (size_t)m * ld;   // m
-  double* coef = diag + m;              // K x m
-  double* ratio = coef + (size_t)K * m; // n
-  // rows of B: the non-candidates, in node order (every lane walks the same list)
-  int n_u = 0;
-  for (int k = 0; k < n; ++k) {
-    if (cand[k]) continue;
-    SOLON_PAR_FOR(c, ld) {
-      B[(size_t)n_u * ld + c] = c < m ? cheb[(size_t)k * ncheb + c] : rho_n[(size_t)(c - m) * n + k];
+                                   double tau, const uint8_t* cand, int n_cand, uint8_t* bad, double* ws,
+                                   TaskRecord* rec) {
+  const int ld = m + K;          // columns: m basis polynomials, K right-hand sides
+  const int n_u = n - n_cand;    // rows: the non-candidates
+  double* B = ws;                            // column-major, ld columns of n_u rows
+  double* norm0 = B + (size_t)n * ld;        // ld
+  double* Rf = norm0 + ld;                   // m x ld
+  double* diag = Rf + (size_t)m * ld;        // m
+  double* coef = diag + m;                   // K x m
+  double* ratio = coef + (size_t)K * m;      // n
+  int* ulist = reinterpret_cast<int*>(ratio + n);   // n
+  SOLON_FOR_THREADS(k, n) {
+    if (!cand[k]) {
+      int pos = 0;
+      for (int o = 0; o < k; ++o) pos += cand[o] ? 0 : 1;
+      ulist[pos] = k;
     }
-    ++n_u;
   }
   SOLON_SYNC();
-  SOLON_PAR_FOR(c, ld) {
-    double sacc = 0.0;
-    for (int i = 0; i < n_u; ++i) sacc = fma(B[(size_t)i * ld + c], B[(size_t)i * ld + c], sacc);
-    norm0[c] = sacc;
+  SOLON_FOR_THREADS(idx, n_u * ld) {
+    const int c = idx / n_u, i = idx - c * n_u, k = ulist[i];
+    B[(size_t)c * n_u + i] = c < m ? cheb[(size_t)k * ncheb + c] : rho_n[(size_t)(c - m) * n + k];
   }
   SOLON_SYNC();
-  mgs_factor(B, n_u, ld, m, ld, norm0, Rf, ld, 0, diag);
-  // back substitution, one projection per lane
-  SOLON_PAR_FOR(kappa, K) {
+  column_norms(B, n_u, n_u, ld, norm0);
+  mgs_factor(B, n_u, n_u, m, ld, norm0, Rf, ld, 0, diag);
+  SOLON_FOR_THREADS(kappa, K) {             // back substitution, one projection per thread
     for (int i = m - 1; i >= 0; --i) {
       double acc = Rf[(size_t)i * ld + m + kappa];
       for (int c = i + 1; c < m; ++c) acc = fma(-Rf[(size_t)i * ld + c], coef[(size_t)kappa * m + c], acc);
@@ -164,7 +181,7 @@ SOLON_HD inline void locate_verify(int n, int m, int K, const double* cheb, int 
     }
   }
   SOLON_SYNC();
-  SOLON_PAR_FOR(k, n) {
+  SOLON_FOR_THREADS(k, n) {
     double worst = 0.0;
     for (int kappa = 0; kappa < K; ++kappa) {
       double q = 0.0;
@@ -177,17 +194,17 @@ SOLON_HD inline void locate_verify(int n, int m, int K, const double* cheb, int 
     bad[k] = ratio[k] > 1.0 ? 1 : 0;
   }
   SOLON_SYNC();
-  int accept = 1, n_flagged = 0;
-  double max_fit = 0.0;
-  for (int k = 0; k < n; ++k) {
-    if (cand[k]) {
-      n_flagged += bad[k];
-    } else {
-      if (bad[k]) accept = 0;
-      max_fit = ratio[k] > max_fit ? ratio[k] : max_fit;
+  if (SOLON_TID == 0) {
+    int accept = 1, n_flagged = 0;
+    double max_fit = 0.0;
+    for (int k = 0; k < n; ++k) {
+      if (cand[k]) {
+        n_flagged += bad[k];
+      } else {
+        if (bad[k]) accept = 0;
+        max_fit = ratio[k] > max_fit ? ratio[k] : max_fit;
+      }
     }
-  }
-  if (SOLON_LANE == 0) {
     rec->accept = accept;
     rec->n_flagged = n_flagged;
     rec->max_fit = max_fit;
@@ -196,7 +213,7 @@ SOLON_HD inline void locate_verify(int n, int m, int K, const double* cheb, int 
 }
 
 // One task: assume exactly t corrupt nodes among the n (finite) nodes of a group.
-//   rho_n   K x n projected values divided by `scale` (so honest values are O(1))
+//   rho_n   K x n projected values divided by the scale (so honest values are O(1))
 //   w       n node scalars;  tau  tolerance in the same normalised units
 //   flags   n bytes out: 1 for candidates that do not fit (the located nodes if accepted)
 //   cand, bad: n bytes of scratch each;  ws: locate_task_ws_doubles(n, m, K, t) doubles
@@ -205,114 +222,113 @@ SOLON_HD inline void locate_task(int n, int m, int K, int t, const double* rho_n
   const int ncheb = m + t + 1;
   double* cheb = ws;                         // n x ncheb
   double* rest = cheb + (size_t)n * ncheb;
-  SOLON_PAR_FOR(k, n) chebyshev_row(w[k], ncheb, cheb + (size_t)k * ncheb);
-  SOLON_PAR_FOR(k, n) cand[k] = 0;
+  SOLON_FOR_THREADS(k, n) {
+    chebyshev_row(w[k], ncheb, cheb + (size_t)k * ncheb);
+    cand[k] = 0;
+  }
   SOLON_SYNC();
   if (t > 0) {
     const int n_num = m + t;
-    const int ncol = K * n_num + t;
-    const int ld = ncol + 1;
+    const int ncol = K * n_num + t;            // unknowns: K numerators, then theta
+    const int ld = ncol + 1;                   // + right-hand side
     const int rows = K * n;
-    double* A = rest;                          // rows x ld
+    double* A = rest;                          // column-major, ld columns of `rows` rows
     double* norm0 = A + (size_t)rows * ld;     // ld
     double* Rt = norm0 + ld;                   // t x (t+1): trailing rows of R, rhs in the last column
     double* diag = Rt + (size_t)t * (t + 1);   // ncol
     double* absE = diag + ncol;                // n
-    SOLON_PAR_FOR(row, rows) {
-      int kappa = row / n, k = row - kappa * n;
-      double rv = rho_n[(size_t)kappa * n + k];
-      double sc = 1.0 / sqrt(1.0 + rv * rv);   // balance rows of very large (corrupt) values
-      double* a = A + (size_t)row * ld;
-      for (int c = 0; c < K * n_num; ++c) a[c] = 0.0;
-      for (int i = 0; i < n_num; ++i) a[kappa * n_num + i] = sc * cheb[(size_t)k * ncheb + i];
-      for (int i = 0; i < t; ++i) a[K * n_num + i] = -sc * rv * cheb[(size_t)k * ncheb + i];
-      a[ncol] = sc * rv * cheb[(size_t)k * ncheb + t];
+    SOLON_FOR_THREADS(idx, rows * ld) {
+      const int c = idx / rows, row = idx - c * rows;
+      const int kappa = row / n, k = row - kappa * n;
+      const double rv = rho_n[(size_t)kappa * n + k];
+      const double sc = 1.0 / sqrt(1.0 + rv * rv);     // balance rows of very large (corrupt) values
+      double val;
+      if (c < K * n_num) {
+        const int blk = c / n_num, i = c - blk * n_num;
+        val = blk == kappa ? sc * cheb[(size_t)k * ncheb + i] : 0.0;
+      } else if (c < ncol) {
+        val = -sc * rv * cheb[(size_t)k * ncheb + (c - K * n_num)];
+      } else {
+        val = sc * rv * cheb[(size_t)k * ncheb + t];
+      }
+      A[idx] = val;
     }
     SOLON_SYNC();
-    SOLON_PAR_FOR(c, ld) {
-      double sacc = 0.0;
-      for (int i = 0; i < rows; ++i) sacc = fma(A[(size_t)i * ld + c], A[(size_t)i * ld + c], sacc);
-      norm0[c] = sacc;
-    }
-    SOLON_SYNC();
+    column_norms(A, rows, rows, ld, norm0);
     const int r_first = ncol - t;
-    mgs_factor(A, rows, ld, ncol, ld, norm0, Rt, t + 1, r_first, diag);
-    // back substitution for the last t unknowns (theta); every lane does the same arithmetic
+    mgs_factor(A, rows, rows, ncol, ld, norm0, Rt, t + 1, r_first, diag);
+    // back substitution for the last t unknowns (theta); every thread does the same arithmetic
     double theta[SOLON_THETA_MAX];
     for (int i = t - 1; i >= 0; --i) {
       double acc = Rt[(size_t)i * (t + 1) + t];
       for (int c = i + 1; c < t; ++c) acc = fma(-Rt[(size_t)i * (t + 1) + c], theta[c], acc);
       theta[i] = diag[r_first + i] > 0.0 ? acc / diag[r_first + i] : 0.0;
     }
-    SOLON_PAR_FOR(k, n) {
+    SOLON_FOR_THREADS(k, n) {
       double e = cheb[(size_t)k * ncheb + t];
       for (int i = 0; i < t; ++i) e = fma(theta[i], cheb[(size_t)k * ncheb + i], e);
-      double ae = fabs(e);
+      const double ae = fabs(e);
       absE[k] = (ae == ae) ? ae : INFINITY;
     }
     SOLON_SYNC();
-    SOLON_PAR_FOR(k, n) {
+    SOLON_FOR_THREADS(k, n) {
       int rank = 0;
-      double mine = absE[k];
+      const double mine = absE[k];
       for (int o = 0; o < n; ++o) rank += (absE[o] < mine || (absE[o] == mine && o < k)) ? 1 : 0;
       cand[k] = rank < t ? 1 : 0;
     }
     SOLON_SYNC();
   }
-  locate_verify(n, m, K, cheb, ncheb, rho_n, tau, cand, bad, rest, rec);
-  SOLON_PAR_FOR(k, n) flags[k] = (cand[k] && bad[k]) ? 1 : 0;
+  locate_verify(n, m, K, cheb, ncheb, rho_n, tau, cand, t, bad, rest, rec);
+  SOLON_FOR_THREADS(k, n) flags[k] = (cand[k] && bad[k]) ? 1 : 0;
   SOLON_SYNC();
 }
 
 // Recovery table for one group: given the trusted nodes (trusted[k] != 0 among n), choose the rows
 // the recovery reads and the weights coeff[j*m + l] of row rec_rows[j] in coordinate l of a chunk,
 // i.e. the least-squares inverse of [W-hat_{m-1}]_{rows,.} (monomial basis, as the encoder used).
-// ws: locate_epilogue_ws_doubles(n, m).  Returns the number of rows (same value in every lane).
+// ws: locate_epilogue_ws_doubles(n, m).  Returns the number of rows (same value in every thread).
 SOLON_HD inline int recovery_table(int n, int m, const double* w, const uint8_t* trusted, int* rec_rows,
                                    double* coeff, double* ws) {
   int n_u = 0;
   for (int k = 0; k < n; ++k) n_u += trusted[k] ? 1 : 0;
   if (n_u < m) return 0;
-  int n_rec = (m <= SOLON_SUBSET_MAX_M) ? m : n_u;
-  // every lane derives the same list; lane 0 stores it
+  const int n_rec = (m <= SOLON_SUBSET_MAX_M) ? m : n_u;
   {
+    // every thread derives the same list; thread 0 stores it
     int seen = 0, next = 0;
     for (int k = 0; k < n && next < n_rec; ++k) {
       if (!trusted[k]) continue;
-      int want = (n_rec == n_u) ? next
-                 : (m == 1 ? (n_u - 1) / 2 : (int)(((long long)next * (n_u - 1) + (m - 1) / 2) / (m - 1)));
+      const int want = (n_rec == n_u) ? next
+                       : (m == 1 ? (n_u - 1) / 2 : (int)(((long long)next * (n_u - 1) + (m - 1) / 2) / (m - 1)));
       if (seen == want) {
-        if (SOLON_LANE == 0) rec_rows[next] = k;
+        if (SOLON_TID == 0) rec_rows[next] = k;
         ++next;
       }
       ++seen;
     }
   }
   SOLON_SYNC();
-  double* V = ws;                          // n_rec x m (becomes Q, un-normalised)
+  double* V = ws;                          // column-major: m columns of n_rec rows (becomes Q, un-normalised)
   double* norm0 = V + (size_t)n_rec * m;   // m
   double* R = norm0 + m;                   // m x m
   double* diag = R + (size_t)m * m;        // m
-  SOLON_PAR_FOR(j, n_rec) {
-    double x = w[rec_rows[j]], p = 1.0;
+  SOLON_FOR_THREADS(j, n_rec) {
+    const double x = w[rec_rows[j]];
+    double p = 1.0;
     for (int l = 0; l < m; ++l) {
-      V[(size_t)j * m + l] = p;
+      V[(size_t)l * n_rec + j] = p;
       p *= x;
     }
   }
   SOLON_SYNC();
-  SOLON_PAR_FOR(l, m) {
-    double sacc = 0.0;
-    for (int j = 0; j < n_rec; ++j) sacc = fma(V[(size_t)j * m + l], V[(size_t)j * m + l], sacc);
-    norm0[l] = sacc;
-  }
-  SOLON_SYNC();
-  mgs_factor(V, n_rec, m, m, m, norm0, R, m, 0, diag);
-  // C = R^{-1} Q^T, one trusted row per lane
-  SOLON_PAR_FOR(j, n_rec) {
+  column_norms(V, n_rec, n_rec, m, norm0);
+  mgs_factor(V, n_rec, n_rec, m, m, norm0, R, m, 0, diag);
+  // C = R^{-1} Q^T, one trusted row per thread
+  SOLON_FOR_THREADS(j, n_rec) {
     double* c = coeff + (size_t)j * m;
     for (int l = m - 1; l >= 0; --l) {
-      double acc = diag[l] > 0.0 ? V[(size_t)j * m + l] / diag[l] : 0.0;
+      double acc = diag[l] > 0.0 ? V[(size_t)l * n_rec + j] / diag[l] : 0.0;
       for (int i = l + 1; i < m; ++i) acc = fma(-R[(size_t)l * m + i], c[i], acc);
       c[l] = diag[l] > 0.0 ? acc / diag[l] : 0.0;
     }
@@ -326,7 +342,7 @@ SOLON_HD inline int recovery_table(int n, int m, const double* w, const uint8_t*
 //   rho: K rows with leading dimension ld_rho, this group's n entries each;  nu, w: n entries
 //   idx[n_eff] original positions of the kept nodes; rho_n (K x n_eff) = rho / scale; w_c their scalars
 //   *tau_eff = tau, or 0 when the median energy is 0 (all-zero data: any deviation counts)
-// scratch: n doubles.  Returns n_eff (same in every lane).
+// scratch: n doubles.  Returns n_eff (same in every thread).
 SOLON_HD inline int locate_prepare(int n, int K, const double* rho, int ld_rho, const double* nu, const double* w,
                                    double tau, int* idx, double* rho_n, double* w_c, double* tau_eff,
                                    double* scratch) {
@@ -335,26 +351,26 @@ SOLON_HD inline int locate_prepare(int n, int K, const double* rho, int ld_rho, 
     bool finite = isfinite(nu[k]);
     for (int kappa = 0; kappa < K; ++kappa) finite = finite && isfinite(rho[(size_t)kappa * ld_rho + k]);
     if (finite) {
-      if (SOLON_LANE == 0) idx[n_eff] = k;
+      if (SOLON_TID == 0) idx[n_eff] = k;
       ++n_eff;
     }
   }
   SOLON_SYNC();
   // lower median of the kept energies by rank counting
-  SOLON_PAR_FOR(i, n_eff) {
-    double mine = nu[idx[i]];
+  SOLON_FOR_THREADS(i, n_eff) {
+    const double mine = nu[idx[i]];
     int rank = 0;
     for (int o = 0; o < n_eff; ++o) {
-      double other = nu[idx[o]];
+      const double other = nu[idx[o]];
       rank += (other < mine || (other == mine && o < i)) ? 1 : 0;
     }
     if (rank == (n_eff - 1) / 2) scratch[0] = mine;
   }
   SOLON_SYNC();
-  double med = n_eff > 0 ? scratch[0] : 0.0;
-  double scale = med > 0.0 ? sqrt(2.0 * med) : 1.0;
+  const double med = n_eff > 0 ? scratch[0] : 0.0;
+  const double scale = med > 0.0 ? sqrt(2.0 * med) : 1.0;
   *tau_eff = med > 0.0 ? tau : 0.0;
-  SOLON_PAR_FOR(i, n_eff) {
+  SOLON_FOR_THREADS(i, n_eff) {
     w_c[i] = w[idx[i]];
     for (int kappa = 0; kappa < K; ++kappa) rho_n[(size_t)kappa * n_eff + i] = rho[(size_t)kappa * ld_rho + idx[i]] / scale;
   }
@@ -391,18 +407,18 @@ SOLON_HD inline int locate_epilogue(int n, int m, int s_eff, int n_eff, const in
       }
     }
   }
-  SOLON_PAR_FOR(k, n) trusted[k] = 0;
+  SOLON_FOR_THREADS(k, n) trusted[k] = 0;
   SOLON_SYNC();
   if (chosen >= 0) {
-    SOLON_PAR_FOR(i, n_eff) trusted[idx[i]] = flags[(size_t)chosen * flags_ld + i] ? 0 : 1;
+    SOLON_FOR_THREADS(i, n_eff) trusted[idx[i]] = flags[(size_t)chosen * flags_ld + i] ? 0 : 1;
   } else {
-    SOLON_PAR_FOR(i, n_eff) trusted[idx[i]] = 1;
+    SOLON_FOR_THREADS(i, n_eff) trusted[idx[i]] = 1;
   }
   SOLON_SYNC();
-  SOLON_PAR_FOR(k, n) mask[k] = trusted[k] ? 0 : 1;
-  int n_rec = recovery_table(n, m, w, trusted, rec_rows, coeff, ws);
+  SOLON_FOR_THREADS(k, n) mask[k] = trusted[k] ? 0 : 1;
+  const int n_rec = recovery_table(n, m, w, trusted, rec_rows, coeff, ws);
   if (n_rec == 0) ok = 0;
-  if (SOLON_LANE == 0) {
+  if (SOLON_TID == 0) {
     *n_rec_out = n_rec;
     *t_out = ok ? chosen + (n - n_eff) : -1;
   }

@@ -184,6 +184,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
   int max_group = 0;
   for (int g = 0; g < q; ++g) max_group = start[g + 1] - start[g] > max_group ? start[g + 1] - start[g] : max_group;
   if (max_group > SOLON_MAX_GROUP) return SOLON_ERR_INVALID_ARG;
+  if ((int64_t)P * m > 16384) return SOLON_ERR_INVALID_ARG;   // recovery table must fit in shared memory
 
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1) {
@@ -208,7 +209,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     return SOLON_ERR_CUDA;
   }
   p->num_sms = prop.multiProcessorCount;
-  p->proj_grid = p->num_sms * 2;
+  p->proj_grid = p->num_sms * 4;
 
   rc = SOLON_OK;
   do {

@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(const float* __re
 
 template <int K>
 static int launch_project_k(solon_plan* plan, const float* received) {
-  int tile_cols = K <= 2 ? 4096 : 2048;
+  int tile_cols = K <= 2 ? 2048 : 1024;
   int64_t range_len = (plan->d_c + plan->proj_grid - 1) / plan->proj_grid;
   range_len = (range_len + 3) / 4 * 4;
   if (range_len < tile_cols) tile_cols = (int)range_len;

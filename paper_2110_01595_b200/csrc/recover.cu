@@ -21,28 +21,16 @@ struct RecoverParams {
   const int* n_rec;      // q
   const int* rec_rows;   // P, group g's rows at [group_start[g], +n_rec[g])
   const double* coeff;   // P x m, same indexing
-  int table_in_smem;
 };
 
-// Gather the per-group lists into one contiguous list.  Returns the number of rows.
-__device__ __forceinline__ int gather_table(const RecoverParams& prm, int* rows_s, double* coeff_s, int* count_s) {
-  if (threadIdx.x == 0) {
-    int total = 0;
-    for (int g = 0; g < prm.q; ++g) total += prm.n_rec[g];
-    *count_s = total;
-  }
+// Copy the locator's tables (group layout, rows per group, row indices, weights) into shared memory.
+__device__ __forceinline__ void load_tables(const RecoverParams& prm, double* coeff_s, int* rows_s, int* start_s,
+                                            int* n_rec_s) {
+  for (int i = threadIdx.x; i < prm.P * prm.m; i += blockDim.x) coeff_s[i] = prm.coeff[i];
+  for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
+  for (int i = threadIdx.x; i <= prm.q; i += blockDim.x) start_s[i] = prm.group_start[i];
+  for (int i = threadIdx.x; i < prm.q; i += blockDim.x) n_rec_s[i] = prm.n_rec[i];
   __syncthreads();
-  // position of entry (g, j) in the packed list = sum of n_rec of the earlier groups + j
-  for (int g = 0, base = 0; g < prm.q; ++g) {
-    const int n = prm.n_rec[g], src = prm.group_start[g];
-    for (int j = threadIdx.x; j < n; j += blockDim.x) rows_s[base + j] = prm.rec_rows[src + j];
-    if (coeff_s) {
-      for (int i = threadIdx.x; i < n * prm.m; i += blockDim.x) coeff_s[(size_t)base * prm.m + i] = prm.coeff[(size_t)src * prm.m + i];
-    }
-    base += n;
-  }
-  __syncthreads();
-  return *count_s;
 }
 
 template <int M, int CPT>
@@ -52,8 +40,9 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
   float* out_s = reinterpret_cast<float*>(smem_raw);                                 // kTileChunks x M
   double* coeff_s = reinterpret_cast<double*>(smem_raw + (size_t)kTileChunks * M * sizeof(float));
   int* rows_s = reinterpret_cast<int*>(coeff_s + (size_t)prm.P * M);
-  __shared__ int count_s;
-  const int n_rows = gather_table(prm, rows_s, coeff_s, &count_s);
+  int* start_s = rows_s + prm.P;
+  int* n_rec_s = start_s + prm.q + 1;
+  load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
   const int tid = threadIdx.x;
 
   for (int64_t c0 = (int64_t)blockIdx.x * kTileChunks; c0 < prm.d_c; c0 += (int64_t)gridDim.x * kTileChunks) {
@@ -66,17 +55,20 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
 #pragma unroll
     for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kRecThreads < prm.d_c;
 
-    for (int j = 0; j < n_rows; ++j) {
-      const float* row = prm.R + (int64_t)rows_s[j] * prm.d_c + c0 + tid;
-      double v[CPT];
+    for (int g = 0; g < prm.q; ++g) {
+      const int base = start_s[g], n = n_rec_s[g];
+      for (int j = 0; j < n; ++j) {
+        const float* row = prm.R + (int64_t)rows_s[base + j] * prm.d_c + c0 + tid;
+        double v[CPT];
 #pragma unroll
-      for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (double)__ldcs(row + i * kRecThreads) : 0.0;
-      const double* cj = coeff_s + (size_t)j * M;
+        for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (double)__ldcs(row + i * kRecThreads) : 0.0;
+        const double* cj = coeff_s + (size_t)(base + j) * M;
 #pragma unroll
-      for (int l = 0; l < M; ++l) {
-        const double c = cj[l];
+        for (int l = 0; l < M; ++l) {
+          const double c = cj[l];
 #pragma unroll
-        for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
+          for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
+        }
       }
     }
 #pragma unroll
@@ -103,14 +95,18 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* coeff_s = reinterpret_cast<double*>(smem_raw);
   int* rows_s = reinterpret_cast<int*>(coeff_s + (size_t)prm.P * prm.m);
-  __shared__ int count_s;
-  const int n_rows = gather_table(prm, rows_s, coeff_s, &count_s);
+  int* start_s = rows_s + prm.P;
+  int* n_rec_s = start_s + prm.q + 1;
+  load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < prm.d; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t p = e / prm.m;
     const int l = (int)(e - p * prm.m);
     double acc = 0.0;
-    for (int j = 0; j < n_rows; ++j)
-      acc = fma(coeff_s[(size_t)j * prm.m + l], (double)prm.R[(int64_t)rows_s[j] * prm.d_c + p], acc);
+    for (int g = 0; g < prm.q; ++g) {
+      const int base = start_s[g], n = n_rec_s[g];
+      for (int j = 0; j < n; ++j)
+        acc = fma(coeff_s[(size_t)(base + j) * prm.m + l], (double)prm.R[(int64_t)rows_s[base + j] * prm.d_c + p], acc);
+    }
     prm.agg[e] = (float)acc;
   }
 }
@@ -118,11 +114,11 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
 template <int M, int CPT>
 static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   size_t smem = (size_t)kRecThreads * CPT * M * sizeof(float) + (size_t)plan->P * M * sizeof(double) +
-                (size_t)plan->P * sizeof(int);
+                (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_kernel<M, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int64_t tiles = (plan->d_c + (int64_t)kRecThreads * CPT - 1) / ((int64_t)kRecThreads * CPT);
-  int64_t cap = (int64_t)plan->num_sms * 8;
+  int64_t cap = (int64_t)plan->num_sms * 3;
   int grid = (int)(tiles < cap ? tiles : cap);
   recover_kernel<M, CPT><<<grid, kRecThreads, smem, plan->stream>>>(prm);
   SOLON_CUDA_TRY(cudaGetLastError());
@@ -142,7 +138,6 @@ int launch_recover(solon_plan* plan, const float* received, float* agg) {
   prm.n_rec = plan->d_n_rec;
   prm.rec_rows = plan->d_rec_rows;
   prm.coeff = plan->d_coeff;
-  prm.table_in_smem = 1;
   plan->launches += 1;
   switch (plan->m) {
     case 1: return launch_recover_m<1, 4>(plan, prm);
@@ -155,7 +150,7 @@ int launch_recover(solon_plan* plan, const float* received, float* agg) {
     case 10: return launch_recover_m<10, 2>(plan, prm);
     default: break;
   }
-  size_t smem = (size_t)plan->P * plan->m * sizeof(double) + (size_t)plan->P * sizeof(int);
+  size_t smem = (size_t)plan->P * plan->m * sizeof(double) + (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int64_t want = (plan->d + kRecThreads - 1) / kRecThreads;

@@ -46,7 +46,9 @@ def test_full_size(name):
         G_s[:, in_range] = G[:, torch.from_numpy(cols[in_range]).cuda()].cpu().numpy()
         Z_s = so.encode(G_s, wl.m, sizes, w)                                       # P x len(chunks)
         got_Z = coded[:, torch.from_numpy(chunks).cuda()].cpu().numpy().astype(np.float64)
-        assert np.all(np.abs(got_Z - Z_s) <= 2.0 ** -24 * 1.0001 * np.abs(Z_s) + 1e-13 * np.abs(G_s).max() * wl.P)
+        bound = so.encode(np.abs(G_s), wl.m, sizes, np.abs(w))                     # sum of |terms|
+        ops = (max(sizes) + wl.m) if wl.m <= 6 else 1                              # float32 roundings, else one
+        assert np.all(np.abs(got_Z - Z_s) <= ops * 2.0 ** -24 * bound * 1.0001 + 1e-45)
         # aggregate at the sampled coordinates against the plain float64 sum
         want_s = so.plain_sum(G_s)[in_range]
         got_s = agg[torch.from_numpy(cols[in_range]).cuda()].cpu().numpy().astype(np.float64)

@@ -29,17 +29,19 @@ def _oracle_plan(wl):
 
 
 def _check_encode(plan, G_cpu, coded_gpu, m, sizes, w):
+    """Coded vectors against the oracle's float64 values.  m > 6: float64 evaluation rounded once (half an ulp).
+    m <= 6: float32 sums and Horner steps, bounded by (r_g + m) roundings of the sum of absolute terms."""
     Z = so.encode(G_cpu.numpy(), m, sizes, w)
     got = coded_gpu.cpu().numpy().astype(np.float64)
-    # float64 evaluation rounded once to float32: half an ulp of the value, plus float64 reordering noise
-    absG = np.abs(G_cpu.numpy()).astype(np.float64)
-    bound = np.zeros_like(Z)
-    for start, size in zip(so.group_starts(sizes), sizes):
-        s_abs = so.group_sum(absG, start, size, m).reshape(-1, m)
-        for k in range(start, start + size):
-            bound[k] = s_abs @ np.abs(w[k]) ** np.arange(m)
+    bound = so.encode(np.abs(G_cpu.numpy()), m, sizes, np.abs(w))          # sum of |terms| of every entry
     err = np.abs(got - Z)
-    assert np.all(err <= 2.0 ** -24 * np.abs(Z) * 1.0001 + 1e-14 * bound + 1e-45), float((err / (np.abs(Z) + 1e-30)).max())
+    if m > 6:
+        assert np.all(err <= 2.0 ** -24 * np.abs(Z) * 1.0001 + 1e-14 * bound + 1e-45), float((err / (np.abs(Z) + 1e-30)).max())
+    else:
+        ops = np.zeros((Z.shape[0], 1))
+        for start, size in zip(so.group_starts(sizes), sizes):
+            ops[start:start + size] = size + m
+        assert np.all(err <= ops * 2.0 ** -24 * bound + 1e-45), float((err / (bound + 1e-30)).max())
     return Z
 
 
