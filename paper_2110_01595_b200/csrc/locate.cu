@@ -35,9 +35,14 @@ struct LocateParams {
 // Workspace carving shared by the device kernel and the host mirror.
 struct GroupScratch {
   int* idx;          // n
+  int* rows_l;       // n      recovery rows (local copy, written out at the end)
   uint8_t* cand;     // n
   uint8_t* bad;      // n
   uint8_t* trusted;  // n
+  uint8_t* mask_l;   // n
+  double* rho_in;    // K x n  staged inputs: every later read hits shared memory, not L2
+  double* nu_in;     // n
+  double* w_in;      // n
   double* rho_n;     // K x n
   double* w_c;       // n
   double* scratch;   // n
@@ -46,16 +51,21 @@ struct GroupScratch {
 
 SOLON_HD static inline size_t group_scratch_doubles(int n, int K) {
   // ints and bytes are carved out of double-sized cells to keep everything 8-byte aligned
-  return (size_t)(n + 1) / 2 + 1 + 3 * ((size_t)n / 8 + 1) + (size_t)(K + 2) * n;
+  return 2 * ((size_t)(n + 1) / 2 + 1) + 4 * ((size_t)n / 8 + 1) + (size_t)(2 * K + 4) * n;
 }
 
 SOLON_HD static inline GroupScratch carve(double* ws, int n, int K) {
   GroupScratch sc;
   double* p = ws;
   sc.idx = reinterpret_cast<int*>(p);            p += (n + 1) / 2 + 1;
+  sc.rows_l = reinterpret_cast<int*>(p);         p += (n + 1) / 2 + 1;
   sc.cand = reinterpret_cast<uint8_t*>(p);       p += n / 8 + 1;
   sc.bad = reinterpret_cast<uint8_t*>(p);        p += n / 8 + 1;
   sc.trusted = reinterpret_cast<uint8_t*>(p);    p += n / 8 + 1;
+  sc.mask_l = reinterpret_cast<uint8_t*>(p);     p += n / 8 + 1;
+  sc.rho_in = p;                                 p += (size_t)K * n;
+  sc.nu_in = p;                                  p += n;
+  sc.w_in = p;                                   p += n;
   sc.rho_n = p;                                  p += (size_t)K * n;
   sc.w_c = p;                                    p += n;
   sc.scratch = p;                                p += n;
@@ -74,6 +84,17 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
   double* ws = prm.use_smem ? smem_ws : prm.ws_global + ((size_t)g * (prm.s + 1) + t) * prm.ws_stride;
   GroupScratch sc = carve(ws, n, prm.K);
   __shared__ unsigned int s_ticket;
+  __shared__ int s_n_rec, s_t_acc;
+
+  // one parallel round trip brings the group's inputs on chip
+  for (int i = tid; i < n; i += kLocThreads) {
+    sc.w_in[i] = prm.w[row0 + i];
+    if (prm.s > 0) {
+      sc.nu_in[i] = prm.nu[row0 + i];
+      for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
+    }
+  }
+  __syncthreads();
 
   TaskRecord* recs = prm.records + (size_t)g * (prm.s + 1);
   uint8_t* flags = prm.task_flags + (size_t)t * prm.P + row0;
@@ -92,8 +113,8 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
     }
     __syncthreads();
   } else {
-    n_eff = locate_prepare(n, prm.K, prm.rho + row0, prm.P, prm.nu + row0, prm.w + row0, prm.tau, sc.idx, sc.rho_n,
-                           sc.w_c, &tau_eff, sc.scratch);
+    n_eff = locate_prepare(n, prm.K, sc.rho_in, n, sc.nu_in, sc.w_in, prm.tau, sc.idx, sc.rho_n, sc.w_c, &tau_eff,
+                           sc.scratch);
   }
   const int s_eff = prm.s - (n - n_eff);
   if (prm.s == 0) {
@@ -124,14 +145,18 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
     flags_l[i] = __ldcg(prm.task_flags + (size_t)tt * prm.P + row0 + k);
   }
   __syncthreads();
-  int* rec_rows_g = prm.rec_rows + row0;
-  const int ok = locate_epilogue(n, prm.m, s_eff, n_eff, sc.idx, prm.w + row0, recs_l, flags_l, n, prm.mask + row0,
-                                 &prm.t_acc[g], rec_rows_g, &prm.n_rec[g], prm.coeff + (size_t)row0 * prm.m,
-                                 sc.trusted, ep_ws);
-  // recovery rows as global node indices
-  const int n_rec = prm.n_rec[g];
-  for (int j = tid; j < n_rec; j += kLocThreads) rec_rows_g[j] += row0;
+  double* coeff_l = ep_ws;                                  // n x m, local copy of the weights
+  double* ep_rest = ep_ws + (size_t)n * prm.m;
+  const int ok = locate_epilogue(n, prm.m, s_eff, n_eff, sc.idx, sc.w_in, recs_l, flags_l, n, sc.mask_l, &s_t_acc,
+                                 sc.rows_l, &s_n_rec, coeff_l, sc.trusted, ep_rest);
+  // write the group's results: mask, recovery rows as global node indices, weights
+  const int n_rec = s_n_rec;
+  for (int k = tid; k < n; k += kLocThreads) prm.mask[row0 + k] = sc.mask_l[k];
+  for (int j = tid; j < n_rec; j += kLocThreads) prm.rec_rows[row0 + j] = sc.rows_l[j] + row0;
+  for (int i = tid; i < n_rec * prm.m; i += kLocThreads) prm.coeff[(size_t)row0 * prm.m + i] = coeff_l[i];
   if (tid == 0) {
+    prm.n_rec[g] = n_rec;
+    prm.t_acc[g] = s_t_acc;
     if (!ok) atomicOr(prm.status, kStatusUndecodable);
     prm.group_ticket[g] = 0u;   // ready for the next decode
   }
@@ -139,7 +164,8 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
 
 size_t locate_ws_doubles(int n, int m, int K, int s) {
   size_t task = locate_task_ws_doubles(n, m, K, s);
-  size_t epi = ((size_t)(s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1 + locate_epilogue_ws_doubles(n, m);
+  size_t epi = ((size_t)(s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1 + (size_t)n * m +
+               locate_epilogue_ws_doubles(n, m);
   return group_scratch_doubles(n, K) + (task > epi ? task : epi) + 8;
 }
 

@@ -71,12 +71,25 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(const float* __re
 #pragma unroll
       for (int kappa = 0; kappa < K; ++kappa) a_rho[kappa] = b_rho[kappa] = 0.0;
       int c = lane;
-      for (; c + 7 * 32 < cols; c += 8 * 32) {
-        float va[8], vb[8];
+      // software pipeline: the loads of the next 8 x 32 columns are in flight while this batch is used
+      float va[8], vb[8], na_[8], nb_[8];
+      bool have = c + 7 * 32 < cols;
+      if (have) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           va[u] = __ldcs(ra + c + u * 32);
           vb[u] = __ldcs(rb + c + u * 32);
+        }
+      }
+      while (have) {
+        const int cn = c + 8 * 32;
+        const bool more = cn + 7 * 32 < cols;
+        if (more) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            na_[u] = __ldcs(ra + cn + u * 32);
+            nb_[u] = __ldcs(rb + cn + u * 32);
+          }
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -90,6 +103,15 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(const float* __re
           a_nu = fmaf(va[u], va[u], a_nu);
           b_nu = fmaf(vb[u], vb[u], b_nu);
         }
+        if (more) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            va[u] = na_[u];
+            vb[u] = nb_[u];
+          }
+        }
+        c = cn;
+        have = more;
       }
       for (; c < cols; c += 32) {
         const float va = __ldcs(ra + c), vb = __ldcs(rb + c);

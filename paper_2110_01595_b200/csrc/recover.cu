@@ -11,6 +11,7 @@
 namespace solon {
 
 constexpr int kRecThreads = 256;
+constexpr int kRowBlock = 5;   // rows whose loads are in flight together
 
 struct RecoverParams {
   const float* R;
@@ -57,17 +58,30 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
 
     for (int g = 0; g < prm.q; ++g) {
       const int base = start_s[g], n = n_rec_s[g];
-      for (int j = 0; j < n; ++j) {
-        const float* row = prm.R + (int64_t)rows_s[base + j] * prm.d_c + c0 + tid;
-        double v[CPT];
+      // rows in blocks of kRowBlock: all loads of a block are issued before its arithmetic
+      for (int j0 = 0; j0 < n; j0 += kRowBlock) {
+        float v[kRowBlock][CPT];
 #pragma unroll
-        for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (double)__ldcs(row + i * kRecThreads) : 0.0;
-        const double* cj = coeff_s + (size_t)(base + j) * M;
+        for (int jj = 0; jj < kRowBlock; ++jj) {
+          const int j = j0 + jj < n ? j0 + jj : n - 1;
+          const float* row = prm.R + (int64_t)rows_s[base + j] * prm.d_c + c0 + tid;
 #pragma unroll
-        for (int l = 0; l < M; ++l) {
-          const double c = cj[l];
+          for (int i = 0; i < CPT; ++i) v[jj][i] = ok[i] ? __ldcs(row + i * kRecThreads) : 0.f;
+        }
 #pragma unroll
-          for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
+        for (int jj = 0; jj < kRowBlock; ++jj) {
+          if (j0 + jj < n) {
+            const double* cj = coeff_s + (size_t)(base + j0 + jj) * M;
+            double dv[CPT];
+#pragma unroll
+            for (int i = 0; i < CPT; ++i) dv[i] = (double)v[jj][i];
+#pragma unroll
+            for (int l = 0; l < M; ++l) {
+              const double c = cj[l];
+#pragma unroll
+              for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, dv[i], acc[i][l]);
+            }
+          }
         }
       }
     }
@@ -118,7 +132,10 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_kernel<M, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int64_t tiles = (plan->d_c + (int64_t)kRecThreads * CPT - 1) / ((int64_t)kRecThreads * CPT);
-  int64_t cap = (int64_t)plan->num_sms * 3;
+  int per_sm = 1;
+  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recover_kernel<M, CPT>, kRecThreads, smem));
+  if (per_sm < 1) per_sm = 1;
+  int64_t cap = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(tiles < cap ? tiles : cap);
   recover_kernel<M, CPT><<<grid, kRecThreads, smem, plan->stream>>>(prm);
   SOLON_CUDA_TRY(cudaGetLastError());
