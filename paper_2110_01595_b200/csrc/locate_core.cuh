@@ -44,8 +44,11 @@
 
 #if defined(__CUDACC__)
 #define SOLON_HD __host__ __device__
+#define SOLON_HD_NOINLINE __host__ __device__ __noinline__   /* one copy of the code: the locator runs once per
+                                                                decode from a cold instruction cache */
 #else
 #define SOLON_HD
+#define SOLON_HD_NOINLINE
 #endif
 
 #define SOLON_SUBSET_MAX_M 6
@@ -96,7 +99,7 @@ SOLON_HD inline void chebyshev_row(double x, int count, double* out) {
 }
 
 // norm0[c] = squared norm of column c of the column-major matrix A (rows x ncols, column stride ldc).
-SOLON_HD inline void column_norms(const double* A, int rows, int ldc, int ncols, double* norm0) {
+SOLON_HD_NOINLINE inline void column_norms(const double* A, int rows, int ldc, int ncols, double* norm0) {
   SOLON_FOR_WARPS(c, ncols) {
     double acc = 0.0;
     SOLON_FOR_LANES(i, rows) acc = fma(A[(size_t)c * ldc + i], A[(size_t)c * ldc + i], acc);
@@ -111,7 +114,7 @@ SOLON_HD inline void column_norms(const double* A, int rows, int ldc, int ncols,
 // R (row-major, leading dimension ldr) receives the rows j >= r_first of the triangular factor,
 // right-hand-side columns included, with entry (j, c) stored at R[(j - r_first) * ldr + c - r_first];
 // diag[j] = ||q_j|| (0 for a numerically dependent column).
-SOLON_HD inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols, const double* norm0,
+SOLON_HD_NOINLINE inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols, const double* norm0,
                                 double* R, int ldr, int r_first, double* diag) {
   for (int j = 0; j < nq; ++j) {
     const double* qj = A + (size_t)j * ldc;
@@ -136,7 +139,7 @@ SOLON_HD inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols,
         const double coef = dot * inv2;
         SOLON_FOR_LANES(i, rows) ac[i] = fma(-coef, qj[i], ac[i]);
       }
-      if (j >= r_first && SOLON_LANE == 0) R[(size_t)(j - r_first) * ldr + (c - r_first)] = dead ? 0.0 : dot / nrm;
+      if (j >= r_first && SOLON_LANE == 0) R[(size_t)(j - r_first) * ldr + (c - r_first)] = dot * (nrm * inv2);
     }
     SOLON_SYNC();
   }

@@ -125,7 +125,8 @@ static int alloc_projection(solon_plan* p) {
   (void)cudaGetLastError();
   p->d_f = nullptr; p->d_partials = nullptr; p->d_rho = nullptr; p->d_locate_ws = nullptr;
   if ((rc = dev_alloc(&p->d_f, (size_t)p->K * p->f_pitch))) return rc;
-  if ((rc = dev_alloc(&p->d_partials, (size_t)p->proj_grid * (p->K + 1) * p->P))) return rc;
+  // per-CTA partial sums followed by the per-bunch sums of the two-level reduction
+  if ((rc = dev_alloc(&p->d_partials, (size_t)(p->proj_grid + p->proj_grid / 16 + 1) * (p->K + 1) * p->P))) return rc;
   if ((rc = dev_alloc(&p->d_rho, (size_t)p->K * p->P))) return rc;
   p->locate_ws_stride = locate_ws_doubles(p->max_group, p->m, p->K, p->s);
   if ((rc = dev_alloc(&p->d_locate_ws, (size_t)p->q * (p->s + 1) * p->locate_ws_stride))) return rc;
@@ -218,7 +219,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     if ((rc = dev_alloc(&p->d_w, P))) break;
     if ((rc = alloc_projection(p))) break;
     if ((rc = dev_alloc(&p->d_nu, P))) break;
-    if ((rc = dev_alloc(&p->d_proj_ticket, 1))) break;
+    if ((rc = dev_alloc(&p->d_proj_ticket, (size_t)p->proj_grid / 16 + 2))) break;
     TaskRecord* recs = nullptr;
     if ((rc = dev_alloc(&recs, (size_t)q * (s + 1)))) break;
     p->d_task_records = recs;
@@ -233,7 +234,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_start, start.data(), (q + 1) * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_of, p->group_of.data(), P * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_w, p->w.data(), P * sizeof(double), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, ((size_t)p->proj_grid / 16 + 2) * sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_group_ticket, 0, q * sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_n_rec, 0, q * sizeof(int));

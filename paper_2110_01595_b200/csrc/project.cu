@@ -5,14 +5,15 @@
 // walks it in tiles, keeps the tile of f in shared memory as float64 and lets each warp stream its own
 // rows (two at a time) against it, so each received byte is read once and f is read once per CTA.
 // Products are exact in float64 and accumulated in float64; nu is accumulated in float32 per lane and
-// in float64 across lanes and tiles.  Per-CTA partial sums go to global memory; the last CTA to
-// finish (atomic ticket, no waiting) adds them in a fixed order, so results are bit-reproducible.
+// in float64 across lanes and tiles.  Per-CTA partial sums go to global memory and are added in a fixed
+// order by the last CTAs to finish (atomic tickets, no waiting), so results are bit-reproducible.
 #include "solon_internal.h"
 
 namespace solon {
 
 constexpr int kProjThreads = 256;
 constexpr int kProjWarps = kProjThreads / 32;
+constexpr int kProjBunch = 16;   // CTAs per first-level reduction
 
 template <int K>
 struct ProjAcc {
@@ -144,35 +145,59 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(const float* __re
   __syncthreads();
   double* mine = partials + (size_t)blockIdx.x * n_acc;
   for (int i = tid; i < n_acc; i += kProjThreads) mine[i] = sacc[i];
+  // Two-level, fixed-order reduction of the per-CTA partial sums with atomic tickets (nobody waits):
+  // the last CTA of every bunch of kProjBunch adds that bunch, the last bunch adds the bunch sums.
+  const unsigned int bunch = blockIdx.x / kProjBunch;
+  const unsigned int n_bunches = (gridDim.x + kProjBunch - 1) / kProjBunch;
+  const unsigned int first = bunch * kProjBunch;
+  const unsigned int members = min((unsigned int)kProjBunch, gridDim.x - first);
+  double* bunch_sums = partials + (size_t)gridDim.x * n_acc;
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_ticket = atomicAdd(ticket, 1u);
+  if (tid == 0) s_ticket = atomicAdd(ticket + 1 + bunch, 1u);
   __syncthreads();
-  if (s_ticket != gridDim.x - 1) return;
-  // last CTA: add the per-CTA partial sums in a fixed order (lane-strided, then a fixed shuffle tree)
+  if (s_ticket != members - 1) return;
   __threadfence();
-  for (int i = warp; i < n_acc; i += kProjWarps) {
+  for (int i = tid; i < n_acc; i += kProjThreads) {
     double acc = 0.0;
-    for (unsigned int b = lane; b < gridDim.x; b += 32) acc += __ldcg(partials + (size_t)b * n_acc + i);
-    acc = warp_sum(acc);
-    if (lane == 0) {
-      if (i < K * P) rho_out[i] = acc;
-      else nu_out[i - K * P] = acc;
-    }
+#pragma unroll 4
+    for (unsigned int b = 0; b < members; ++b) acc += __ldcg(partials + (size_t)(first + b) * n_acc + i);
+    bunch_sums[(size_t)bunch * n_acc + i] = acc;
   }
-  if (tid == 0) *ticket = 0u;   // ready for the next decode
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    ticket[1 + bunch] = 0u;   // ready for the next decode
+    s_ticket = atomicAdd(ticket, 1u);
+  }
+  __syncthreads();
+  if (s_ticket != n_bunches - 1) return;
+  __threadfence();
+  for (int i = tid; i < n_acc; i += kProjThreads) {
+    double acc = 0.0;
+#pragma unroll 4
+    for (unsigned int b = 0; b < n_bunches; ++b) acc += __ldcg(bunch_sums + (size_t)b * n_acc + i);
+    if (i < K * P) rho_out[i] = acc;
+    else nu_out[i - K * P] = acc;
+  }
+  if (tid == 0) *ticket = 0u;
 }
 
 template <int K>
 static int launch_project_k(solon_plan* plan, const float* received) {
   int tile_cols = K <= 2 ? 2048 : 1024;
-  int64_t range_len = (plan->d_c + plan->proj_grid - 1) / plan->proj_grid;
-  range_len = (range_len + 3) / 4 * 4;
-  if (range_len < tile_cols) tile_cols = (int)range_len;
   size_t smem = (size_t)K * tile_cols * sizeof(double) + (size_t)(K + 1) * plan->P * sizeof(double);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(project_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  project_kernel<K><<<plan->proj_grid, kProjThreads, smem, plan->stream>>>(
+  // one wave: as many CTAs as are resident at once (the partial-sum buffer holds plan->proj_grid of them)
+  int per_sm = 1;
+  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, project_kernel<K>, kProjThreads, smem));
+  int grid = plan->num_sms * (per_sm < 1 ? 1 : per_sm);
+  if (grid > plan->proj_grid) grid = plan->proj_grid;
+  int64_t range_len = (plan->d_c + grid - 1) / grid;
+  range_len = (range_len + 3) / 4 * 4;
+  if (range_len < tile_cols) tile_cols = (int)range_len;
+  project_kernel<K><<<grid, kProjThreads, smem, plan->stream>>>(
       received, plan->d_f, plan->f_pitch, plan->P, plan->d_c, range_len, tile_cols, plan->d_partials, plan->d_rho,
       plan->d_nu, plan->d_proj_ticket);
   SOLON_CUDA_TRY(cudaGetLastError());

@@ -3,8 +3,8 @@
 //
 // One pass over the trusted rows the locator selected (m per group when m <= 6, else all trusted rows).
 // Each thread owns a few chunks, loads one float per row and chunk (coalesced along the chunk axis),
-// accumulates the m outputs of each chunk in float64 registers, and the tile is written back through
-// shared memory as contiguous 128-bit stores.  The rows and weights come from device memory written by
+// accumulates the m outputs of each chunk in float64 registers, and every warp writes its run of chunks
+// back through its own shared-memory buffer as contiguous 128-bit stores.  The rows and weights come from device memory written by
 // the locator kernel, so no host round trip separates the two.
 #include "solon_internal.h"
 
@@ -37,16 +37,21 @@ __device__ __forceinline__ void load_tables(const RecoverParams& prm, double* co
 template <int M, int CPT>
 __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  constexpr int kTileChunks = kRecThreads * CPT;
-  float* out_s = reinterpret_cast<float*>(smem_raw);                                 // kTileChunks x M
-  double* coeff_s = reinterpret_cast<double*>(smem_raw + (size_t)kTileChunks * M * sizeof(float));
+  constexpr int kWarpChunks = 32 * CPT;                      // chunks one warp handles per step
+  constexpr int kWarps = kRecThreads / 32;
+  float* out_all = reinterpret_cast<float*>(smem_raw);       // per warp: kWarpChunks x M
+  double* coeff_s = reinterpret_cast<double*>(smem_raw + (size_t)kWarps * kWarpChunks * M * sizeof(float));
   int* rows_s = reinterpret_cast<int*>(coeff_s + (size_t)prm.P * M);
   int* start_s = rows_s + prm.P;
   int* n_rec_s = start_s + prm.q + 1;
   load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
-  const int tid = threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* out_s = out_all + (size_t)warp * kWarpChunks * M;
 
-  for (int64_t c0 = (int64_t)blockIdx.x * kTileChunks; c0 < prm.d_c; c0 += (int64_t)gridDim.x * kTileChunks) {
+  // Warps run independently of each other (no CTA barrier below): while one waits for its loads another
+  // does arithmetic or stores.
+  const int64_t stride = (int64_t)gridDim.x * kWarps * kWarpChunks;
+  for (int64_t c0 = ((int64_t)blockIdx.x * kWarps + warp) * kWarpChunks; c0 < prm.d_c; c0 += stride) {
     double acc[CPT][M];
 #pragma unroll
     for (int i = 0; i < CPT; ++i)
@@ -54,7 +59,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
       for (int l = 0; l < M; ++l) acc[i][l] = 0.0;
     bool ok[CPT];
 #pragma unroll
-    for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kRecThreads < prm.d_c;
+    for (int i = 0; i < CPT; ++i) ok[i] = c0 + lane + i * 32 < prm.d_c;
 
     for (int g = 0; g < prm.q; ++g) {
       const int base = start_s[g], n = n_rec_s[g];
@@ -64,9 +69,9 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
 #pragma unroll
         for (int jj = 0; jj < kRowBlock; ++jj) {
           const int j = j0 + jj < n ? j0 + jj : n - 1;
-          const float* row = prm.R + (int64_t)rows_s[base + j] * prm.d_c + c0 + tid;
+          const float* row = prm.R + (int64_t)rows_s[base + j] * prm.d_c + c0 + lane;
 #pragma unroll
-          for (int i = 0; i < CPT; ++i) v[jj][i] = ok[i] ? __ldcs(row + i * kRecThreads) : 0.f;
+          for (int i = 0; i < CPT; ++i) v[jj][i] = ok[i] ? __ldcs(row + i * 32) : 0.f;
         }
 #pragma unroll
         for (int jj = 0; jj < kRowBlock; ++jj) {
@@ -88,19 +93,19 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
 #pragma unroll
     for (int i = 0; i < CPT; ++i)
 #pragma unroll
-      for (int l = 0; l < M; ++l) out_s[(size_t)(tid + i * kRecThreads) * M + l] = (float)acc[i][l];
-    __syncthreads();
-    // contiguous write-back of the tile: floats [c0 M, min((c0 + tile) M, d))
+      for (int l = 0; l < M; ++l) out_s[(size_t)(lane + i * 32) * M + l] = (float)acc[i][l];
+    __syncwarp();
+    // contiguous write-back: floats [c0 M, min((c0 + kWarpChunks) M, d)); c0 M is a multiple of 4
     const int64_t o0 = c0 * M;
-    int64_t o1 = o0 + (int64_t)kTileChunks * M;
+    int64_t o1 = o0 + (int64_t)kWarpChunks * M;
     if (o1 > prm.d) o1 = prm.d;
     const int count = (int)(o1 - o0);
-    const int vec = count / 4;                       // o0 is a multiple of 4 (tile of 256 * CPT chunks)
+    const int vec = count / 4;
     float4* dst4 = reinterpret_cast<float4*>(prm.agg + o0);
     const float4* src4 = reinterpret_cast<const float4*>(out_s);
-    for (int i = tid; i < vec; i += kRecThreads) dst4[i] = src4[i];
-    for (int i = vec * 4 + tid; i < count; i += kRecThreads) prm.agg[o0 + i] = out_s[i];
-    __syncthreads();
+    for (int i = lane; i < vec; i += 32) dst4[i] = src4[i];
+    for (int i = vec * 4 + lane; i < count; i += 32) prm.agg[o0 + i] = out_s[i];
+    __syncwarp();
   }
 }
 
@@ -131,6 +136,7 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
                 (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_kernel<M, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  static_assert((32 * CPT) % 4 == 0, "warp tiles must start on a 16-byte boundary of the output");
   int64_t tiles = (plan->d_c + (int64_t)kRecThreads * CPT - 1) / ((int64_t)kRecThreads * CPT);
   int per_sm = 1;
   SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recover_kernel<M, CPT>, kRecThreads, smem));
