@@ -188,6 +188,30 @@ int solon_plan_get_projections(solon_plan* plan, double* rho /* host, K * P */, 
  * Capacities: n_rec and t hold q ints, rec_rows P ints, coeff P * m doubles. */
 int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows, double* coeff);
 
+/* Projections without any allocation.  (The paper has no counterpart: this entry point exists for
+ * callers of this library that are not allowed to allocate device memory at the moment they need
+ * the projections - for example a service whose whole device memory has already been handed to its
+ * own pool, or a step loop that must not run into the device-wide synchronisation an allocation
+ * implies.  solon_plan_create allocates, so such callers cannot use a plan.)
+ *
+ * Computes what the first kernel of solon_decode computes: rho[kappa * P + k] = sum_p
+ * f[kappa * f_pitch + p] * received[k * d_c + p] and nu[k] = sum_p received[k * d_c + p]^2.
+ *   received  device, P x d_c float32          f    device, K rows of f_pitch floats (f_pitch >= d_c,
+ *   rho       device, K x P float64 (output)        a multiple of 4; base 16-byte aligned; entries
+ *   nu        device, P float64 (output)            beyond d_c in a row are ignored)
+ * The kernel's scratch (per-block partial sums and completion counters, about 1.3 MB) is a fixed
+ * array inside the library's device image, so every GPU that loads the library holds it until the
+ * process exits.  Limits: (K + 1) * P <= 512 and K <= 4; larger problems get SOLON_ERR_INVALID_ARG.
+ * Nothing is allocated or freed, here or in any routine this calls.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the one array: two
+ * calls whose kernels may overlap on the GPU (different streams, no ordering) race on it and
+ * corrupt each other's sums; calls on one stream, or otherwise ordered, are fine.  The counters are
+ * cleared at the start of every call; the partial sums are fully rewritten by every call.
+ * Enqueued on `cuda_stream`; does not synchronise. */
+int solon_project_noalloc(const float* received, const float* f, int64_t f_pitch, int P, int64_t d_c,
+                          int K, double* rho, double* nu, void* cuda_stream);
+
 /* Number of kernels the library launched on behalf of this plan since creation. */
 int64_t solon_plan_kernel_launches(const solon_plan* plan);
 

@@ -55,6 +55,7 @@ SIGNATURES = {
     "solon_plan_get_projections": (c_int, [c_void_p, POINTER(c_double), POINTER(c_double)]),
     "solon_plan_get_recovery": (c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_double)]),
     "solon_plan_kernel_launches": (c_int64, [c_void_p]),
+    "solon_project_noalloc": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int64, c_int, c_void_p, c_void_p, c_void_p]),
 }
 
 _lib = None
@@ -131,6 +132,26 @@ def solon_locate_host(rho: np.ndarray, nu: np.ndarray, w_g: np.ndarray, m: int, 
     if status not in (OK, ERR_UNDECODABLE):
         raise SolonError(status, "solon_locate_host")
     return status, mask, t.value, rows[:n_rec.value].copy(), coeff[:n_rec.value * m].reshape(n_rec.value, m).copy()
+
+
+def solon_project_noalloc(received, f, rho, nu, stream=None) -> int:
+    """Projections through the entry point that allocates nothing.
+
+    received: P x d_c float32 CUDA tensor; f: K x f_pitch float32 CUDA tensor (f_pitch >= d_c, multiple of 4);
+    rho (K x P) and nu (P): float64 CUDA tensors the caller has already allocated.  Returns the status code.
+    """
+    import torch
+
+    P, d_c = received.shape
+    K, f_pitch = f.shape
+    for t, dt in ((received, torch.float32), (f, torch.float32), (rho, torch.float64), (nu, torch.float64)):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == dt):
+            raise ValueError("solon_project_noalloc takes contiguous CUDA tensors (float32 in, float64 out)")
+    if tuple(rho.shape) != (K, P) or tuple(nu.shape) != (P,):
+        raise ValueError("rho must be K x P and nu must have P entries")
+    stream = stream if stream is not None else torch.cuda.current_stream()
+    return lib().solon_project_noalloc(c_void_p(received.data_ptr()), c_void_p(f.data_ptr()), f_pitch, P, d_c, K,
+                                       c_void_p(rho.data_ptr()), c_void_p(nu.data_ptr()), c_void_p(stream.cuda_stream))
 
 
 # ------------------------------------------------------------------ plan

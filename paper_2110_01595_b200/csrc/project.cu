@@ -7,6 +7,8 @@
 // Products are exact in float64 and accumulated in float64; nu is accumulated in float32 per lane and
 // in float64 across lanes and tiles.  Per-CTA partial sums go to global memory and are added in a fixed
 // order by the last CTAs to finish (atomic tickets, no waiting), so results are bit-reproducible.
+#include <mutex>
+
 #include "solon_internal.h"
 
 namespace solon {
@@ -215,4 +217,82 @@ int launch_project(solon_plan* plan, const float* received) {
   }
 }
 
+// ---- projections without any allocation ------------------------------------------------------------
+//
+// Scratch for solon_project_noalloc: the per-CTA partial sums, the per-bunch sums and the tickets of
+// project_kernel, in a file-scope device array instead of plan-owned cudaMalloc memory.  Every GPU that
+// loads the library holds these bytes until the process exits.
+constexpr int kNoAllocMaxCtas = 296;                                   // grid cap of the no-allocation variant
+constexpr int kNoAllocMaxSums = 512;                                   // (K + 1) * P
+constexpr int kNoAllocBunches = kNoAllocMaxCtas / kProjBunch + 1;
+constexpr size_t kNoAllocPartialBytes = (size_t)(kNoAllocMaxCtas + kNoAllocBunches) * kNoAllocMaxSums * sizeof(double);
+constexpr size_t kNoAllocTicketBytes = 256;                            // 1 + kNoAllocBunches counters, padded
+static_assert((1 + kNoAllocBunches) * sizeof(unsigned int) <= kNoAllocTicketBytes, "ticket area too small");
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocPartialBytes + kNoAllocTicketBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+static std::mutex g_noalloc_mutex;
+static unsigned char* g_noalloc_ptr[kNoAllocMaxDevices];               // device address of the array, per device
+
+// In host code the array's name is only a handle; the device address comes from cudaGetSymbolAddress,
+// asked once per device while that device is current.
+static int noalloc_scratch_address(unsigned char** out) {
+  int device = -1;
+  SOLON_CUDA_TRY(cudaGetDevice(&device));
+  if (device < 0 || device >= kNoAllocMaxDevices) return SOLON_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[device]) {
+    void* ptr = nullptr;
+    SOLON_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    if (!ptr) return SOLON_ERR_CUDA;
+    g_noalloc_ptr[device] = static_cast<unsigned char*>(ptr);
+  }
+  *out = g_noalloc_ptr[device];
+  return SOLON_OK;
+}
+
+template <int K>
+static int launch_project_noalloc_k(const float* received, const float* f, int64_t f_pitch, int P, int64_t d_c,
+                                    double* rho, double* nu, cudaStream_t stream, unsigned char* scratch) {
+  int tile_cols = K <= 2 ? 2048 : 1024;
+  size_t smem = (size_t)K * tile_cols * sizeof(double) + (size_t)(K + 1) * P * sizeof(double);
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(project_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  int device = 0, num_sms = 0, per_sm = 1;
+  SOLON_CUDA_TRY(cudaGetDevice(&device));
+  SOLON_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device));
+  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, project_kernel<K>, kProjThreads, smem));
+  int grid = num_sms * (per_sm < 1 ? 1 : per_sm);
+  if (grid > kNoAllocMaxCtas) grid = kNoAllocMaxCtas;
+  int64_t range_len = (d_c + grid - 1) / grid;
+  range_len = (range_len + 3) / 4 * 4;
+  if (range_len < tile_cols) tile_cols = (int)range_len;
+  double* partials = reinterpret_cast<double*>(scratch);
+  unsigned int* ticket = reinterpret_cast<unsigned int*>(scratch + kNoAllocPartialBytes);
+  // the tickets must start at zero; the partial sums are fully rewritten by every launch
+  SOLON_CUDA_TRY(cudaMemsetAsync(ticket, 0, kNoAllocTicketBytes, stream));
+  project_kernel<K><<<grid, kProjThreads, smem, stream>>>(received, f, f_pitch, P, d_c, range_len, tile_cols, partials,
+                                                          rho, nu, ticket);
+  SOLON_CUDA_TRY(cudaGetLastError());
+  return SOLON_OK;
+}
+
 }  // namespace solon
+
+extern "C" int solon_project_noalloc(const float* received, const float* f, int64_t f_pitch, int P, int64_t d_c, int K,
+                                     double* rho, double* nu, void* cuda_stream) {
+  using namespace solon;
+  if (!received || !f || !rho || !nu) return SOLON_ERR_INVALID_ARG;
+  if (P < 1 || d_c < 1 || K < 1 || K > SOLON_MAX_PROJECTIONS) return SOLON_ERR_INVALID_ARG;
+  if ((int64_t)(K + 1) * P > kNoAllocMaxSums) return SOLON_ERR_INVALID_ARG;      // beyond the static scratch
+  if (f_pitch < d_c || (f_pitch & 3) || ((uintptr_t)f & 15) || ((uintptr_t)received & 3)) return SOLON_ERR_INVALID_ARG;
+  unsigned char* scratch = nullptr;
+  int rc = noalloc_scratch_address(&scratch);
+  if (rc) return rc;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  switch (K) {
+    case 1: return launch_project_noalloc_k<1>(received, f, f_pitch, P, d_c, rho, nu, stream, scratch);
+    case 2: return launch_project_noalloc_k<2>(received, f, f_pitch, P, d_c, rho, nu, stream, scratch);
+    case 3: return launch_project_noalloc_k<3>(received, f, f_pitch, P, d_c, rho, nu, stream, scratch);
+    default: return launch_project_noalloc_k<4>(received, f, f_pitch, P, d_c, rho, nu, stream, scratch);
+  }
+}
