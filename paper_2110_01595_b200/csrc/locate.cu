@@ -13,9 +13,13 @@ namespace solon {
 
 struct LocateParams {
   const int* group_start;
-  const double* w;
+  const double* w;       // P node scalars
   const double* rho;     // K x P
   const double* nu;      // P
+  const double* qb;      // per group n_g x n_g orthonormal polynomial tables, group g at qb_off[g]
+  const int64_t* qb_off; // q
+  const double* mt;      // q x m x m
+  const double* tch;     // P x (s + 1)
   int P, m, s, K;
   double tau;
   TaskRecord* records;   // q x (s + 1)
@@ -34,41 +38,37 @@ struct LocateParams {
 
 // Workspace carving shared by the device kernel and the host mirror.
 struct GroupScratch {
-  int* idx;          // n
   int* rows_l;       // n      recovery rows (local copy, written out at the end)
   uint8_t* cand;     // n
   uint8_t* bad;      // n
   uint8_t* trusted;  // n
   uint8_t* mask_l;   // n
+  uint8_t* forced;   // n
   double* rho_in;    // K x n  staged inputs: every later read hits shared memory, not L2
   double* nu_in;     // n
-  double* w_in;      // n
   double* rho_n;     // K x n
-  double* w_c;       // n
-  double* scratch;   // n
+  double* scratch;   // K + 2
   double* task_ws;   // rest
 };
 
 SOLON_HD static inline size_t group_scratch_doubles(int n, int K) {
   // ints and bytes are carved out of double-sized cells to keep everything 8-byte aligned
-  return 2 * ((size_t)(n + 1) / 2 + 1) + 4 * ((size_t)n / 8 + 1) + (size_t)(2 * K + 4) * n;
+  return ((size_t)(n + 1) / 2 + 1) + 5 * ((size_t)n / 8 + 1) + (size_t)(2 * K + 1) * n + K + 2;
 }
 
 SOLON_HD static inline GroupScratch carve(double* ws, int n, int K) {
   GroupScratch sc;
   double* p = ws;
-  sc.idx = reinterpret_cast<int*>(p);            p += (n + 1) / 2 + 1;
   sc.rows_l = reinterpret_cast<int*>(p);         p += (n + 1) / 2 + 1;
   sc.cand = reinterpret_cast<uint8_t*>(p);       p += n / 8 + 1;
   sc.bad = reinterpret_cast<uint8_t*>(p);        p += n / 8 + 1;
   sc.trusted = reinterpret_cast<uint8_t*>(p);    p += n / 8 + 1;
   sc.mask_l = reinterpret_cast<uint8_t*>(p);     p += n / 8 + 1;
+  sc.forced = reinterpret_cast<uint8_t*>(p);     p += n / 8 + 1;
   sc.rho_in = p;                                 p += (size_t)K * n;
   sc.nu_in = p;                                  p += n;
-  sc.w_in = p;                                   p += n;
   sc.rho_n = p;                                  p += (size_t)K * n;
-  sc.w_c = p;                                    p += n;
-  sc.scratch = p;                                p += n;
+  sc.scratch = p;                                p += K + 2;
   sc.task_ws = p;
   return sc;
 }
@@ -85,25 +85,18 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
   GroupScratch sc = carve(ws, n, prm.K);
   __shared__ unsigned int s_ticket;
   __shared__ int s_n_rec, s_t_acc;
-
-  // one parallel round trip brings the group's inputs on chip
-  for (int i = tid; i < n; i += kLocThreads) {
-    sc.w_in[i] = prm.w[row0 + i];
-    if (prm.s > 0) {
-      sc.nu_in[i] = prm.nu[row0 + i];
-      for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
-    }
-  }
-  __syncthreads();
+  GroupTables tb;
+  tb.Qb = prm.qb + prm.qb_off[g];
+  tb.Mt = prm.mt + (size_t)g * prm.m * prm.m;
+  tb.Tch = prm.tch + (size_t)row0 * (prm.s + 1);
+  tb.w = prm.w + row0;
 
   TaskRecord* recs = prm.records + (size_t)g * (prm.s + 1);
   uint8_t* flags = prm.task_flags + (size_t)t * prm.P + row0;
-  double tau_eff = 0.0;
-  int n_eff = n;
   if (prm.s == 0) {
     // pure compression code: nothing to locate, every node is trusted
     for (int k = tid; k < n; k += kLocThreads) {
-      sc.idx[k] = k;
+      sc.forced[k] = 0;
       flags[k] = 0;
     }
     if (tid == 0) {
@@ -113,17 +106,15 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
     }
     __syncthreads();
   } else {
-    n_eff = locate_prepare(n, prm.K, sc.rho_in, n, sc.nu_in, sc.w_in, prm.tau, sc.idx, sc.rho_n, sc.w_c, &tau_eff,
-                           sc.scratch);
-  }
-  const int s_eff = prm.s - (n - n_eff);
-  if (prm.s == 0) {
-  } else if (t <= s_eff && n_eff >= prm.m + 2 * t) {
-    locate_task(n_eff, prm.m, prm.K, t, sc.rho_n, sc.w_c, tau_eff, flags, sc.cand, sc.bad, sc.task_ws, &recs[t]);
-  } else if (tid == 0) {
-    recs[t].accept = 0;
-    recs[t].n_flagged = 0;
-    recs[t].max_fit = INFINITY;
+    // one parallel round trip brings the group's projected values on chip
+    for (int i = tid; i < n; i += kLocThreads) {
+      sc.nu_in[i] = prm.nu[row0 + i];
+      for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
+    }
+    __syncthreads();
+    double tau_eff = 0.0;
+    locate_prepare(n, prm.K, sc.rho_in, sc.nu_in, prm.tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
+    locate_task(tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, flags, sc.cand, sc.bad, sc.task_ws, &recs[t]);
   }
   __threadfence();
   __syncthreads();
@@ -147,8 +138,8 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
   __syncthreads();
   double* coeff_l = ep_ws;                                  // n x m, local copy of the weights
   double* ep_rest = ep_ws + (size_t)n * prm.m;
-  const int ok = locate_epilogue(n, prm.m, s_eff, n_eff, sc.idx, sc.w_in, recs_l, flags_l, n, sc.mask_l, &s_t_acc,
-                                 sc.rows_l, &s_n_rec, coeff_l, sc.trusted, ep_rest);
+  const int ok = locate_epilogue(tb, n, prm.m, prm.s, sc.forced, recs_l, flags_l, n, sc.mask_l, &s_t_acc, sc.rows_l,
+                                 &s_n_rec, coeff_l, sc.trusted, ep_rest);
   // write the group's results: mask, recovery rows as global node indices, weights
   const int n_rec = s_n_rec;
   for (int k = tid; k < n; k += kLocThreads) prm.mask[row0 + k] = sc.mask_l[k];
@@ -165,8 +156,67 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
 size_t locate_ws_doubles(int n, int m, int K, int s) {
   size_t task = locate_task_ws_doubles(n, m, K, s);
   size_t epi = ((size_t)(s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1 + (size_t)n * m +
-               locate_epilogue_ws_doubles(n, m);
+               locate_epilogue_ws_doubles(n, m, s);
   return group_scratch_doubles(n, K) + (task > epi ? task : epi) + 8;
+}
+
+// Tables of one group (host, once per plan): the orthonormal polynomials q_0..q_{n-1} on the nodes
+// (Gram-Schmidt, twice, of the Chebyshev polynomials T_0..T_{n-1} evaluated at the nodes), the monomial
+// coefficients of q_0..q_{m-1}, and T_0..T_s at the nodes.
+void build_group_tables(int n, int m, int s, const double* w, double* Qb, double* Mt, double* Tch) {
+  typedef long double real;
+  std::vector<real> T((size_t)n * n), Q((size_t)n * n), R((size_t)n * n, 0.0L);   // column-major n x n
+  for (int k = 0; k < n; ++k) {
+    real t0 = 1.0L, t1 = (real)w[k];
+    for (int i = 0; i < n; ++i) {
+      T[(size_t)i * n + k] = t0;
+      real t2 = 2.0L * (real)w[k] * t1 - t0;
+      t0 = t1;
+      t1 = t2;
+    }
+  }
+  Q = T;
+  for (int j = 0; j < n; ++j) {
+    for (int pass = 0; pass < 2; ++pass) {
+      for (int i = 0; i < j; ++i) {
+        real dot = 0.0L;
+        for (int k = 0; k < n; ++k) dot += Q[(size_t)i * n + k] * Q[(size_t)j * n + k];
+        for (int k = 0; k < n; ++k) Q[(size_t)j * n + k] -= dot * Q[(size_t)i * n + k];
+        R[(size_t)i * n + j] += dot;           // R[i][j], row-major
+      }
+    }
+    real nrm = 0.0L;
+    for (int k = 0; k < n; ++k) nrm += Q[(size_t)j * n + k] * Q[(size_t)j * n + k];
+    nrm = sqrtl(nrm);
+    R[(size_t)j * n + j] = nrm;
+    for (int k = 0; k < n; ++k) Q[(size_t)j * n + k] = nrm > 0.0L ? Q[(size_t)j * n + k] / nrm : 0.0L;
+  }
+  for (size_t i = 0; i < (size_t)n * n; ++i) Qb[i] = (double)Q[i];
+  // q_i = sum_{j<=i} Rinv[j][i] T_j (T = Q R); T_j = sum_l C[l][j] w^l with integer C from the recurrence
+  std::vector<real> Rinv((size_t)m * m, 0.0L), C((size_t)m * m, 0.0L);
+  for (int i = 0; i < m; ++i) {
+    Rinv[(size_t)i * m + i] = 1.0L / R[(size_t)i * n + i];
+    for (int r = i - 1; r >= 0; --r) {
+      real acc = 0.0L;
+      for (int c = r + 1; c <= i; ++c) acc += R[(size_t)r * n + c] * Rinv[(size_t)c * m + i];
+      Rinv[(size_t)r * m + i] = -acc / R[(size_t)r * n + r];
+    }
+  }
+  for (int j = 0; j < m; ++j) {
+    if (j == 0) C[0] = 1.0L;
+    else if (j == 1) C[(size_t)1 * m + 1] = 1.0L;
+    else
+      for (int l = 0; l <= j; ++l)
+        C[(size_t)l * m + j] = (l > 0 ? 2.0L * C[(size_t)(l - 1) * m + (j - 1)] : 0.0L) - C[(size_t)l * m + (j - 2)];
+  }
+  for (int l = 0; l < m; ++l)
+    for (int i = 0; i < m; ++i) {
+      real acc = 0.0L;
+      for (int j = 0; j <= i; ++j) acc += C[(size_t)l * m + j] * Rinv[(size_t)j * m + i];
+      Mt[(size_t)l * m + i] = (double)acc;
+    }
+  for (int k = 0; k < n; ++k)
+    for (int i = 0; i <= s; ++i) Tch[(size_t)k * (s + 1) + i] = i < n ? (double)T[(size_t)i * n + k] : 0.0;
 }
 
 int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
@@ -175,6 +225,10 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
   prm.w = plan->d_w;
   prm.rho = plan->d_rho;
   prm.nu = plan->d_nu;
+  prm.qb = plan->d_qb;
+  prm.qb_off = plan->d_qb_off;
+  prm.mt = plan->d_mt;
+  prm.tch = plan->d_tch;
   prm.P = plan->P; prm.m = plan->m; prm.s = plan->s; prm.K = plan->K;
   prm.tau = plan->tau;
   prm.records = reinterpret_cast<TaskRecord*>(plan->d_task_records);
@@ -211,25 +265,31 @@ extern "C" int solon_locate_host(int n, int m, int s, int K, const double* rho, 
   if (n < 1 || n > SOLON_MAX_GROUP || m < 1 || m > SOLON_MAX_M || s < 0 || s > SOLON_MAX_S || K < 1 ||
       K > SOLON_MAX_PROJECTIONS || n < 2 * s + m)
     return SOLON_ERR_INVALID_ARG;
+  std::vector<double> Qb((size_t)n * n), Mt((size_t)m * m), Tch((size_t)n * (s + 1));
+  build_group_tables(n, m, s, w_g, Qb.data(), Mt.data(), Tch.data());
+  GroupTables tb;
+  tb.Qb = Qb.data();
+  tb.Mt = Mt.data();
+  tb.Tch = Tch.data();
+  tb.w = w_g;
   std::vector<double> ws(group_scratch_doubles(n, K) + locate_task_ws_doubles(n, m, K, s) +
-                         locate_epilogue_ws_doubles(n, m) + 64);
+                         locate_epilogue_ws_doubles(n, m, s) + 64);
   GroupScratch sc = carve(ws.data(), n, K);
   std::vector<TaskRecord> recs(s + 1);
   std::vector<uint8_t> flags((size_t)(s + 1) * n, 0);
   double tau_eff = 0.0;
-  const int n_eff = locate_prepare(n, K, rho, n, nu, w_g, tau, sc.idx, sc.rho_n, sc.w_c, &tau_eff, sc.scratch);
-  const int s_eff = s - (n - n_eff);
-  for (int t = 0; t <= s; ++t) {
-    if (t <= s_eff && n_eff >= m + 2 * t) {
-      locate_task(n_eff, m, K, t, sc.rho_n, sc.w_c, tau_eff, flags.data() + (size_t)t * n, sc.cand, sc.bad, sc.task_ws,
-                  &recs[t]);
-    } else {
-      recs[t].accept = 0;
-      recs[t].n_flagged = 0;
-      recs[t].max_fit = INFINITY;
-    }
+  if (s > 0) {
+    locate_prepare(n, K, rho, nu, tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
+    for (int t = 0; t <= s; ++t)
+      locate_task(tb, n, m, K, t, s, sc.rho_n, sc.forced, tau_eff, flags.data() + (size_t)t * n, sc.cand, sc.bad,
+                  sc.task_ws, &recs[t]);
+  } else {
+    for (int k = 0; k < n; ++k) sc.forced[k] = 0;
+    recs[0].accept = 1;
+    recs[0].n_flagged = 0;
+    recs[0].max_fit = 0.0;
   }
-  const int ok = locate_epilogue(n, m, s_eff, n_eff, sc.idx, w_g, recs.data(), flags.data(), n, mask, t_out, rec_rows,
-                                 n_rec, coeff, sc.trusted, sc.task_ws);
+  const int ok = locate_epilogue(tb, n, m, s, sc.forced, recs.data(), flags.data(), n, mask, t_out, rec_rows, n_rec,
+                                 coeff, sc.trusted, sc.task_ws);
   return ok ? SOLON_OK : SOLON_ERR_UNDECODABLE;
 }

@@ -1,21 +1,26 @@
 // Locator (phi) and recovery-table (psi) arithmetic of Solon's decoder, Section 3.4, in float64.
 //
-// One source, two builds.  On the device every function is executed by one CTA: matrices live in
-// shared memory column by column, a warp owns columns (SOLON_FOR_WARPS), its lanes own rows
-// (SOLON_FOR_LANES, partial sums combined by lane_sum), element-wise work is spread over all threads
-// (SOLON_FOR_THREADS) and SOLON_SYNC is the CTA barrier.  On the host the same code runs serially
-// (one warp of one lane), which is what solon_locate_host exposes for CPU tests.
+// One source, two builds.  On the device every function is executed by one CTA: a warp owns columns
+// (SOLON_FOR_WARPS), its lanes own rows (SOLON_FOR_LANES, partial sums combined by lane_sum),
+// element-wise work is spread over all threads (SOLON_FOR_THREADS) and SOLON_SYNC is the CTA barrier.
+// On the host the same code runs serially (one warp of one lane), which is what solon_locate_host
+// exposes for CPU tests.
 //
 // Reading of the paper's exact-arithmetic locator used here:
-//   * the error count is tried incrementally, t = 0..s; for each t the rational-interpolation
-//     system of Section 3.4 is solved with the K projections sharing one denominator;
-//   * polynomials are expanded in Chebyshev polynomials T_i instead of monomials (the same
-//     rational function, a better conditioned system); the denominator is T_t + sum theta_i T_i;
-//   * the t nodes where the denominator is smallest are the candidates; a degree-(m-1) fit on the
-//     remaining nodes must reproduce every remaining node within tau (relative to
-//     sqrt(2 median nu)), which replaces the paper's "P_j(w_i) != r_i" test;
+//   * the error count is tried incrementally, t = 0..s; for each t the rational-interpolation system
+//     of Section 3.4, N_kappa(w_k) = rho_kappa,k E(w_k) with deg N_kappa < m + t and E monic of degree t,
+//     is solved in the least-squares sense with the K projections sharing E;
+//   * the node scalars are fixed by the plan, so an orthonormal basis q_0, q_1, ... of the polynomials
+//     on a group's nodes (q_i of degree i) is tabulated once.  The numerators are eliminated by
+//     projecting on the complement of the polynomials of degree < m + t (columns m+t.. of the table):
+//     only the t coefficients of E remain unknown, E = T_t + sum_i theta_i T_i in Chebyshev polynomials;
+//   * the t nodes where E is smallest are the candidates; a degree-(m-1) fit on the remaining nodes
+//     must reproduce every remaining node within tau (relative to sqrt(2 median nu)), which replaces
+//     the paper's "P_j(w_i) != r_i" test.  The refit is obtained from the fit over all nodes by the
+//     deletion (downdating) identity  r = e + H[:,V] (I - H[V,V])^{-1} e[V],  H = Q_m Q_m^T;
 //   * the inverse of the block decoder is the least-squares inverse over the rows it reads:
-//     m well-spread trusted rows when m <= SOLON_SUBSET_MAX_M, all trusted rows otherwise.
+//     m well-spread trusted rows when m <= SOLON_SUBSET_MAX_M (Lagrange form), all trusted rows
+//     otherwise (the same deletion identity applied to the coefficient map).
 #pragma once
 
 #include <math.h>
@@ -44,15 +49,13 @@
 
 #if defined(__CUDACC__)
 #define SOLON_HD __host__ __device__
-#define SOLON_HD_NOINLINE __host__ __device__ __noinline__   /* one copy of the code: the locator runs once per
-                                                                decode from a cold instruction cache */
 #else
 #define SOLON_HD
-#define SOLON_HD_NOINLINE
 #endif
 
 #define SOLON_SUBSET_MAX_M 6
 #define SOLON_THETA_MAX 16   /* largest error count per group (SOLON_MAX_S) */
+#define SOLON_RHO_CLAMP 1e8  /* projected values beyond this multiple of the group's median are clamped */
 
 namespace solon {
 
@@ -65,6 +68,14 @@ SOLON_HD inline double lane_sum(double x) {
   return x;
 }
 
+// Tables of one group, fixed at plan time (functions of the node scalars only).
+struct GroupTables {
+  const double* Qb;    // n x n, column-major: Qb[j * n + k] = q_j(w_k), orthonormal columns, deg q_j = j
+  const double* Mt;    // m x m, row-major: q_i(w) = sum_l Mt[l * m + i] w^l  (i < m)
+  const double* Tch;   // n x (s + 1), row-major: Tch[k * (s + 1) + i] = T_i(w_k)
+  const double* w;     // n node scalars
+};
+
 // One (group, t) record written by locate_task and read by the group's epilogue.
 struct TaskRecord {
   int accept;      // 1 if every node outside the candidates fits the polynomial
@@ -72,34 +83,22 @@ struct TaskRecord {
   double max_fit;  // largest |residual| / tolerance over the non-candidates (best-guess ranking)
 };
 
-// Doubles of workspace one task needs (group of n nodes, K projections, t errors).
+// Doubles of workspace one task needs (group of n nodes, K projections, up to t errors).
 SOLON_HD inline size_t locate_task_ws_doubles(int n, int m, int K, int t) {
-  size_t ncheb = (size_t)m + t + 1;
-  size_t ncol = (size_t)K * (m + t) + t;
-  size_t rows = (size_t)K * n;
-  size_t solve = rows * (ncol + 1) + (ncol + 1) + (size_t)t * (t + 1) + ncol + n;
-  size_t fit = (size_t)n * (m + K) + (m + K) + (size_t)m * (m + K) + m + (size_t)K * m + n + (size_t)n / 2 + 2;
-  return (size_t)n * ncheb + (solve > fit ? solve : fit) + 8;
+  size_t rows = (size_t)K * n;                              // upper bound of K (n - m - t)
+  size_t solve = rows * (t + 1) + (t + 1) + (size_t)t * (t + 1) + t + n;
+  size_t fit = (size_t)K * m + (size_t)K * n + 3 * (size_t)t * t + (size_t)K * t + n + (size_t)(t + n) / 2 + 4;
+  return solve + fit + 16;
 }
 
 // Doubles of workspace the epilogue needs.
-SOLON_HD inline size_t locate_epilogue_ws_doubles(int n, int m) {
-  return (size_t)n * m + (size_t)m * m + 2 * (size_t)m + 64;
-}
-
-// T_i(x) for i = 0..count-1 into out[0..count).
-SOLON_HD inline void chebyshev_row(double x, int count, double* out) {
-  double t0 = 1.0, t1 = x;
-  for (int i = 0; i < count; ++i) {
-    out[i] = t0;
-    double t2 = 2.0 * x * t1 - t0;
-    t0 = t1;
-    t1 = t2;
-  }
+SOLON_HD inline size_t locate_epilogue_ws_doubles(int n, int m, int s) {
+  size_t t = (size_t)s;     // untrusted nodes the all-rows table is built for: at most s
+  return 3 * t * t + t * (size_t)n + (size_t)m * n + (size_t)n + 64;
 }
 
 // norm0[c] = squared norm of column c of the column-major matrix A (rows x ncols, column stride ldc).
-SOLON_HD_NOINLINE inline void column_norms(const double* A, int rows, int ldc, int ncols, double* norm0) {
+SOLON_HD inline void column_norms(const double* A, int rows, int ldc, int ncols, double* norm0) {
   SOLON_FOR_WARPS(c, ncols) {
     double acc = 0.0;
     SOLON_FOR_LANES(i, rows) acc = fma(A[(size_t)c * ldc + i], A[(size_t)c * ldc + i], acc);
@@ -111,11 +110,10 @@ SOLON_HD_NOINLINE inline void column_norms(const double* A, int rows, int ldc, i
 
 // Modified Gram-Schmidt on the first `nq` columns of the column-major matrix A, applied to all
 // `ncols` columns (the trailing ones are right-hand sides).  Columns stay un-normalised.
-// R (row-major, leading dimension ldr) receives the rows j >= r_first of the triangular factor,
-// right-hand-side columns included, with entry (j, c) stored at R[(j - r_first) * ldr + c - r_first];
+// R (row-major, leading dimension ldr) receives the triangular factor, right-hand sides included;
 // diag[j] = ||q_j|| (0 for a numerically dependent column).
-SOLON_HD_NOINLINE inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols, const double* norm0,
-                                double* R, int ldr, int r_first, double* diag) {
+SOLON_HD inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols, const double* norm0, double* R,
+                                int ldr, double* diag) {
   for (int j = 0; j < nq; ++j) {
     const double* qj = A + (size_t)j * ldc;
     double acc = 0.0;
@@ -126,7 +124,7 @@ SOLON_HD_NOINLINE inline void mgs_factor(double* A, int rows, int ldc, int nq, i
     const double inv2 = dead ? 0.0 : 1.0 / nrm2;
     if (SOLON_TID == 0) {
       diag[j] = nrm;
-      if (j >= r_first) R[(size_t)(j - r_first) * ldr + (j - r_first)] = nrm;
+      R[(size_t)j * ldr + j] = nrm;
     }
     const int todo = ncols - (j + 1);
     SOLON_FOR_WARPS(cc, todo) {
@@ -139,62 +137,125 @@ SOLON_HD_NOINLINE inline void mgs_factor(double* A, int rows, int ldc, int nq, i
         const double coef = dot * inv2;
         SOLON_FOR_LANES(i, rows) ac[i] = fma(-coef, qj[i], ac[i]);
       }
-      if (j >= r_first && SOLON_LANE == 0) R[(size_t)(j - r_first) * ldr + (c - r_first)] = dot * (nrm * inv2);
+      if (SOLON_LANE == 0) R[(size_t)j * ldr + c] = dot * (nrm * inv2);
     }
     SOLON_SYNC();
   }
 }
 
+// In-place inverse of the symmetric positive definite t x t matrix S (row-major) by Gauss-Jordan
+// elimination on [S | I] held in `aug` (t x 2t, row-major); one thread per column of the pair.
+// No pivoting is needed for a positive definite matrix.
+SOLON_HD inline void spd_inverse(double* S, int t, double* aug) {
+  const int w2 = 2 * t;
+  SOLON_FOR_THREADS(idx, t * w2) {
+    const int r = idx / w2, c = idx - r * w2;
+    aug[idx] = c < t ? S[(size_t)r * t + c] : (c - t == r ? 1.0 : 0.0);
+  }
+  SOLON_SYNC();
+  for (int p = 0; p < t; ++p) {
+    const double piv = aug[(size_t)p * w2 + p];
+    const double inv = piv != 0.0 ? 1.0 / piv : 0.0;
+    // columns other than p: scale the pivot row, eliminate column p from the other rows
+    SOLON_FOR_THREADS(c, w2) {
+      if (c == p) continue;
+      const double top = aug[(size_t)p * w2 + c] * inv;
+      for (int r = 0; r < t; ++r) {
+        if (r == p) continue;
+        aug[(size_t)r * w2 + c] = fma(-aug[(size_t)r * w2 + p], top, aug[(size_t)r * w2 + c]);
+      }
+      aug[(size_t)p * w2 + c] = top;
+    }
+    SOLON_SYNC();       // column p has been read by everyone
+    SOLON_FOR_THREADS(r, t) aug[(size_t)r * w2 + p] = r == p ? 1.0 : 0.0;
+    SOLON_SYNC();
+  }
+  SOLON_FOR_THREADS(idx, t * t) {
+    const int r = idx / t, c = idx - r * t;
+    S[idx] = aug[(size_t)r * w2 + t + c];
+  }
+  SOLON_SYNC();
+}
+
+// S <- (I - H[V,V])^{-1} for the node list V (nv nodes), H = Q_m Q_m^T.
+SOLON_HD inline void deletion_inverse(const GroupTables& tb, int n, int m, const int* V, int nv, double* S, double* aug) {
+  SOLON_FOR_THREADS(idx, nv * nv) {
+    const int a = idx / nv, b = idx - a * nv;
+    double h = 0.0;
+    for (int i = 0; i < m; ++i) h = fma(tb.Qb[(size_t)i * n + V[a]], tb.Qb[(size_t)i * n + V[b]], h);
+    S[idx] = (a == b ? 1.0 : 0.0) - h;
+  }
+  SOLON_SYNC();
+  spd_inverse(S, nv, aug);
+}
+
 // Verification: fit a degree-(m-1) polynomial to every projection on the non-candidates and test
-// all nodes.  cheb: n x ncheb table of T_i(w_k); rho_n: K x n projected values divided by the
-// scale; cand[k] != 0 marks the n_cand candidates.  bad[k] receives 1 where some projection is off by
-// more than tau (or is not a number).  Returns through rec.
-SOLON_HD inline void locate_verify(int n, int m, int K, const double* cheb, int ncheb, const double* rho_n,
-                                   double tau, const uint8_t* cand, int n_cand, uint8_t* bad, double* ws,
+// all nodes.  cand[k] != 0 marks the n_cand candidates; forced[k] != 0 marks nodes that are corrupt by
+// inspection (they never fit).  bad[k] receives 1 where some projection is off by more than tau.
+SOLON_HD inline void locate_verify(const GroupTables& tb, int n, int m, int K, const double* rho_n, double tau,
+                                   const uint8_t* cand, int n_cand, const uint8_t* forced, uint8_t* bad, double* ws,
                                    TaskRecord* rec) {
-  const int ld = m + K;          // columns: m basis polynomials, K right-hand sides
-  const int n_u = n - n_cand;    // rows: the non-candidates
-  double* B = ws;                            // column-major, ld columns of n_u rows
-  double* norm0 = B + (size_t)n * ld;        // ld
-  double* Rf = norm0 + ld;                   // m x ld
-  double* diag = Rf + (size_t)m * ld;        // m
-  double* coef = diag + m;                   // K x m
-  double* ratio = coef + (size_t)K * m;      // n
-  int* ulist = reinterpret_cast<int*>(ratio + n);   // n
+  const int t = n_cand;
+  double* coef = ws;                         // K x m   c = Q_m^T rho
+  double* e = coef + (size_t)K * m;          // K x n   e = rho - Q_m c (fit over all nodes)
+  double* S = e + (size_t)K * n;             // t x t
+  double* aug = S + (size_t)t * t;           // t x 2t
+  double* x = aug + 2 * (size_t)t * t;       // K x t   leave-out residuals of the candidates
+  double* ratio = x + (size_t)K * t;         // n
+  int* vlist = reinterpret_cast<int*>(ratio + n);   // t candidates in node order
+  int* vpos = vlist + t;                            // n: position of node k in vlist
   SOLON_FOR_THREADS(k, n) {
-    if (!cand[k]) {
-      int pos = 0;
-      for (int o = 0; o < k; ++o) pos += cand[o] ? 0 : 1;
-      ulist[pos] = k;
+    int pos = 0;
+    for (int o = 0; o < k; ++o) pos += cand[o] ? 1 : 0;
+    vpos[k] = pos;
+    if (cand[k]) vlist[pos] = k;
+  }
+  SOLON_FOR_THREADS(idx, K * m) {
+    const int kappa = idx / m, i = idx - kappa * m;
+    double acc = 0.0;
+    for (int k = 0; k < n; ++k) acc = fma(tb.Qb[(size_t)i * n + k], rho_n[(size_t)kappa * n + k], acc);
+    coef[idx] = acc;
+  }
+  SOLON_SYNC();
+  SOLON_FOR_THREADS(idx, K * n) {
+    const int kappa = idx / n, k = idx - kappa * n;
+    double acc = rho_n[idx];
+    for (int i = 0; i < m; ++i) acc = fma(-tb.Qb[(size_t)i * n + k], coef[(size_t)kappa * m + i], acc);
+    e[idx] = acc;
+  }
+  SOLON_SYNC();
+  if (t > 0) {
+    deletion_inverse(tb, n, m, vlist, t, S, aug);
+    SOLON_FOR_THREADS(idx, K * t) {
+      const int kappa = idx / t, a = idx - kappa * t;
+      double acc = 0.0;
+      for (int b = 0; b < t; ++b) acc = fma(S[(size_t)a * t + b], e[(size_t)kappa * n + vlist[b]], acc);
+      x[idx] = acc;
     }
+    SOLON_SYNC();
   }
-  SOLON_SYNC();
-  SOLON_FOR_THREADS(idx, n_u * ld) {
-    const int c = idx / n_u, i = idx - c * n_u, k = ulist[i];
-    B[(size_t)c * n_u + i] = c < m ? cheb[(size_t)k * ncheb + c] : rho_n[(size_t)(c - m) * n + k];
-  }
-  SOLON_SYNC();
-  column_norms(B, n_u, n_u, ld, norm0);
-  mgs_factor(B, n_u, n_u, m, ld, norm0, Rf, ld, 0, diag);
-  SOLON_FOR_THREADS(kappa, K) {             // back substitution, one projection per thread
-    for (int i = m - 1; i >= 0; --i) {
-      double acc = Rf[(size_t)i * ld + m + kappa];
-      for (int c = i + 1; c < m; ++c) acc = fma(-Rf[(size_t)i * ld + c], coef[(size_t)kappa * m + c], acc);
-      coef[(size_t)kappa * m + i] = diag[i] > 0.0 ? acc / diag[i] : 0.0;
-    }
-  }
-  SOLON_SYNC();
   SOLON_FOR_THREADS(k, n) {
     double worst = 0.0;
     for (int kappa = 0; kappa < K; ++kappa) {
-      double q = 0.0;
-      for (int i = 0; i < m; ++i) q = fma(coef[(size_t)kappa * m + i], cheb[(size_t)k * ncheb + i], q);
-      double res = fabs(rho_n[(size_t)kappa * n + k] - q);
+      double res;
+      if (cand[k]) {
+        res = x[(size_t)kappa * t + vpos[k]];
+      } else {
+        res = e[(size_t)kappa * n + k];
+        for (int b = 0; b < t; ++b) {
+          double h = 0.0;
+          for (int i = 0; i < m; ++i) h = fma(tb.Qb[(size_t)i * n + k], tb.Qb[(size_t)i * n + vlist[b]], h);
+          res = fma(h, x[(size_t)kappa * t + b], res);
+        }
+      }
+      res = fabs(res);
       if (!(res == res)) res = INFINITY;
       worst = res > worst ? res : worst;
     }
-    ratio[k] = tau > 0.0 ? worst / tau : (worst > 0.0 ? INFINITY : 0.0);
-    bad[k] = ratio[k] > 1.0 ? 1 : 0;
+    double rt = tau > 0.0 ? worst / tau : (worst > 0.0 ? INFINITY : 0.0);
+    if (forced[k]) rt = INFINITY;
+    ratio[k] = rt;
+    bad[k] = rt > 1.0 ? 1 : 0;
   }
   SOLON_SYNC();
   if (SOLON_TID == 0) {
@@ -215,62 +276,51 @@ SOLON_HD inline void locate_verify(int n, int m, int K, const double* cheb, int 
   SOLON_SYNC();
 }
 
-// One task: assume exactly t corrupt nodes among the n (finite) nodes of a group.
-//   rho_n   K x n projected values divided by the scale (so honest values are O(1))
-//   w       n node scalars;  tau  tolerance in the same normalised units
+// One task: assume exactly t corrupt nodes among the n nodes of a group.
+//   rho_n   K x n projected values divided by the scale (0 for forced nodes)
+//   s       the plan's s (row stride of tb.Tch is s + 1);  tau  tolerance in the same normalised units
 //   flags   n bytes out: 1 for candidates that do not fit (the located nodes if accepted)
 //   cand, bad: n bytes of scratch each;  ws: locate_task_ws_doubles(n, m, K, t) doubles
-SOLON_HD inline void locate_task(int n, int m, int K, int t, const double* rho_n, const double* w, double tau,
-                                 uint8_t* flags, uint8_t* cand, uint8_t* bad, double* ws, TaskRecord* rec) {
-  const int ncheb = m + t + 1;
-  double* cheb = ws;                         // n x ncheb
-  double* rest = cheb + (size_t)n * ncheb;
-  SOLON_FOR_THREADS(k, n) {
-    chebyshev_row(w[k], ncheb, cheb + (size_t)k * ncheb);
-    cand[k] = 0;
-  }
+SOLON_HD inline void locate_task(const GroupTables& tb, int n, int m, int K, int t, int s, const double* rho_n,
+                                 const uint8_t* forced, double tau, uint8_t* flags, uint8_t* cand, uint8_t* bad,
+                                 double* ws, TaskRecord* rec) {
+  const int ldt = s + 1;
+  SOLON_FOR_THREADS(k, n) cand[k] = 0;
   SOLON_SYNC();
+  double* rest = ws;
   if (t > 0) {
-    const int n_num = m + t;
-    const int ncol = K * n_num + t;            // unknowns: K numerators, then theta
-    const int ld = ncol + 1;                   // + right-hand side
-    const int rows = K * n;
-    double* A = rest;                          // column-major, ld columns of `rows` rows
+    const int nperp = n - m - t;               // complement of the polynomials of degree < m + t
+    const int rows = K * nperp;
+    const int ld = t + 1;                      // t unknowns theta, then the right-hand side
+    double* A = ws;                            // column-major, ld columns of `rows` rows
     double* norm0 = A + (size_t)rows * ld;     // ld
-    double* Rt = norm0 + ld;                   // t x (t+1): trailing rows of R, rhs in the last column
-    double* diag = Rt + (size_t)t * (t + 1);   // ncol
-    double* absE = diag + ncol;                // n
+    double* Rt = norm0 + ld;                   // t x (t + 1)
+    double* diag = Rt + (size_t)t * (t + 1);   // t
+    double* absE = diag + t;                   // n
+    rest = absE + n;
+    // A[(kappa, j), i] = sum_k q_{m+t+j}(w_k) rho_kappa,k T_i(w_k); the last column carries -(...) T_t
     SOLON_FOR_THREADS(idx, rows * ld) {
-      const int c = idx / rows, row = idx - c * rows;
-      const int kappa = row / n, k = row - kappa * n;
-      const double rv = rho_n[(size_t)kappa * n + k];
-      const double sc = 1.0 / sqrt(1.0 + rv * rv);     // balance rows of very large (corrupt) values
-      double val;
-      if (c < K * n_num) {
-        const int blk = c / n_num, i = c - blk * n_num;
-        val = blk == kappa ? sc * cheb[(size_t)k * ncheb + i] : 0.0;
-      } else if (c < ncol) {
-        val = -sc * rv * cheb[(size_t)k * ncheb + (c - K * n_num)];
-      } else {
-        val = sc * rv * cheb[(size_t)k * ncheb + t];
-      }
-      A[idx] = val;
+      const int i = idx / rows, row = idx - i * rows;
+      const int kappa = row / nperp, j = row - kappa * nperp;
+      const double* q = tb.Qb + (size_t)(m + t + j) * n;
+      double acc = 0.0;
+      for (int k = 0; k < n; ++k) acc = fma(q[k] * rho_n[(size_t)kappa * n + k], tb.Tch[(size_t)k * ldt + i], acc);
+      A[idx] = i < t ? acc : -acc;
     }
     SOLON_SYNC();
     column_norms(A, rows, rows, ld, norm0);
-    const int r_first = ncol - t;
-    mgs_factor(A, rows, rows, ncol, ld, norm0, Rt, t + 1, r_first, diag);
-    // back substitution for the last t unknowns (theta); every thread does the same arithmetic
+    mgs_factor(A, rows, rows, t, ld, norm0, Rt, t + 1, diag);
+    // back substitution for theta; every thread does the same arithmetic
     double theta[SOLON_THETA_MAX];
     for (int i = t - 1; i >= 0; --i) {
       double acc = Rt[(size_t)i * (t + 1) + t];
       for (int c = i + 1; c < t; ++c) acc = fma(-Rt[(size_t)i * (t + 1) + c], theta[c], acc);
-      theta[i] = diag[r_first + i] > 0.0 ? acc / diag[r_first + i] : 0.0;
+      theta[i] = diag[i] > 0.0 ? acc / diag[i] : 0.0;
     }
     SOLON_FOR_THREADS(k, n) {
-      double e = cheb[(size_t)k * ncheb + t];
-      for (int i = 0; i < t; ++i) e = fma(theta[i], cheb[(size_t)k * ncheb + i], e);
-      const double ae = fabs(e);
+      double ev = tb.Tch[(size_t)k * ldt + t];
+      for (int i = 0; i < t; ++i) ev = fma(theta[i], tb.Tch[(size_t)k * ldt + i], ev);
+      const double ae = fabs(ev);
       absE[k] = (ae == ae) ? ae : INFINITY;
     }
     SOLON_SYNC();
@@ -282,7 +332,7 @@ SOLON_HD inline void locate_task(int n, int m, int K, int t, const double* rho_n
     }
     SOLON_SYNC();
   }
-  locate_verify(n, m, K, cheb, ncheb, rho_n, tau, cand, t, bad, rest, rec);
+  locate_verify(tb, n, m, K, rho_n, tau, cand, t, forced, bad, rest, rec);
   SOLON_FOR_THREADS(k, n) flags[k] = (cand[k] && bad[k]) ? 1 : 0;
   SOLON_SYNC();
 }
@@ -290,19 +340,22 @@ SOLON_HD inline void locate_task(int n, int m, int K, int t, const double* rho_n
 // Recovery table for one group: given the trusted nodes (trusted[k] != 0 among n), choose the rows
 // the recovery reads and the weights coeff[j*m + l] of row rec_rows[j] in coordinate l of a chunk,
 // i.e. the least-squares inverse of [W-hat_{m-1}]_{rows,.} (monomial basis, as the encoder used).
-// ws: locate_epilogue_ws_doubles(n, m).  Returns the number of rows (same value in every thread).
-SOLON_HD inline int recovery_table(int n, int m, const double* w, const uint8_t* trusted, int* rec_rows,
+// ws: locate_epilogue_ws_doubles(n, m, s).  Returns the number of rows (same value in every thread),
+// 0 if fewer than m nodes are trusted or (all-rows form) more than s are not.
+SOLON_HD inline int recovery_table(const GroupTables& tb, int n, int m, int s, const uint8_t* trusted, int* rec_rows,
                                    double* coeff, double* ws) {
   int n_u = 0;
   for (int k = 0; k < n; ++k) n_u += trusted[k] ? 1 : 0;
   if (n_u < m) return 0;
-  const int n_rec = (m <= SOLON_SUBSET_MAX_M) ? m : n_u;
+  const bool subset = m <= SOLON_SUBSET_MAX_M;
+  if (!subset && n - n_u > s) return 0;
+  const int n_rec = subset ? m : n_u;
   {
     // every thread derives the same list; thread 0 stores it
     int seen = 0, next = 0;
     for (int k = 0; k < n && next < n_rec; ++k) {
       if (!trusted[k]) continue;
-      const int want = (n_rec == n_u) ? next
+      const int want = !subset ? next
                        : (m == 1 ? (n_u - 1) / 2 : (int)(((long long)next * (n_u - 1) + (m - 1) / 2) / (m - 1)));
       if (seen == want) {
         if (SOLON_TID == 0) rec_rows[next] = k;
@@ -312,118 +365,174 @@ SOLON_HD inline int recovery_table(int n, int m, const double* w, const uint8_t*
     }
   }
   SOLON_SYNC();
-  double* V = ws;                          // column-major: m columns of n_rec rows (becomes Q, un-normalised)
-  double* norm0 = V + (size_t)n_rec * m;   // m
-  double* R = norm0 + m;                   // m x m
-  double* diag = R + (size_t)m * m;        // m
-  SOLON_FOR_THREADS(j, n_rec) {
-    const double x = w[rec_rows[j]];
-    double p = 1.0;
-    for (int l = 0; l < m; ++l) {
-      V[(size_t)l * n_rec + j] = p;
-      p *= x;
+  if (subset) {
+    // Lagrange form of the inverse Vandermonde: row j holds the monomial coefficients of
+    // L_j(w) = prod_{i != j} (w - x_i) / (x_j - x_i), built by multiplying one factor at a time.
+    SOLON_FOR_THREADS(j, m) {
+      double* c = coeff + (size_t)j * m;
+      const double xj = tb.w[rec_rows[j]];
+      for (int l = 0; l < m; ++l) c[l] = 0.0;
+      c[0] = 1.0;
+      int deg = 0;
+      double denom = 1.0;
+      for (int i = 0; i < m; ++i) {
+        if (i == j) continue;
+        const double xi = tb.w[rec_rows[i]];
+        for (int l = deg + 1; l >= 1; --l) c[l] = fma(-xi, c[l], c[l - 1]);   // times (w - x_i)
+        c[0] = -xi * c[0];
+        ++deg;
+        denom *= xj - xi;
+      }
+      const double inv = 1.0 / denom;
+      for (int l = 0; l < m; ++l) c[l] *= inv;
+    }
+    SOLON_SYNC();
+    return n_rec;
+  }
+  // All trusted rows: coefficients in the orthonormal basis after deleting the untrusted nodes V,
+  //   c' = (Q_U^T + Q_V^T (I - H_VV)^{-1} H_VU) z_U,  then monomial coefficients  y = Mt c'.
+  const int nv = n - n_u;
+  double* S = ws;                               // nv x nv
+  double* aug = S + (size_t)nv * nv;            // nv x 2nv
+  double* Z = aug + 2 * (size_t)nv * nv;        // nv x n_u:  S^{-1} H_VU
+  double* Wc = Z + (size_t)nv * n_u;            // m x n_u:   Q_U^T + Q_V^T Z
+  int* vlist = reinterpret_cast<int*>(Wc + (size_t)m * n_u);   // nv
+  SOLON_FOR_THREADS(k, n) {
+    if (!trusted[k]) {
+      int pos = 0;
+      for (int o = 0; o < k; ++o) pos += trusted[o] ? 0 : 1;
+      vlist[pos] = k;
     }
   }
   SOLON_SYNC();
-  column_norms(V, n_rec, n_rec, m, norm0);
-  mgs_factor(V, n_rec, n_rec, m, m, norm0, R, m, 0, diag);
-  // C = R^{-1} Q^T, one trusted row per thread
-  SOLON_FOR_THREADS(j, n_rec) {
-    double* c = coeff + (size_t)j * m;
-    for (int l = m - 1; l >= 0; --l) {
-      double acc = diag[l] > 0.0 ? V[(size_t)l * n_rec + j] / diag[l] : 0.0;
-      for (int i = l + 1; i < m; ++i) acc = fma(-R[(size_t)l * m + i], c[i], acc);
-      c[l] = diag[l] > 0.0 ? acc / diag[l] : 0.0;
+  if (nv > 0) {
+    deletion_inverse(tb, n, m, vlist, nv, S, aug);
+    SOLON_FOR_THREADS(idx, nv * n_u) {
+      const int a = idx / n_u, u = idx - a * n_u;
+      double acc = 0.0;
+      for (int b = 0; b < nv; ++b) {
+        double h = 0.0;
+        for (int i = 0; i < m; ++i) h = fma(tb.Qb[(size_t)i * n + vlist[b]], tb.Qb[(size_t)i * n + rec_rows[u]], h);
+        acc = fma(S[(size_t)a * nv + b], h, acc);
+      }
+      Z[idx] = acc;
     }
+    SOLON_SYNC();
+  }
+  SOLON_FOR_THREADS(idx, m * n_u) {
+    const int i = idx / n_u, u = idx - i * n_u;
+    double acc = tb.Qb[(size_t)i * n + rec_rows[u]];
+    for (int a = 0; a < nv; ++a) acc = fma(tb.Qb[(size_t)i * n + vlist[a]], Z[(size_t)a * n_u + u], acc);
+    Wc[idx] = acc;
+  }
+  SOLON_SYNC();
+  SOLON_FOR_THREADS(idx, n_u * m) {
+    const int u = idx / m, l = idx - u * m;
+    double acc = 0.0;
+    for (int i = 0; i < m; ++i) acc = fma(tb.Mt[(size_t)l * m + i], Wc[(size_t)i * n_u + u], acc);
+    coeff[(size_t)u * m + l] = acc;
   }
   SOLON_SYNC();
   return n_rec;
 }
 
-// Group preparation shared by all tasks of a group: drop nodes whose projected values or energy are
-// not finite (such nodes are corrupt by inspection), scale the rest.
-//   rho: K rows with leading dimension ld_rho, this group's n entries each;  nu, w: n entries
-//   idx[n_eff] original positions of the kept nodes; rho_n (K x n_eff) = rho / scale; w_c their scalars
-//   *tau_eff = tau, or 0 when the median energy is 0 (all-zero data: any deviation counts)
-// scratch: n doubles.  Returns n_eff (same in every thread).
-SOLON_HD inline int locate_prepare(int n, int K, const double* rho, int ld_rho, const double* nu, const double* w,
-                                   double tau, int* idx, double* rho_n, double* w_c, double* tau_eff,
-                                   double* scratch) {
-  int n_eff = 0;
-  for (int k = 0; k < n; ++k) {
+// Group preparation shared by all tasks of a group.
+//   rho (K x n), nu (n): this group's projected values and energies
+//   forced[k] = 1 for nodes whose values are not finite (corrupt by inspection; their rho_n is 0)
+//   rho_n = rho / sqrt(2 median nu), clamped to +-SOLON_RHO_CLAMP medians of |rho| per projection
+//   *tau_eff = tau, or (median energy 0: all-zero data, any deviation counts) 1e-10 of the largest |rho|
+// scratch: K + 2 doubles.
+SOLON_HD inline void locate_prepare(int n, int K, const double* rho, const double* nu, double tau, uint8_t* forced,
+                                    double* rho_n, double* tau_eff, double* scratch) {
+  SOLON_FOR_THREADS(k, n) {
     bool finite = isfinite(nu[k]);
-    for (int kappa = 0; kappa < K; ++kappa) finite = finite && isfinite(rho[(size_t)kappa * ld_rho + k]);
-    if (finite) {
-      if (SOLON_TID == 0) idx[n_eff] = k;
-      ++n_eff;
+    for (int kappa = 0; kappa < K; ++kappa) finite = finite && isfinite(rho[(size_t)kappa * n + k]);
+    forced[k] = finite ? 0 : 1;
+  }
+  SOLON_FOR_THREADS(i, K + 1) scratch[i] = 0.0;
+  SOLON_SYNC();
+  int n_fin = 0;
+  for (int k = 0; k < n; ++k) n_fin += forced[k] ? 0 : 1;
+  // lower medians by rank counting among the finite nodes: scratch[0] <- median nu,
+  // scratch[1 + kappa] <- median |rho_kappa|
+  SOLON_FOR_THREADS(idx, (K + 1) * n) {
+    const int which = idx / n, i = idx - which * n;
+    if (!forced[i]) {
+      const double* src = which == 0 ? nu : rho + (size_t)(which - 1) * n;
+      const double mine = fabs(src[i]);
+      int rank = 0;
+      for (int o = 0; o < n; ++o) {
+        if (forced[o]) continue;
+        const double other = fabs(src[o]);
+        rank += (other < mine || (other == mine && o < i)) ? 1 : 0;
+      }
+      if (rank == (n_fin - 1) / 2) scratch[which] = mine;
     }
   }
   SOLON_SYNC();
-  // lower median of the kept energies by rank counting
-  SOLON_FOR_THREADS(i, n_eff) {
-    const double mine = nu[idx[i]];
-    int rank = 0;
-    for (int o = 0; o < n_eff; ++o) {
-      const double other = nu[idx[o]];
-      rank += (other < mine || (other == mine && o < i)) ? 1 : 0;
-    }
-    if (rank == (n_eff - 1) / 2) scratch[0] = mine;
-  }
-  SOLON_SYNC();
-  const double med = n_eff > 0 ? scratch[0] : 0.0;
+  const double med = n_fin > 0 ? scratch[0] : 0.0;
   const double scale = med > 0.0 ? sqrt(2.0 * med) : 1.0;
-  *tau_eff = med > 0.0 ? tau : 0.0;
-  SOLON_FOR_THREADS(i, n_eff) {
-    w_c[i] = w[idx[i]];
-    for (int kappa = 0; kappa < K; ++kappa) rho_n[(size_t)kappa * n_eff + i] = rho[(size_t)kappa * ld_rho + idx[i]] / scale;
+  if (med > 0.0) {
+    *tau_eff = tau;
+  } else {
+    // all-zero honest data: any deviation counts, down to the rounding of the largest value present
+    double big = 0.0;
+    for (int idx = 0; idx < K * n; ++idx) {
+      const double v = forced[idx % n] ? 0.0 : fabs(rho[idx]);
+      big = v > big ? v : big;
+    }
+    *tau_eff = 1e-10 * big;
+  }
+  SOLON_FOR_THREADS(idx, K * n) {
+    const int kappa = idx / n, i = idx - kappa * n;
+    double v = forced[i] ? 0.0 : rho[idx];
+    const double cap = scratch[1 + kappa] * SOLON_RHO_CLAMP;
+    if (cap > 0.0) v = v > cap ? cap : (v < -cap ? -cap : v);
+    rho_n[idx] = v / scale;
   }
   SOLON_SYNC();
-  return n_eff;
 }
 
 // Group epilogue: pick the smallest accepted error count (else the best-fitting guess), write the
-// mask over the group's n original nodes, and build the recovery table from the trusted nodes.
-//   recs[s_eff+1], flags[(s_eff+1) x flags_ld] from the tasks (s_eff < 0: more non-finite nodes than s)
-//   trusted: n bytes scratch; ws: locate_epilogue_ws_doubles(n, m)
-// Returns 1 if the group decoded, 0 if not.  *t_out: corrupt nodes assumed (-1 if undecodable).
-SOLON_HD inline int locate_epilogue(int n, int m, int s_eff, int n_eff, const int* idx, const double* w,
+// mask over the group's n nodes, and build the recovery table from the trusted nodes.
+//   recs[s+1], flags[(s+1) x flags_ld] from the tasks; forced from locate_prepare
+//   trusted: n bytes scratch; ws: locate_epilogue_ws_doubles(n, m, s)
+// Returns 1 if the group decoded, 0 if not.  *t_out: corrupt nodes located (-1 if undecodable).
+SOLON_HD inline int locate_epilogue(const GroupTables& tb, int n, int m, int s, const uint8_t* forced,
                                     const TaskRecord* recs, const uint8_t* flags, int flags_ld, uint8_t* mask,
                                     int* t_out, int* rec_rows, int* n_rec_out, double* coeff, uint8_t* trusted,
                                     double* ws) {
-  int chosen = -1, ok = 0;
-  if (s_eff >= 0) {
-    for (int t = 0; t <= s_eff; ++t) {
-      if (recs[t].accept) {
+  int chosen = 0, ok = 0;
+  for (int t = 0; t <= s; ++t) {
+    if (recs[t].accept) {
+      chosen = t;
+      ok = 1;
+      break;
+    }
+  }
+  if (!ok) {
+    double best = INFINITY;
+    for (int t = 0; t <= s; ++t) {
+      if (recs[t].max_fit < best) {
+        best = recs[t].max_fit;
         chosen = t;
-        ok = 1;
-        break;
-      }
-    }
-    if (!ok) {
-      double best = INFINITY;
-      chosen = 0;
-      for (int t = 0; t <= s_eff; ++t) {
-        if (recs[t].max_fit < best) {
-          best = recs[t].max_fit;
-          chosen = t;
-        }
       }
     }
   }
-  SOLON_FOR_THREADS(k, n) trusted[k] = 0;
-  SOLON_SYNC();
-  if (chosen >= 0) {
-    SOLON_FOR_THREADS(i, n_eff) trusted[idx[i]] = flags[(size_t)chosen * flags_ld + i] ? 0 : 1;
-  } else {
-    SOLON_FOR_THREADS(i, n_eff) trusted[idx[i]] = 1;
+  SOLON_FOR_THREADS(k, n) {
+    const uint8_t corrupt = (flags[(size_t)chosen * flags_ld + k] || forced[k]) ? 1 : 0;
+    trusted[k] = corrupt ? 0 : 1;
+    mask[k] = corrupt;
   }
   SOLON_SYNC();
-  SOLON_FOR_THREADS(k, n) mask[k] = trusted[k] ? 0 : 1;
-  const int n_rec = recovery_table(n, m, w, trusted, rec_rows, coeff, ws);
+  int n_bad = 0;
+  for (int k = 0; k < n; ++k) n_bad += trusted[k] ? 0 : 1;
+  if (n_bad > s) ok = 0;
+  const int n_rec = recovery_table(tb, n, m, s, trusted, rec_rows, coeff, ws);
   if (n_rec == 0) ok = 0;
   if (SOLON_TID == 0) {
     *n_rec_out = n_rec;
-    *t_out = ok ? chosen + (n - n_eff) : -1;
+    *t_out = ok ? n_bad : -1;
   }
   SOLON_SYNC();
   return ok;
