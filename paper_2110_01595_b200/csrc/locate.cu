@@ -28,6 +28,7 @@ struct LocateParams {
   double* ws_global;     // q x (s + 1) x ws_stride, used when shared memory is too small
   size_t ws_stride;
   int use_smem;
+  int stage_tables;      // copy the group's tables to shared memory (after ws_stride doubles of workspace)
   uint8_t* mask;         // P (caller's buffer)
   int* t_acc;            // q
   int* n_rec;            // q
@@ -90,6 +91,19 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
   tb.Mt = prm.mt + (size_t)g * prm.m * prm.m;
   tb.Tch = prm.tch + (size_t)row0 * (prm.s + 1);
   tb.w = prm.w + row0;
+  if (prm.stage_tables) {
+    // small groups: one coalesced pass brings the plan's tables on chip, so the dependent reads of the
+    // solver never wait on L2 or HBM (the tables are evicted by the streaming kernels between decodes)
+    double* qb_s = smem_ws + prm.ws_stride;
+    double* tch_s = qb_s + (size_t)n * n;
+    double* w_s = tch_s + (size_t)n * (prm.s + 1);
+    for (int i = tid; i < n * n; i += kLocThreads) qb_s[i] = tb.Qb[i];
+    for (int i = tid; i < n * (prm.s + 1); i += kLocThreads) tch_s[i] = tb.Tch[i];
+    for (int i = tid; i < n; i += kLocThreads) w_s[i] = tb.w[i];
+    tb.Qb = qb_s;
+    tb.Tch = tch_s;
+    tb.w = w_s;
+  }
 
   TaskRecord* recs = prm.records + (size_t)g * (prm.s + 1);
   uint8_t* flags = prm.task_flags + (size_t)t * prm.P + row0;
@@ -246,6 +260,12 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
   if (need > plan->locate_ws_stride * sizeof(double)) return SOLON_ERR_INTERNAL;
   prm.use_smem = need <= 96 * 1024 ? 1 : 0;
   size_t smem = prm.use_smem ? need : 0;
+  const size_t tables = ((size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
+  prm.stage_tables = (prm.use_smem && smem + tables <= 160 * 1024) ? 1 : 0;
+  if (prm.stage_tables) {
+    prm.ws_stride = need / sizeof(double);      // the tables follow the workspace in shared memory
+    smem += tables;
+  }
   if (prm.use_smem && smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(plan->s + 1, plan->q);

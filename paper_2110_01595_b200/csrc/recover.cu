@@ -3,7 +3,8 @@
 //
 // One pass over the trusted rows the locator selected (m per group when m <= 6, else all trusted rows).
 // Each thread owns a few chunks, loads one float per row and chunk (coalesced along the chunk axis),
-// accumulates the m outputs of each chunk in float64 registers, and every warp writes its run of chunks
+// accumulates the m outputs of each chunk in registers (float32 for m <= 6, where the weights are small;
+// float64 above, where they reach 10^3 and cancel), and every warp writes its run of chunks
 // back through its own shared-memory buffer as contiguous 128-bit stores.  The rows and weights come from device memory written by
 // the locator kernel, so no host round trip separates the two.
 #include "solon_internal.h"
@@ -25,23 +26,25 @@ struct RecoverParams {
 };
 
 // Copy the locator's tables (group layout, rows per group, row indices, weights) into shared memory.
-__device__ __forceinline__ void load_tables(const RecoverParams& prm, double* coeff_s, int* rows_s, int* start_s,
+template <typename Acc>
+__device__ __forceinline__ void load_tables(const RecoverParams& prm, Acc* coeff_s, int* rows_s, int* start_s,
                                             int* n_rec_s) {
-  for (int i = threadIdx.x; i < prm.P * prm.m; i += blockDim.x) coeff_s[i] = prm.coeff[i];
+  for (int i = threadIdx.x; i < prm.P * prm.m; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
   for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
   for (int i = threadIdx.x; i <= prm.q; i += blockDim.x) start_s[i] = prm.group_start[i];
   for (int i = threadIdx.x; i < prm.q; i += blockDim.x) n_rec_s[i] = prm.n_rec[i];
   __syncthreads();
 }
 
-template <int M, int CPT>
+template <int M, int CPT, typename Acc>
 __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int kWarpChunks = 32 * CPT;                      // chunks one warp handles per step
   constexpr int kWarps = kRecThreads / 32;
   float* out_all = reinterpret_cast<float*>(smem_raw);       // per warp: kWarpChunks x M
-  double* coeff_s = reinterpret_cast<double*>(smem_raw + (size_t)kWarps * kWarpChunks * M * sizeof(float));
-  int* rows_s = reinterpret_cast<int*>(coeff_s + (size_t)prm.P * M);
+  Acc* coeff_s = reinterpret_cast<Acc*>(smem_raw + (size_t)kWarps * kWarpChunks * M * sizeof(float));
+  int* rows_s = reinterpret_cast<int*>(smem_raw + (size_t)kWarps * kWarpChunks * M * sizeof(float) +
+                                       (size_t)prm.P * M * sizeof(double));
   int* start_s = rows_s + prm.P;
   int* n_rec_s = start_s + prm.q + 1;
   load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
@@ -52,11 +55,11 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
   // does arithmetic or stores.
   const int64_t stride = (int64_t)gridDim.x * kWarps * kWarpChunks;
   for (int64_t c0 = ((int64_t)blockIdx.x * kWarps + warp) * kWarpChunks; c0 < prm.d_c; c0 += stride) {
-    double acc[CPT][M];
+    Acc acc[CPT][M];
 #pragma unroll
     for (int i = 0; i < CPT; ++i)
 #pragma unroll
-      for (int l = 0; l < M; ++l) acc[i][l] = 0.0;
+      for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
     bool ok[CPT];
 #pragma unroll
     for (int i = 0; i < CPT; ++i) ok[i] = c0 + lane + i * 32 < prm.d_c;
@@ -76,13 +79,13 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
 #pragma unroll
         for (int jj = 0; jj < kRowBlock; ++jj) {
           if (j0 + jj < n) {
-            const double* cj = coeff_s + (size_t)(base + j0 + jj) * M;
-            double dv[CPT];
+            const Acc* cj = coeff_s + (size_t)(base + j0 + jj) * M;
+            Acc dv[CPT];
 #pragma unroll
-            for (int i = 0; i < CPT; ++i) dv[i] = (double)v[jj][i];
+            for (int i = 0; i < CPT; ++i) dv[i] = (Acc)v[jj][i];
 #pragma unroll
             for (int l = 0; l < M; ++l) {
-              const double c = cj[l];
+              const Acc c = cj[l];
 #pragma unroll
               for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, dv[i], acc[i][l]);
             }
@@ -130,20 +133,20 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   }
 }
 
-template <int M, int CPT>
+template <int M, int CPT, typename Acc>
 static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   size_t smem = (size_t)kRecThreads * CPT * M * sizeof(float) + (size_t)plan->P * M * sizeof(double) +
                 (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
-  SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_kernel<M, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_kernel<M, CPT, Acc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   static_assert((32 * CPT) % 4 == 0, "warp tiles must start on a 16-byte boundary of the output");
   int64_t tiles = (plan->d_c + (int64_t)kRecThreads * CPT - 1) / ((int64_t)kRecThreads * CPT);
   int per_sm = 1;
-  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recover_kernel<M, CPT>, kRecThreads, smem));
+  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recover_kernel<M, CPT, Acc>, kRecThreads, smem));
   if (per_sm < 1) per_sm = 1;
   int64_t cap = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(tiles < cap ? tiles : cap);
-  recover_kernel<M, CPT><<<grid, kRecThreads, smem, plan->stream>>>(prm);
+  recover_kernel<M, CPT, Acc><<<grid, kRecThreads, smem, plan->stream>>>(prm);
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }
@@ -163,14 +166,14 @@ int launch_recover(solon_plan* plan, const float* received, float* agg) {
   prm.coeff = plan->d_coeff;
   plan->launches += 1;
   switch (plan->m) {
-    case 1: return launch_recover_m<1, 4>(plan, prm);
-    case 2: return launch_recover_m<2, 4>(plan, prm);
-    case 3: return launch_recover_m<3, 4>(plan, prm);
-    case 4: return launch_recover_m<4, 4>(plan, prm);
-    case 5: return launch_recover_m<5, 4>(plan, prm);
-    case 6: return launch_recover_m<6, 2>(plan, prm);
-    case 8: return launch_recover_m<8, 2>(plan, prm);
-    case 10: return launch_recover_m<10, 2>(plan, prm);
+    case 1: return launch_recover_m<1, 4, float>(plan, prm);
+    case 2: return launch_recover_m<2, 4, float>(plan, prm);
+    case 3: return launch_recover_m<3, 4, float>(plan, prm);
+    case 4: return launch_recover_m<4, 4, float>(plan, prm);
+    case 5: return launch_recover_m<5, 4, float>(plan, prm);
+    case 6: return launch_recover_m<6, 2, float>(plan, prm);
+    case 8: return launch_recover_m<8, 2, double>(plan, prm);
+    case 10: return launch_recover_m<10, 2, double>(plan, prm);
     default: break;
   }
   size_t smem = (size_t)plan->P * plan->m * sizeof(double) + (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
