@@ -311,6 +311,88 @@ def run_ours(args, wl):
     dist_util.shutdown()
 
 
+def run_sweep(args):
+    """The grid P in {15,45,105} x s in {1,3,5} x m in {1,2,5,10} x d: s random nodes send N(0,100^2).
+
+    Every point is checked (mask equal to the attacked set; aggregate against a float64 device-side sum of the
+    partition gradients, the definition of the result) and timed with CUDA events; GB/s figures use each
+    kernel's algorithmic bytes.  One JSON line per point goes to the file; one summary line is printed.
+    """
+    from paper_2110_01595_b200 import binding, build
+
+    torch.cuda.set_device(0)
+    build.build()
+    peak, peak_kind = measured_peak()
+    ds = tuple(int(x) for x in args.sweep_d.split(","))
+    points = synth.sweep_points(ds)
+    worst_err, failures, rows = 0.0, 0, []
+    with open(args.sweep, "a") as out:
+        for wl in points:
+            G = synth.make_grads(wl, "cuda")
+            plan = binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed)
+            coded = plan.encode(G)
+            nodes = synth.byzantine_nodes(wl)
+            byz_rows = synth.byzantine_rows(wl, coded, nodes)
+            agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+            mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
+
+            def step(ev=None):
+                if ev:
+                    ev[0].record()
+                plan.encode(G, coded)
+                if ev:
+                    ev[1].record()
+                for i, k in enumerate(nodes):
+                    coded[k].copy_(byz_rows[i])
+                if ev:
+                    ev[2].record()
+                plan.decode(coded, agg, mask)
+                if ev:
+                    ev[3].record()
+
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            n_steps = max(3, min(args.steps, 10))
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_steps)]
+            for ev in evs:
+                step(ev)
+            torch.cuda.synchronize()
+            status = plan.decode_status()
+            enc_ms = float(np.median([e[0].elapsed_time(e[1]) for e in evs]))
+            dec_ms = float(np.median([e[2].elapsed_time(e[3]) for e in evs]))
+            n_rec = int(plan.recovery()[0].sum())
+            enc_b, proj_b, rec_b = algorithmic_bytes(wl, n_rec)
+            ref = G.sum(dim=0, dtype=torch.float64)
+            scale = float(ref.abs().max())
+            err = float((agg.double() - ref).abs().max()) / scale
+            mask_ok = mask.nonzero().flatten().tolist() == nodes
+            ok = bool(status == 0 and mask_ok and err <= 1e-4)
+            failures += 0 if ok else 1
+            worst_err = max(worst_err, err)
+            total_b = enc_b + proj_b + rec_b
+            row = {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "q": plan.q, "ok": ok,
+                   "status": status, "mask_exact": mask_ok, "agg_err": err, "encode_ms": enc_ms, "decode_ms": dec_ms,
+                   "gradient_gbs": wl.P * wl.d * 4 / ((enc_ms + dec_ms) * 1e-3) / 1e9,
+                   "hbm_gbs": total_b / ((enc_ms + dec_ms) * 1e-3) / 1e9,
+                   "frac_of_peak": total_b / ((enc_ms + dec_ms) * 1e-3) / 1e9 / peak,
+                   "frac_of_8TBs": total_b / ((enc_ms + dec_ms) * 1e-3) / 1e9 / 8000.0,
+                   "encode_gbs": enc_b / (enc_ms * 1e-3) / 1e9, "decodes_per_s": 1e3 / dec_ms}
+            out.write(json.dumps(row) + "\n")
+            out.flush()
+            rows.append(row)
+            plan.close()
+            del G, coded, byz_rows, agg, mask, ref, plan
+            torch.cuda.empty_cache()
+    big = [r for r in rows if r["d"] >= 10_000_000]
+    summary = {"sweep_points": len(rows), "failures": failures, "worst_agg_err": worst_err, "peak_gbs": peak,
+               "peak_kind": peak_kind,
+               "median_frac_of_peak_d_ge_10M": float(np.median([r["frac_of_peak"] for r in big])) if big else None,
+               "min_frac_of_8TBs_d_ge_10M": min((r["frac_of_8TBs"] for r in big), default=None),
+               "max_frac_of_8TBs_d_ge_10M": max((r["frac_of_8TBs"] for r in big), default=None)}
+    print(json.dumps(summary), flush=True)
+
+
 # DRAM bytes (read + write) per encode launch from an ncu capture, by workload; None = not captured for this build.
 TRAFFIC: dict = {}
 
@@ -325,6 +407,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default=None, metavar="FILE",
+                    help="run the (P, s, m, d) grid instead: one JSON line per point is appended to FILE, a summary is printed")
+    ap.add_argument("--sweep-d", default="1000000,10000000,50000000", help="gradient lengths of the grid")
     ap.add_argument("--oracle-d", type=int, default=None,
                     help="coordinates per gradient in the oracle's sample (default: 16M for the cpu_baseline leg, "
                          "2M per step for --impl reference)")
@@ -340,8 +425,9 @@ def main():
         raise SystemExit("the lsq configuration is a parity case, not a bench workload")
     if args.oracle_d is None:
         args.oracle_d = 2_000_000 if args.impl == "reference" else 16_000_000
-    if args.oracle_d is None:
-        args.oracle_d = 2_000_000 if args.impl == "reference" else 16_000_000
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args, wl)
     else:
