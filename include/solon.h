@@ -212,6 +212,14 @@ int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows,
 int solon_project_noalloc(const float* received, const float* f, int64_t f_pitch, int P, int64_t d_c,
                           int K, double* rho, double* nu, void* cuda_stream);
 
+/* Per-kernel timing with CUDA events on the plan's stream.  When switched on, solon_encode and
+ * solon_decode record an event before and after each of their kernels; solon_plan_get_timings
+ * synchronises the stream and returns the durations of the most recent calls in milliseconds:
+ * ms[0] encode, ms[1] projections, ms[2] locator, ms[3] recovery (0 for a kernel not yet run).
+ * Off by default (the events cost a few microseconds per call). */
+int solon_plan_set_profiling(solon_plan* plan, int on);
+int solon_plan_get_timings(solon_plan* plan, float* ms /* host, 4 */);
+
 /* Number of kernels the library launched on behalf of this plan since creation. */
 int64_t solon_plan_kernel_launches(const solon_plan* plan);
 

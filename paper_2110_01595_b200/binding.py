@@ -55,6 +55,8 @@ SIGNATURES = {
     "solon_plan_get_projections": (c_int, [c_void_p, POINTER(c_double), POINTER(c_double)]),
     "solon_plan_get_recovery": (c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_double)]),
     "solon_plan_kernel_launches": (c_int64, [c_void_p]),
+    "solon_plan_set_profiling": (c_int, [c_void_p, c_int]),
+    "solon_plan_get_timings": (c_int, [c_void_p, POINTER(c_float)]),
     "solon_project_noalloc": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_int64, c_int, c_void_p, c_void_p, c_void_p]),
 }
 
@@ -230,6 +232,15 @@ class Plan:
         f = np.zeros((self.K, self.d_c), dtype=np.float32)
         _check(lib().solon_plan_get_projection_vectors(self._h, _dptr(f, c_float)), "solon_plan_get_projection_vectors")
         return f
+
+    def set_profiling(self, on: bool) -> None:
+        _check(lib().solon_plan_set_profiling(self._h, 1 if on else 0), "solon_plan_set_profiling")
+
+    def timings(self) -> dict:
+        """Milliseconds of the most recent encode / projection / locator / recovery kernels (profiling on)."""
+        ms = np.zeros(4, dtype=np.float32)
+        _check(lib().solon_plan_get_timings(self._h, _dptr(ms, c_float)), "solon_plan_get_timings")
+        return {"encode": float(ms[0]), "project": float(ms[1]), "locate": float(ms[2]), "recover": float(ms[3])}
 
     def kernel_launches(self) -> int:
         return int(lib().solon_plan_kernel_launches(self._h))

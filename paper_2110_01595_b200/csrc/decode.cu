@@ -6,12 +6,23 @@ using namespace solon;
 
 extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask) {
   if (!plan || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
-  if (((uintptr_t)received & 3) || ((uintptr_t)agg_grad & 15)) return SOLON_ERR_INVALID_ARG;
+  if (((uintptr_t)received & 15) || ((uintptr_t)agg_grad & 15)) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), plan->stream));
   int rc;
+  const bool prof = plan->profiling != 0;
+  auto mark = [&](int i) -> int {
+    if (!prof) return SOLON_OK;
+    SOLON_CUDA_TRY(cudaEventRecord(plan->ev[i], plan->stream));
+    plan->ev_valid[i] = 1;
+    return SOLON_OK;
+  };
+  if ((rc = mark(2))) return rc;
   if (plan->s > 0 && (rc = launch_project(plan, received))) return rc;   // s = 0: nothing to locate
+  if ((rc = mark(3))) return rc;
   if ((rc = launch_locate(plan, byz_mask))) return rc;
-  return launch_recover(plan, received, agg_grad);
+  if ((rc = mark(4))) return rc;
+  if ((rc = launch_recover(plan, received, agg_grad))) return rc;
+  return mark(5);
 }
 
 template <typename T>

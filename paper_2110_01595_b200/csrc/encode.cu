@@ -456,5 +456,14 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
 extern "C" int solon_encode(solon_plan* plan, const float* partition_grads, float* coded) {
   if (!plan || !partition_grads || !coded) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)partition_grads & 15) || ((uintptr_t)coded & 3)) return SOLON_ERR_INVALID_ARG;
-  return solon::launch_encode(plan, partition_grads, coded);
+  if (plan->profiling) {
+    SOLON_CUDA_TRY(cudaEventRecord(plan->ev[0], plan->stream));
+    plan->ev_valid[0] = 1;
+  }
+  int rc = solon::launch_encode(plan, partition_grads, coded);
+  if (rc == SOLON_OK && plan->profiling) {
+    SOLON_CUDA_TRY(cudaEventRecord(plan->ev[1], plan->stream));
+    plan->ev_valid[1] = 1;
+  }
+  return rc;
 }

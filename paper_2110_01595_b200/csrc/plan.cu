@@ -115,6 +115,8 @@ static void free_device(solon_plan* p) {
   cudaFree(p->d_task_records); cudaFree(p->d_task_flags); cudaFree(p->d_group_ticket); cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status);
   cudaFree(p->d_resid);
+  for (int i = 0; i < 6; ++i)
+    if (p->ev[i]) cudaEventDestroy(p->ev[i]);
   cudaFree(p->d_stage_grads); cudaFree(p->d_stage_coded); cudaFree(p->d_stage_agg); cudaFree(p->d_stage_mask);
   (void)cudaGetLastError();
 }
@@ -373,6 +375,27 @@ int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows,
       memcpy(coeff + out * plan->m, cf.data() + (size_t)(base + j) * plan->m, plan->m * sizeof(double));
     }
   }
+  return SOLON_OK;
+}
+
+int solon_plan_set_profiling(solon_plan* plan, int on) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  if (on && !plan->ev[0]) {
+    for (int i = 0; i < 6; ++i) SOLON_CUDA_TRY(cudaEventCreate(&plan->ev[i]));
+  }
+  plan->profiling = on ? 1 : 0;
+  return SOLON_OK;
+}
+
+int solon_plan_get_timings(solon_plan* plan, float* ms) {
+  if (!plan || !ms) return SOLON_ERR_INVALID_ARG;
+  for (int i = 0; i < 4; ++i) ms[i] = 0.f;
+  if (!plan->ev[0]) return SOLON_OK;
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  if (plan->ev_valid[0] && plan->ev_valid[1]) SOLON_CUDA_TRY(cudaEventElapsedTime(&ms[0], plan->ev[0], plan->ev[1]));
+  for (int i = 0; i < 3; ++i)
+    if (plan->ev_valid[2 + i] && plan->ev_valid[3 + i])
+      SOLON_CUDA_TRY(cudaEventElapsedTime(&ms[1 + i], plan->ev[2 + i], plan->ev[3 + i]));
   return SOLON_OK;
 }
 

@@ -1,18 +1,17 @@
 // Recovery kernel: the block decoder psi of Section 3.4 applied to every chunk, fused with the final sum
 // of Algorithm 1:  agg[p m + l] = sum_g sum_{j in rows_g} coeff_g[j][l] * R[rows_g[j]][p],  truncated to d.
 //
-// One pass over the trusted rows the locator selected (m per group when m <= 6, else all trusted rows).
-// Each thread owns a few chunks, loads one float per row and chunk (coalesced along the chunk axis),
-// accumulates the m outputs of each chunk in registers (float32 for m <= 6, where the weights are small;
-// float64 above, where they reach 10^3 and cancel), and every warp writes its run of chunks
-// back through its own shared-memory buffer as contiguous 128-bit stores.  The rows and weights come from device memory written by
-// the locator kernel, so no host round trip separates the two.
+// One pass over the trusted rows the locator selected (m per group when m <= 6, else all trusted rows),
+// streamed through shared memory with bulk asynchronous copies (see recover_kernel).  The m outputs of
+// each chunk are accumulated in registers: float32 for m <= 6, where the weights are small; float64
+// above, where they reach 10^3 and cancel.  The rows and weights come from device memory written by the
+// locator kernel, so no host round trip separates the two.
 #include "solon_internal.h"
+#include "stream_pipe.cuh"
 
 namespace solon {
 
 constexpr int kRecThreads = 256;
-constexpr int kRowBlock = 5;   // rows whose loads are in flight together
 
 struct RecoverParams {
   const float* R;
@@ -36,25 +35,113 @@ __device__ __forceinline__ void load_tables(const RecoverParams& prm, Acc* coeff
   __syncthreads();
 }
 
-template <int M, int CPT, typename Acc>
-__global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  constexpr int kWarpChunks = 32 * CPT;                      // chunks one warp handles per step
-  constexpr int kWarps = kRecThreads / 32;
-  float* out_all = reinterpret_cast<float*>(smem_raw);       // per warp: kWarpChunks x M
-  Acc* coeff_s = reinterpret_cast<Acc*>(smem_raw + (size_t)kWarps * kWarpChunks * M * sizeof(float));
-  int* rows_s = reinterpret_cast<int*>(smem_raw + (size_t)kWarps * kWarpChunks * M * sizeof(float) +
-                                       (size_t)prm.P * M * sizeof(double));
-  int* start_s = rows_s + prm.P;
-  int* n_rec_s = start_s + prm.q + 1;
-  load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float* out_s = out_all + (size_t)warp * kWarpChunks * M;
+// Packed list of the rows the recovery reads (all groups, in group order) and their weights.
+template <typename Acc>
+__device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_p, Acc* coeff_p, int* count_s) {
+  // positions by a serial prefix over the groups (q is small), then a parallel copy
+  if (threadIdx.x == 0) {
+    int total = 0;
+    for (int g = 0; g < prm.q; ++g) total += prm.n_rec[g];
+    *count_s = total;
+  }
+  for (int g = 0, base = 0; g < prm.q; ++g) {
+    const int n = prm.n_rec[g], src = prm.group_start[g];
+    for (int j = threadIdx.x; j < n; j += blockDim.x) rows_p[base + j] = prm.rec_rows[src + j];
+    for (int i = threadIdx.x; i < n * prm.m; i += blockDim.x) coeff_p[(size_t)base * prm.m + i] = (Acc)prm.coeff[(size_t)src * prm.m + i];
+    base += n;
+  }
+  __syncthreads();
+  return *count_s;
+}
 
-  // Warps run independently of each other (no CTA barrier below): while one waits for its loads another
-  // does arithmetic or stores.
-  const int64_t stride = (int64_t)gridDim.x * kWarps * kWarpChunks;
-  for (int64_t c0 = ((int64_t)blockIdx.x * kWarps + warp) * kWarpChunks; c0 < prm.d_c; c0 += stride) {
+// Bytes reserved for the P x M weight table in shared memory, rounded up to 16.
+__host__ __device__ inline size_t recover_coeff_bytes(int P, int M) { return ((size_t)P * M * sizeof(double) + 15) & ~(size_t)15; }
+
+constexpr int kRecConsumers = 256;
+constexpr int kRecPipeThreads = kRecConsumers + 32;   // + one producer warp
+
+struct RecoverPipe {
+  int row_batch;     // rows per stage
+  int stages;
+  int slot_floats;   // shared-memory floats per row slot (multiple of 4)
+  int* status;
+};
+
+// Streaming kernel: a producer warp moves the selected rows, tile by tile and a few rows at a time, into a
+// shared-memory ring with bulk asynchronous copies; consumer threads own CPT chunks each, take one float per
+// row from the ring, apply the row's m weights, and every consumer warp writes its runs of chunks back
+// through its own shared buffer as contiguous 128-bit stores.
+template <int M, int CPT, typename Acc>
+__global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams prm, RecoverPipe pp) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  constexpr int kTileChunks = kRecConsumers * CPT;
+  const int tid = threadIdx.x;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
+  uint64_t* empty_bar = full_bar + pp.stages;
+  int* abort_flag = reinterpret_cast<int*>(empty_bar + pp.stages);
+  int* count_s = abort_flag + 1;
+  // every region starts on a 16-byte boundary (128-bit shared loads, bulk-copy destinations)
+  Acc* coeff_p = reinterpret_cast<Acc*>(smem_raw + 256);                                  // P x M
+  int* rows_p = reinterpret_cast<int*>(smem_raw + 256 + recover_coeff_bytes(prm.P, M));   // P
+  float* out_all = reinterpret_cast<float*>(rows_p + ((prm.P + 3) & ~3));                 // 8 warps x 32 x M
+  float* ring = out_all + (size_t)(kRecConsumers / 32) * 32 * M;                          // 32 M floats: 128 M bytes
+  const size_t stage_floats = (size_t)pp.row_batch * pp.slot_floats;
+
+  if (tid == 0) {
+    for (int s = 0; s < pp.stages; ++s) {
+      pipe::mbar_init(&full_bar[s], 32);
+      pipe::mbar_init(&empty_bar[s], kRecConsumers / 32);
+    }
+    *abort_flag = 0;
+    pipe::fence_barrier_init();
+  }
+  const int n_rows = pack_tables(prm, rows_p, coeff_p, count_s);
+  const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
+  const int64_t total_floats = (int64_t)prm.P * prm.d_c;
+
+  if (tid >= kRecConsumers) {
+    const int lane = tid - kRecConsumers;
+    uint32_t it = 0;
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      const int64_t c0 = tile * kTileChunks;
+      int64_t c1 = c0 + kTileChunks;
+      if (c1 > prm.d_c) c1 = prm.d_c;
+      for (int b0 = 0; b0 < n_rows; b0 += pp.row_batch, ++it) {
+        const int stage = it % pp.stages;
+        const uint32_t phase = (it / pp.stages) & 1;
+        if (it >= (uint32_t)pp.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
+        const int nb = min(pp.row_batch, n_rows - b0);
+        if (lane < nb) {
+          const int64_t first = (int64_t)rows_p[b0 + lane] * prm.d_c + c0;
+          const int64_t last = first + (c1 - c0);
+          const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
+          int64_t a1 = (last + 3) & ~(int64_t)3;
+          const int64_t safe_end = total_floats & ~(int64_t)3;      // bulk copies stay inside the matrix
+          if (a1 > safe_end) a1 = safe_end;
+          float* slot = ring + stage * stage_floats + (size_t)lane * pp.slot_floats;
+          const uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
+          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.R[e];   // <= 3 floats
+          if (bytes) {
+            pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
+            pipe::bulk_load(slot, prm.R + a0, bytes, &full_bar[stage]);
+          } else {
+            pipe::mbar_arrive(&full_bar[stage]);
+          }
+        } else {
+          pipe::mbar_arrive(&full_bar[stage]);
+        }
+      }
+    }
+    if (*(volatile int*)abort_flag) pipe::drain_delay();
+    return;
+  }
+
+  const int lane = tid & 31, warp = tid >> 5;
+  float* out_s = out_all + (size_t)warp * 32 * M;
+  const int dc_mod4 = (int)(prm.d_c & 3);
+  uint32_t it = 0;
+  for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const int64_t c0 = tile * kTileChunks;
     Acc acc[CPT][M];
 #pragma unroll
     for (int i = 0; i < CPT; ++i)
@@ -62,53 +149,49 @@ __global__ void __launch_bounds__(kRecThreads) recover_kernel(RecoverParams prm)
       for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
     bool ok[CPT];
 #pragma unroll
-    for (int i = 0; i < CPT; ++i) ok[i] = c0 + lane + i * 32 < prm.d_c;
+    for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kRecConsumers < prm.d_c;
 
-    for (int g = 0; g < prm.q; ++g) {
-      const int base = start_s[g], n = n_rec_s[g];
-      // rows in blocks of kRowBlock: all loads of a block are issued before its arithmetic
-      for (int j0 = 0; j0 < n; j0 += kRowBlock) {
-        float v[kRowBlock][CPT];
+    for (int b0 = 0; b0 < n_rows; b0 += pp.row_batch, ++it) {
+      const int stage = it % pp.stages;
+      const uint32_t phase = (it / pp.stages) & 1;
+      pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
+      const int nb = min(pp.row_batch, n_rows - b0);
+      const float* slot = ring + stage * stage_floats + tid;
+      for (int j = 0; j < nb; ++j) {
+        const int shift = ((((rows_p[b0 + j] & 3) * dc_mod4) + (int)(c0 & 3)) & 3);   // (row * d_c + c0) mod 4
+        const float* src = slot + shift;
+        Acc v[CPT];
 #pragma unroll
-        for (int jj = 0; jj < kRowBlock; ++jj) {
-          const int j = j0 + jj < n ? j0 + jj : n - 1;
-          const float* row = prm.R + (int64_t)rows_s[base + j] * prm.d_c + c0 + lane;
+        for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (Acc)src[i * kRecConsumers] : (Acc)0;
+        const Acc* cj = coeff_p + (size_t)(b0 + j) * M;
 #pragma unroll
-          for (int i = 0; i < CPT; ++i) v[jj][i] = ok[i] ? __ldcs(row + i * 32) : 0.f;
+        for (int l = 0; l < M; ++l) {
+          const Acc c = cj[l];
+#pragma unroll
+          for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
         }
-#pragma unroll
-        for (int jj = 0; jj < kRowBlock; ++jj) {
-          if (j0 + jj < n) {
-            const Acc* cj = coeff_s + (size_t)(base + j0 + jj) * M;
-            Acc dv[CPT];
-#pragma unroll
-            for (int i = 0; i < CPT; ++i) dv[i] = (Acc)v[jj][i];
-#pragma unroll
-            for (int l = 0; l < M; ++l) {
-              const Acc c = cj[l];
-#pragma unroll
-              for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, dv[i], acc[i][l]);
-            }
-          }
-        }
+        slot += pp.slot_floats;
       }
+      __syncwarp();
+      if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
     }
+    // write-back: for each i the warp's 32 chunks are contiguous, 32 M floats starting on a 16-byte boundary
 #pragma unroll
-    for (int i = 0; i < CPT; ++i)
+    for (int i = 0; i < CPT; ++i) {
 #pragma unroll
-      for (int l = 0; l < M; ++l) out_s[(size_t)(lane + i * 32) * M + l] = (float)acc[i][l];
-    __syncwarp();
-    // contiguous write-back: floats [c0 M, min((c0 + kWarpChunks) M, d)); c0 M is a multiple of 4
-    const int64_t o0 = c0 * M;
-    int64_t o1 = o0 + (int64_t)kWarpChunks * M;
-    if (o1 > prm.d) o1 = prm.d;
-    const int count = (int)(o1 - o0);
-    const int vec = count / 4;
-    float4* dst4 = reinterpret_cast<float4*>(prm.agg + o0);
-    const float4* src4 = reinterpret_cast<const float4*>(out_s);
-    for (int i = lane; i < vec; i += 32) dst4[i] = src4[i];
-    for (int i = vec * 4 + lane; i < count; i += 32) prm.agg[o0 + i] = out_s[i];
-    __syncwarp();
+      for (int l = 0; l < M; ++l) out_s[lane * M + l] = (float)acc[i][l];
+      __syncwarp();
+      const int64_t o0 = (c0 + (int64_t)i * kRecConsumers + warp * 32) * M;
+      int64_t o1 = o0 + 32 * M;
+      if (o1 > prm.d) o1 = prm.d;
+      const int count = o1 > o0 ? (int)(o1 - o0) : 0;
+      const int vec = count / 4;
+      float4* dst4 = reinterpret_cast<float4*>(prm.agg + o0);
+      const float4* src4 = reinterpret_cast<const float4*>(out_s);
+      for (int e = lane; e < vec; e += 32) dst4[e] = src4[e];
+      for (int e = vec * 4 + lane; e < count; e += 32) prm.agg[o0 + e] = out_s[e];
+      __syncwarp();
+    }
   }
 }
 
@@ -135,18 +218,41 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
 
 template <int M, int CPT, typename Acc>
 static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
-  size_t smem = (size_t)kRecThreads * CPT * M * sizeof(float) + (size_t)plan->P * M * sizeof(double) +
-                (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
-  if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
-  SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_kernel<M, CPT, Acc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  static_assert((32 * CPT) % 4 == 0, "warp tiles must start on a 16-byte boundary of the output");
-  int64_t tiles = (plan->d_c + (int64_t)kRecThreads * CPT - 1) / ((int64_t)kRecThreads * CPT);
+  constexpr int kTileChunks = kRecConsumers * CPT;
+  RecoverPipe pp;
+  pp.status = plan->d_status;
+  pp.slot_floats = kTileChunks + 8;
+  const size_t slot_bytes = (size_t)pp.slot_floats * 4;
+  const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + (size_t)((plan->P + 3) & ~3) * sizeof(int) +
+                       (size_t)(kRecConsumers / 32) * 32 * M * sizeof(float);
+  // the locator may select up to all P rows (large m) or as few as q m; batches of about 20 KB
+  int row_batch = (int)((size_t)20 * 1024 / slot_bytes);
+  if (row_batch < 1) row_batch = 1;
+  if (row_batch > 32) row_batch = 32;
+  const int max_rows = M <= 6 ? plan->q * M : plan->P;
+  if (row_batch > max_rows) row_batch = max_rows;
+  {
+    int nb = (max_rows + row_batch - 1) / row_batch;     // an even split of the expected row count
+    row_batch = (max_rows + nb - 1) / nb;
+  }
+  const size_t per_cta = (size_t)227 * 1024 / 2 - 1024;
+  int stages = 4;
+  while (stages > 2 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --stages;
+  while (row_batch > 1 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --row_batch;
+  const size_t smem = fixed + (size_t)stages * row_batch * slot_bytes;
+  if (smem > (size_t)226 * 1024) return SOLON_ERR_INVALID_ARG;
+  pp.row_batch = row_batch;
+  pp.stages = stages;
+  auto kernel = recover_kernel<M, CPT, Acc>;
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  static_assert((32 * M * 4) % 16 == 0, "warp runs must start on a 16-byte boundary of the output");
+  int64_t tiles = (plan->d_c + kTileChunks - 1) / kTileChunks;
   int per_sm = 1;
-  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recover_kernel<M, CPT, Acc>, kRecThreads, smem));
+  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kRecPipeThreads, smem));
   if (per_sm < 1) per_sm = 1;
   int64_t cap = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(tiles < cap ? tiles : cap);
-  recover_kernel<M, CPT, Acc><<<grid, kRecThreads, smem, plan->stream>>>(prm);
+  kernel<<<grid, kRecPipeThreads, smem, plan->stream>>>(prm, pp);
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }

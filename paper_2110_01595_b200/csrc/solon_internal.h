@@ -83,6 +83,11 @@ struct solon_plan {
   double* d_coeff;         // P x m
   int* d_status;           // [0] status bits of the last decode, [1] sticky bits (expired waits)
 
+  // optional per-kernel timing: events [0,1] around encode, [2..5] before/after the decode kernels
+  int profiling;
+  cudaEvent_t ev[6];
+  int ev_valid[6];
+
   // lsq workspace
   float* d_resid;          // P * lsq_rows
   int64_t resid_capacity;
