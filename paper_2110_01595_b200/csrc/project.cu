@@ -30,7 +30,7 @@ __device__ __forceinline__ double warp_sum(double v) {
 }
 
 template <int K>
-__global__ void __launch_bounds__(kProjThreads) project_kernel(const float* __restrict__ R, const float* __restrict__ f,
+__global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* __restrict__ R, const float* __restrict__ f,
                                                                int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
                                                                int tile_cols, double* __restrict__ partials,
                                                                double* __restrict__ rho_out, double* __restrict__ nu_out,
