@@ -1,9 +1,9 @@
 // Locator kernel (phi of Section 3.4) and recovery table (the inverse inside psi), on the device, plus
 // the host mirror solon_locate_host built from the same source (locate_core.cuh).
 //
-// Grid (s + 1, q): CTA (t, g) assumes exactly t corrupt nodes in group g.  All error
-// counts are tried concurrently; the last CTA of a group to finish (atomic ticket, nobody waits) picks
-// the smallest accepted count, writes the group's part of the mask and builds the recovery table.
+// One CTA per group; warp t of it assumes exactly t corrupt nodes, so all error counts are tried
+// concurrently.  The CTA then picks the smallest accepted count, writes the group's part of the mask and
+// builds the recovery table.
 #include <vector>
 
 #include "locate_core.cuh"
@@ -17,18 +17,16 @@ struct LocateParams {
   const double* rho;     // K x P
   const double* nu;      // P
   const double* qb;      // per group n_g x n_g orthonormal polynomial tables, group g at qb_off[g]
+  const double* hm;      // per group n_g x n_g projector tables, same offsets
   const int64_t* qb_off; // q
   const double* mt;      // q x m x m
   const double* tch;     // P x (s + 1)
   int P, m, s, K;
   double tau;
-  TaskRecord* records;   // q x (s + 1)
-  uint8_t* task_flags;   // (s + 1) x P
-  unsigned int* group_ticket;   // q
-  double* ws_global;     // q x (s + 1) x ws_stride, used when shared memory is too small
+  double* ws_global;     // q x ws_stride doubles, used when shared memory is too small
   size_t ws_stride;
   int use_smem;
-  int stage_tables;      // copy the group's tables to shared memory (after ws_stride doubles of workspace)
+  int stage_tables;      // copy the group's tables to shared memory (they follow the workspace)
   uint8_t* mask;         // P (caller's buffer)
   int* t_acc;            // q
   int* n_rec;            // q
@@ -37,57 +35,70 @@ struct LocateParams {
   int* status;
 };
 
-// Workspace carving shared by the device kernel and the host mirror.
+// Workspace of one group, shared by the device kernel and the host mirror.
 struct GroupScratch {
-  int* rows_l;       // n      recovery rows (local copy, written out at the end)
-  uint8_t* cand;     // n
-  uint8_t* bad;      // n
-  uint8_t* trusted;  // n
-  uint8_t* mask_l;   // n
-  uint8_t* forced;   // n
-  double* rho_in;    // K x n  staged inputs: every later read hits shared memory, not L2
-  double* nu_in;     // n
-  double* rho_n;     // K x n
-  double* scratch;   // K + 2
-  double* task_ws;   // rest
+  int* rows_l;           // n      recovery rows (local copy, written out at the end)
+  uint8_t* trusted;      // n
+  uint8_t* mask_l;       // n
+  uint8_t* forced;       // n
+  uint8_t* flags;        // (s + 1) x n   located nodes per error count
+  TaskRecord* recs;      // s + 1
+  double* rho_in;        // K x n  staged inputs
+  double* nu_in;         // n
+  double* rho_n;         // K x n
+  double* scratch;       // K + 2
+  double* coeff_l;       // n x m
+  double* tasks;         // (s + 1) x task_stride, reused by the epilogue
+  size_t task_stride;
 };
 
-SOLON_HD static inline size_t group_scratch_doubles(int n, int K) {
-  // ints and bytes are carved out of double-sized cells to keep everything 8-byte aligned
-  return ((size_t)(n + 1) / 2 + 1) + 5 * ((size_t)n / 8 + 1) + (size_t)(2 * K + 1) * n + K + 2;
+// cand / bad bytes followed by the task's doubles
+SOLON_HD static inline size_t task_stride_doubles(int n, int m, int K, int s) {
+  return 2 * ((size_t)n / 8 + 1) + locate_task_ws_doubles(n, m, K, s);
 }
 
-SOLON_HD static inline GroupScratch carve(double* ws, int n, int K) {
+SOLON_HD static inline size_t group_ws_doubles(int n, int m, int K, int s) {
+  size_t tasks = (size_t)(s + 1) * task_stride_doubles(n, m, K, s);
+  size_t epi = locate_epilogue_ws_doubles(n, m, s);
+  return ((size_t)(n + 1) / 2 + 1) + 3 * ((size_t)n / 8 + 1) + ((size_t)(s + 1) * n / 8 + 1) + 2 * (size_t)(s + 1) +
+         (size_t)(2 * K + 1) * n + K + 2 + (size_t)n * m + (tasks > epi ? tasks : epi) + 8;
+}
+
+SOLON_HD static inline GroupScratch carve(double* ws, int n, int m, int K, int s) {
   GroupScratch sc;
   double* p = ws;
   sc.rows_l = reinterpret_cast<int*>(p);         p += (n + 1) / 2 + 1;
-  sc.cand = reinterpret_cast<uint8_t*>(p);       p += n / 8 + 1;
-  sc.bad = reinterpret_cast<uint8_t*>(p);        p += n / 8 + 1;
   sc.trusted = reinterpret_cast<uint8_t*>(p);    p += n / 8 + 1;
   sc.mask_l = reinterpret_cast<uint8_t*>(p);     p += n / 8 + 1;
   sc.forced = reinterpret_cast<uint8_t*>(p);     p += n / 8 + 1;
+  sc.flags = reinterpret_cast<uint8_t*>(p);      p += (size_t)(s + 1) * n / 8 + 1;
+  sc.recs = reinterpret_cast<TaskRecord*>(p);    p += 2 * (size_t)(s + 1);
   sc.rho_in = p;                                 p += (size_t)K * n;
   sc.nu_in = p;                                  p += n;
   sc.rho_n = p;                                  p += (size_t)K * n;
   sc.scratch = p;                                p += K + 2;
-  sc.task_ws = p;
+  sc.coeff_l = p;                                p += (size_t)n * m;
+  sc.tasks = p;
+  sc.task_stride = task_stride_doubles(n, m, K, s);
   return sc;
 }
 
-constexpr int kLocThreads = 256;
-
-__global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
+// One CTA per group, one warp per error count: warp t assumes exactly t corrupt nodes, all counts are tried
+// at the same time with warp-level synchronisation only; afterwards the whole CTA picks the smallest
+// accepted count, writes the group's part of the mask and builds the recovery table.  No CTA waits on
+// another one.
+__global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocateParams prm) {
   extern __shared__ __align__(16) double smem_ws[];
-  const int t = blockIdx.x, g = blockIdx.y;
-  const int tid = threadIdx.x;
+  const int g = blockIdx.x;
+  const int tid = threadIdx.x, n_threads = blockDim.x;
   const int row0 = prm.group_start[g];
   const int n = prm.group_start[g + 1] - row0;
-  double* ws = prm.use_smem ? smem_ws : prm.ws_global + ((size_t)g * (prm.s + 1) + t) * prm.ws_stride;
-  GroupScratch sc = carve(ws, n, prm.K);
-  __shared__ unsigned int s_ticket;
+  double* ws = prm.use_smem ? smem_ws : prm.ws_global + (size_t)g * prm.ws_stride;
+  GroupScratch sc = carve(ws, n, prm.m, prm.K, prm.s);
   __shared__ int s_n_rec, s_t_acc;
   GroupTables tb;
   tb.Qb = prm.qb + prm.qb_off[g];
+  tb.Hm = prm.hm + prm.qb_off[g];
   tb.Mt = prm.mt + (size_t)g * prm.m * prm.m;
   tb.Tch = prm.tch + (size_t)row0 * (prm.s + 1);
   tb.w = prm.w + row0;
@@ -95,89 +106,69 @@ __global__ void __launch_bounds__(kLocThreads) locate_kernel(LocateParams prm) {
     // small groups: one coalesced pass brings the plan's tables on chip, so the dependent reads of the
     // solver never wait on L2 or HBM (the tables are evicted by the streaming kernels between decodes)
     double* qb_s = smem_ws + prm.ws_stride;
-    double* tch_s = qb_s + (size_t)n * n;
+    double* hm_s = qb_s + (size_t)n * n;
+    double* tch_s = hm_s + (size_t)n * n;
     double* w_s = tch_s + (size_t)n * (prm.s + 1);
-    for (int i = tid; i < n * n; i += kLocThreads) qb_s[i] = tb.Qb[i];
-    for (int i = tid; i < n * (prm.s + 1); i += kLocThreads) tch_s[i] = tb.Tch[i];
-    for (int i = tid; i < n; i += kLocThreads) w_s[i] = tb.w[i];
+    for (int i = tid; i < n * n; i += n_threads) {
+      qb_s[i] = tb.Qb[i];
+      hm_s[i] = tb.Hm[i];
+    }
+    for (int i = tid; i < n * (prm.s + 1); i += n_threads) tch_s[i] = tb.Tch[i];
+    for (int i = tid; i < n; i += n_threads) w_s[i] = tb.w[i];
     tb.Qb = qb_s;
+    tb.Hm = hm_s;
     tb.Tch = tch_s;
     tb.w = w_s;
   }
-
-  TaskRecord* recs = prm.records + (size_t)g * (prm.s + 1);
-  uint8_t* flags = prm.task_flags + (size_t)t * prm.P + row0;
+  const Team cta = Team::cta();
   if (prm.s == 0) {
     // pure compression code: nothing to locate, every node is trusted
-    for (int k = tid; k < n; k += kLocThreads) {
+    for (int k = tid; k < n; k += n_threads) {
       sc.forced[k] = 0;
-      flags[k] = 0;
+      sc.flags[k] = 0;
     }
     if (tid == 0) {
-      recs[0].accept = 1;
-      recs[0].n_flagged = 0;
-      recs[0].max_fit = 0.0;
+      sc.recs[0].accept = 1;
+      sc.recs[0].n_flagged = 0;
+      sc.recs[0].max_fit = 0.0;
     }
-    __syncthreads();
   } else {
     // one parallel round trip brings the group's projected values on chip
-    for (int i = tid; i < n; i += kLocThreads) {
+    for (int i = tid; i < n; i += n_threads) {
       sc.nu_in[i] = prm.nu[row0 + i];
       for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
     }
     __syncthreads();
     double tau_eff = 0.0;
-    locate_prepare(n, prm.K, sc.rho_in, sc.nu_in, prm.tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
-    locate_task(tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, flags, sc.cand, sc.bad, sc.task_ws, &recs[t]);
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_ticket = atomicAdd(&prm.group_ticket[g], 1u);
-  __syncthreads();
-  if (s_ticket != (unsigned int)prm.s) return;
-  __threadfence();
-  // Group epilogue.  Records and flags written by the other CTAs are read through L2.
-  TaskRecord* recs_l = reinterpret_cast<TaskRecord*>(sc.task_ws);                  // s + 1 records
-  uint8_t* flags_l = reinterpret_cast<uint8_t*>(recs_l + (prm.s + 1));             // (s + 1) x n
-  double* ep_ws = sc.task_ws + ((size_t)(prm.s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1;
-  for (int i = tid; i <= prm.s; i += kLocThreads) {
-    recs_l[i].accept = __ldcg(&recs[i].accept);
-    recs_l[i].n_flagged = __ldcg(&recs[i].n_flagged);
-    recs_l[i].max_fit = __ldcg(&recs[i].max_fit);
-  }
-  for (int i = tid; i < (prm.s + 1) * n; i += kLocThreads) {
-    int tt = i / n, k = i - tt * n;
-    flags_l[i] = __ldcg(prm.task_flags + (size_t)tt * prm.P + row0 + k);
+    locate_prepare(cta, n, prm.K, sc.rho_in, sc.nu_in, prm.tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
+    const int t = tid >> 5;                       // this warp's error count
+    double* task = sc.tasks + (size_t)t * sc.task_stride;
+    uint8_t* cand = reinterpret_cast<uint8_t*>(task);
+    uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
+    locate_task(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n,
+                cand, bad, task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
   }
   __syncthreads();
-  double* coeff_l = ep_ws;                                  // n x m, local copy of the weights
-  double* ep_rest = ep_ws + (size_t)n * prm.m;
-  const int ok = locate_epilogue(tb, n, prm.m, prm.s, sc.forced, recs_l, flags_l, n, sc.mask_l, &s_t_acc, sc.rows_l,
-                                 &s_n_rec, coeff_l, sc.trusted, ep_rest);
+  const int ok = locate_epilogue(cta, tb, n, prm.m, prm.s, sc.forced, sc.recs, sc.flags, n, sc.mask_l, &s_t_acc, sc.rows_l,
+                                 &s_n_rec, sc.coeff_l, sc.trusted, sc.tasks);
   // write the group's results: mask, recovery rows as global node indices, weights
   const int n_rec = s_n_rec;
-  for (int k = tid; k < n; k += kLocThreads) prm.mask[row0 + k] = sc.mask_l[k];
-  for (int j = tid; j < n_rec; j += kLocThreads) prm.rec_rows[row0 + j] = sc.rows_l[j] + row0;
-  for (int i = tid; i < n_rec * prm.m; i += kLocThreads) prm.coeff[(size_t)row0 * prm.m + i] = coeff_l[i];
+  for (int k = tid; k < n; k += n_threads) prm.mask[row0 + k] = sc.mask_l[k];
+  for (int j = tid; j < n_rec; j += n_threads) prm.rec_rows[row0 + j] = sc.rows_l[j] + row0;
+  for (int i = tid; i < n_rec * prm.m; i += n_threads) prm.coeff[(size_t)row0 * prm.m + i] = sc.coeff_l[i];
   if (tid == 0) {
     prm.n_rec[g] = n_rec;
     prm.t_acc[g] = s_t_acc;
     if (!ok) atomicOr(prm.status, kStatusUndecodable);
-    prm.group_ticket[g] = 0u;   // ready for the next decode
   }
 }
 
-size_t locate_ws_doubles(int n, int m, int K, int s) {
-  size_t task = locate_task_ws_doubles(n, m, K, s);
-  size_t epi = ((size_t)(s + 1) * (sizeof(TaskRecord) + (size_t)n) + 7) / 8 + 1 + (size_t)n * m +
-               locate_epilogue_ws_doubles(n, m, s);
-  return group_scratch_doubles(n, K) + (task > epi ? task : epi) + 8;
-}
+size_t locate_ws_doubles(int n, int m, int K, int s) { return group_ws_doubles(n, m, K, s); }
 
 // Tables of one group (host, once per plan): the orthonormal polynomials q_0..q_{n-1} on the nodes
 // (Gram-Schmidt, twice, of the Chebyshev polynomials T_0..T_{n-1} evaluated at the nodes), the monomial
 // coefficients of q_0..q_{m-1}, and T_0..T_s at the nodes.
-void build_group_tables(int n, int m, int s, const double* w, double* Qb, double* Mt, double* Tch) {
+void build_group_tables(int n, int m, int s, const double* w, double* Qb, double* Hm, double* Mt, double* Tch) {
   typedef long double real;
   std::vector<real> T((size_t)n * n), Q((size_t)n * n), R((size_t)n * n, 0.0L);   // column-major n x n
   for (int k = 0; k < n; ++k) {
@@ -206,6 +197,12 @@ void build_group_tables(int n, int m, int s, const double* w, double* Qb, double
     for (int k = 0; k < n; ++k) Q[(size_t)j * n + k] = nrm > 0.0L ? Q[(size_t)j * n + k] / nrm : 0.0L;
   }
   for (size_t i = 0; i < (size_t)n * n; ++i) Qb[i] = (double)Q[i];
+  for (int a = 0; a < n; ++a)
+    for (int b = 0; b < n; ++b) {
+      real h = 0.0L;
+      for (int i = 0; i < m && i < n; ++i) h += Q[(size_t)i * n + a] * Q[(size_t)i * n + b];
+      Hm[(size_t)a * n + b] = (double)h;
+    }
   // q_i = sum_{j<=i} Rinv[j][i] T_j (T = Q R); T_j = sum_l C[l][j] w^l with integer C from the recurrence
   std::vector<real> Rinv((size_t)m * m, 0.0L), C((size_t)m * m, 0.0L);
   for (int i = 0; i < m; ++i) {
@@ -240,14 +237,12 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
   prm.rho = plan->d_rho;
   prm.nu = plan->d_nu;
   prm.qb = plan->d_qb;
+  prm.hm = plan->d_hm;
   prm.qb_off = plan->d_qb_off;
   prm.mt = plan->d_mt;
   prm.tch = plan->d_tch;
   prm.P = plan->P; prm.m = plan->m; prm.s = plan->s; prm.K = plan->K;
   prm.tau = plan->tau;
-  prm.records = reinterpret_cast<TaskRecord*>(plan->d_task_records);
-  prm.task_flags = plan->d_task_flags;
-  prm.group_ticket = plan->d_group_ticket;
   prm.ws_global = plan->d_locate_ws;
   prm.ws_stride = plan->locate_ws_stride;
   prm.mask = byz_mask;
@@ -258,18 +253,17 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
   prm.status = plan->d_status;
   size_t need = locate_ws_doubles(plan->max_group, plan->m, plan->K, plan->s) * sizeof(double);
   if (need > plan->locate_ws_stride * sizeof(double)) return SOLON_ERR_INTERNAL;
-  prm.use_smem = need <= 96 * 1024 ? 1 : 0;
+  prm.use_smem = need <= 128 * 1024 ? 1 : 0;
   size_t smem = prm.use_smem ? need : 0;
-  const size_t tables = ((size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
-  prm.stage_tables = (prm.use_smem && smem + tables <= 160 * 1024) ? 1 : 0;
+  const size_t tables = (2 * (size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
+  prm.stage_tables = (prm.use_smem && smem + tables <= 200 * 1024) ? 1 : 0;
   if (prm.stage_tables) {
     prm.ws_stride = need / sizeof(double);      // the tables follow the workspace in shared memory
     smem += tables;
   }
-  if (prm.use_smem && smem > 48 * 1024)
+  if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  dim3 grid(plan->s + 1, plan->q);
-  locate_kernel<<<grid, kLocThreads, smem, plan->stream>>>(prm);
+  locate_kernel<<<plan->q, 32 * (plan->s + 1), smem, plan->stream>>>(prm);
   plan->launches += 1;
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
@@ -285,31 +279,34 @@ extern "C" int solon_locate_host(int n, int m, int s, int K, const double* rho, 
   if (n < 1 || n > SOLON_MAX_GROUP || m < 1 || m > SOLON_MAX_M || s < 0 || s > SOLON_MAX_S || K < 1 ||
       K > SOLON_MAX_PROJECTIONS || n < 2 * s + m)
     return SOLON_ERR_INVALID_ARG;
-  std::vector<double> Qb((size_t)n * n), Mt((size_t)m * m), Tch((size_t)n * (s + 1));
-  build_group_tables(n, m, s, w_g, Qb.data(), Mt.data(), Tch.data());
+  std::vector<double> Qb((size_t)n * n), Hm((size_t)n * n), Mt((size_t)m * m), Tch((size_t)n * (s + 1));
+  build_group_tables(n, m, s, w_g, Qb.data(), Hm.data(), Mt.data(), Tch.data());
   GroupTables tb;
   tb.Qb = Qb.data();
+  tb.Hm = Hm.data();
   tb.Mt = Mt.data();
   tb.Tch = Tch.data();
   tb.w = w_g;
-  std::vector<double> ws(group_scratch_doubles(n, K) + locate_task_ws_doubles(n, m, K, s) +
-                         locate_epilogue_ws_doubles(n, m, s) + 64);
-  GroupScratch sc = carve(ws.data(), n, K);
-  std::vector<TaskRecord> recs(s + 1);
-  std::vector<uint8_t> flags((size_t)(s + 1) * n, 0);
+  std::vector<double> ws(group_ws_doubles(n, m, K, s) + 64);
+  GroupScratch sc = carve(ws.data(), n, m, K, s);
+  const Team tm = Team::serial();
   double tau_eff = 0.0;
   if (s > 0) {
-    locate_prepare(n, K, rho, nu, tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
-    for (int t = 0; t <= s; ++t)
-      locate_task(tb, n, m, K, t, s, sc.rho_n, sc.forced, tau_eff, flags.data() + (size_t)t * n, sc.cand, sc.bad,
-                  sc.task_ws, &recs[t]);
+    locate_prepare(tm, n, K, rho, nu, tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
+    for (int t = 0; t <= s; ++t) {
+      double* task = sc.tasks + (size_t)t * sc.task_stride;
+      uint8_t* cand = reinterpret_cast<uint8_t*>(task);
+      uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
+      locate_task(tm, tb, n, m, K, t, s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n, cand, bad,
+                  task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
+    }
   } else {
-    for (int k = 0; k < n; ++k) sc.forced[k] = 0;
-    recs[0].accept = 1;
-    recs[0].n_flagged = 0;
-    recs[0].max_fit = 0.0;
+    for (int k = 0; k < n; ++k) sc.forced[k] = sc.flags[k] = 0;
+    sc.recs[0].accept = 1;
+    sc.recs[0].n_flagged = 0;
+    sc.recs[0].max_fit = 0.0;
   }
-  const int ok = locate_epilogue(tb, n, m, s, sc.forced, recs.data(), flags.data(), n, mask, t_out, rec_rows, n_rec,
-                                 coeff, sc.trusted, sc.task_ws);
+  const int ok = locate_epilogue(tm, tb, n, m, s, sc.forced, sc.recs, sc.flags, n, mask, t_out, rec_rows, n_rec, coeff,
+                                 sc.trusted, sc.tasks);
   return ok ? SOLON_OK : SOLON_ERR_UNDECODABLE;
 }

@@ -26,32 +26,41 @@
 #include <math.h>
 #include <stdint.h>
 
-#if defined(__CUDA_ARCH__)
-#define SOLON_TID ((int)threadIdx.x)
-#define SOLON_NTHREADS ((int)blockDim.x)
-#define SOLON_LANE ((int)(threadIdx.x & 31))
-#define SOLON_NLANES 32
-#define SOLON_WARP ((int)(threadIdx.x >> 5))
-#define SOLON_NWARPS ((int)(blockDim.x >> 5))
-#define SOLON_SYNC() __syncthreads()
-#else
-#define SOLON_TID 0
-#define SOLON_NTHREADS 1
-#define SOLON_LANE 0
-#define SOLON_NLANES 1
-#define SOLON_WARP 0
-#define SOLON_NWARPS 1
-#define SOLON_SYNC() ((void)0)
-#endif
-#define SOLON_FOR_THREADS(i, n) for (int i = SOLON_TID; i < (n); i += SOLON_NTHREADS)
-#define SOLON_FOR_WARPS(i, n) for (int i = SOLON_WARP; i < (n); i += SOLON_NWARPS)
-#define SOLON_FOR_LANES(i, n) for (int i = SOLON_LANE; i < (n); i += SOLON_NLANES)
-
 #if defined(__CUDACC__)
 #define SOLON_HD __host__ __device__
 #else
 #define SOLON_HD
 #endif
+
+// The threads that execute a routine together: a whole CTA, one warp of it, or (host) a single thread.
+struct Team {
+  int tid, nthreads;   // index and count of the threads of the team
+  int lane, nlanes;    // lane inside the warp
+  int warp, nwarps;    // warp inside the team
+  SOLON_HD void sync() const {
+#if defined(__CUDA_ARCH__)
+    if (nwarps == 1) __syncwarp();
+    else __syncthreads();   // a team of several warps is always the whole CTA
+#endif
+  }
+#if defined(__CUDACC__)
+  static __device__ Team cta() {
+    return Team{(int)threadIdx.x, (int)blockDim.x, (int)(threadIdx.x & 31), 32, (int)(threadIdx.x >> 5), (int)(blockDim.x >> 5)};
+  }
+  static __device__ Team own_warp() { return Team{(int)(threadIdx.x & 31), 32, (int)(threadIdx.x & 31), 32, 0, 1}; }
+#endif
+  static Team serial() { return Team{0, 1, 0, 1, 0, 1}; }
+};
+#define SOLON_TID (tm.tid)
+#define SOLON_NTHREADS (tm.nthreads)
+#define SOLON_LANE (tm.lane)
+#define SOLON_NLANES (tm.nlanes)
+#define SOLON_WARP (tm.warp)
+#define SOLON_NWARPS (tm.nwarps)
+#define SOLON_SYNC() tm.sync()
+#define SOLON_FOR_THREADS(i, n) for (int i = SOLON_TID; i < (n); i += SOLON_NTHREADS)
+#define SOLON_FOR_WARPS(i, n) for (int i = SOLON_WARP; i < (n); i += SOLON_NWARPS)
+#define SOLON_FOR_LANES(i, n) for (int i = SOLON_LANE; i < (n); i += SOLON_NLANES)
 
 #define SOLON_SUBSET_MAX_M 6
 #define SOLON_THETA_MAX 16   /* largest error count per group (SOLON_MAX_S) */
@@ -71,6 +80,7 @@ SOLON_HD inline double lane_sum(double x) {
 // Tables of one group, fixed at plan time (functions of the node scalars only).
 struct GroupTables {
   const double* Qb;    // n x n, column-major: Qb[j * n + k] = q_j(w_k), orthonormal columns, deg q_j = j
+  const double* Hm;    // n x n, row-major: H = Q_m Q_m^T, the projector on the polynomials of degree < m
   const double* Mt;    // m x m, row-major: q_i(w) = sum_l Mt[l * m + i] w^l  (i < m)
   const double* Tch;   // n x (s + 1), row-major: Tch[k * (s + 1) + i] = T_i(w_k)
   const double* w;     // n node scalars
@@ -85,10 +95,11 @@ struct TaskRecord {
 
 // Doubles of workspace one task needs (group of n nodes, K projections, up to t errors).
 SOLON_HD inline size_t locate_task_ws_doubles(int n, int m, int K, int t) {
+  (void)m;
   size_t rows = (size_t)K * n;                              // upper bound of K (n - m - t)
-  size_t solve = rows * (t + 1) + (t + 1) + (size_t)t * (t + 1) + t + n;
-  size_t fit = (size_t)K * m + (size_t)K * n + 3 * (size_t)t * t + (size_t)K * t + n + (size_t)(t + n) / 2 + 4;
-  return solve + fit + 16;
+  size_t solve = rows * (t + 1) + (t + 1) + (size_t)t * (t + 1) + t;
+  size_t fit = (size_t)K * n + 3 * (size_t)t * t + (size_t)K * t + n;
+  return (size_t)n + (size_t)(t + n) / 2 + 1 + (solve > fit ? solve : fit) + 16;
 }
 
 // Doubles of workspace the epilogue needs.
@@ -98,7 +109,7 @@ SOLON_HD inline size_t locate_epilogue_ws_doubles(int n, int m, int s) {
 }
 
 // norm0[c] = squared norm of column c of the column-major matrix A (rows x ncols, column stride ldc).
-SOLON_HD inline void column_norms(const double* A, int rows, int ldc, int ncols, double* norm0) {
+SOLON_HD inline void column_norms(const Team& tm, const double* A, int rows, int ldc, int ncols, double* norm0) {
   SOLON_FOR_WARPS(c, ncols) {
     double acc = 0.0;
     SOLON_FOR_LANES(i, rows) acc = fma(A[(size_t)c * ldc + i], A[(size_t)c * ldc + i], acc);
@@ -112,7 +123,7 @@ SOLON_HD inline void column_norms(const double* A, int rows, int ldc, int ncols,
 // `ncols` columns (the trailing ones are right-hand sides).  Columns stay un-normalised.
 // R (row-major, leading dimension ldr) receives the triangular factor, right-hand sides included;
 // diag[j] = ||q_j|| (0 for a numerically dependent column).
-SOLON_HD inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols, const double* norm0, double* R,
+SOLON_HD inline void mgs_factor(const Team& tm, double* A, int rows, int ldc, int nq, int ncols, const double* norm0, double* R,
                                 int ldr, double* diag) {
   for (int j = 0; j < nq; ++j) {
     const double* qj = A + (size_t)j * ldc;
@@ -146,7 +157,7 @@ SOLON_HD inline void mgs_factor(double* A, int rows, int ldc, int nq, int ncols,
 // In-place inverse of the symmetric positive definite t x t matrix S (row-major) by Gauss-Jordan
 // elimination on [S | I] held in `aug` (t x 2t, row-major); one thread per column of the pair.
 // No pivoting is needed for a positive definite matrix.
-SOLON_HD inline void spd_inverse(double* S, int t, double* aug) {
+SOLON_HD inline void spd_inverse(const Team& tm, double* S, int t, double* aug) {
   const int w2 = 2 * t;
   SOLON_FOR_THREADS(idx, t * w2) {
     const int r = idx / w2, c = idx - r * w2;
@@ -177,55 +188,61 @@ SOLON_HD inline void spd_inverse(double* S, int t, double* aug) {
   SOLON_SYNC();
 }
 
-// S <- (I - H[V,V])^{-1} for the node list V (nv nodes), H = Q_m Q_m^T.
-SOLON_HD inline void deletion_inverse(const GroupTables& tb, int n, int m, const int* V, int nv, double* S, double* aug) {
+// S <- (I - H[V,V])^{-1} for the node list V (nv nodes), H = Q_m Q_m^T (tabulated).
+SOLON_HD inline void deletion_inverse(const Team& tm, const GroupTables& tb, int n, const int* V, int nv, double* S, double* aug) {
   SOLON_FOR_THREADS(idx, nv * nv) {
     const int a = idx / nv, b = idx - a * nv;
-    double h = 0.0;
-    for (int i = 0; i < m; ++i) h = fma(tb.Qb[(size_t)i * n + V[a]], tb.Qb[(size_t)i * n + V[b]], h);
-    S[idx] = (a == b ? 1.0 : 0.0) - h;
+    S[idx] = (a == b ? 1.0 : 0.0) - tb.Hm[(size_t)V[a] * n + V[b]];
   }
   SOLON_SYNC();
-  spd_inverse(S, nv, aug);
+  spd_inverse(tm, S, nv, aug);
 }
 
 // Verification: fit a degree-(m-1) polynomial to every projection on the non-candidates and test
-// all nodes.  cand[k] != 0 marks the n_cand candidates; forced[k] != 0 marks nodes that are corrupt by
-// inspection (they never fit).  bad[k] receives 1 where some projection is off by more than tau.
-SOLON_HD inline void locate_verify(const GroupTables& tb, int n, int m, int K, const double* rho_n, double tau,
-                                   const uint8_t* cand, int n_cand, const uint8_t* forced, uint8_t* bad, double* ws,
-                                   TaskRecord* rec) {
-  const int t = n_cand;
-  double* coef = ws;                         // K x m   c = Q_m^T rho
-  double* e = coef + (size_t)K * m;          // K x n   e = rho - Q_m c (fit over all nodes)
+// all nodes.  cand[k] != 0 marks the t candidates, vlist[0..t) lists them and vpos[k] is a candidate's
+// position in that list; forced[k] != 0 marks nodes that are corrupt by inspection (they never fit).
+// bad[k] receives 1 where some projection is off by more than tau.
+SOLON_HD inline void locate_verify(const Team& tm, const GroupTables& tb, int n, int K, const double* rho_n, double tau,
+                                   const uint8_t* cand, int t, const int* vlist, const int* vpos, const uint8_t* forced,
+                                   uint8_t* bad, double* ws, TaskRecord* rec) {
+  double* e = ws;                            // K x n   residual of the fit over all nodes: rho - H rho
   double* S = e + (size_t)K * n;             // t x t
   double* aug = S + (size_t)t * t;           // t x 2t
   double* x = aug + 2 * (size_t)t * t;       // K x t   leave-out residuals of the candidates
   double* ratio = x + (size_t)K * t;         // n
-  int* vlist = reinterpret_cast<int*>(ratio + n);   // t candidates in node order
-  int* vpos = vlist + t;                            // n: position of node k in vlist
-  SOLON_FOR_THREADS(k, n) {
-    int pos = 0;
-    for (int o = 0; o < k; ++o) pos += cand[o] ? 1 : 0;
-    vpos[k] = pos;
-    if (cand[k]) vlist[pos] = k;
-  }
-  SOLON_FOR_THREADS(idx, K * m) {
-    const int kappa = idx / m, i = idx - kappa * m;
-    double acc = 0.0;
-    for (int k = 0; k < n; ++k) acc = fma(tb.Qb[(size_t)i * n + k], rho_n[(size_t)kappa * n + k], acc);
-    coef[idx] = acc;
-  }
-  SOLON_SYNC();
   SOLON_FOR_THREADS(idx, K * n) {
     const int kappa = idx / n, k = idx - kappa * n;
-    double acc = rho_n[idx];
-    for (int i = 0; i < m; ++i) acc = fma(-tb.Qb[(size_t)i * n + k], coef[(size_t)kappa * m + i], acc);
-    e[idx] = acc;
+    const double* h = tb.Hm + (size_t)k * n;
+    const double* r = rho_n + (size_t)kappa * n;
+    double a0 = r[k], a1 = 0.0;
+    int j = 0;
+    for (; j + 1 < n; j += 2) {
+      a0 = fma(-h[j], r[j], a0);
+      a1 = fma(-h[j + 1], r[j + 1], a1);
+    }
+    if (j < n) a0 = fma(-h[j], r[j], a0);
+    e[idx] = a0 + a1;
   }
   SOLON_SYNC();
-  if (t > 0) {
-    deletion_inverse(tb, n, m, vlist, t, S, aug);
+  if (t == 1) {
+    // one deleted node v: x = e_v / (1 - H_vv), every thread computes it for itself
+    const int v = vlist[0];
+    const double sinv = 1.0 / (1.0 - tb.Hm[(size_t)v * n + v]);
+    SOLON_FOR_THREADS(kappa, K) x[kappa] = sinv * e[(size_t)kappa * n + v];
+    SOLON_SYNC();
+  } else if (t == 2) {
+    const int v0 = vlist[0], v1 = vlist[1];
+    const double s00 = 1.0 - tb.Hm[(size_t)v0 * n + v0], s11 = 1.0 - tb.Hm[(size_t)v1 * n + v1];
+    const double s01 = -tb.Hm[(size_t)v0 * n + v1];
+    const double idet = 1.0 / (s00 * s11 - s01 * s01);
+    SOLON_FOR_THREADS(kappa, K) {
+      const double e0 = e[(size_t)kappa * n + v0], e1 = e[(size_t)kappa * n + v1];
+      x[(size_t)kappa * 2] = (s11 * e0 - s01 * e1) * idet;
+      x[(size_t)kappa * 2 + 1] = (s00 * e1 - s01 * e0) * idet;
+    }
+    SOLON_SYNC();
+  } else if (t > 2) {
+    deletion_inverse(tm, tb, n, vlist, t, S, aug);
     SOLON_FOR_THREADS(idx, K * t) {
       const int kappa = idx / t, a = idx - kappa * t;
       double acc = 0.0;
@@ -234,6 +251,7 @@ SOLON_HD inline void locate_verify(const GroupTables& tb, int n, int m, int K, c
     }
     SOLON_SYNC();
   }
+  const double inv_tau = tau > 0.0 ? 1.0 / tau : 0.0;
   SOLON_FOR_THREADS(k, n) {
     double worst = 0.0;
     for (int kappa = 0; kappa < K; ++kappa) {
@@ -242,80 +260,186 @@ SOLON_HD inline void locate_verify(const GroupTables& tb, int n, int m, int K, c
         res = x[(size_t)kappa * t + vpos[k]];
       } else {
         res = e[(size_t)kappa * n + k];
-        for (int b = 0; b < t; ++b) {
-          double h = 0.0;
-          for (int i = 0; i < m; ++i) h = fma(tb.Qb[(size_t)i * n + k], tb.Qb[(size_t)i * n + vlist[b]], h);
-          res = fma(h, x[(size_t)kappa * t + b], res);
-        }
+        for (int b = 0; b < t; ++b) res = fma(tb.Hm[(size_t)k * n + vlist[b]], x[(size_t)kappa * t + b], res);
       }
       res = fabs(res);
       if (!(res == res)) res = INFINITY;
       worst = res > worst ? res : worst;
     }
-    double rt = tau > 0.0 ? worst / tau : (worst > 0.0 ? INFINITY : 0.0);
+    double rt = tau > 0.0 ? worst * inv_tau : (worst > 0.0 ? INFINITY : 0.0);
     if (forced[k]) rt = INFINITY;
     ratio[k] = rt;
     bad[k] = rt > 1.0 ? 1 : 0;
   }
   SOLON_SYNC();
+  // every thread scans the verdicts (no branches on loaded values); thread 0 stores the record
+  int rejected = 0, n_flagged = 0;
+  double max_fit = 0.0;
+  for (int k = 0; k < n; ++k) {
+    const int c = cand[k] ? 1 : 0, b = bad[k] ? 1 : 0;
+    n_flagged += c & b;
+    rejected += (1 - c) & b;
+    const double rk = c ? 0.0 : ratio[k];
+    max_fit = rk > max_fit ? rk : max_fit;
+  }
   if (SOLON_TID == 0) {
-    int accept = 1, n_flagged = 0;
-    double max_fit = 0.0;
-    for (int k = 0; k < n; ++k) {
-      if (cand[k]) {
-        n_flagged += bad[k];
-      } else {
-        if (bad[k]) accept = 0;
-        max_fit = ratio[k] > max_fit ? ratio[k] : max_fit;
-      }
-    }
-    rec->accept = accept;
+    rec->accept = rejected == 0 ? 1 : 0;
     rec->n_flagged = n_flagged;
     rec->max_fit = max_fit;
   }
-  SOLON_SYNC();
 }
+
+#define SOLON_FAST_T 5         /* error counts handled by the register-resident solver */
+#if defined(__CUDA_ARCH__)
+#define SOLON_FAST_RPL 2       /* rows per lane it can hold */
+#else
+#define SOLON_FAST_RPL 64
+#endif
 
 // One task: assume exactly t corrupt nodes among the n nodes of a group.
 //   rho_n   K x n projected values divided by the scale (0 for forced nodes)
 //   s       the plan's s (row stride of tb.Tch is s + 1);  tau  tolerance in the same normalised units
 //   flags   n bytes out: 1 for candidates that do not fit (the located nodes if accepted)
 //   cand, bad: n bytes of scratch each;  ws: locate_task_ws_doubles(n, m, K, t) doubles
-SOLON_HD inline void locate_task(const GroupTables& tb, int n, int m, int K, int t, int s, const double* rho_n,
+SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, int m, int K, int t, int s, const double* rho_n,
                                  const uint8_t* forced, double tau, uint8_t* flags, uint8_t* cand, uint8_t* bad,
                                  double* ws, TaskRecord* rec) {
   const int ldt = s + 1;
-  SOLON_FOR_THREADS(k, n) cand[k] = 0;
+  double* absE = ws;                         // n
+  int* vlist = reinterpret_cast<int*>(absE + n);   // t
+  int* vpos = vlist + t;                            // n
+  double* rest = absE + n + (size_t)(t + n) / 2 + 1;
+  SOLON_FOR_THREADS(k, n) {
+    cand[k] = 0;
+    vpos[k] = 0;
+  }
   SOLON_SYNC();
-  double* rest = ws;
   if (t > 0) {
     const int nperp = n - m - t;               // complement of the polynomials of degree < m + t
     const int rows = K * nperp;
-    const int ld = t + 1;                      // t unknowns theta, then the right-hand side
-    double* A = ws;                            // column-major, ld columns of `rows` rows
-    double* norm0 = A + (size_t)rows * ld;     // ld
-    double* Rt = norm0 + ld;                   // t x (t + 1)
-    double* diag = Rt + (size_t)t * (t + 1);   // t
-    double* absE = diag + t;                   // n
-    rest = absE + n;
-    // A[(kappa, j), i] = sum_k q_{m+t+j}(w_k) rho_kappa,k T_i(w_k); the last column carries -(...) T_t
-    SOLON_FOR_THREADS(idx, rows * ld) {
-      const int i = idx / rows, row = idx - i * rows;
-      const int kappa = row / nperp, j = row - kappa * nperp;
-      const double* q = tb.Qb + (size_t)(m + t + j) * n;
-      double acc = 0.0;
-      for (int k = 0; k < n; ++k) acc = fma(q[k] * rho_n[(size_t)kappa * n + k], tb.Tch[(size_t)k * ldt + i], acc);
-      A[idx] = i < t ? acc : -acc;
-    }
-    SOLON_SYNC();
-    column_norms(A, rows, rows, ld, norm0);
-    mgs_factor(A, rows, rows, t, ld, norm0, Rt, t + 1, diag);
-    // back substitution for theta; every thread does the same arithmetic
     double theta[SOLON_THETA_MAX];
-    for (int i = t - 1; i >= 0; --i) {
-      double acc = Rt[(size_t)i * (t + 1) + t];
-      for (int c = i + 1; c < t; ++c) acc = fma(-Rt[(size_t)i * (t + 1) + c], theta[c], acc);
-      theta[i] = diag[i] > 0.0 ? acc / diag[i] : 0.0;
+    if (tm.nwarps == 1 && t <= SOLON_FAST_T && rows <= SOLON_FAST_RPL * tm.nlanes) {
+      // Small system: every lane keeps its rows of [A | b] in registers.  Row (kappa, j), column i:
+      //   sum_k q_{m+t+j}(w_k) rho_kappa,k T_i(w_k);  the last column carries -(...) T_t.
+      // One combined lane reduction per Gram-Schmidt step yields the norm and all inner products.
+      double a[SOLON_FAST_RPL][SOLON_FAST_T + 1];
+      const int rpl = (rows + tm.nlanes - 1) / tm.nlanes;
+#pragma unroll
+      for (int rr = 0; rr < SOLON_FAST_RPL; ++rr) {
+        const int row = tm.lane + rr * tm.nlanes;
+#pragma unroll
+        for (int i = 0; i <= SOLON_FAST_T; ++i) a[rr][i] = 0.0;
+        if (rr < rpl && row < rows) {
+          const int kappa = row / nperp, j = row - kappa * nperp;
+          const double* q = tb.Qb + (size_t)(m + t + j) * n;
+          for (int k = 0; k < n; ++k) {
+            const double qr = q[k] * rho_n[(size_t)kappa * n + k];
+#pragma unroll
+            for (int i = 0; i <= SOLON_FAST_T; ++i)
+              if (i <= t) a[rr][i] = fma(qr, tb.Tch[(size_t)k * ldt + i], a[rr][i]);
+          }
+#pragma unroll
+          for (int i = 0; i <= SOLON_FAST_T; ++i)
+            if (i == t) a[rr][i] = -a[rr][i];
+        }
+      }
+      double R[SOLON_FAST_T][SOLON_FAST_T + 1], diag[SOLON_FAST_T], norm0[SOLON_FAST_T];
+#pragma unroll
+      for (int j = 0; j < SOLON_FAST_T; ++j) {
+        double v = 0.0;
+#pragma unroll
+        for (int rr = 0; rr < SOLON_FAST_RPL; ++rr) v = fma(a[rr][j], a[rr][j], v);
+        norm0[j] = v;
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+#if defined(__CUDA_ARCH__)
+        double tmp[SOLON_FAST_T];
+#pragma unroll
+        for (int j = 0; j < SOLON_FAST_T; ++j) tmp[j] = __shfl_xor_sync(0xffffffffu, norm0[j], off);
+#pragma unroll
+        for (int j = 0; j < SOLON_FAST_T; ++j) norm0[j] += tmp[j];
+#endif
+      }
+#pragma unroll
+      for (int j = 0; j < SOLON_FAST_T; ++j) {
+        diag[j] = 0.0;
+#pragma unroll
+        for (int c = 0; c <= SOLON_FAST_T; ++c) R[j][c] = 0.0;
+        if (j < t) {
+          double d[SOLON_FAST_T + 1];      // d[c] = a_j . a_c for c >= j (d[j] is the squared norm)
+#pragma unroll
+          for (int c = 0; c <= SOLON_FAST_T; ++c) {
+            double v = 0.0;
+            if (c >= j && c <= t) {
+#pragma unroll
+              for (int rr = 0; rr < SOLON_FAST_RPL; ++rr) v = fma(a[rr][j], a[rr][c], v);
+            }
+            d[c] = v;
+          }
+#if defined(__CUDA_ARCH__)
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            double tmp[SOLON_FAST_T + 1];
+#pragma unroll
+            for (int c = 0; c <= SOLON_FAST_T; ++c) tmp[c] = __shfl_xor_sync(0xffffffffu, d[c], off);
+#pragma unroll
+            for (int c = 0; c <= SOLON_FAST_T; ++c) d[c] += tmp[c];
+          }
+#endif
+          const double nrm2 = d[j];
+          const bool dead = !(nrm2 > norm0[j] * 1e-26) || !(nrm2 > 0.0);
+          const double nrm = dead ? 0.0 : sqrt(nrm2);
+          const double inv2 = dead ? 0.0 : 1.0 / nrm2;
+          diag[j] = nrm;
+#pragma unroll
+          for (int c = 0; c <= SOLON_FAST_T; ++c) {
+            if (c > j && c <= t) {
+              const double coef = d[c] * inv2;
+#pragma unroll
+              for (int rr = 0; rr < SOLON_FAST_RPL; ++rr) a[rr][c] = fma(-coef, a[rr][j], a[rr][c]);
+              R[j][c] = d[c] * (nrm * inv2);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int i = SOLON_FAST_T - 1; i >= 0; --i) {
+        if (i < t) {
+          double acc = 0.0;
+#pragma unroll
+          for (int c = 0; c <= SOLON_FAST_T; ++c)
+            if (c == t) acc = R[i][c];
+#pragma unroll
+          for (int c = 0; c < SOLON_FAST_T; ++c)
+            if (c > i && c < t) acc = fma(-R[i][c], theta[c], acc);
+          theta[i] = diag[i] > 0.0 ? acc / diag[i] : 0.0;
+        }
+      }
+    } else {
+      const int ld = t + 1;                      // t unknowns theta, then the right-hand side
+      double* A = rest;                          // column-major, ld columns of `rows` rows
+      double* norm0 = A + (size_t)rows * ld;     // ld
+      double* Rt = norm0 + ld;                   // t x (t + 1)
+      double* diag = Rt + (size_t)t * (t + 1);   // t
+      SOLON_FOR_THREADS(idx, rows * ld) {
+        const int i = idx / rows, row = idx - i * rows;
+        const int kappa = row / nperp, j = row - kappa * nperp;
+        const double* q = tb.Qb + (size_t)(m + t + j) * n;
+        double acc = 0.0;
+        for (int k = 0; k < n; ++k) acc = fma(q[k] * rho_n[(size_t)kappa * n + k], tb.Tch[(size_t)k * ldt + i], acc);
+        A[idx] = i < t ? acc : -acc;
+      }
+      SOLON_SYNC();
+      column_norms(tm, A, rows, rows, ld, norm0);
+      mgs_factor(tm, A, rows, rows, t, ld, norm0, Rt, t + 1, diag);
+      // back substitution for theta; every thread does the same arithmetic
+      for (int i = t - 1; i >= 0; --i) {
+        double acc = Rt[(size_t)i * (t + 1) + t];
+        for (int c = i + 1; c < t; ++c) acc = fma(-Rt[(size_t)i * (t + 1) + c], theta[c], acc);
+        theta[i] = diag[i] > 0.0 ? acc / diag[i] : 0.0;
+      }
+      SOLON_SYNC();     // A is reused by the verification below
     }
     SOLON_FOR_THREADS(k, n) {
       double ev = tb.Tch[(size_t)k * ldt + t];
@@ -327,12 +451,19 @@ SOLON_HD inline void locate_task(const GroupTables& tb, int n, int m, int K, int
     SOLON_FOR_THREADS(k, n) {
       int rank = 0;
       const double mine = absE[k];
-      for (int o = 0; o < n; ++o) rank += (absE[o] < mine || (absE[o] == mine && o < k)) ? 1 : 0;
-      cand[k] = rank < t ? 1 : 0;
+      for (int o = 0; o < n; ++o) {
+        const double other = absE[o];
+        rank += (other < mine || (other == mine && o < k)) ? 1 : 0;
+      }
+      if (rank < t) {
+        cand[k] = 1;
+        vlist[rank] = k;
+        vpos[k] = rank;
+      }
     }
     SOLON_SYNC();
   }
-  locate_verify(tb, n, m, K, rho_n, tau, cand, t, forced, bad, rest, rec);
+  locate_verify(tm, tb, n, K, rho_n, tau, cand, t, vlist, vpos, forced, bad, rest, rec);
   SOLON_FOR_THREADS(k, n) flags[k] = (cand[k] && bad[k]) ? 1 : 0;
   SOLON_SYNC();
 }
@@ -342,7 +473,7 @@ SOLON_HD inline void locate_task(const GroupTables& tb, int n, int m, int K, int
 // i.e. the least-squares inverse of [W-hat_{m-1}]_{rows,.} (monomial basis, as the encoder used).
 // ws: locate_epilogue_ws_doubles(n, m, s).  Returns the number of rows (same value in every thread),
 // 0 if fewer than m nodes are trusted or (all-rows form) more than s are not.
-SOLON_HD inline int recovery_table(const GroupTables& tb, int n, int m, int s, const uint8_t* trusted, int* rec_rows,
+SOLON_HD inline int recovery_table(const Team& tm, const GroupTables& tb, int n, int m, int s, const uint8_t* trusted, int* rec_rows,
                                    double* coeff, double* ws) {
   int n_u = 0;
   for (int k = 0; k < n; ++k) n_u += trusted[k] ? 1 : 0;
@@ -356,7 +487,7 @@ SOLON_HD inline int recovery_table(const GroupTables& tb, int n, int m, int s, c
     for (int k = 0; k < n && next < n_rec; ++k) {
       if (!trusted[k]) continue;
       const int want = !subset ? next
-                       : (m == 1 ? (n_u - 1) / 2 : (int)(((long long)next * (n_u - 1) + (m - 1) / 2) / (m - 1)));
+                       : (m == 1 ? (n_u - 1) / 2 : (next * (n_u - 1) + (m - 1) / 2) / (m - 1));
       if (seen == want) {
         if (SOLON_TID == 0) rec_rows[next] = k;
         ++next;
@@ -369,22 +500,23 @@ SOLON_HD inline int recovery_table(const GroupTables& tb, int n, int m, int s, c
     // Lagrange form of the inverse Vandermonde: row j holds the monomial coefficients of
     // L_j(w) = prod_{i != j} (w - x_i) / (x_j - x_i), built by multiplying one factor at a time.
     SOLON_FOR_THREADS(j, m) {
-      double* c = coeff + (size_t)j * m;
+      double c[SOLON_SUBSET_MAX_M];
+#pragma unroll
+      for (int l = 0; l < SOLON_SUBSET_MAX_M; ++l) c[l] = l == 0 ? 1.0 : 0.0;
       const double xj = tb.w[rec_rows[j]];
-      for (int l = 0; l < m; ++l) c[l] = 0.0;
-      c[0] = 1.0;
-      int deg = 0;
       double denom = 1.0;
       for (int i = 0; i < m; ++i) {
         if (i == j) continue;
         const double xi = tb.w[rec_rows[i]];
-        for (int l = deg + 1; l >= 1; --l) c[l] = fma(-xi, c[l], c[l - 1]);   // times (w - x_i)
+#pragma unroll
+        for (int l = SOLON_SUBSET_MAX_M - 1; l >= 1; --l) c[l] = fma(-xi, c[l], c[l - 1]);   // times (w - x_i)
         c[0] = -xi * c[0];
-        ++deg;
         denom *= xj - xi;
       }
       const double inv = 1.0 / denom;
-      for (int l = 0; l < m; ++l) c[l] *= inv;
+#pragma unroll
+      for (int l = 0; l < SOLON_SUBSET_MAX_M; ++l)
+        if (l < m) coeff[(size_t)j * m + l] = c[l] * inv;
     }
     SOLON_SYNC();
     return n_rec;
@@ -406,7 +538,7 @@ SOLON_HD inline int recovery_table(const GroupTables& tb, int n, int m, int s, c
   }
   SOLON_SYNC();
   if (nv > 0) {
-    deletion_inverse(tb, n, m, vlist, nv, S, aug);
+    deletion_inverse(tm, tb, n, vlist, nv, S, aug);
     SOLON_FOR_THREADS(idx, nv * n_u) {
       const int a = idx / n_u, u = idx - a * n_u;
       double acc = 0.0;
@@ -442,7 +574,7 @@ SOLON_HD inline int recovery_table(const GroupTables& tb, int n, int m, int s, c
 //   rho_n = rho / sqrt(2 median nu), clamped to +-SOLON_RHO_CLAMP medians of |rho| per projection
 //   *tau_eff = tau, or (median energy 0: all-zero data, any deviation counts) 1e-10 of the largest |rho|
 // scratch: K + 2 doubles.
-SOLON_HD inline void locate_prepare(int n, int K, const double* rho, const double* nu, double tau, uint8_t* forced,
+SOLON_HD inline void locate_prepare(const Team& tm, int n, int K, const double* rho, const double* nu, double tau, uint8_t* forced,
                                     double* rho_n, double* tau_eff, double* scratch) {
   SOLON_FOR_THREADS(k, n) {
     bool finite = isfinite(nu[k]);
@@ -498,7 +630,7 @@ SOLON_HD inline void locate_prepare(int n, int K, const double* rho, const doubl
 //   recs[s+1], flags[(s+1) x flags_ld] from the tasks; forced from locate_prepare
 //   trusted: n bytes scratch; ws: locate_epilogue_ws_doubles(n, m, s)
 // Returns 1 if the group decoded, 0 if not.  *t_out: corrupt nodes located (-1 if undecodable).
-SOLON_HD inline int locate_epilogue(const GroupTables& tb, int n, int m, int s, const uint8_t* forced,
+SOLON_HD inline int locate_epilogue(const Team& tm, const GroupTables& tb, int n, int m, int s, const uint8_t* forced,
                                     const TaskRecord* recs, const uint8_t* flags, int flags_ld, uint8_t* mask,
                                     int* t_out, int* rec_rows, int* n_rec_out, double* coeff, uint8_t* trusted,
                                     double* ws) {
@@ -528,7 +660,7 @@ SOLON_HD inline int locate_epilogue(const GroupTables& tb, int n, int m, int s, 
   int n_bad = 0;
   for (int k = 0; k < n; ++k) n_bad += trusted[k] ? 0 : 1;
   if (n_bad > s) ok = 0;
-  const int n_rec = recovery_table(tb, n, m, s, trusted, rec_rows, coeff, ws);
+  const int n_rec = recovery_table(tm, tb, n, m, s, trusted, rec_rows, coeff, ws);
   if (n_rec == 0) ok = 0;
   if (SOLON_TID == 0) {
     *n_rec_out = n_rec;

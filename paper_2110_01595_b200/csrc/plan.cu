@@ -110,7 +110,7 @@ static int dev_alloc(T** ptr, size_t count) {
 
 static void free_device(solon_plan* p) {
   cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f);
-  cudaFree(p->d_qb); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
+  cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_task_records); cudaFree(p->d_task_flags); cudaFree(p->d_group_ticket); cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status);
@@ -132,7 +132,7 @@ static int alloc_projection(solon_plan* p) {
   if ((rc = dev_alloc(&p->d_partials, (size_t)(p->proj_grid + p->proj_grid / 16 + 1) * (p->K + 1) * p->P))) return rc;
   if ((rc = dev_alloc(&p->d_rho, (size_t)p->K * p->P))) return rc;
   p->locate_ws_stride = locate_ws_doubles(p->max_group, p->m, p->K, p->s);
-  if ((rc = dev_alloc(&p->d_locate_ws, (size_t)p->q * (p->s + 1) * p->locate_ws_stride))) return rc;
+  if ((rc = dev_alloc(&p->d_locate_ws, (size_t)p->q * p->locate_ws_stride))) return rc;
   return SOLON_OK;
 }
 
@@ -228,15 +228,17 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
       qb_off[g] = qb_total;
       qb_total += (int64_t)n_g * n_g;
     }
-    std::vector<double> h_qb(qb_total), h_mt((size_t)q * m * m), h_tch((size_t)P * (s + 1));
+    std::vector<double> h_qb(qb_total), h_hm(qb_total), h_mt((size_t)q * m * m), h_tch((size_t)P * (s + 1));
     for (int g = 0; g < q; ++g)
       build_group_tables(start[g + 1] - start[g], m, s, p->w.data() + start[g], h_qb.data() + qb_off[g],
-                         h_mt.data() + (size_t)g * m * m, h_tch.data() + (size_t)start[g] * (s + 1));
+                         h_hm.data() + qb_off[g], h_mt.data() + (size_t)g * m * m, h_tch.data() + (size_t)start[g] * (s + 1));
     if ((rc = dev_alloc(&p->d_qb, (size_t)qb_total))) break;
+    if ((rc = dev_alloc(&p->d_hm, (size_t)qb_total))) break;
     if ((rc = dev_alloc(&p->d_qb_off, q))) break;
     if ((rc = dev_alloc(&p->d_mt, h_mt.size()))) break;
     if ((rc = dev_alloc(&p->d_tch, h_tch.size()))) break;
     if (cudaMemcpy(p->d_qb, h_qb.data(), h_qb.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(p->d_hm, h_hm.data(), h_hm.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(p->d_qb_off, qb_off.data(), q * sizeof(int64_t), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(p->d_mt, h_mt.data(), h_mt.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(p->d_tch, h_tch.data(), h_tch.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess) {

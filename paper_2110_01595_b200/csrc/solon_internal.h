@@ -58,6 +58,7 @@ struct solon_plan {
   int* d_group_of;         // P
   double* d_w;             // P (float64 node scalars)
   double* d_qb;            // per group n_g x n_g orthonormal polynomial tables (locator)
+  double* d_hm;            // per group n_g x n_g projectors on the polynomials of degree < m (same offsets)
   int64_t* d_qb_off;       // q offsets into d_qb
   double* d_mt;            // q x m x m monomial coefficients of the first m orthonormal polynomials
   double* d_tch;           // P x (s + 1) Chebyshev polynomials at the nodes
@@ -112,8 +113,8 @@ int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w,
 // Doubles of workspace one locator CTA needs for a group of n nodes.
 size_t locate_ws_doubles(int n, int m, int K, int s);
 
-// Host: locator tables of one group (n x n Qb column-major, m x m Mt, n x (s + 1) Tch).
-void build_group_tables(int n, int m, int s, const double* w, double* Qb, double* Mt, double* Tch);
+// Host: locator tables of one group (n x n Qb column-major, n x n Hm, m x m Mt, n x (s + 1) Tch).
+void build_group_tables(int n, int m, int s, const double* w, double* Qb, double* Hm, double* Mt, double* Tch);
 
 // Host-side layout rules (also used by the plan-free helpers).
 int check_params(int P, int s, int m, int r, int64_t d);
