@@ -121,6 +121,8 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
     tb.w = w_s;
   }
   const Team cta = Team::cta();
+  pdl_trigger();   // the recovery kernel may be scheduled early; it waits for this grid before reading the table
+  pdl_wait();      // the projections are complete and visible (everything above only read plan tables)
   if (prm.s == 0) {
     // pure compression code: nothing to locate, every node is trusted
     for (int k = tid; k < n; k += n_threads) {
@@ -263,10 +265,8 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
   }
   if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  locate_kernel<<<plan->q, 32 * (plan->s + 1), smem, plan->stream>>>(prm);
   plan->launches += 1;
-  SOLON_CUDA_TRY(cudaGetLastError());
-  return SOLON_OK;
+  return launch_dependent(locate_kernel, dim3(plan->q), dim3(32 * (plan->s + 1)), smem, plan->stream, prm);
 }
 
 }  // namespace solon

@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
   __shared__ unsigned int s_ticket;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_acc = (K + 1) * P;
+  pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading rho
   for (int i = tid; i < n_acc; i += kProjThreads) sacc[i] = 0.0;
 
   const int64_t c_begin = (int64_t)blockIdx.x * range_len;

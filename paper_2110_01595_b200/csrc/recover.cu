@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     *abort_flag = 0;
     pipe::fence_barrier_init();
   }
+  pdl_wait();   // the locator's mask and table are complete and visible; nothing above touched global memory
   const int n_rows = pack_tables(prm, rows_p, coeff_p, count_s);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
@@ -252,9 +253,7 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   if (per_sm < 1) per_sm = 1;
   int64_t cap = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(tiles < cap ? tiles : cap);
-  kernel<<<grid, kRecPipeThreads, smem, plan->stream>>>(prm, pp);
-  SOLON_CUDA_TRY(cudaGetLastError());
-  return SOLON_OK;
+  return launch_dependent(kernel, dim3(grid), dim3(kRecPipeThreads), smem, plan->stream, prm, pp);
 }
 
 int launch_recover(solon_plan* plan, const float* received, float* agg) {

@@ -102,6 +102,35 @@ struct solon_plan {
 
 namespace solon {
 
+// Programmatic dependent launch (sm_90+): a kernel launched with launch_dependent may start while the kernel
+// before it in the stream is still running, once every CTA of that kernel has called pdl_trigger (or exited);
+// it must call pdl_wait before it reads anything the earlier kernel wrote or writes anything it may still
+// read.  pdl_wait returns when the earlier kernel has completed and its writes are visible.
+#if defined(__CUDACC__)
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                   Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return SOLON_ERR_CUDA;
+  }
+  return SOLON_OK;
+}
+#endif
+
 // Kernel launchers (each enqueues on plan->stream and returns a solon_status).
 int launch_fill_projection(solon_plan* plan);
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
