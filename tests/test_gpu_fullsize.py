@@ -66,3 +66,25 @@ def test_full_size(name):
             lim = np.sqrt((f.astype(np.float64) ** 2).sum(1))[:, None] * np.sqrt(o_nu)[None, :]
             assert np.all(np.abs(rho - o_rho) <= 1e-11 * lim)
             assert np.allclose(nu, o_nu, rtol=1e-4)
+
+
+@pytest.mark.parametrize("P,s,m,d", [(105, 5, 10, 10_000_000), (15, 1, 10, 10_000_000), (105, 1, 1, 10_000_000),
+                                     (45, 5, 2, 10_000_000), (15, 5, 5, 50_000_000)])
+def test_sweep_points_full_size(P, s, m, d):
+    """Sweep points at bench size: mask exact, aggregate against the float64 definition at sampled coordinates
+    (oracle) and everywhere (device-side float64 sum)."""
+    wl = synth.Workload(f"sweep_P{P}_s{s}_m{m}_d{d}", P, s, m, d, "normal", 1.0, "gaussian", s, 7000 + P + 10 * s + m)
+    G = synth.make_grads(wl, "cuda")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.cpu().numpy().nonzero()[0].tolist() == nodes
+        ref = G.sum(dim=0, dtype=torch.float64)
+        scale = float(ref.abs().max())
+        assert float((agg.double() - ref).abs().max()) <= AGG_TOL * scale
+        cols = np.unique(np.concatenate([np.random.default_rng(wl.seed).integers(0, d, size=2000), [0, d - 1]]))
+        G_s = G[:, torch.from_numpy(cols).cuda()].cpu().numpy()
+        got = agg[torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.float64)
+        assert np.abs(got - so.plain_sum(G_s)).max() <= AGG_TOL * scale
