@@ -88,3 +88,33 @@ def test_sweep_points_full_size(P, s, m, d):
         G_s = G[:, torch.from_numpy(cols).cuda()].cpu().numpy()
         got = agg[torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.float64)
         assert np.abs(got - so.plain_sum(G_s)).max() <= AGG_TOL * scale
+
+
+def test_config_lsq_full_size():
+    """The least-squares configuration as specified: P=15, s=1, m=3, d=100000, 256 rows per partition, w = 0.
+    With w = 0 the gradient of a column needs only that column of X, so the oracle checks sampled columns."""
+    wl = synth.WORKLOADS["lsq"]
+    X, y, wvec = synth.make_lsq_problem(wl, "cuda")
+    assert float(wvec.abs().max()) == 0.0
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        G = plan.lsq_grads(X, y, wvec, rows=wl.lsq_rows)
+        cols = np.unique(np.concatenate([np.random.default_rng(1).integers(0, wl.d, size=300), [0, wl.d - 1]]))
+        ct = torch.from_numpy(cols).cuda()
+        X_s = X[:, ct].cpu().numpy()
+        want_G = so.lsq_grads(X_s, y.cpu().numpy(), np.zeros(len(cols), dtype=np.float32), wl.lsq_rows)   # P x len(cols)
+        got_G = G[:, ct].cpu().numpy().astype(np.float64)
+        bound = np.zeros_like(want_G)
+        ya = np.abs(y.cpu().numpy()).astype(np.float64)
+        for i in range(wl.P):
+            rows = slice(i * wl.lsq_rows, (i + 1) * wl.lsq_rows)
+            bound[i] = np.abs(X_s[rows]).astype(np.float64).T @ ya[rows]
+        assert np.all(np.abs(got_G - want_G) <= 3e-7 * bound + 1e-30)
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.cpu().numpy().nonzero()[0].tolist() == nodes and len(nodes) == 1
+        # aggregate against the oracle's own float64 gradients at the sampled columns; scale from the device sum
+        scale = float(G.sum(dim=0, dtype=torch.float64).abs().max())
+        got = agg[ct].cpu().numpy().astype(np.float64)
+        assert np.abs(got - want_G.sum(0)).max() <= AGG_TOL * scale
