@@ -289,9 +289,10 @@ def run_ours(args, wl):
     line = {
         "metric": METRIC, "value": total_units / (max_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32 in/out, f64 arithmetic", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32" if wl.m <= 6 else "f64", "data": "synthetic",
         "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "n_byz": len(nodes),
-                   "attack": wl.attack, "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * wl.d * 4 / 1e9),
+                   "attack": wl.attack,
+                   "arithmetic": "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64", "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * wl.d * 4 / 1e9),
                    "parallelism": "independent problems per GPU, no collective"},
         "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
                      "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(wl.name),

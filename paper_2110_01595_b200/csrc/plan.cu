@@ -112,7 +112,7 @@ static void free_device(solon_plan* p) {
   cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f);
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
-  cudaFree(p->d_task_records); cudaFree(p->d_task_flags); cudaFree(p->d_group_ticket); cudaFree(p->d_locate_ws);
+  cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status);
   cudaFree(p->d_resid);
   for (int i = 0; i < 6; ++i)
@@ -249,11 +249,6 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     if ((rc = alloc_projection(p))) break;
     if ((rc = dev_alloc(&p->d_nu, P))) break;
     if ((rc = dev_alloc(&p->d_proj_ticket, (size_t)p->proj_grid / 16 + 2))) break;
-    TaskRecord* recs = nullptr;
-    if ((rc = dev_alloc(&recs, (size_t)q * (s + 1)))) break;
-    p->d_task_records = recs;
-    if ((rc = dev_alloc(&p->d_task_flags, (size_t)(s + 1) * P))) break;
-    if ((rc = dev_alloc(&p->d_group_ticket, q))) break;
     if ((rc = dev_alloc(&p->d_t_acc, q))) break;
     if ((rc = dev_alloc(&p->d_n_rec, q))) break;
     if ((rc = dev_alloc(&p->d_rec_rows, P))) break;
@@ -264,7 +259,6 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_of, p->group_of.data(), P * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_w, p->w.data(), P * sizeof(double), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, ((size_t)p->proj_grid / 16 + 2) * sizeof(unsigned int));
-    if (e == cudaSuccess) e = cudaMemset(p->d_group_ticket, 0, q * sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_n_rec, 0, q * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_t_acc, 0, q * sizeof(int));

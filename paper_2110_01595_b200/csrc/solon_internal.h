@@ -73,10 +73,7 @@ struct solon_plan {
   unsigned int* d_proj_ticket;   // 1
 
   // locator workspace / outputs
-  void* d_task_records;    // q x (s + 1) TaskRecord
-  uint8_t* d_task_flags;   // (s + 1) x P
-  unsigned int* d_group_ticket;  // q
-  double* d_locate_ws;     // q x (s + 1) x locate_ws_stride doubles (global fallback workspace)
+  double* d_locate_ws;     // q x locate_ws_stride doubles (workspace of groups too large for shared memory)
   size_t locate_ws_stride;
   int* d_t_acc;            // q
   int* d_n_rec;            // q
