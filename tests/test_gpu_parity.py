@@ -161,6 +161,10 @@ def test_config_lsq_small():
     (23, 1, 3, 23, 777),      # r = P, one odd-sized group
     (40, 2, 12, 20, 3000),    # m = 12 (generic kernels), two groups of 20
     (128, 1, 2, 128, 513),    # largest group the locator handles
+    (256, 1, 2, 4, 10_007),   # 64 groups of four
+    (1024, 1, 1, 3, 517),     # most nodes allowed: 341 groups of three (one of four)
+    (126, 16, 1, 126, 300),   # most adversaries per group allowed
+    (40, 3, 8, 20, 4_001),    # m = 8: float64 paths, all-rows inverse
 ])
 def test_edge_shapes(P, s, m, r, d):
     wl = synth.Workload("edge", P, s, m, d, "normal", 1.0, "gaussian", s, 99)
