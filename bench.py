@@ -170,7 +170,8 @@ def run_reference(args, wl):
     sample = f"first {small.d} of {wl.d} coordinates of every partition gradient, all {wl.P} nodes"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
+        "scaling": "strong" if sp is not None else "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "sample_d": small.d},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
@@ -195,9 +196,24 @@ def run_ours(args, wl):
 
     import dataclasses
 
-    wl_rank = dataclasses.replace(wl, seed=wl.seed + 17 * rank)      # every rank its own problem
-    G = synth.make_grads(wl_rank, "cuda")
-    plan = binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl_rank.seed)
+    sp = None
+    if args.sharded:
+        # one problem for all ranks: rank i holds the coordinates [lo_i, hi_i) of every gradient; the decode's
+        # single exchange is an all-reduce of (K + 1) x P float64 values between the projection and the locator
+        from paper_2110_01595_b200 import sharded
+
+        sp = sharded.ShardedPlan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed, rank=rank, world=world)
+        G_all = synth.make_grads(wl, "cuda")
+        G = G_all[:, sp.lo:sp.hi].contiguous()
+        del G_all
+        whole, wl_rank = wl, wl
+        wl = dataclasses.replace(wl, d=sp.d_local)               # this rank's share, for the byte counts below
+        plan = sp.plan
+    else:
+        whole = wl
+        wl_rank = dataclasses.replace(wl, seed=wl.seed + 17 * rank)      # every rank its own problem
+        G = synth.make_grads(wl_rank, "cuda")
+        plan = binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl_rank.seed)
     coded = plan.encode(G)
     nodes = synth.byzantine_nodes(wl_rank)
     byz_rows = synth.byzantine_rows(wl_rank, coded, nodes)
@@ -214,7 +230,10 @@ def run_ours(args, wl):
             coded[k].copy_(byz_rows[i])                       # the adversary: plain device-to-device copies
         if events is not None:
             events[2].record()
-        plan.decode(coded, agg, mask)
+        if sp is not None:
+            sp.decode(coded, agg, mask)
+        else:
+            plan.decode(coded, agg, mask)
         if events is not None:
             events[3].record()
 
@@ -256,7 +275,7 @@ def run_ours(args, wl):
 
     # end to end through the host-buffer entry point: pinned host memory in, host results out
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and sp is None:
         G_host = torch.empty((wl.P, wl.d), dtype=torch.float32).pin_memory()
         G_host.copy_(G)
         rows_host = byz_rows.cpu().pin_memory() if nodes else torch.empty((0, wl.d_c))
@@ -288,14 +307,16 @@ def run_ours(args, wl):
     path_gbs = total_b / ((enc_ms + dec_ms) * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": total_units / (max_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True,
+        "scaling": "strong" if sp is not None else "weak",
         "vs_baseline": None, "dtype": "f32" if wl.m <= 6 else "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "n_byz": len(nodes),
+        "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": whole.d, "n_byz": len(nodes),
                    "attack": wl.attack,
                    "arithmetic": "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64", "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * wl.d * 4 / 1e9),
-                   "parallelism": "independent problems per GPU, no collective"},
+                   "parallelism": ("one problem, coordinates sharded over the GPUs, one all-reduce of (K+1) x P float64 per decode"
+                                   if sp is not None else "independent problems per GPU, no collective")},
         "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(wl.name),
+                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(wl.name) if sp is None else None,
                      "algorithmic_bytes": enc_b, "ms": enc_ms},
         "path": {"encode_ms": enc_ms, "decode_ms": dec_ms, "decodes_per_s": 1e3 / dec_ms, "algorithmic_bytes": total_b,
                  "hbm_gbs": path_gbs, "frac_of_peak": path_gbs / peak, "frac_of_8TBs": path_gbs / 8000.0},
@@ -303,7 +324,7 @@ def run_ours(args, wl):
         "e2e": e2e,
         "gpu_launches": int(launches),
     }
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and sp is None:
         small, G_s, nodes_s, rows_s, f_s = oracle_sample(wl, args.oracle_d, "cpu")
         dt = oracle_step_seconds(small, G_s, nodes_s, rows_s, f_s)
         line["cpu_baseline"] = {"value": small.P * small.d * 4 / dt / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
@@ -410,6 +431,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="with --gpus N: ONE problem whose coordinates are spread over the N GPUs (strong scaling; the "
+                         "decode's only exchange is a small all-reduce) instead of N independent problems; no e2e leg")
     ap.add_argument("--sweep", default=None, metavar="FILE",
                     help="run the (P, s, m, d) grid instead: one JSON line per point is appended to FILE, a summary is printed")
     ap.add_argument("--sweep-d", default="1000000,10000000,50000000", help="gradient lengths of the grid")

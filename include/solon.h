@@ -155,6 +155,26 @@ int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8
  * SOLON_ERR_UNDECODABLE, SOLON_ERR_INTERNAL or SOLON_ERR_CUDA. */
 int solon_decode_status(solon_plan* plan);
 
+/* The decode in two halves, for a coded matrix whose COLUMNS are spread over several devices.
+ * Equation (1)'s locator needs only the projected values rho = f R, and f R is a sum over
+ * columns; so each device projects the columns it holds with its own f, the K x P values (and
+ * the P row energies) are summed over the devices by whatever collective the caller has, and
+ * every device then runs the same locator on the same sums and recovers its own columns
+ * (Algorithm 1 applied to a column block of Y_j; the chunks of Section 3.4 are independent).
+ * Each device uses a plan built for the columns it owns (same P, s, m, r; d = its share, a
+ * multiple of m except on the last device; different seeds).
+ *
+ * solon_decode_project: first kernel only.
+ *   received  device, P x d_c        rho  device, K x P float64 (output)    nu  device, P float64 (output)
+ * With s = 0 nothing is launched and rho, nu are left untouched.
+ * solon_decode_finish: locator and recovery from the given rho and nu (device; the caller's sums).
+ *   received, agg_grad, byz_mask as in solon_decode.
+ * solon_decode(plan, R, u, mask) equals solon_decode_project followed by solon_decode_finish on
+ * the same buffers.  Status is read with solon_decode_status after solon_decode_finish. */
+int solon_decode_project(solon_plan* plan, const float* received, double* rho, double* nu);
+int solon_decode_finish(solon_plan* plan, const double* rho, const double* nu, const float* received,
+                        float* agg_grad, uint8_t* byz_mask);
+
 /* Least-squares partition gradients g_i = X_i^T (X_i w - y_i) (the paper accepts any method that
  * needs a sum of per-partition functions, Section 1; this one feeds the encode step).
  *   X      device, (P * rows) x d; partition i owns rows [i rows, (i+1) rows)

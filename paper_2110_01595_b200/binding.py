@@ -50,6 +50,8 @@ SIGNATURES = {
     "solon_encode": (c_int, [c_void_p, c_void_p, c_void_p]),
     "solon_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_decode_status": (c_int, [c_void_p]),
+    "solon_decode_project": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
+    "solon_decode_finish": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_lsq_grads": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_step_host": (c_int, [c_void_p, c_void_p, c_int, POINTER(c_int), c_void_p, c_void_p, c_void_p]),
     "solon_plan_get_projections": (c_int, [c_void_p, POINTER(c_double), POINTER(c_double)]),
@@ -269,6 +271,27 @@ class Plan:
             byz_mask = torch.empty(self.P, dtype=torch.uint8, device=received.device)
         _check(lib().solon_decode(self._h, self._dev(received, (self.P, self.d_c)), self._dev(agg_grad, (self.d,)),
                                   self._dev(byz_mask, (self.P,), torch.uint8)), "solon_decode")
+        return agg_grad, byz_mask
+
+    def decode_project(self, received, rho, nu):
+        """First half of the decode: rho (K x P) and nu (P), float64 device tensors, receive this plan's projections."""
+        torch = self._torch
+        _check(lib().solon_decode_project(self._h, self._dev(received, (self.P, self.d_c)),
+                                          self._dev(rho, (self.K, self.P), torch.float64),
+                                          self._dev(nu, (self.P,), torch.float64)), "solon_decode_project")
+        return rho, nu
+
+    def decode_finish(self, rho, nu, received, agg_grad=None, byz_mask=None):
+        """Second half: locator and recovery from the given (summed) projections."""
+        torch = self._torch
+        if agg_grad is None:
+            agg_grad = torch.empty(self.d, dtype=torch.float32, device=received.device)
+        if byz_mask is None:
+            byz_mask = torch.empty(self.P, dtype=torch.uint8, device=received.device)
+        _check(lib().solon_decode_finish(self._h, self._dev(rho, (self.K, self.P), torch.float64),
+                                         self._dev(nu, (self.P,), torch.float64),
+                                         self._dev(received, (self.P, self.d_c)), self._dev(agg_grad, (self.d,)),
+                                         self._dev(byz_mask, (self.P,), torch.uint8)), "solon_decode_finish")
         return agg_grad, byz_mask
 
     def decode_status(self) -> int:

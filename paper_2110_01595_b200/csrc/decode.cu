@@ -25,6 +25,24 @@ extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_
   return mark(5);
 }
 
+extern "C" int solon_decode_project(solon_plan* plan, const float* received, double* rho, double* nu) {
+  if (!plan || !received || !rho || !nu) return SOLON_ERR_INVALID_ARG;
+  if (((uintptr_t)received & 15) || ((uintptr_t)rho & 7) || ((uintptr_t)nu & 7)) return SOLON_ERR_INVALID_ARG;
+  if (plan->s == 0) return SOLON_OK;
+  return launch_project(plan, received, rho, nu);
+}
+
+extern "C" int solon_decode_finish(solon_plan* plan, const double* rho, const double* nu, const float* received,
+                                   float* agg_grad, uint8_t* byz_mask) {
+  if (!plan || !rho || !nu || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
+  if (((uintptr_t)received & 15) || ((uintptr_t)agg_grad & 15) || ((uintptr_t)rho & 7) || ((uintptr_t)nu & 7))
+    return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), plan->stream));
+  int rc;
+  if ((rc = launch_locate(plan, byz_mask, rho, nu))) return rc;
+  return launch_recover(plan, received, agg_grad);
+}
+
 template <typename T>
 static int stage_alloc(T** ptr, size_t count) {
   if (*ptr) return SOLON_OK;

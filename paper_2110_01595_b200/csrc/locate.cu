@@ -232,12 +232,12 @@ void build_group_tables(int n, int m, int s, const double* w, double* Qb, double
     for (int i = 0; i <= s; ++i) Tch[(size_t)k * (s + 1) + i] = i < n ? (double)T[(size_t)i * n + k] : 0.0;
 }
 
-int launch_locate(solon_plan* plan, uint8_t* byz_mask) {
+int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const double* nu) {
   LocateParams prm;
   prm.group_start = plan->d_group_start;
   prm.w = plan->d_w;
-  prm.rho = plan->d_rho;
-  prm.nu = plan->d_nu;
+  prm.rho = rho ? rho : plan->d_rho;
+  prm.nu = nu ? nu : plan->d_nu;
   prm.qb = plan->d_qb;
   prm.hm = plan->d_hm;
   prm.qb_off = plan->d_qb_off;

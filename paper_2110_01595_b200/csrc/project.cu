@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
 }
 
 template <int K>
-static int launch_project_k(solon_plan* plan, const float* received) {
+static int launch_project_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
   int tile_cols = K <= 2 ? 2048 : 1024;
   size_t smem = (size_t)K * tile_cols * sizeof(double) + (size_t)(K + 1) * plan->P * sizeof(double);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
@@ -201,19 +201,21 @@ static int launch_project_k(solon_plan* plan, const float* received) {
   range_len = (range_len + 3) / 4 * 4;
   if (range_len < tile_cols) tile_cols = (int)range_len;
   project_kernel<K><<<grid, kProjThreads, smem, plan->stream>>>(
-      received, plan->d_f, plan->f_pitch, plan->P, plan->d_c, range_len, tile_cols, plan->d_partials, plan->d_rho,
-      plan->d_nu, plan->d_proj_ticket);
+      received, plan->d_f, plan->f_pitch, plan->P, plan->d_c, range_len, tile_cols, plan->d_partials, rho_out,
+      nu_out, plan->d_proj_ticket);
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }
 
-int launch_project(solon_plan* plan, const float* received) {
+int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
+  if (!rho_out) rho_out = plan->d_rho;
+  if (!nu_out) nu_out = plan->d_nu;
   plan->launches += 1;
   switch (plan->K) {
-    case 1: return launch_project_k<1>(plan, received);
-    case 2: return launch_project_k<2>(plan, received);
-    case 3: return launch_project_k<3>(plan, received);
-    case 4: return launch_project_k<4>(plan, received);
+    case 1: return launch_project_k<1>(plan, received, rho_out, nu_out);
+    case 2: return launch_project_k<2>(plan, received, rho_out, nu_out);
+    case 3: return launch_project_k<3>(plan, received, rho_out, nu_out);
+    case 4: return launch_project_k<4>(plan, received, rho_out, nu_out);
     default: return SOLON_ERR_INVALID_ARG;
   }
 }

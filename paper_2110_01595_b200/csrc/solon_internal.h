@@ -131,8 +131,9 @@ static inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 blo
 // Kernel launchers (each enqueues on plan->stream and returns a solon_status).
 int launch_fill_projection(solon_plan* plan);
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
-int launch_project(solon_plan* plan, const float* received);
-int launch_locate(solon_plan* plan, uint8_t* byz_mask);
+// rho_out / nu_out (and rho / nu below): device buffers, or nullptr for the plan's own
+int launch_project(solon_plan* plan, const float* received, double* rho_out = nullptr, double* nu_out = nullptr);
+int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho = nullptr, const double* nu = nullptr);
 int launch_recover(solon_plan* plan, const float* received, float* agg);
 int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w, float* grads);
 
