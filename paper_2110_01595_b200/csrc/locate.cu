@@ -26,6 +26,8 @@ struct LocateParams {
   double* ws_global;     // q x ws_stride doubles, used when shared memory is too small
   size_t ws_stride;
   int use_smem;
+  unsigned long long* tile_counter;   // work counter of the recovery kernel, zeroed here
+  int warm;               // run the solver once on made-up values before waiting for the projections
   int stage_tables;      // copy the group's tables to shared memory (they follow the workspace)
   uint8_t* mask;         // P (caller's buffer)
   int* t_acc;            // q
@@ -122,46 +124,67 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   }
   const Team cta = Team::cta();
   pdl_trigger();   // the recovery kernel may be scheduled early; it waits for this grid before reading the table
-  pdl_wait();      // the projections are complete and visible (everything above only read plan tables)
-  if (prm.s == 0) {
-    // pure compression code: nothing to locate, every node is trusted
-    for (int k = tid; k < n; k += n_threads) {
-      sc.forced[k] = 0;
-      sc.flags[k] = 0;
+  // Two passes over the same code.  Pass 0 (small problems only) runs before the projections exist, on made-up
+  // values with s corrupt nodes, and writes nothing outside this CTA's scratch: between two decodes gigabytes
+  // stream through L2, so the solver's instructions would otherwise be fetched from HBM line by line on the
+  // critical path; this way they are fetched while the projection kernel is still streaming.  Pass 1 is the
+  // decode proper.
+#pragma unroll 1
+  for (int pass = prm.warm ? 0 : 1; pass < 2; ++pass) {
+    if (pass == 1) {
+      pdl_wait();   // the projections are complete and visible (everything above only read plan tables)
+      if (g == 0 && tid == 0) *prm.tile_counter = 0ULL;   // the recovery kernel reads it only after this grid is done
     }
-    if (tid == 0) {
-      sc.recs[0].accept = 1;
-      sc.recs[0].n_flagged = 0;
-      sc.recs[0].max_fit = 0.0;
-    }
-  } else {
-    // one parallel round trip brings the group's projected values on chip
-    for (int i = tid; i < n; i += n_threads) {
-      sc.nu_in[i] = prm.nu[row0 + i];
-      for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
+    if (prm.s == 0) {
+      // pure compression code: nothing to locate, every node is trusted
+      for (int k = tid; k < n; k += n_threads) {
+        sc.forced[k] = 0;
+        sc.flags[k] = 0;
+      }
+      if (tid == 0) {
+        sc.recs[0].accept = 1;
+        sc.recs[0].n_flagged = 0;
+        sc.recs[0].max_fit = 0.0;
+      }
+    } else {
+      // one parallel round trip brings the group's projected values on chip
+      for (int i = tid; i < n; i += n_threads) {
+        if (pass == 1) {
+          sc.nu_in[i] = prm.nu[row0 + i];
+          for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
+        } else {
+          sc.nu_in[i] = 1.0;
+          for (int kappa = 0; kappa < prm.K; ++kappa)
+            sc.rho_in[(size_t)kappa * n + i] = 1.0 + (prm.m > 1 ? (kappa + 1) * tb.w[i] : 0.0) + (i < prm.s ? 3.0 * (i + 1) : 0.0);
+        }
+      }
+      __syncthreads();
+      double tau_eff = 0.0;
+      locate_prepare(cta, n, prm.K, sc.rho_in, sc.nu_in, prm.tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
+      const int t = tid >> 5;                       // this warp's error count
+      double* task = sc.tasks + (size_t)t * sc.task_stride;
+      uint8_t* cand = reinterpret_cast<uint8_t*>(task);
+      uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
+      locate_task(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n,
+                  cand, bad, task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
     }
     __syncthreads();
-    double tau_eff = 0.0;
-    locate_prepare(cta, n, prm.K, sc.rho_in, sc.nu_in, prm.tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
-    const int t = tid >> 5;                       // this warp's error count
-    double* task = sc.tasks + (size_t)t * sc.task_stride;
-    uint8_t* cand = reinterpret_cast<uint8_t*>(task);
-    uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
-    locate_task(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n,
-                cand, bad, task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
-  }
-  __syncthreads();
-  const int ok = locate_epilogue(cta, tb, n, prm.m, prm.s, sc.forced, sc.recs, sc.flags, n, sc.mask_l, &s_t_acc, sc.rows_l,
-                                 &s_n_rec, sc.coeff_l, sc.trusted, sc.tasks);
-  // write the group's results: mask, recovery rows as global node indices, weights
-  const int n_rec = s_n_rec;
-  for (int k = tid; k < n; k += n_threads) prm.mask[row0 + k] = sc.mask_l[k];
-  for (int j = tid; j < n_rec; j += n_threads) prm.rec_rows[row0 + j] = sc.rows_l[j] + row0;
-  for (int i = tid; i < n_rec * prm.m; i += n_threads) prm.coeff[(size_t)row0 * prm.m + i] = sc.coeff_l[i];
-  if (tid == 0) {
-    prm.n_rec[g] = n_rec;
-    prm.t_acc[g] = s_t_acc;
-    if (!ok) atomicOr(prm.status, kStatusUndecodable);
+    const int ok = locate_epilogue(cta, tb, n, prm.m, prm.s, sc.forced, sc.recs, sc.flags, n, sc.mask_l, &s_t_acc, sc.rows_l,
+                                   &s_n_rec, sc.coeff_l, sc.trusted, sc.tasks);
+    if (pass == 0) {
+      __syncthreads();
+      continue;
+    }
+    // write the group's results: mask, recovery rows as global node indices, weights
+    const int n_rec = s_n_rec;
+    for (int k = tid; k < n; k += n_threads) prm.mask[row0 + k] = sc.mask_l[k];
+    for (int j = tid; j < n_rec; j += n_threads) prm.rec_rows[row0 + j] = sc.rows_l[j] + row0;
+    for (int i = tid; i < n_rec * prm.m; i += n_threads) prm.coeff[(size_t)row0 * prm.m + i] = sc.coeff_l[i];
+    if (tid == 0) {
+      prm.n_rec[g] = n_rec;
+      prm.t_acc[g] = s_t_acc;
+      if (!ok) atomicOr(prm.status, kStatusUndecodable);
+    }
   }
 }
 
@@ -253,9 +276,11 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   prm.rec_rows = plan->d_rec_rows;
   prm.coeff = plan->d_coeff;
   prm.status = plan->d_status;
+  prm.tile_counter = plan->d_tile_counter;
   size_t need = locate_ws_doubles(plan->max_group, plan->m, plan->K, plan->s) * sizeof(double);
   if (need > plan->locate_ws_stride * sizeof(double)) return SOLON_ERR_INTERNAL;
   prm.use_smem = need <= 128 * 1024 ? 1 : 0;
+  prm.warm = (plan->max_group <= 64 && plan->s <= 5) ? 1 : 0;
   size_t smem = prm.use_smem ? need : 0;
   const size_t tables = (2 * (size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
   prm.stage_tables = (prm.use_smem && smem + tables <= 200 * 1024) ? 1 : 0;

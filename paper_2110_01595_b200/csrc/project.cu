@@ -197,6 +197,9 @@ static int launch_project_k(solon_plan* plan, const float* received, double* rho
   SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, project_kernel<K>, kProjThreads, smem));
   int grid = plan->num_sms * (per_sm < 1 ? 1 : per_sm);
   if (grid > plan->proj_grid) grid = plan->proj_grid;
+  // leave one slot per group free: the locator's CTAs (launched as dependents) then become resident while this
+  // kernel streams and use the time to stage their tables and fetch their code
+  if (plan->q <= plan->num_sms && grid >= 4 * plan->q) grid -= plan->q;
   int64_t range_len = (plan->d_c + grid - 1) / grid;
   range_len = (range_len + 3) / 4 * 4;
   if (range_len < tile_cols) tile_cols = (int)range_len;

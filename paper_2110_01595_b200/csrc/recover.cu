@@ -35,20 +35,24 @@ __device__ __forceinline__ void load_tables(const RecoverParams& prm, Acc* coeff
   __syncthreads();
 }
 
-// Packed list of the rows the recovery reads (all groups, in group order) and their weights.
+// The locator's tables, brought on chip in ONE parallel round trip (every load is independent of every other),
+// then the list of the table slots in use (all groups, in group order) built from the on-chip copies:
+//   coeff_s[slot * m + l], rows_s[slot] for slot in [group_start[g], group_start[g] + n_rec[g]); slots_s[i] = i-th
+//   slot in use.  Returns the number of slots in use.  start_s, n_rec_s: q + 1 and q ints of scratch.
 template <typename Acc>
-__device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_p, Acc* coeff_p, int* count_s) {
-  // positions by a serial prefix over the groups (q is small), then a parallel copy
-  if (threadIdx.x == 0) {
-    int total = 0;
-    for (int g = 0; g < prm.q; ++g) total += prm.n_rec[g];
-    *count_s = total;
-  }
-  for (int g = 0, base = 0; g < prm.q; ++g) {
-    const int n = prm.n_rec[g], src = prm.group_start[g];
-    for (int j = threadIdx.x; j < n; j += blockDim.x) rows_p[base + j] = prm.rec_rows[src + j];
-    for (int i = threadIdx.x; i < n * prm.m; i += blockDim.x) coeff_p[(size_t)base * prm.m + i] = (Acc)prm.coeff[(size_t)src * prm.m + i];
-    base += n;
+__device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_s, Acc* coeff_s, int* slots_s, int* start_s,
+                                           int* n_rec_s, int* count_s) {
+  for (int i = threadIdx.x; i < prm.P * prm.m; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
+  for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
+  for (int i = threadIdx.x; i <= prm.q; i += blockDim.x) start_s[i] = prm.group_start[i];
+  for (int i = threadIdx.x; i < prm.q; i += blockDim.x) n_rec_s[i] = prm.n_rec[i];
+  __syncthreads();
+  for (int g = threadIdx.x; g < prm.q; g += blockDim.x) {
+    int base = 0;
+    for (int o = 0; o < g; ++o) base += n_rec_s[o];
+    const int n = n_rec_s[g], src = start_s[g];
+    for (int j = 0; j < n; ++j) slots_s[base + j] = src + j;
+    if (g == prm.q - 1) *count_s = base + n;
   }
   __syncthreads();
   return *count_s;
@@ -64,6 +68,7 @@ struct RecoverPipe {
   int row_batch;     // rows per stage
   int stages;
   int slot_floats;   // shared-memory floats per row slot (multiple of 4)
+  unsigned long long* tile_counter;   // next tile to hand out; zero at launch
   int* status;
 };
 
@@ -78,12 +83,17 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + pp.stages;
-  int* abort_flag = reinterpret_cast<int*>(empty_bar + pp.stages);
+  long long* tile_of = reinterpret_cast<long long*>(empty_bar + pp.stages);   // per stage: tile of the batch it holds
+  int* b0_of = reinterpret_cast<int*>(tile_of + pp.stages);                  // per stage: first row of that batch
+  int* abort_flag = b0_of + pp.stages;
   int* count_s = abort_flag + 1;
   // every region starts on a 16-byte boundary (128-bit shared loads, bulk-copy destinations)
   Acc* coeff_p = reinterpret_cast<Acc*>(smem_raw + 256);                                  // P x M
   int* rows_p = reinterpret_cast<int*>(smem_raw + 256 + recover_coeff_bytes(prm.P, M));   // P
-  float* out_all = reinterpret_cast<float*>(rows_p + ((prm.P + 3) & ~3));                 // 8 warps x 32 x M
+  int* slots_p = rows_p + ((prm.P + 3) & ~3);                                             // P
+  int* start_s = slots_p + ((prm.P + 3) & ~3);                                            // q + 1
+  int* n_rec_s = start_s + ((prm.q + 4) & ~3);                                            // q
+  float* out_all = reinterpret_cast<float*>(n_rec_s + ((prm.q + 3) & ~3));                // 8 warps x 32 x M
   float* ring = out_all + (size_t)(kRecConsumers / 32) * 32 * M;                          // 32 M floats: 128 M bytes
   const size_t stage_floats = (size_t)pp.row_batch * pp.slot_floats;
 
@@ -96,24 +106,36 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     pipe::fence_barrier_init();
   }
   pdl_wait();   // the locator's mask and table are complete and visible; nothing above touched global memory
-  const int n_rows = pack_tables(prm, rows_p, coeff_p, count_s);
+  const int n_rows = pack_tables(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
 
+  // Tiles are handed out through a global counter (zeroed by the locator kernel), not by a fixed stride: SMs do
+  // not all draw the same bandwidth (those of the fuller GPCs get about a third less), and with equal shares the
+  // slow ones finish long after the rest.  The producer announces every batch's tile in tile_of[stage]; a
+  // negative tile ends the stream.
   if (tid >= kRecConsumers) {
     const int lane = tid - kRecConsumers;
     uint32_t it = 0;
-    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    long long tile = 0;
+    if (lane == 0) tile = (long long)atomicAdd(pp.tile_counter, 1ULL);
+    tile = __shfl_sync(0xffffffffu, tile, 0);
+    while (tile < n_tiles) {
       const int64_t c0 = tile * kTileChunks;
       int64_t c1 = c0 + kTileChunks;
       if (c1 > prm.d_c) c1 = prm.d_c;
-      for (int b0 = 0; b0 < n_rows; b0 += pp.row_batch, ++it) {
+      int b0 = 0;
+      do {
         const int stage = it % pp.stages;
         const uint32_t phase = (it / pp.stages) & 1;
         if (it >= (uint32_t)pp.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
         const int nb = min(pp.row_batch, n_rows - b0);
+        if (lane == 0) {
+          tile_of[stage] = tile;
+          b0_of[stage] = b0;
+        }
         if (lane < nb) {
-          const int64_t first = (int64_t)rows_p[b0 + lane] * prm.d_c + c0;
+          const int64_t first = (int64_t)rows_p[slots_p[b0 + lane]] * prm.d_c + c0;
           const int64_t last = first + (c1 - c0);
           const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
           int64_t a1 = (last + 3) & ~(int64_t)3;
@@ -131,7 +153,19 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
         } else {
           pipe::mbar_arrive(&full_bar[stage]);
         }
-      }
+        b0 += pp.row_batch;
+        ++it;
+      } while (b0 < n_rows);
+      // claim late: a tile claimed ahead of time is a tile a faster SM can no longer take
+      if (lane == 0) tile = (long long)atomicAdd(pp.tile_counter, 1ULL);
+      tile = __shfl_sync(0xffffffffu, tile, 0);
+    }
+    {
+      const int stage = it % pp.stages;
+      const uint32_t phase = (it / pp.stages) & 1;
+      if (it >= (uint32_t)pp.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
+      if (lane == 0) tile_of[stage] = -1;
+      pipe::mbar_arrive(&full_bar[stage]);
     }
     if (*(volatile int*)abort_flag) pipe::drain_delay();
     return;
@@ -140,43 +174,47 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
   const int lane = tid & 31, warp = tid >> 5;
   float* out_s = out_all + (size_t)warp * 32 * M;
   const int dc_mod4 = (int)(prm.d_c & 3);
-  uint32_t it = 0;
-  for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+  Acc acc[CPT][M];
+  bool ok[CPT];
+  for (uint32_t it = 0;; ++it) {
+    const int stage = it % pp.stages;
+    const uint32_t phase = (it / pp.stages) & 1;
+    pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
+    const long long tile = *(volatile long long*)&tile_of[stage];
+    if (tile < 0 || *(volatile int*)abort_flag) break;
+    const int b0 = *(volatile int*)&b0_of[stage];
     const int64_t c0 = tile * kTileChunks;
-    Acc acc[CPT][M];
+    if (b0 == 0) {
 #pragma unroll
-    for (int i = 0; i < CPT; ++i)
+      for (int i = 0; i < CPT; ++i) {
 #pragma unroll
-      for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
-    bool ok[CPT];
-#pragma unroll
-    for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kRecConsumers < prm.d_c;
-
-    for (int b0 = 0; b0 < n_rows; b0 += pp.row_batch, ++it) {
-      const int stage = it % pp.stages;
-      const uint32_t phase = (it / pp.stages) & 1;
-      pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
-      const int nb = min(pp.row_batch, n_rows - b0);
-      const float* slot = ring + stage * stage_floats + tid;
-      for (int j = 0; j < nb; ++j) {
-        const int shift = ((((rows_p[b0 + j] & 3) * dc_mod4) + (int)(c0 & 3)) & 3);   // (row * d_c + c0) mod 4
-        const float* src = slot + shift;
-        Acc v[CPT];
-#pragma unroll
-        for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (Acc)src[i * kRecConsumers] : (Acc)0;
-        const Acc* cj = coeff_p + (size_t)(b0 + j) * M;
-#pragma unroll
-        for (int l = 0; l < M; ++l) {
-          const Acc c = cj[l];
-#pragma unroll
-          for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
-        }
-        slot += pp.slot_floats;
+        for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
+        ok[i] = c0 + tid + i * kRecConsumers < prm.d_c;
       }
-      __syncwarp();
-      if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
     }
-    // write-back: for each i the warp's 32 chunks are contiguous, 32 M floats starting on a 16-byte boundary
+    const int nb = min(pp.row_batch, n_rows - b0);
+    const float* slot = ring + stage * stage_floats + tid;
+    for (int j = 0; j < nb; ++j) {
+      const int sl = slots_p[b0 + j];
+      const int shift = ((((rows_p[sl] & 3) * dc_mod4) + (int)(c0 & 3)) & 3);   // (row * d_c + c0) mod 4
+      const float* src = slot + shift;
+      Acc v[CPT];
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (Acc)src[i * kRecConsumers] : (Acc)0;
+      const Acc* cj = coeff_p + (size_t)sl * M;
+#pragma unroll
+      for (int l = 0; l < M; ++l) {
+        const Acc c = cj[l];
+#pragma unroll
+        for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
+      }
+      slot += pp.slot_floats;
+    }
+    __syncwarp();
+    if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
+    if (b0 + pp.row_batch < n_rows) continue;
+    // last batch of the tile: write back; for each i the warp's 32 chunks are contiguous, 32 M floats starting
+    // on a 16-byte boundary
 #pragma unroll
     for (int i = 0; i < CPT; ++i) {
 #pragma unroll
@@ -198,7 +236,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
 
 // Any m: one thread per output coordinate (slower; used for compression ratios without a specialisation).
 __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverParams prm) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   double* coeff_s = reinterpret_cast<double*>(smem_raw);
   int* rows_s = reinterpret_cast<int*>(coeff_s + (size_t)prm.P * prm.m);
   int* start_s = rows_s + prm.P;
@@ -224,7 +262,8 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   pp.status = plan->d_status;
   pp.slot_floats = kTileChunks + 8;
   const size_t slot_bytes = (size_t)pp.slot_floats * 4;
-  const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + (size_t)((plan->P + 3) & ~3) * sizeof(int) +
+  const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + 2 * (size_t)((plan->P + 3) & ~3) * sizeof(int) +
+                       (size_t)(((plan->q + 4) & ~3) + ((plan->q + 3) & ~3)) * sizeof(int) +
                        (size_t)(kRecConsumers / 32) * 32 * M * sizeof(float);
   // the locator may select up to all P rows (large m) or as few as q m; batches of about 20 KB
   int row_batch = (int)((size_t)20 * 1024 / slot_bytes);
@@ -240,6 +279,12 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   int stages = 4;
   while (stages > 2 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --stages;
   while (row_batch > 1 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --row_batch;
+  {
+    // few tiles per CTA: a deep ring would claim most of them up front and leave the counter nothing to balance
+    const int64_t n_tiles_all = (plan->d_c + kTileChunks - 1) / kTileChunks;
+    const int batches_per_tile = (max_rows + row_batch - 1) / row_batch;
+    if (n_tiles_all < (int64_t)plan->num_sms * 4 * 16 && stages > batches_per_tile + 1) stages = batches_per_tile + 1;
+  }
   const size_t smem = fixed + (size_t)stages * row_batch * slot_bytes;
   if (smem > (size_t)226 * 1024) return SOLON_ERR_INVALID_ARG;
   pp.row_batch = row_batch;
@@ -253,6 +298,7 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   if (per_sm < 1) per_sm = 1;
   int64_t cap = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(tiles < cap ? tiles : cap);
+  pp.tile_counter = plan->d_tile_counter;
   return launch_dependent(kernel, dim3(grid), dim3(kRecPipeThreads), smem, plan->stream, prm, pp);
 }
 
@@ -270,17 +316,21 @@ int launch_recover(solon_plan* plan, const float* received, float* agg) {
   prm.rec_rows = plan->d_rec_rows;
   prm.coeff = plan->d_coeff;
   plan->launches += 1;
+#define SOLON_RECOVER_CASE(M_, CPT_, ACC_) \
+  case M_:                                 \
+    return launch_recover_m<M_, CPT_, ACC_>(plan, prm);
   switch (plan->m) {
-    case 1: return launch_recover_m<1, 4, float>(plan, prm);
-    case 2: return launch_recover_m<2, 4, float>(plan, prm);
-    case 3: return launch_recover_m<3, 4, float>(plan, prm);
-    case 4: return launch_recover_m<4, 4, float>(plan, prm);
-    case 5: return launch_recover_m<5, 4, float>(plan, prm);
-    case 6: return launch_recover_m<6, 2, float>(plan, prm);
-    case 8: return launch_recover_m<8, 2, double>(plan, prm);
-    case 10: return launch_recover_m<10, 2, double>(plan, prm);
+    SOLON_RECOVER_CASE(1, 4, float)
+    SOLON_RECOVER_CASE(2, 4, float)
+    SOLON_RECOVER_CASE(3, 4, float)
+    SOLON_RECOVER_CASE(4, 4, float)
+    SOLON_RECOVER_CASE(5, 4, float)
+    SOLON_RECOVER_CASE(6, 2, float)
+    SOLON_RECOVER_CASE(8, 2, double)
+    SOLON_RECOVER_CASE(10, 2, double)
     default: break;
   }
+#undef SOLON_RECOVER_CASE
   size_t smem = (size_t)plan->P * plan->m * sizeof(double) + (size_t)(plan->P + 2 * plan->q + 2) * sizeof(int);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(recover_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

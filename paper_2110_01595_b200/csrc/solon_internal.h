@@ -80,6 +80,7 @@ struct solon_plan {
   int* d_rec_rows;         // P   (global node index of the j-th recovery row of group g at start[g] + j)
   double* d_coeff;         // P x m
   int* d_status;           // [0] status bits of the last decode, [1] sticky bits (expired waits)
+  unsigned long long* d_tile_counter;   // the recovery kernel's next tile; the locator kernel zeroes it
 
   // optional per-kernel timing: events [0,1] around encode, [2..5] before/after the decode kernels
   int profiling;
