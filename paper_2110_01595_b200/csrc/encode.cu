@@ -36,6 +36,7 @@ struct EncodeParams {
   int stages;
   int slot_floats;        // shared-memory floats per row slot (multiple of 4)
   int64_t tiles_per_group;
+  unsigned long long* tile_counter;   // [0] next tile to hand out, [1] CTAs that have left; both zero at launch
   int* status;            // device status words: [1] collects wait-expiry bits
 };
 
@@ -219,7 +220,9 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + prm.stages;
-  int* abort_flag = reinterpret_cast<int*>(empty_bar + prm.stages);
+  long long* tile_of = reinterpret_cast<long long*>(empty_bar + prm.stages);   // per stage: tile of the batch it holds
+  int* b0_of = reinterpret_cast<int*>(tile_of + prm.stages);                  // per stage: first row of that batch
+  int* abort_flag = b0_of + prm.stages;
   Acc* w_s = reinterpret_cast<Acc*>(smem_raw + 256);                       // all P node scalars
   float* ring = reinterpret_cast<float*>(smem_raw + 256 + (((size_t)prm.P * sizeof(Acc) + 15) & ~(size_t)15));
   const size_t stage_floats = (size_t)prm.row_batch * prm.slot_floats;
@@ -237,10 +240,17 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 
   const int64_t total_tiles = prm.tiles_per_group * prm.q;
 
+  // Tiles are handed out through a global counter, not by a fixed stride: the SMs do not all draw the same
+  // bandwidth (those of the fuller GPCs get less), and with equal shares the slow ones finish long after the
+  // rest.  The producer announces every batch's tile in tile_of[stage]; a negative tile ends the stream.  The
+  // last CTA to leave puts the counters back to zero for the next launch.
   if (tid >= kEncConsumers) {
     const int lane = tid - kEncConsumers;
     uint32_t it = 0;
-    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    long long tile = 0;
+    if (lane == 0) tile = (long long)atomicAdd(prm.tile_counter, 1ULL);
+    tile = __shfl_sync(0xffffffffu, tile, 0);
+    while (tile < total_tiles) {
       const int g = (int)(tile / prm.tiles_per_group);
       const int64_t ct = tile - (int64_t)g * prm.tiles_per_group;
       const int row0 = prm.group_start[g], r_g = prm.group_start[g + 1] - row0;
@@ -252,6 +262,10 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
         const uint32_t phase = (it / prm.stages) & 1;
         if (it >= (uint32_t)prm.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, prm.status + 1);
         const int nb = min(prm.row_batch, r_g - b0);
+        if (lane == 0) {
+          tile_of[stage] = tile;
+          b0_of[stage] = b0;
+        }
         if (lane < nb) {
           const int64_t first = (int64_t)(row0 + b0 + lane) * prm.d + e0;
           const int64_t last = first + (e1 - e0);
@@ -272,59 +286,81 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
           pipe::mbar_arrive(&full_bar[stage]);
         }
       }
+      if (lane == 0) tile = (long long)atomicAdd(prm.tile_counter, 1ULL);
+      tile = __shfl_sync(0xffffffffu, tile, 0);
+    }
+    {
+      const int stage = it % prm.stages;
+      const uint32_t phase = (it / prm.stages) & 1;
+      if (it >= (uint32_t)prm.stages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, prm.status + 1);
+      if (lane == 0) tile_of[stage] = -1;
+      pipe::mbar_arrive(&full_bar[stage]);
+    }
+    if (lane == 0) {
+      __threadfence();   // this CTA's last claim is ordered before its departure
+      if (atomicAdd(prm.tile_counter + 1, 1ULL) == (unsigned long long)gridDim.x - 1) {
+        prm.tile_counter[0] = 0ULL;   // every CTA has made its last claim
+        prm.tile_counter[1] = 0ULL;
+      }
     }
     if (*(volatile int*)abort_flag) pipe::drain_delay();
     return;
   }
 
-  uint32_t it = 0;
   const int d_mod4 = (int)(prm.d & 3);
-  for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-    const int g = (int)(tile / prm.tiles_per_group);
-    const int64_t ct = tile - (int64_t)g * prm.tiles_per_group;
-    const int row0 = prm.group_start[g], r_g = prm.group_start[g + 1] - row0;
-    const int64_t e0 = ct * kTileFloats;
-    const int valid = (int)((prm.d - e0) < kTileFloats ? (prm.d - e0) : kTileFloats);
-    const bool full_tile = valid == kTileFloats;
-    Acc acc[CPT][M];
+  Acc acc[CPT][M];
+  int row0 = 0, r_g = 0, valid = 0;
+  int64_t e0 = 0, ct = 0;
+  for (uint32_t it = 0;; ++it) {
+    const int stage = it % prm.stages;
+    const uint32_t phase = (it / prm.stages) & 1;
+    pipe::mbar_wait(&full_bar[stage], phase, abort_flag, prm.status + 1);
+    const long long tile = *(volatile long long*)&tile_of[stage];
+    if (tile < 0 || *(volatile int*)abort_flag) break;
+    const int b0 = *(volatile int*)&b0_of[stage];
+    if (b0 == 0) {
+      const int g = (int)(tile / prm.tiles_per_group);
+      ct = tile - (int64_t)g * prm.tiles_per_group;
+      row0 = prm.group_start[g];
+      r_g = prm.group_start[g + 1] - row0;
+      e0 = ct * kTileFloats;
+      valid = (int)((prm.d - e0) < kTileFloats ? (prm.d - e0) : kTileFloats);
 #pragma unroll
-    for (int i = 0; i < CPT; ++i)
+      for (int i = 0; i < CPT; ++i)
 #pragma unroll
-      for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
-
-    for (int b0 = 0; b0 < r_g; b0 += prm.row_batch, ++it) {
-      const int stage = it % prm.stages;
-      const uint32_t phase = (it / prm.stages) & 1;
-      pipe::mbar_wait(&full_bar[stage], phase, abort_flag, prm.status + 1);
-      const int nb = min(prm.row_batch, r_g - b0);
-      const float* slot = ring + stage * stage_floats + tid * M;
-      int shift = ((((row0 + b0) & 3) * d_mod4) + (int)(e0 & 3)) & 3;        // (row * d + e0) mod 4
-      if (full_tile) {
-        for (int j = 0; j < nb; ++j) {
-          const float* src = slot + shift;
-#pragma unroll
-          for (int i = 0; i < CPT; ++i)
-#pragma unroll
-            for (int l = 0; l < M; ++l) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
-          slot += prm.slot_floats;
-          shift = (shift + d_mod4) & 3;
-        }
-      } else {
-        for (int j = 0; j < nb; ++j) {
-          const float* src = slot + shift;
-#pragma unroll
-          for (int i = 0; i < CPT; ++i)
-#pragma unroll
-            for (int l = 0; l < M; ++l)
-              if ((tid + i * kEncConsumers) * M + l < valid) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
-          slot += prm.slot_floats;
-          shift = (shift + d_mod4) & 3;
-        }
-      }
-      __syncwarp();
-      if ((tid & 31) == 0) pipe::mbar_arrive(&empty_bar[stage]);
+        for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
     }
+    const bool full_tile = valid == kTileFloats;
+    const int nb = min(prm.row_batch, r_g - b0);
+    const float* slot = ring + stage * stage_floats + tid * M;
+    int shift = ((((row0 + b0) & 3) * d_mod4) + (int)(e0 & 3)) & 3;        // (row * d + e0) mod 4
+    if (full_tile) {
+      for (int j = 0; j < nb; ++j) {
+        const float* src = slot + shift;
+#pragma unroll
+        for (int i = 0; i < CPT; ++i)
+#pragma unroll
+          for (int l = 0; l < M; ++l) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
+        slot += prm.slot_floats;
+        shift = (shift + d_mod4) & 3;
+      }
+    } else {
+      for (int j = 0; j < nb; ++j) {
+        const float* src = slot + shift;
+#pragma unroll
+        for (int i = 0; i < CPT; ++i)
+#pragma unroll
+          for (int l = 0; l < M; ++l)
+            if ((tid + i * kEncConsumers) * M + l < valid) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
+        slot += prm.slot_floats;
+        shift = (shift + d_mod4) & 3;
+      }
+    }
+    __syncwarp();
+    if ((tid & 31) == 0) pipe::mbar_arrive(&empty_bar[stage]);
+    if (b0 + prm.row_batch < r_g) continue;
 
+    // last batch of the tile: one Horner evaluation per node of the group, coalesced stores
     const int64_t c0 = ct * kTileChunks;
     float* out = prm.coded + (int64_t)row0 * prm.d_c + c0 + tid;
     bool ok[CPT];
@@ -439,6 +475,7 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   prm.d_c = plan->d_c;
   prm.total_floats = (int64_t)plan->P * plan->d;
   prm.status = plan->d_status;
+  prm.tile_counter = plan->d_tile_counter + 1;
   plan->launches += 1;
   switch (plan->m) {
     case 1: return launch_encode_direct<1, 4, float, 3>(plan, prm);

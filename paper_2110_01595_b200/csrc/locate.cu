@@ -26,6 +26,10 @@ struct LocateParams {
   double* ws_global;     // q x ws_stride doubles, used when shared memory is too small
   size_t ws_stride;
   int use_smem;
+  const double* bunch_sums;   // n_bunches x (K + 1) x P partial sums of the projection kernel (rho rows, then nu)
+  int n_bunches;              // 0: rho and nu are final
+  double* rho_w;              // with n_bunches > 0 the sums are also written here (K x P) and to nu_w (P)
+  double* nu_w;
   unsigned long long* tile_counter;   // work counter of the recovery kernel, zeroed here
   int warm;               // run the solver once on made-up values before waiting for the projections
   int stage_tables;      // copy the group's tables to shared memory (they follow the workspace)
@@ -89,6 +93,8 @@ SOLON_HD static inline GroupScratch carve(double* ws, int n, int m, int K, int s
 // at the same time with warp-level synchronisation only; afterwards the whole CTA picks the smallest
 // accepted count, writes the group's part of the mask and builds the recovery table.  No CTA waits on
 // another one.
+constexpr int kGatherBatch = 20;   // bunch sums fetched at once per column (the projection kernel leaves 37 on 148 SMs: two rounds)
+
 __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocateParams prm) {
   extern __shared__ __align__(16) double smem_ws[];
   const int g = blockIdx.x;
@@ -148,8 +154,36 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       }
     } else {
       // one parallel round trip brings the group's projected values on chip
+      if (prm.n_bunches > 0) {
+        // last level of the projection kernel's reduction, for this group's columns only: a thread fetches all
+        // bunch sums of its column at once and adds them in bunch order.  (Pass 0 runs this too, on whatever
+        // the buffer holds, only to have the code on chip; its values are replaced below.)
+        const int n_cols = (prm.K + 1) * n;
+        const size_t n_acc = (size_t)(prm.K + 1) * prm.P;
+        for (int c = tid; c < n_cols; c += n_threads) {
+          const int which = c / n, i = c - which * n;
+          const double* src = prm.bunch_sums + (size_t)which * prm.P + row0 + i;
+          double acc = 0.0;
+          for (int b0 = 0; b0 < prm.n_bunches; b0 += kGatherBatch) {
+            double v[kGatherBatch];
+#pragma unroll
+            for (int u = 0; u < kGatherBatch; ++u) v[u] = b0 + u < prm.n_bunches ? __ldcg(src + (size_t)(b0 + u) * n_acc) : 0.0;
+#pragma unroll
+            for (int u = 0; u < kGatherBatch; ++u) acc += v[u];
+          }
+          if (which < prm.K) {
+            sc.rho_in[(size_t)which * n + i] = acc;
+            if (pass == 1) prm.rho_w[(size_t)which * prm.P + row0 + i] = acc;
+          } else {
+            sc.nu_in[i] = acc;
+            if (pass == 1) prm.nu_w[row0 + i] = acc;
+          }
+        }
+        __syncthreads();
+      }
       for (int i = tid; i < n; i += n_threads) {
         if (pass == 1) {
+          if (prm.n_bunches > 0) continue;
           sc.nu_in[i] = prm.nu[row0 + i];
           for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
         } else {
@@ -165,8 +199,9 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       double* task = sc.tasks + (size_t)t * sc.task_stride;
       uint8_t* cand = reinterpret_cast<uint8_t*>(task);
       uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
-      locate_task(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n,
-                  cand, bad, task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
+      if (t <= prm.s)      // warps beyond s + 1 only help with the CTA-wide steps
+        locate_task(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n,
+                    cand, bad, task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
     }
     __syncthreads();
     const int ok = locate_epilogue(cta, tb, n, prm.m, prm.s, sc.forced, sc.recs, sc.flags, n, sc.mask_l, &s_t_acc, sc.rows_l,
@@ -261,6 +296,12 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   prm.w = plan->d_w;
   prm.rho = rho ? rho : plan->d_rho;
   prm.nu = nu ? nu : plan->d_nu;
+  // the decode proper: the projection kernel stopped one level short and left its bunch sums
+  const bool fused = !rho && !nu && plan->s > 0 && plan->proj_bunches > 0;
+  prm.bunch_sums = fused ? plan->proj_bunch_sums : nullptr;
+  prm.n_bunches = fused ? plan->proj_bunches : 0;
+  prm.rho_w = plan->d_rho;
+  prm.nu_w = plan->d_nu;
   prm.qb = plan->d_qb;
   prm.hm = plan->d_hm;
   prm.qb_off = plan->d_qb_off;
@@ -291,7 +332,10 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   plan->launches += 1;
-  return launch_dependent(locate_kernel, dim3(plan->q), dim3(32 * (plan->s + 1)), smem, plan->stream, prm);
+  // one warp per error count, at least four for the CTA-wide steps (four still fit, at 128 registers a thread, in the
+  // slot the projection kernel leaves free, so the CTA is resident early)
+  const int warps = plan->s + 1 < 4 ? 4 : plan->s + 1;
+  return launch_dependent(locate_kernel, dim3(plan->q), dim3(32 * warps), smem, plan->stream, prm);
 }
 
 }  // namespace solon

@@ -254,14 +254,14 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     if ((rc = dev_alloc(&p->d_rec_rows, P))) break;
     if ((rc = dev_alloc(&p->d_coeff, (size_t)P * m))) break;
     if ((rc = dev_alloc(&p->d_status, 2))) break;
-    if ((rc = dev_alloc(&p->d_tile_counter, 1))) break;
+    if ((rc = dev_alloc(&p->d_tile_counter, 4))) break;
     cudaError_t e = cudaSuccess;
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_start, start.data(), (q + 1) * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_of, p->group_of.data(), P * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_w, p->w.data(), P * sizeof(double), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, ((size_t)p->proj_grid / 16 + 2) * sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 2 * sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(p->d_tile_counter, 0, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(p->d_tile_counter, 0, 4 * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(p->d_n_rec, 0, q * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_t_acc, 0, q * sizeof(int));
     if (e != cudaSuccess) { (void)cudaGetLastError(); rc = SOLON_ERR_CUDA; break; }

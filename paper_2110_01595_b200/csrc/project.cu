@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
                                                                int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
                                                                int tile_cols, double* __restrict__ partials,
                                                                double* __restrict__ rho_out, double* __restrict__ nu_out,
-                                                               unsigned int* ticket) {
+                                                               unsigned int* ticket, int final_reduce) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* fs = reinterpret_cast<double*>(smem_raw);            // K x tile_cols
   double* sacc = fs + (size_t)K * tile_cols;                  // P x (K + 1)
@@ -162,10 +162,20 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
   if (s_ticket != members - 1) return;
   __threadfence();
   for (int i = tid; i < n_acc; i += kProjThreads) {
+    double v[kProjBunch];
+#pragma unroll
+    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b)     // all loads in flight at once, then a fixed order
+      v[b] = b < members ? __ldcg(partials + (size_t)(first + b) * n_acc + i) : 0.0;
     double acc = 0.0;
-#pragma unroll 4
-    for (unsigned int b = 0; b < members; ++b) acc += __ldcg(partials + (size_t)(first + b) * n_acc + i);
+#pragma unroll
+    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b) acc += v[b];
     bunch_sums[(size_t)bunch * n_acc + i] = acc;
+  }
+  if (!final_reduce) {
+    // the locator kernel adds the bunch sums itself (it needs them on chip anyway): nothing more to do here
+    __syncthreads();
+    if (tid == 0) ticket[1 + bunch] = 0u;   // ready for the next decode
+    return;
   }
   __threadfence();
   __syncthreads();
@@ -187,7 +197,7 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
 }
 
 template <int K>
-static int launch_project_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
+static int launch_project_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out, int final_reduce) {
   int tile_cols = K <= 2 ? 2048 : 1024;
   size_t smem = (size_t)K * tile_cols * sizeof(double) + (size_t)(K + 1) * plan->P * sizeof(double);
   if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
@@ -205,20 +215,24 @@ static int launch_project_k(solon_plan* plan, const float* received, double* rho
   if (range_len < tile_cols) tile_cols = (int)range_len;
   project_kernel<K><<<grid, kProjThreads, smem, plan->stream>>>(
       received, plan->d_f, plan->f_pitch, plan->P, plan->d_c, range_len, tile_cols, plan->d_partials, rho_out,
-      nu_out, plan->d_proj_ticket);
+      nu_out, plan->d_proj_ticket, final_reduce);
+  plan->proj_bunches = final_reduce ? 0 : (grid + kProjBunch - 1) / kProjBunch;
+  plan->proj_bunch_sums = plan->d_partials + (size_t)grid * (K + 1) * plan->P;
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }
 
 int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
+  // no output buffers: the decode proper, whose locator kernel adds the last level of partial sums itself
+  const int final_reduce = (rho_out || nu_out) ? 1 : 0;
   if (!rho_out) rho_out = plan->d_rho;
   if (!nu_out) nu_out = plan->d_nu;
   plan->launches += 1;
   switch (plan->K) {
-    case 1: return launch_project_k<1>(plan, received, rho_out, nu_out);
-    case 2: return launch_project_k<2>(plan, received, rho_out, nu_out);
-    case 3: return launch_project_k<3>(plan, received, rho_out, nu_out);
-    case 4: return launch_project_k<4>(plan, received, rho_out, nu_out);
+    case 1: return launch_project_k<1>(plan, received, rho_out, nu_out, final_reduce);
+    case 2: return launch_project_k<2>(plan, received, rho_out, nu_out, final_reduce);
+    case 3: return launch_project_k<3>(plan, received, rho_out, nu_out, final_reduce);
+    case 4: return launch_project_k<4>(plan, received, rho_out, nu_out, final_reduce);
     default: return SOLON_ERR_INVALID_ARG;
   }
 }
@@ -277,7 +291,7 @@ static int launch_project_noalloc_k(const float* received, const float* f, int64
   // the tickets must start at zero; the partial sums are fully rewritten by every launch
   SOLON_CUDA_TRY(cudaMemsetAsync(ticket, 0, kNoAllocTicketBytes, stream));
   project_kernel<K><<<grid, kProjThreads, smem, stream>>>(received, f, f_pitch, P, d_c, range_len, tile_cols, partials,
-                                                          rho, nu, ticket);
+                                                          rho, nu, ticket, 1);
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }

@@ -68,6 +68,8 @@ struct solon_plan {
   // projection workspace
   int proj_grid;           // CTAs of the projection kernel = number of partial sums
   double* d_partials;      // proj_grid x (K + 1) x P
+  int proj_bunches;        // > 0: the last projection launch left this many bunch sums for the locator to add
+  const double* proj_bunch_sums;   // proj_bunches x (K + 1) x P
   double* d_rho;           // K x P
   double* d_nu;            // P
   unsigned int* d_proj_ticket;   // 1
@@ -80,7 +82,8 @@ struct solon_plan {
   int* d_rec_rows;         // P   (global node index of the j-th recovery row of group g at start[g] + j)
   double* d_coeff;         // P x m
   int* d_status;           // [0] status bits of the last decode, [1] sticky bits (expired waits)
-  unsigned long long* d_tile_counter;   // the recovery kernel's next tile; the locator kernel zeroes it
+  unsigned long long* d_tile_counter;   // [0] the recovery kernel's next tile (the locator kernel zeroes it);
+                                        // [1], [2] the encode kernel's next tile and departed CTAs (it zeroes them itself)
 
   // optional per-kernel timing: events [0,1] around encode, [2..5] before/after the decode kernels
   int profiling;
