@@ -1,15 +1,16 @@
 // Detection projections (Section 3.4): rho[kappa][k] = f_kappa . R_k for the K random vectors f_kappa
 // and all P received rows, plus the row energies nu[k] = ||R_k||^2 that scale the locator's tolerance.
 //
-// One pass over the P x d_c received matrix.  Every CTA owns one contiguous range of the chunk axis,
-// walks it in tiles, keeps the tile of f in shared memory as float64 and lets each warp stream its own
-// rows (two at a time) against it, so each received byte is read once and f is read once per CTA.
-// Products are exact in float64 and accumulated in float64; nu is accumulated in float32 per lane and
-// in float64 across lanes and tiles.  Per-CTA partial sums go to global memory and are added in a fixed
-// order by the last CTAs to finish (atomic tickets, no waiting), so results are bit-reproducible.
+// One pass over the P x d_c received matrix.  Every CTA owns one contiguous range of the chunk axis.
+// Two forms: the plan's decode uses the streaming kernel (rows and f brought through a shared-memory ring by
+// bulk copies, float32 products in short runs, float64 sums: see project_pipe_kernel); the entry point that
+// allocates nothing uses the direct kernel (each warp loads its own rows, the tile of f in shared memory as
+// float64, every product and sum in float64).  Per-CTA partial sums go to global memory and are added in a
+// fixed order by the last CTAs to finish (atomic tickets, no waiting), so results are bit-reproducible.
 #include <mutex>
 
 #include "solon_internal.h"
+#include "stream_pipe.cuh"
 
 namespace solon {
 
@@ -29,6 +30,59 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
+// Two-level, fixed-order reduction of the per-CTA partial sums with atomic tickets (nobody waits): every CTA
+// has written its n_acc sums to partials[blockIdx.x]; the last CTA of every bunch of kProjBunch adds that
+// bunch, and (final_reduce) the last bunch adds the bunch sums into rho_out / nu_out.  Called by all threads.
+__device__ __forceinline__ void reduce_partials(double* __restrict__ partials, int n_acc, int KP, double* __restrict__ rho_out,
+                                                double* __restrict__ nu_out, unsigned int* ticket, int final_reduce) {
+  __shared__ unsigned int s_ticket;
+  const int tid = threadIdx.x, n_threads = blockDim.x;
+  const unsigned int bunch = blockIdx.x / kProjBunch;
+  const unsigned int n_bunches = (gridDim.x + kProjBunch - 1) / kProjBunch;
+  const unsigned int first = bunch * kProjBunch;
+  const unsigned int members = min((unsigned int)kProjBunch, gridDim.x - first);
+  double* bunch_sums = partials + (size_t)gridDim.x * n_acc;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_ticket = atomicAdd(ticket + 1 + bunch, 1u);
+  __syncthreads();
+  if (s_ticket != members - 1) return;
+  __threadfence();
+  for (int i = tid; i < n_acc; i += n_threads) {
+    double v[kProjBunch];
+#pragma unroll
+    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b)     // all loads in flight at once, then a fixed order
+      v[b] = b < members ? __ldcg(partials + (size_t)(first + b) * n_acc + i) : 0.0;
+    double acc = 0.0;
+#pragma unroll
+    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b) acc += v[b];
+    bunch_sums[(size_t)bunch * n_acc + i] = acc;
+  }
+  if (!final_reduce) {
+    // the locator kernel adds the bunch sums itself (it needs them on chip anyway): nothing more to do here
+    __syncthreads();
+    if (tid == 0) ticket[1 + bunch] = 0u;   // ready for the next decode
+    return;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    ticket[1 + bunch] = 0u;   // ready for the next decode
+    s_ticket = atomicAdd(ticket, 1u);
+  }
+  __syncthreads();
+  if (s_ticket != n_bunches - 1) return;
+  __threadfence();
+  for (int i = tid; i < n_acc; i += n_threads) {
+    double acc = 0.0;
+#pragma unroll 4
+    for (unsigned int b = 0; b < n_bunches; ++b) acc += __ldcg(bunch_sums + (size_t)b * n_acc + i);
+    if (i < KP) rho_out[i] = acc;
+    else nu_out[i - KP] = acc;
+  }
+  if (tid == 0) *ticket = 0u;
+}
+
 template <int K>
 __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* __restrict__ R, const float* __restrict__ f,
                                                                int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
@@ -38,7 +92,6 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* fs = reinterpret_cast<double*>(smem_raw);            // K x tile_cols
   double* sacc = fs + (size_t)K * tile_cols;                  // P x (K + 1)
-  __shared__ unsigned int s_ticket;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_acc = (K + 1) * P;
   pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading rho
@@ -148,74 +201,228 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
   __syncthreads();
   double* mine = partials + (size_t)blockIdx.x * n_acc;
   for (int i = tid; i < n_acc; i += kProjThreads) mine[i] = sacc[i];
-  // Two-level, fixed-order reduction of the per-CTA partial sums with atomic tickets (nobody waits):
-  // the last CTA of every bunch of kProjBunch adds that bunch, the last bunch adds the bunch sums.
-  const unsigned int bunch = blockIdx.x / kProjBunch;
-  const unsigned int n_bunches = (gridDim.x + kProjBunch - 1) / kProjBunch;
-  const unsigned int first = bunch * kProjBunch;
-  const unsigned int members = min((unsigned int)kProjBunch, gridDim.x - first);
-  double* bunch_sums = partials + (size_t)gridDim.x * n_acc;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_ticket = atomicAdd(ticket + 1 + bunch, 1u);
-  __syncthreads();
-  if (s_ticket != members - 1) return;
-  __threadfence();
-  for (int i = tid; i < n_acc; i += kProjThreads) {
-    double v[kProjBunch];
+  reduce_partials(partials, n_acc, K * P, rho_out, nu_out, ticket, final_reduce);
+}
+
+// ---- streaming form: rows and f come through shared memory by bulk copies ------------------------------------
+//
+// A producer warp moves, per stage, one column slice of up to kPipeRows received rows plus the same slice of the
+// K projection vectors into a shared-memory ring (cp.async.bulk, completion on an mbarrier), so hundreds of KB
+// per SM are in flight without occupying registers.  The P rows are cut into equal batches of at most kPipeRows;
+// within a batch consumer warp w owns rows w, w + 8, w + 16, w + 24 (those that exist), walks the slice 32 columns
+// at a time reusing each f value for all its rows, and keeps its sums across all slices of the CTA's column range:
+// products and short runs (8 steps) in float32, everything else in float64.  The rounding this adds (at most
+// 8 * 2^-24 of sum |f_p R_kp|, the size of the float32 rounding the coded vectors already carry) is a hundred times
+// below the locator's tolerance.  A row is summed by exactly one warp in a fixed order: bit-reproducible.
+constexpr int kPipeRows = 32;                       // rows per stage: up to four per consumer warp
+constexpr int kPipeConsumers = 256;
+constexpr int kPipeWarps = kPipeConsumers / 32;
+constexpr int kPipeThreads = kPipeConsumers + 32;   // + one producer warp
+constexpr int kPipeStages = 2;
+
+struct ProjPipe {
+  int slice_cols;     // columns per stage (multiple of 32)
+  int slot_floats;    // slice_cols + 8: room for the alignment shift and the rounded-up end
+  int batch_rows;     // rows per batch (<= kPipeRows), the same for all batches but the last
+  int* status;
+};
+
+// One slice for the NR rows of this warp: rows[j] point at column 0 of the slice in the warp's j-th row.
+template <int K, int NR>
+__device__ __forceinline__ void pipe_consume(const float* const* rows, const float* fs, int slot_floats, int cols, int lane,
+                                             double (*rho)[K], double* nu) {
+  for (int c = lane; c < cols; c += 8 * 32) {
+    float sr[NR][K], sn[NR];
 #pragma unroll
-    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b)     // all loads in flight at once, then a fixed order
-      v[b] = b < members ? __ldcg(partials + (size_t)(first + b) * n_acc + i) : 0.0;
-    double acc = 0.0;
+    for (int j = 0; j < NR; ++j) {
+      sn[j] = 0.f;
 #pragma unroll
-    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b) acc += v[b];
-    bunch_sums[(size_t)bunch * n_acc + i] = acc;
+      for (int kappa = 0; kappa < K; ++kappa) sr[j][kappa] = 0.f;
+    }
+    const int steps = (cols - c + 31) / 32;      // 8 except at the ragged end of the range
+    if (steps >= 8) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int cc = c + u * 32;
+        float fv[K];
+#pragma unroll
+        for (int kappa = 0; kappa < K; ++kappa) fv[kappa] = fs[(size_t)kappa * slot_floats + cc];
+#pragma unroll
+        for (int j = 0; j < NR; ++j) {
+          const float v = rows[j][cc];
+#pragma unroll
+          for (int kappa = 0; kappa < K; ++kappa) sr[j][kappa] = fmaf(fv[kappa], v, sr[j][kappa]);
+          sn[j] = fmaf(v, v, sn[j]);
+        }
+      }
+    } else {
+      for (int cc = c; cc < cols; cc += 32) {
+        float fv[K];
+#pragma unroll
+        for (int kappa = 0; kappa < K; ++kappa) fv[kappa] = fs[(size_t)kappa * slot_floats + cc];
+#pragma unroll
+        for (int j = 0; j < NR; ++j) {
+          const float v = rows[j][cc];
+#pragma unroll
+          for (int kappa = 0; kappa < K; ++kappa) sr[j][kappa] = fmaf(fv[kappa], v, sr[j][kappa]);
+          sn[j] = fmaf(v, v, sn[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < NR; ++j) {
+#pragma unroll
+      for (int kappa = 0; kappa < K; ++kappa) rho[j][kappa] += (double)sr[j][kappa];
+      nu[j] += (double)sn[j];
+    }
   }
-  if (!final_reduce) {
-    // the locator kernel adds the bunch sums itself (it needs them on chip anyway): nothing more to do here
-    __syncthreads();
-    if (tid == 0) ticket[1 + bunch] = 0u;   // ready for the next decode
-    return;
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    ticket[1 + bunch] = 0u;   // ready for the next decode
-    s_ticket = atomicAdd(ticket, 1u);
-  }
-  __syncthreads();
-  if (s_ticket != n_bunches - 1) return;
-  __threadfence();
-  for (int i = tid; i < n_acc; i += kProjThreads) {
-    double acc = 0.0;
-#pragma unroll 4
-    for (unsigned int b = 0; b < n_bunches; ++b) acc += __ldcg(bunch_sums + (size_t)b * n_acc + i);
-    if (i < K * P) rho_out[i] = acc;
-    else nu_out[i - K * P] = acc;
-  }
-  if (tid == 0) *ticket = 0u;
 }
 
 template <int K>
-static int launch_project_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out, int final_reduce) {
-  int tile_cols = K <= 2 ? 2048 : 1024;
-  size_t smem = (size_t)K * tile_cols * sizeof(double) + (size_t)(K + 1) * plan->P * sizeof(double);
-  if (smem > 200 * 1024) return SOLON_ERR_INVALID_ARG;
-  SOLON_CUDA_TRY(cudaFuncSetAttribute(project_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  // one wave: as many CTAs as are resident at once (the partial-sum buffer holds plan->proj_grid of them)
-  int per_sm = 1;
-  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, project_kernel<K>, kProjThreads, smem));
-  int grid = plan->num_sms * (per_sm < 1 ? 1 : per_sm);
+__global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const float* __restrict__ R, const float* __restrict__ f,
+                                                                     int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
+                                                                     ProjPipe pp, double* __restrict__ partials,
+                                                                     double* __restrict__ rho_out, double* __restrict__ nu_out,
+                                                                     unsigned int* ticket, int final_reduce) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
+  uint64_t* empty_bar = full_bar + kPipeStages;
+  int* abort_flag = reinterpret_cast<int*>(empty_bar + kPipeStages);
+  float* ring = reinterpret_cast<float*>(smem_raw + 128);
+  const size_t stage_floats = (size_t)(pp.batch_rows + K) * pp.slot_floats;   // the rows of a batch, then f
+  const int n_acc = (K + 1) * P;
+  pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading the sums
+  if (tid == 0) {
+    for (int s = 0; s < kPipeStages; ++s) {
+      pipe::mbar_init(&full_bar[s], 32);
+      pipe::mbar_init(&empty_bar[s], kPipeWarps);
+    }
+    *abort_flag = 0;
+    pipe::fence_barrier_init();
+  }
+  __syncthreads();
+
+  const int64_t c_begin = (int64_t)blockIdx.x * range_len;     // multiple of 4
+  int64_t c_end = c_begin + range_len;
+  if (c_end > d_c) c_end = d_c;
+  const int64_t total_floats = (int64_t)P * d_c;
+  double* mine = partials + (size_t)blockIdx.x * n_acc;
+
+  if (tid >= kPipeConsumers) {
+    const int lane = tid - kPipeConsumers;
+    uint32_t it = 0;
+    for (int b0 = 0; b0 < P; b0 += pp.batch_rows) {
+      const int nb = min(pp.batch_rows, P - b0);
+      for (int64_t c0 = c_begin; c0 < c_end; c0 += pp.slice_cols, ++it) {
+        const int stage = it % kPipeStages;
+        const uint32_t phase = (it / kPipeStages) & 1;
+        if (it >= (uint32_t)kPipeStages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
+        const int64_t cols = (c_end - c0) < pp.slice_cols ? (c_end - c0) : pp.slice_cols;
+        float* stage_base = ring + stage * stage_floats;
+        uint32_t row_bytes = 0, f_bytes = 0;
+        const float* row_src = nullptr;
+        float* slot = stage_base + (size_t)lane * pp.slot_floats;
+        if (lane < nb) {
+          const int64_t first = (int64_t)(b0 + lane) * d_c + c0;
+          const int64_t last = first + cols;
+          const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
+          int64_t a1 = (last + 3) & ~(int64_t)3;
+          const int64_t safe_end = total_floats & ~(int64_t)3;      // bulk copies stay inside the matrix
+          if (a1 > safe_end) a1 = safe_end;
+          row_bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
+          row_src = R + a0;
+          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = R[e];   // <= 3 floats
+        }
+        // the first K lanes also bring the slice of f (16-byte aligned rows padded to a multiple of 4 floats)
+        if (lane < K) f_bytes = (uint32_t)(((cols + 3) & ~(int64_t)3) * 4);
+        if (row_bytes + f_bytes) pipe::mbar_arrive_expect_tx(&full_bar[stage], row_bytes + f_bytes);
+        else pipe::mbar_arrive(&full_bar[stage]);
+        if (row_bytes) pipe::bulk_load(slot, row_src, row_bytes, &full_bar[stage]);
+        if (f_bytes)
+          pipe::bulk_load(stage_base + (size_t)(pp.batch_rows + lane) * pp.slot_floats, f + (int64_t)lane * f_pitch + c0, f_bytes,
+                          &full_bar[stage]);
+      }
+    }
+    if (*(volatile int*)abort_flag) pipe::drain_delay();
+  } else {
+    const int lane = tid & 31, warp = tid >> 5;
+    const int dc_mod4 = (int)(d_c & 3);
+    uint32_t it = 0;
+    for (int b0 = 0; b0 < P; b0 += pp.batch_rows) {
+      const int nb = min(pp.batch_rows, P - b0);
+      const int nr = warp < nb ? (nb - warp + kPipeWarps - 1) / kPipeWarps : 0;    // rows warp, warp + 8, ... below nb
+      int shift[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) shift[j] = (((b0 + warp + 8 * j) & 3) * dc_mod4) & 3;   // (row * d_c + c0) mod 4
+      double rho[4][K], nu[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        nu[j] = 0.0;
+#pragma unroll
+        for (int kappa = 0; kappa < K; ++kappa) rho[j][kappa] = 0.0;
+      }
+      for (int64_t c0 = c_begin; c0 < c_end; c0 += pp.slice_cols, ++it) {
+        const int stage = it % kPipeStages;
+        const uint32_t phase = (it / kPipeStages) & 1;
+        pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
+        const int cols = (int)((c_end - c0) < pp.slice_cols ? (c_end - c0) : pp.slice_cols);
+        const float* base = ring + stage * stage_floats;
+        const float* fs = base + (size_t)pp.batch_rows * pp.slot_floats;
+        const float* rows[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) rows[j] = base + (size_t)(warp + 8 * j) * pp.slot_floats + shift[j];
+        if (nr == 4) pipe_consume<K, 4>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+        else if (nr == 3) pipe_consume<K, 3>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+        else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+        else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+        __syncwarp();
+        if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (j < nr) {
+          const int row = b0 + warp + 8 * j;
+#pragma unroll
+          for (int kappa = 0; kappa < K; ++kappa) {
+            const double t = warp_sum(rho[j][kappa]);
+            if (lane == 0) mine[(size_t)kappa * P + row] = t;
+          }
+          const double t = warp_sum(nu[j]);
+          if (lane == 0) mine[(size_t)K * P + row] = t;
+        }
+      }
+    }
+  }
+  reduce_partials(partials, n_acc, K * P, rho_out, nu_out, ticket, final_reduce);
+}
+
+template <int K>
+static int launch_project_pipe_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out, int final_reduce) {
+  ProjPipe pp;
+  pp.status = plan->d_status;
+  // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
+  const size_t per_cta = (size_t)227 * 1024 / 2 - 1024 - 128;
+  const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
+  pp.batch_rows = (plan->P + n_batches - 1) / n_batches;
+  int slice = (int)(per_cta / ((size_t)kPipeStages * (pp.batch_rows + K) * 4)) - 8;
+  slice = slice / 32 * 32;
+  if (slice > 2048) slice = 2048;
+  int grid = plan->num_sms * 2;
   if (grid > plan->proj_grid) grid = plan->proj_grid;
   // leave one slot per group free: the locator's CTAs (launched as dependents) then become resident while this
   // kernel streams and use the time to stage their tables and fetch their code
-  if (plan->q <= plan->num_sms && grid >= 4 * plan->q) grid -= plan->q;
+  if (plan->q <= plan->num_sms / 2 && grid >= 4 * plan->q) grid -= plan->q;
   int64_t range_len = (plan->d_c + grid - 1) / grid;
   range_len = (range_len + 3) / 4 * 4;
-  if (range_len < tile_cols) tile_cols = (int)range_len;
-  project_kernel<K><<<grid, kProjThreads, smem, plan->stream>>>(
-      received, plan->d_f, plan->f_pitch, plan->P, plan->d_c, range_len, tile_cols, plan->d_partials, rho_out,
-      nu_out, plan->d_proj_ticket, final_reduce);
+  if (range_len < slice) slice = (int)((range_len + 31) / 32 * 32);
+  pp.slice_cols = slice;
+  pp.slot_floats = slice + 8;
+  const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows + K) * pp.slot_floats * sizeof(float);
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  project_pipe_kernel<K><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->f_pitch, plan->P, plan->d_c,
+                                                                     range_len, pp, plan->d_partials, rho_out, nu_out,
+                                                                     plan->d_proj_ticket, final_reduce);
   plan->proj_bunches = final_reduce ? 0 : (grid + kProjBunch - 1) / kProjBunch;
   plan->proj_bunch_sums = plan->d_partials + (size_t)grid * (K + 1) * plan->P;
   SOLON_CUDA_TRY(cudaGetLastError());
@@ -229,10 +436,10 @@ int launch_project(solon_plan* plan, const float* received, double* rho_out, dou
   if (!nu_out) nu_out = plan->d_nu;
   plan->launches += 1;
   switch (plan->K) {
-    case 1: return launch_project_k<1>(plan, received, rho_out, nu_out, final_reduce);
-    case 2: return launch_project_k<2>(plan, received, rho_out, nu_out, final_reduce);
-    case 3: return launch_project_k<3>(plan, received, rho_out, nu_out, final_reduce);
-    case 4: return launch_project_k<4>(plan, received, rho_out, nu_out, final_reduce);
+    case 1: return launch_project_pipe_k<1>(plan, received, rho_out, nu_out, final_reduce);
+    case 2: return launch_project_pipe_k<2>(plan, received, rho_out, nu_out, final_reduce);
+    case 3: return launch_project_pipe_k<3>(plan, received, rho_out, nu_out, final_reduce);
+    case 4: return launch_project_pipe_k<4>(plan, received, rho_out, nu_out, final_reduce);
     default: return SOLON_ERR_INVALID_ARG;
   }
 }

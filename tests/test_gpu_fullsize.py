@@ -64,7 +64,8 @@ def test_full_size(name):
             rho, nu = plan.projections()
             o_rho, o_nu = so.project(R, f), so.row_energy(R)
             lim = np.sqrt((f.astype(np.float64) ** 2).sum(1))[:, None] * np.sqrt(o_nu)[None, :]
-            assert np.all(np.abs(rho - o_rho) <= 1e-11 * lim)
+            # float32 runs of eight terms inside the kernel: at most 8 * 2^-24 of sum |f_p R_kp| <= ||f|| ||R_k||
+            assert np.all(np.abs(rho - o_rho) <= 8 * 2.0 ** -24 * 1.01 * lim)
             assert np.allclose(nu, o_nu, rtol=1e-4)
 
 

@@ -1,6 +1,6 @@
 """GPU parity: the CUDA path, called through the C-ABI binding, against the float64 oracle on the same
 seeded inputs.  Bars: Byzantine mask bit-exact; aggregate within 1e-4 of ||sum||_inf; coded vectors within
-one float32 rounding of the oracle's float64 values; projections to float64 accuracy."""
+one float32 rounding of the oracle's float64 values; projections within the float32 runs the kernel states."""
 
 import dataclasses
 
@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
 
 AGG_TOL = 1e-4          # max |agg_gpu - agg*| / ||agg*||_inf
 TAU = 1e-5              # the library's default detection tolerance, also given to the oracle
+RHO_TOL = 8 * 2.0 ** -24 * 1.01   # projections: worst case of the kernel's float32 runs, relative to ||f|| ||R_k||
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -82,7 +83,9 @@ def _run_case(wl, n_byz=None, check_intermediates=True):
             o_nu = so.row_energy(R)
             f64 = f.astype(np.float64)
             lim = np.sqrt((f64 ** 2).sum(1))[:, None] * np.sqrt(o_nu)[None, :]
-            assert np.all(np.abs(rho - o_rho) <= 1e-12 * lim + 1e-300)
+            # products and runs of eight terms in float32, the rest in float64: |error| <= 8 * 2^-24 * sum |f_p R_kp|,
+            # and sum |f_p R_kp| <= ||f|| ||R_k||
+            assert np.all(np.abs(rho - o_rho) <= RHO_TOL * lim + 1e-300)
             assert np.allclose(nu, o_nu, rtol=1e-4)
             n_rec, t_acc, rows, coeff = plan.recovery()
             starts = so.group_starts(sizes)
