@@ -321,7 +321,9 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   size_t need = locate_ws_doubles(plan->max_group, plan->m, plan->K, plan->s) * sizeof(double);
   if (need > plan->locate_ws_stride * sizeof(double)) return SOLON_ERR_INTERNAL;
   prm.use_smem = need <= 128 * 1024 ? 1 : 0;
-  prm.warm = (plan->max_group <= 64 && plan->s <= 5) ? 1 : 0;
+  // the warm-up pass pays when it ends before the projections do: small solver, long projection pass (the pass takes
+  // 35-50 us beside a streaming kernel; the projection kernel moves about 6 GB per ms)
+  prm.warm = (plan->max_group <= 64 && plan->s <= 5 && (double)plan->P * (double)plan->d_c * 4.0 >= 350e6) ? 1 : 0;
   size_t smem = prm.use_smem ? need : 0;
   const size_t tables = (2 * (size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
   prm.stage_tables = (prm.use_smem && smem + tables <= 200 * 1024) ? 1 : 0;

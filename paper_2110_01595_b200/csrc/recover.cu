@@ -49,8 +49,9 @@ __device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_s
   __syncthreads();
   for (int g = threadIdx.x; g < prm.q; g += blockDim.x) {
     int base = 0;
-    for (int o = 0; o < g; ++o) base += n_rec_s[o];
-    const int n = n_rec_s[g], src = start_s[g];
+    for (int o = 0; o < g; ++o) base += min(max(n_rec_s[o], 0), start_s[o + 1] - start_s[o]);
+    const int src = start_s[g];
+    const int n = min(max(n_rec_s[g], 0), start_s[g + 1] - src);   // never more than the group has nodes
     for (int j = 0; j < n; ++j) slots_s[base + j] = src + j;
     if (g == prm.q - 1) *count_s = base + n;
   }
