@@ -217,6 +217,7 @@ def run_ours(args, wl):
     coded = plan.encode(G)
     nodes = synth.byzantine_nodes(wl_rank)
     byz_rows = synth.byzantine_rows(wl_rank, coded, nodes)
+    nodes_dev = torch.tensor(nodes, dtype=torch.long, device="cuda")
     agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
     mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
 
@@ -226,8 +227,8 @@ def run_ours(args, wl):
         plan.encode(G, coded)
         if events is not None:
             events[1].record()
-        for i, k in enumerate(nodes):
-            coded[k].copy_(byz_rows[i])                       # the adversary: plain device-to-device copies
+        if nodes:
+            coded.index_copy_(0, nodes_dev, byz_rows)         # the adversary: one device-to-device row copy
         if events is not None:
             events[2].record()
         if sp is not None:
@@ -355,6 +356,7 @@ def run_sweep(args):
             coded = plan.encode(G)
             nodes = synth.byzantine_nodes(wl)
             byz_rows = synth.byzantine_rows(wl, coded, nodes)
+            nodes_dev = torch.tensor(nodes, dtype=torch.long, device="cuda")
             agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
             mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
 
@@ -364,8 +366,8 @@ def run_sweep(args):
                 plan.encode(G, coded)
                 if ev:
                     ev[1].record()
-                for i, k in enumerate(nodes):
-                    coded[k].copy_(byz_rows[i])
+                if nodes:
+                    coded.index_copy_(0, nodes_dev, byz_rows)
                 if ev:
                     ev[2].record()
                 plan.decode(coded, agg, mask)
