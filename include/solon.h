@@ -112,6 +112,16 @@ int solon_plan_reseed(solon_plan* plan, uint64_t seed);
  * thirty times the rounding noise of float32 coded vectors. */
 int solon_plan_set_tolerance(solon_plan* plan, double tau);
 
+/* Early locator.  Any subset of the columns gives a valid random projection, so solon_decode lets
+ * the locator kernel start on the projection of the first eighth (about) of every column range
+ * while the projection kernel is still streaming the rest, and afterwards only checks, on the final
+ * projections, that the set it found is exactly the set of nodes that do not fit; if that check
+ * fails (an attacker who spared those columns) the whole locator runs as it would have anyway.
+ * Results do not depend on the mode.  mode 0: never; 1 (default): when the projection pass is long
+ * enough to hide the early run (P * d_c * 4 bytes >= 300 MB) and the solver is small (groups of at
+ * most 64 nodes, s <= 5); 2: whenever the solver is small. */
+int solon_plan_set_early_locator(solon_plan* plan, int mode);
+
 /* Rows per partition for solon_lsq_grads (default 256). */
 int solon_plan_set_lsq_rows(solon_plan* plan, int rows_per_partition);
 
@@ -207,6 +217,11 @@ int solon_plan_get_projections(solon_plan* plan, double* rho /* host, K * P */, 
  * coeff[j*m + l]), and the accepted error count t[g] (-1 if the group was undecodable).
  * Capacities: n_rec and t hold q ints, rec_rows P ints, coeff P * m doubles. */
 int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows, double* coeff);
+
+/* Outcome of the early locator in the last solon_decode, one int per group (host, q entries):
+ * 0 no early run, 1 the early answer was confirmed on the final projections, 2 it was not (the
+ * whole locator ran), 3 the bounded wait for the partial projection expired (the whole locator ran). */
+int solon_plan_get_early_outcome(solon_plan* plan, int* outcome);
 
 /* Projections without any allocation.  (The paper has no counterpart: this entry point exists for
  * callers of this library that are not allowed to allocate device memory at the moment they need

@@ -38,6 +38,7 @@ SIGNATURES = {
     "solon_plan_set_num_projections": (c_int, [c_void_p, c_int]),
     "solon_plan_reseed": (c_int, [c_void_p, c_uint64]),
     "solon_plan_set_tolerance": (c_int, [c_void_p, c_double]),
+    "solon_plan_set_early_locator": (c_int, [c_void_p, c_int]),
     "solon_plan_set_lsq_rows": (c_int, [c_void_p, c_int]),
     "solon_plan_dc": (c_int64, [c_void_p]),
     "solon_plan_num_groups": (c_int, [c_void_p]),
@@ -56,6 +57,7 @@ SIGNATURES = {
     "solon_step_host": (c_int, [c_void_p, c_void_p, c_int, POINTER(c_int), c_void_p, c_void_p, c_void_p]),
     "solon_plan_get_projections": (c_int, [c_void_p, POINTER(c_double), POINTER(c_double)]),
     "solon_plan_get_recovery": (c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_double)]),
+    "solon_plan_get_early_outcome": (c_int, [c_void_p, POINTER(c_int)]),
     "solon_plan_kernel_launches": (c_int64, [c_void_p]),
     "solon_plan_set_profiling": (c_int, [c_void_p, c_int]),
     "solon_plan_get_timings": (c_int, [c_void_p, POINTER(c_float)]),
@@ -206,6 +208,16 @@ class Plan:
 
     def set_tolerance(self, tau: float) -> None:
         _check(lib().solon_plan_set_tolerance(self._h, tau), "solon_plan_set_tolerance")
+
+    def set_early_locator(self, mode: int) -> None:
+        """0: never start the locator on a partial projection; 1 (default): when the projection pass is long; 2: always."""
+        _check(lib().solon_plan_set_early_locator(self._h, mode), "solon_plan_set_early_locator")
+
+    def early_outcome(self) -> np.ndarray:
+        """Per group: 0 no early run, 1 early answer confirmed, 2 not confirmed, 3 wait expired (last decode)."""
+        out = np.zeros(self.q, dtype=np.int32)
+        _check(lib().solon_plan_get_early_outcome(self._h, _dptr(out, c_int)), "solon_plan_get_early_outcome")
+        return out
 
     def set_lsq_rows(self, rows: int) -> None:
         _check(lib().solon_plan_set_lsq_rows(self._h, rows), "solon_plan_set_lsq_rows")

@@ -30,8 +30,12 @@ struct LocateParams {
   int n_bunches;              // 0: rho and nu are final
   double* rho_w;              // with n_bunches > 0 the sums are also written here (K x P) and to nu_w (P)
   double* nu_w;
+  const double* bunch_a;      // same shape as bunch_sums: the sums over part A of the projection kernel's column ranges
+  const unsigned long long* progress;   // bunches whose part-A sums are complete (cumulative over launches)
+  unsigned long long progress_target;   // its value once this decode's part A is complete
+  int* early;                 // q: outcome of the early run per group (see solon_plan_get_early_outcome)
+  int spec;                   // work on part A while the projection kernel streams part B, then only check the result
   unsigned long long* tile_counter;   // work counter of the recovery kernel, zeroed here
-  int warm;               // run the solver once on made-up values before waiting for the projections
   int stage_tables;      // copy the group's tables to shared memory (they follow the workspace)
   uint8_t* mask;         // P (caller's buffer)
   int* t_acc;            // q
@@ -93,6 +97,12 @@ SOLON_HD static inline GroupScratch carve(double* ws, int n, int m, int K, int s
 // at the same time with warp-level synchronisation only; afterwards the whole CTA picks the smallest
 // accepted count, writes the group's part of the mask and builds the recovery table.  No CTA waits on
 // another one.
+__device__ __forceinline__ unsigned long long pipe_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
 constexpr int kGatherBatch = 20;   // bunch sums fetched at once per column (the projection kernel leaves 37 on 148 SMs: two rounds)
 
 __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocateParams prm) {
@@ -130,16 +140,49 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   }
   const Team cta = Team::cta();
   pdl_trigger();   // the recovery kernel may be scheduled early; it waits for this grid before reading the table
-  // Two passes over the same code.  Pass 0 (small problems only) runs before the projections exist, on made-up
-  // values with s corrupt nodes, and writes nothing outside this CTA's scratch: between two decodes gigabytes
-  // stream through L2, so the solver's instructions would otherwise be fetched from HBM line by line on the
-  // critical path; this way they are fetched while the projection kernel is still streaming.  Pass 1 is the
-  // decode proper.
+  // Up to three passes over the same code; the last one is the decode proper, after the projections are complete.
+  // The others (prm.spec) run while the projection kernel is still streaming and write nothing outside this CTA's
+  // scratch.  Pass 0: that kernel announces the sums over part A of its column ranges early - a random projection
+  // of those columns, as good as any for locating whoever lies there - and the whole locator runs on them.  The last
+  // pass then only checks, on the final sums, that the set found is exactly the set of nodes that do not fit
+  // (locate_check): the mask and the recovery table depend on that set alone.  If the check fails (an attacker who
+  // spared part A, a timed-out wait) it runs the whole locator as usual.  Pass 1 rehearses that check on the part-A
+  // sums: between decodes gigabytes stream through L2, and pass 0's solver has pushed the few instructions of the
+  // check out of the SM's instruction cache again, so without it each step of the check would wait for HBM.
+  __shared__ int s_ready, s_spec_ok;
+  if (tid == 0) {
+    s_spec_ok = 0;
+    s_ready = 0;
+  }
 #pragma unroll 1
-  for (int pass = prm.warm ? 0 : 1; pass < 2; ++pass) {
-    if (pass == 1) {
+  for (int pass = prm.spec ? 0 : 2; pass < 3; ++pass) {
+    const bool spec0 = pass == 0;
+    const bool last = pass == 2;
+    if (pass == 1 && !s_spec_ok) continue;     // nothing to rehearse
+    if (last) {
       pdl_wait();   // the projections are complete and visible (everything above only read plan tables)
       if (g == 0 && tid == 0) *prm.tile_counter = 0ULL;   // the recovery kernel reads it only after this grid is done
+    }
+    if (spec0) {
+      // wait (bounded: 2 ms) until every bunch of the projection kernel has added up its part A.  That kernel was
+      // resident as a whole before this one could start and never waits for anything, so the count always comes.
+      if (tid == 0) {
+        int ready = 0;
+        const unsigned long long t_start = pipe_timer_ns();
+        for (;;) {
+          unsigned long long seen;
+          asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(prm.progress) : "memory");
+          if (seen >= prm.progress_target) {
+            ready = 1;
+            break;
+          }
+          if (pipe_timer_ns() - t_start > 2000000ull) break;
+          __nanosleep(200);
+        }
+        s_ready = ready;
+      }
+      __syncthreads();
+      if (!s_ready) continue;      // nothing to go on: pass 1 does all the work
     }
     if (prm.s == 0) {
       // pure compression code: nothing to locate, every node is trusted
@@ -156,13 +199,13 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       // one parallel round trip brings the group's projected values on chip
       if (prm.n_bunches > 0) {
         // last level of the projection kernel's reduction, for this group's columns only: a thread fetches all
-        // bunch sums of its column at once and adds them in bunch order.  (Pass 0 runs this too, on whatever
-        // the buffer holds, only to have the code on chip; its values are replaced below.)
+        // bunch sums of its column at once and adds them in bunch order
         const int n_cols = (prm.K + 1) * n;
         const size_t n_acc = (size_t)(prm.K + 1) * prm.P;
+        const double* sums = last ? prm.bunch_sums : prm.bunch_a;
         for (int c = tid; c < n_cols; c += n_threads) {
           const int which = c / n, i = c - which * n;
-          const double* src = prm.bunch_sums + (size_t)which * prm.P + row0 + i;
+          const double* src = sums + (size_t)which * prm.P + row0 + i;
           double acc = 0.0;
           for (int b0 = 0; b0 < prm.n_bunches; b0 += kGatherBatch) {
             double v[kGatherBatch];
@@ -173,28 +216,46 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
           }
           if (which < prm.K) {
             sc.rho_in[(size_t)which * n + i] = acc;
-            if (pass == 1) prm.rho_w[(size_t)which * prm.P + row0 + i] = acc;
+            if (last) prm.rho_w[(size_t)which * prm.P + row0 + i] = acc;
           } else {
             sc.nu_in[i] = acc;
-            if (pass == 1) prm.nu_w[row0 + i] = acc;
+            if (last) prm.nu_w[row0 + i] = acc;
           }
         }
         __syncthreads();
       }
       for (int i = tid; i < n; i += n_threads) {
-        if (pass == 1) {
+        if (last) {
           if (prm.n_bunches > 0) continue;
           sc.nu_in[i] = prm.nu[row0 + i];
           for (int kappa = 0; kappa < prm.K; ++kappa) sc.rho_in[(size_t)kappa * n + i] = prm.rho[(size_t)kappa * prm.P + row0 + i];
-        } else {
-          sc.nu_in[i] = 1.0;
-          for (int kappa = 0; kappa < prm.K; ++kappa)
-            sc.rho_in[(size_t)kappa * n + i] = 1.0 + (prm.m > 1 ? (kappa + 1) * tb.w[i] : 0.0) + (i < prm.s ? 3.0 * (i + 1) : 0.0);
         }
       }
       __syncthreads();
       double tau_eff = 0.0;
       locate_prepare(cta, n, prm.K, sc.rho_in, sc.nu_in, prm.tau, sc.forced, sc.rho_n, &tau_eff, sc.scratch);
+      bool confirmed = false;
+      if (pass >= 1 && s_spec_ok) {
+        // the set found on part A, checked on the final sums by the whole CTA
+        uint8_t* cand = reinterpret_cast<uint8_t*>(sc.tasks);
+        uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
+        confirmed = locate_check(cta, tb, n, prm.K, prm.s, sc.rho_n, sc.forced, tau_eff, sc.mask_l, cand, bad,
+                                 sc.tasks + 2 * ((size_t)n / 8 + 1), &sc.recs[0]) != 0;
+      }
+      if (pass == 1) continue;     // the rehearsal ends here, whatever the check said
+      if (confirmed) {
+        // mask, recovery rows and weights of pass 0 stand as they are
+        for (int k = tid; k < n; k += n_threads) prm.mask[row0 + k] = sc.mask_l[k];
+        const int n_rec = s_n_rec;
+        for (int j = tid; j < n_rec; j += n_threads) prm.rec_rows[row0 + j] = sc.rows_l[j] + row0;
+        for (int i = tid; i < n_rec * prm.m; i += n_threads) prm.coeff[(size_t)row0 * prm.m + i] = sc.coeff_l[i];
+        if (tid == 0) {
+          prm.n_rec[g] = n_rec;
+          prm.t_acc[g] = s_t_acc;
+          prm.early[g] = 1;
+        }
+        return;
+      }
       const int t = tid >> 5;                       // this warp's error count
       double* task = sc.tasks + (size_t)t * sc.task_stride;
       uint8_t* cand = reinterpret_cast<uint8_t*>(task);
@@ -207,6 +268,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
     const int ok = locate_epilogue(cta, tb, n, prm.m, prm.s, sc.forced, sc.recs, sc.flags, n, sc.mask_l, &s_t_acc, sc.rows_l,
                                    &s_n_rec, sc.coeff_l, sc.trusted, sc.tasks);
     if (pass == 0) {
+      if (tid == 0) s_spec_ok = (spec0 && ok && prm.s > 0) ? 1 : 0;
       __syncthreads();
       continue;
     }
@@ -218,6 +280,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
     if (tid == 0) {
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
+      prm.early[g] = !prm.spec ? 0 : (s_ready ? 2 : 3);
       if (!ok) atomicOr(prm.status, kStatusUndecodable);
     }
   }
@@ -302,6 +365,10 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   prm.n_bunches = fused ? plan->proj_bunches : 0;
   prm.rho_w = plan->d_rho;
   prm.nu_w = plan->d_nu;
+  prm.bunch_a = fused ? plan->proj_bunch_a : nullptr;
+  prm.progress = plan->d_proj_progress;
+  prm.progress_target = plan->proj_progress_target;
+  prm.early = plan->d_early;
   prm.qb = plan->d_qb;
   prm.hm = plan->d_hm;
   prm.qb_off = plan->d_qb_off;
@@ -321,9 +388,11 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   size_t need = locate_ws_doubles(plan->max_group, plan->m, plan->K, plan->s) * sizeof(double);
   if (need > plan->locate_ws_stride * sizeof(double)) return SOLON_ERR_INTERNAL;
   prm.use_smem = need <= 128 * 1024 ? 1 : 0;
-  // the warm-up pass pays when it ends before the projections do: small solver, long projection pass (the pass takes
-  // 35-50 us beside a streaming kernel; the projection kernel moves about 6 GB per ms)
-  prm.warm = (plan->max_group <= 64 && plan->s <= 5 && (double)plan->P * (double)plan->d_c * 4.0 >= 350e6) ? 1 : 0;
+  // working ahead on part A pays for a small solver beside a long projection pass (about 6 GB per ms); otherwise it
+  // would still be at it when the projections end
+  const bool small_solver = plan->max_group <= 64 && plan->s <= 5;
+  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 300e6;
+  prm.spec = (fused && small_solver && (plan->early_locator == 2 || (plan->early_locator == 1 && long_pass))) ? 1 : 0;
   size_t smem = prm.use_smem ? need : 0;
   const size_t tables = (2 * (size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
   prm.stage_tables = (prm.use_smem && smem + tables <= 200 * 1024) ? 1 : 0;

@@ -468,6 +468,33 @@ SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, i
   SOLON_SYNC();
 }
 
+// Check of a given set: is `mask_in` (n bytes, at most s set) exactly the set of nodes that do not fit the
+// polynomial refitted on all the others?  This is the acceptance test of locate_task for candidates that are known
+// in advance.  cand, bad: n bytes of scratch each; ws: locate_task_ws_doubles(n, m, K, s) doubles.
+// Every thread gets the same answer.
+SOLON_HD inline int locate_check(const Team& tm, const GroupTables& tb, int n, int K, int s, const double* rho_n,
+                                 const uint8_t* forced, double tau, const uint8_t* mask_in, uint8_t* cand, uint8_t* bad,
+                                 double* ws, TaskRecord* rec) {
+  int t = 0;
+  for (int k = 0; k < n; ++k) t += mask_in[k] ? 1 : 0;
+  if (t > s) return 0;
+  double* absE = ws;                                // same layout as locate_task
+  int* vlist = reinterpret_cast<int*>(absE + n);    // t
+  int* vpos = vlist + t;                            // n
+  double* rest = absE + n + (size_t)(t + n) / 2 + 1;
+  SOLON_FOR_THREADS(k, n) {
+    int pos = 0;
+    for (int o = 0; o < k; ++o) pos += mask_in[o] ? 1 : 0;
+    cand[k] = mask_in[k] ? 1 : 0;
+    vpos[k] = mask_in[k] ? pos : 0;
+    if (mask_in[k]) vlist[pos] = k;
+  }
+  SOLON_SYNC();
+  locate_verify(tm, tb, n, K, rho_n, tau, cand, t, vlist, vpos, forced, bad, rest, rec);
+  SOLON_SYNC();
+  return (rec->accept && rec->n_flagged == t) ? 1 : 0;
+}
+
 // Recovery table for one group: given the trusted nodes (trusted[k] != 0 among n), choose the rows
 // the recovery reads and the weights coeff[j*m + l] of row rec_rows[j] in coordinate l of a chunk,
 // i.e. the least-squares inverse of [W-hat_{m-1}]_{rows,.} (monomial basis, as the encoder used).

@@ -113,7 +113,7 @@ static void free_device(solon_plan* p) {
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_locate_ws);
-  cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_tile_counter);
+  cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress);
   cudaFree(p->d_resid);
   for (int i = 0; i < 6; ++i)
     if (p->ev[i]) cudaEventDestroy(p->ev[i]);
@@ -128,8 +128,8 @@ static int alloc_projection(solon_plan* p) {
   (void)cudaGetLastError();
   p->d_f = nullptr; p->d_partials = nullptr; p->d_rho = nullptr; p->d_locate_ws = nullptr;
   if ((rc = dev_alloc(&p->d_f, (size_t)p->K * p->f_pitch))) return rc;
-  // per-CTA partial sums followed by the per-bunch sums of the two-level reduction
-  if ((rc = dev_alloc(&p->d_partials, (size_t)(p->proj_grid + p->proj_grid / 16 + 1) * (p->K + 1) * p->P))) return rc;
+  // per-CTA partial sums of the two parts of every column range, then the per-bunch sums of part A and of the whole
+  if ((rc = dev_alloc(&p->d_partials, 2 * (size_t)(p->proj_grid + p->proj_grid / 16 + 1) * (p->K + 1) * p->P))) return rc;
   if ((rc = dev_alloc(&p->d_rho, (size_t)p->K * p->P))) return rc;
   p->locate_ws_stride = locate_ws_doubles(p->max_group, p->m, p->K, p->s);
   if ((rc = dev_alloc(&p->d_locate_ws, (size_t)p->q * p->locate_ws_stride))) return rc;
@@ -214,6 +214,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
   }
   p->num_sms = prop.multiProcessorCount;
   p->proj_grid = p->num_sms * 4;
+  p->early_locator = 1;
 
   rc = SOLON_OK;
   do {
@@ -248,20 +249,24 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
     }
     if ((rc = alloc_projection(p))) break;
     if ((rc = dev_alloc(&p->d_nu, P))) break;
-    if ((rc = dev_alloc(&p->d_proj_ticket, (size_t)p->proj_grid / 16 + 2))) break;
+    if ((rc = dev_alloc(&p->d_proj_ticket, 2 * ((size_t)p->proj_grid / 16 + 2)))) break;
     if ((rc = dev_alloc(&p->d_t_acc, q))) break;
     if ((rc = dev_alloc(&p->d_n_rec, q))) break;
     if ((rc = dev_alloc(&p->d_rec_rows, P))) break;
     if ((rc = dev_alloc(&p->d_coeff, (size_t)P * m))) break;
     if ((rc = dev_alloc(&p->d_status, 2))) break;
     if ((rc = dev_alloc(&p->d_tile_counter, 4))) break;
+    if ((rc = dev_alloc(&p->d_early, (size_t)q))) break;
+    if ((rc = dev_alloc(&p->d_proj_progress, 2))) break;
     cudaError_t e = cudaSuccess;
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_start, start.data(), (q + 1) * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_of, p->group_of.data(), P * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_w, p->w.data(), P * sizeof(double), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, ((size_t)p->proj_grid / 16 + 2) * sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_proj_ticket, 0, 2 * ((size_t)p->proj_grid / 16 + 2) * sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_tile_counter, 0, 4 * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(p->d_early, 0, q * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_proj_progress, 0, 2 * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(p->d_n_rec, 0, q * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_t_acc, 0, q * sizeof(int));
     if (e != cudaSuccess) { (void)cudaGetLastError(); rc = SOLON_ERR_CUDA; break; }
@@ -306,6 +311,19 @@ int solon_plan_reseed(solon_plan* plan, uint64_t seed) {
   if (!plan) return SOLON_ERR_INVALID_ARG;
   plan->seed = seed;
   return launch_fill_projection(plan);
+}
+
+int solon_plan_set_early_locator(solon_plan* plan, int mode) {
+  if (!plan || mode < 0 || mode > 2) return SOLON_ERR_INVALID_ARG;
+  plan->early_locator = mode;
+  return SOLON_OK;
+}
+
+int solon_plan_get_early_outcome(solon_plan* plan, int* outcome) {
+  if (!plan || !outcome) return SOLON_ERR_INVALID_ARG;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(outcome, plan->d_early, (size_t)plan->q * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  return SOLON_OK;
 }
 
 int solon_plan_set_tolerance(solon_plan* plan, double tau) {

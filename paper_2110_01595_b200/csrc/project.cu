@@ -224,6 +224,8 @@ struct ProjPipe {
   int slice_cols;     // columns per stage (multiple of 32)
   int slot_floats;    // slice_cols + 8: room for the alignment shift and the rounded-up end
   int batch_rows;     // rows per batch (<= kPipeRows), the same for all batches but the last
+  int64_t part_a_cols;                // columns of part A in every CTA's range (whole slices)
+  unsigned long long* progress;       // [0] bunches whose part-A sums are complete, counted over all launches
   int* status;
 };
 
@@ -278,6 +280,48 @@ __device__ __forceinline__ void pipe_consume(const float* const* rows, const flo
   }
 }
 
+// Sums of one bunch of kProjBunch CTAs, added in a fixed order by the last of them to arrive (atomic ticket, nobody
+// waits).  Called by n_threads threads of the CTA that synchronise through Sync; every one of them gets the same
+// answer: whether this CTA was the one that completed the bunch.  bunch_out[i] = add_in[i] + sum over members.
+struct SyncAll {
+  __device__ __forceinline__ static void sync() { __syncthreads(); }
+};
+struct SyncConsumers {
+  __device__ __forceinline__ static void sync() { pipe::named_barrier_sync(1, 256); }
+};
+
+template <class Sync>
+__device__ __forceinline__ bool bunch_reduce(const double* __restrict__ partials, const double* add_in, double* __restrict__ bunch_out,
+                                             int n_acc, unsigned int* bunch_ticket, unsigned int* s_flag, int tid, int n_threads) {
+  const unsigned int bunch = blockIdx.x / kProjBunch;
+  const unsigned int first = bunch * kProjBunch;
+  const unsigned int members = min((unsigned int)kProjBunch, gridDim.x - first);
+  __threadfence();
+  Sync::sync();
+  if (tid == 0) *s_flag = atomicAdd(bunch_ticket + bunch, 1u);
+  Sync::sync();
+  const bool last = *s_flag == members - 1;
+  if (!last) return false;
+  __threadfence();
+  for (int i = tid; i < n_acc; i += n_threads) {
+    double v[kProjBunch];
+#pragma unroll
+    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b)     // all loads in flight at once, then a fixed order
+      v[b] = b < members ? __ldcg(partials + (size_t)(first + b) * n_acc + i) : 0.0;
+    double acc = add_in ? __ldcg(add_in + (size_t)bunch * n_acc + i) : 0.0;
+#pragma unroll
+    for (unsigned int b = 0; b < (unsigned int)kProjBunch; ++b) acc += v[b];
+    bunch_out[(size_t)bunch * n_acc + i] = acc;
+  }
+  __threadfence();
+  Sync::sync();
+  if (tid == 0) bunch_ticket[bunch] = 0u;   // ready for the next launch
+  return true;
+}
+
+// The CTA's column range is walked in two parts.  Part A (the first eighth or so) is summed, reduced over the
+// bunches and announced (progress[0]) on its own, so that the locator kernel can already work on a projection of
+// those columns - it is a random projection like any other - while part B streams; the final sums are A + B.
 template <int K>
 __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const float* __restrict__ R, const float* __restrict__ f,
                                                                      int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
@@ -285,6 +329,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
                                                                      double* __restrict__ rho_out, double* __restrict__ nu_out,
                                                                      unsigned int* ticket, int final_reduce) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ unsigned int s_flag;
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + kPipeStages;
@@ -292,7 +337,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
   float* ring = reinterpret_cast<float*>(smem_raw + 128);
   const size_t stage_floats = (size_t)(pp.batch_rows + K) * pp.slot_floats;   // the rows of a batch, then f
   const int n_acc = (K + 1) * P;
-  pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading the sums
+  pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading the final sums
   if (tid == 0) {
     for (int s = 0; s < kPipeStages; ++s) {
       pipe::mbar_init(&full_bar[s], 32);
@@ -306,42 +351,50 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
   const int64_t c_begin = (int64_t)blockIdx.x * range_len;     // multiple of 4
   int64_t c_end = c_begin + range_len;
   if (c_end > d_c) c_end = d_c;
+  int64_t c_mid = c_begin + pp.part_a_cols;                    // part_a_cols is a multiple of the slice width
+  if (c_mid > c_end) c_mid = c_end;
   const int64_t total_floats = (int64_t)P * d_c;
-  double* mine = partials + (size_t)blockIdx.x * n_acc;
+  const unsigned int n_bunches = (gridDim.x + kProjBunch - 1) / kProjBunch;
+  double* part_sums[2] = {partials + (size_t)blockIdx.x * n_acc, partials + ((size_t)gridDim.x + blockIdx.x) * n_acc};
+  double* bunch_a = partials + 2 * (size_t)gridDim.x * n_acc;
+  double* bunch_f = bunch_a + (size_t)n_bunches * n_acc;
 
   if (tid >= kPipeConsumers) {
     const int lane = tid - kPipeConsumers;
     uint32_t it = 0;
-    for (int b0 = 0; b0 < P; b0 += pp.batch_rows) {
-      const int nb = min(pp.batch_rows, P - b0);
-      for (int64_t c0 = c_begin; c0 < c_end; c0 += pp.slice_cols, ++it) {
-        const int stage = it % kPipeStages;
-        const uint32_t phase = (it / kPipeStages) & 1;
-        if (it >= (uint32_t)kPipeStages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
-        const int64_t cols = (c_end - c0) < pp.slice_cols ? (c_end - c0) : pp.slice_cols;
-        float* stage_base = ring + stage * stage_floats;
-        uint32_t row_bytes = 0, f_bytes = 0;
-        const float* row_src = nullptr;
-        float* slot = stage_base + (size_t)lane * pp.slot_floats;
-        if (lane < nb) {
-          const int64_t first = (int64_t)(b0 + lane) * d_c + c0;
-          const int64_t last = first + cols;
-          const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
-          int64_t a1 = (last + 3) & ~(int64_t)3;
-          const int64_t safe_end = total_floats & ~(int64_t)3;      // bulk copies stay inside the matrix
-          if (a1 > safe_end) a1 = safe_end;
-          row_bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
-          row_src = R + a0;
-          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = R[e];   // <= 3 floats
+    for (int part = 0; part < 2; ++part) {
+      const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
+      for (int b0 = 0; b0 < P && lo < hi; b0 += pp.batch_rows) {
+        const int nb = min(pp.batch_rows, P - b0);
+        for (int64_t c0 = lo; c0 < hi; c0 += pp.slice_cols, ++it) {
+          const int stage = it % kPipeStages;
+          const uint32_t phase = (it / kPipeStages) & 1;
+          if (it >= (uint32_t)kPipeStages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
+          const int64_t cols = (hi - c0) < pp.slice_cols ? (hi - c0) : pp.slice_cols;
+          float* stage_base = ring + stage * stage_floats;
+          uint32_t row_bytes = 0, f_bytes = 0;
+          const float* row_src = nullptr;
+          float* slot = stage_base + (size_t)lane * pp.slot_floats;
+          if (lane < nb) {
+            const int64_t first = (int64_t)(b0 + lane) * d_c + c0;
+            const int64_t last = first + cols;
+            const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
+            int64_t a1 = (last + 3) & ~(int64_t)3;
+            const int64_t safe_end = total_floats & ~(int64_t)3;      // bulk copies stay inside the matrix
+            if (a1 > safe_end) a1 = safe_end;
+            row_bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
+            row_src = R + a0;
+            for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = R[e];   // <= 3 floats
+          }
+          // the first K lanes also bring the slice of f (16-byte aligned rows padded to a multiple of 4 floats)
+          if (lane < K) f_bytes = (uint32_t)(((cols + 3) & ~(int64_t)3) * 4);
+          if (row_bytes + f_bytes) pipe::mbar_arrive_expect_tx(&full_bar[stage], row_bytes + f_bytes);
+          else pipe::mbar_arrive(&full_bar[stage]);
+          if (row_bytes) pipe::bulk_load(slot, row_src, row_bytes, &full_bar[stage]);
+          if (f_bytes)
+            pipe::bulk_load(stage_base + (size_t)(pp.batch_rows + lane) * pp.slot_floats, f + (int64_t)lane * f_pitch + c0, f_bytes,
+                            &full_bar[stage]);
         }
-        // the first K lanes also bring the slice of f (16-byte aligned rows padded to a multiple of 4 floats)
-        if (lane < K) f_bytes = (uint32_t)(((cols + 3) & ~(int64_t)3) * 4);
-        if (row_bytes + f_bytes) pipe::mbar_arrive_expect_tx(&full_bar[stage], row_bytes + f_bytes);
-        else pipe::mbar_arrive(&full_bar[stage]);
-        if (row_bytes) pipe::bulk_load(slot, row_src, row_bytes, &full_bar[stage]);
-        if (f_bytes)
-          pipe::bulk_load(stage_base + (size_t)(pp.batch_rows + lane) * pp.slot_floats, f + (int64_t)lane * f_pitch + c0, f_bytes,
-                          &full_bar[stage]);
       }
     }
     if (*(volatile int*)abort_flag) pipe::drain_delay();
@@ -349,58 +402,89 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
     const int lane = tid & 31, warp = tid >> 5;
     const int dc_mod4 = (int)(d_c & 3);
     uint32_t it = 0;
-    for (int b0 = 0; b0 < P; b0 += pp.batch_rows) {
-      const int nb = min(pp.batch_rows, P - b0);
-      const int nr = warp < nb ? (nb - warp + kPipeWarps - 1) / kPipeWarps : 0;    // rows warp, warp + 8, ... below nb
-      int shift[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) shift[j] = (((b0 + warp + 8 * j) & 3) * dc_mod4) & 3;   // (row * d_c + c0) mod 4
-      double rho[4][K], nu[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        nu[j] = 0.0;
-#pragma unroll
-        for (int kappa = 0; kappa < K; ++kappa) rho[j][kappa] = 0.0;
+    for (int part = 0; part < 2; ++part) {
+      const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
+      double* mine = part_sums[part];
+      if (lo >= hi) {
+        for (int i = tid; i < n_acc; i += kPipeConsumers) mine[i] = 0.0;      // nothing of this part in this CTA's range
       }
-      for (int64_t c0 = c_begin; c0 < c_end; c0 += pp.slice_cols, ++it) {
-        const int stage = it % kPipeStages;
-        const uint32_t phase = (it / kPipeStages) & 1;
-        pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
-        const int cols = (int)((c_end - c0) < pp.slice_cols ? (c_end - c0) : pp.slice_cols);
-        const float* base = ring + stage * stage_floats;
-        const float* fs = base + (size_t)pp.batch_rows * pp.slot_floats;
-        const float* rows[4];
+      for (int b0 = 0; b0 < P && lo < hi; b0 += pp.batch_rows) {
+        const int nb = min(pp.batch_rows, P - b0);
+        const int nr = warp < nb ? (nb - warp + kPipeWarps - 1) / kPipeWarps : 0;    // rows warp, warp + 8, ... below nb
+        int shift[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) rows[j] = base + (size_t)(warp + 8 * j) * pp.slot_floats + shift[j];
-        if (nr == 4) pipe_consume<K, 4>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
-        else if (nr == 3) pipe_consume<K, 3>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
-        else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
-        else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
-        __syncwarp();
-        if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
-      }
+        for (int j = 0; j < 4; ++j) shift[j] = (((b0 + warp + 8 * j) & 3) * dc_mod4) & 3;   // (row * d_c + c0) mod 4
+        double rho[4][K], nu[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (j < nr) {
-          const int row = b0 + warp + 8 * j;
+        for (int j = 0; j < 4; ++j) {
+          nu[j] = 0.0;
 #pragma unroll
-          for (int kappa = 0; kappa < K; ++kappa) {
-            const double t = warp_sum(rho[j][kappa]);
-            if (lane == 0) mine[(size_t)kappa * P + row] = t;
-          }
-          const double t = warp_sum(nu[j]);
-          if (lane == 0) mine[(size_t)K * P + row] = t;
+          for (int kappa = 0; kappa < K; ++kappa) rho[j][kappa] = 0.0;
         }
+        for (int64_t c0 = lo; c0 < hi; c0 += pp.slice_cols, ++it) {
+          const int stage = it % kPipeStages;
+          const uint32_t phase = (it / kPipeStages) & 1;
+          pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
+          const int cols = (int)((hi - c0) < pp.slice_cols ? (hi - c0) : pp.slice_cols);
+          const float* base = ring + stage * stage_floats;
+          const float* fs = base + (size_t)pp.batch_rows * pp.slot_floats;
+          const float* rows[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) rows[j] = base + (size_t)(warp + 8 * j) * pp.slot_floats + shift[j];
+          if (nr == 4) pipe_consume<K, 4>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+          else if (nr == 3) pipe_consume<K, 3>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+          else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+          else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+          __syncwarp();
+          if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (j < nr) {
+            const int row = b0 + warp + 8 * j;
+#pragma unroll
+            for (int kappa = 0; kappa < K; ++kappa) {
+              const double t = warp_sum(rho[j][kappa]);
+              if (lane == 0) mine[(size_t)kappa * P + row] = t;
+            }
+            const double t = warp_sum(nu[j]);
+            if (lane == 0) mine[(size_t)K * P + row] = t;
+          }
+        }
+      }
+      if (part == 0) {
+        // part A is complete in this CTA: the consumers alone (the producer is already fetching part B) add their
+        // bunch if they are the last of it, and tell the locator kernel
+        const bool done = bunch_reduce<SyncConsumers>(partials, nullptr, bunch_a, n_acc, ticket + 1 + n_bunches, &s_flag, tid,
+                                                      kPipeConsumers);
+        if (done && tid == 0) atomicAdd(pp.progress, 1ULL);
       }
     }
   }
-  reduce_partials(partials, n_acc, K * P, rho_out, nu_out, ticket, final_reduce);
+  // final sums of a bunch = its part-A sums + its members' part-B sums
+  const bool done = bunch_reduce<SyncAll>(partials + (size_t)gridDim.x * n_acc, bunch_a, bunch_f, n_acc, ticket + 1, &s_flag, tid,
+                                          kPipeThreads);
+  if (!done || !final_reduce) return;
+  // the last bunch to finish adds the bunch sums
+  if (tid == 0) s_flag = atomicAdd(ticket, 1u);
+  __syncthreads();
+  if (s_flag != n_bunches - 1) return;
+  __threadfence();
+  for (int i = tid; i < n_acc; i += kPipeThreads) {
+    double acc = 0.0;
+#pragma unroll 4
+    for (unsigned int b = 0; b < n_bunches; ++b) acc += __ldcg(bunch_f + (size_t)b * n_acc + i);
+    if (i < K * P) rho_out[i] = acc;
+    else nu_out[i - K * P] = acc;
+  }
+  if (tid == 0) *ticket = 0u;
 }
 
 template <int K>
 static int launch_project_pipe_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out, int final_reduce) {
   ProjPipe pp;
   pp.status = plan->d_status;
+  pp.progress = plan->d_proj_progress;
   // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
   const size_t per_cta = (size_t)227 * 1024 / 2 - 1024 - 128;
   const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
@@ -411,20 +495,28 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   int grid = plan->num_sms * 2;
   if (grid > plan->proj_grid) grid = plan->proj_grid;
   // leave one slot per group free: the locator's CTAs (launched as dependents) then become resident while this
-  // kernel streams and use the time to stage their tables and fetch their code
+  // kernel streams and use the time to stage their tables and work on part A
   if (plan->q <= plan->num_sms / 2 && grid >= 4 * plan->q) grid -= plan->q;
   int64_t range_len = (plan->d_c + grid - 1) / grid;
   range_len = (range_len + 3) / 4 * 4;
   if (range_len < slice) slice = (int)((range_len + 31) / 32 * 32);
   pp.slice_cols = slice;
   pp.slot_floats = slice + 8;
+  // part A: about an eighth of the range, whole slices, at least one
+  int64_t a_slices = range_len / slice / 8;
+  if (a_slices < 1) a_slices = 1;
+  pp.part_a_cols = a_slices * slice;
   const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows + K) * pp.slot_floats * sizeof(float);
   SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   project_pipe_kernel<K><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->f_pitch, plan->P, plan->d_c,
                                                                      range_len, pp, plan->d_partials, rho_out, nu_out,
                                                                      plan->d_proj_ticket, final_reduce);
-  plan->proj_bunches = final_reduce ? 0 : (grid + kProjBunch - 1) / kProjBunch;
-  plan->proj_bunch_sums = plan->d_partials + (size_t)grid * (K + 1) * plan->P;
+  const int n_bunches = (grid + kProjBunch - 1) / kProjBunch;
+  const size_t n_acc = (size_t)(K + 1) * plan->P;
+  plan->proj_bunches = final_reduce ? 0 : n_bunches;
+  plan->proj_bunch_a = plan->d_partials + 2 * (size_t)grid * n_acc;
+  plan->proj_bunch_sums = plan->proj_bunch_a + (size_t)n_bunches * n_acc;
+  plan->proj_progress_target += (unsigned long long)n_bunches;     // progress[0] after this launch's part A
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }

@@ -68,8 +68,12 @@ struct solon_plan {
   // projection workspace
   int proj_grid;           // CTAs of the projection kernel = number of partial sums
   double* d_partials;      // proj_grid x (K + 1) x P
+  int early_locator;       // 0 never, 1 by size, 2 whenever the solver is small (solon_plan_set_early_locator)
   int proj_bunches;        // > 0: the last projection launch left this many bunch sums for the locator to add
-  const double* proj_bunch_sums;   // proj_bunches x (K + 1) x P
+  const double* proj_bunch_sums;   // proj_bunches x (K + 1) x P: final sums
+  const double* proj_bunch_a;      // same shape: sums over part A of the column ranges only
+  unsigned long long* d_proj_progress;          // [0] bunches done with part A, cumulative over launches
+  unsigned long long proj_progress_target;      // its value once the most recent launch's part A is complete
   double* d_rho;           // K x P
   double* d_nu;            // P
   unsigned int* d_proj_ticket;   // 1
@@ -81,6 +85,7 @@ struct solon_plan {
   int* d_n_rec;            // q
   int* d_rec_rows;         // P   (global node index of the j-th recovery row of group g at start[g] + j)
   double* d_coeff;         // P x m
+  int* d_early;            // q: 0 no early run, 1 early answer confirmed, 2 not confirmed, 3 the wait for part A expired
   int* d_status;           // [0] status bits of the last decode, [1] sticky bits (expired waits)
   unsigned long long* d_tile_counter;   // [0] the recovery kernel's next tile (the locator kernel zeroes it);
                                         // [1], [2] the encode kernel's next tile and departed CTAs (it zeroes them itself)
