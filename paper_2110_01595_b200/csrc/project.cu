@@ -351,7 +351,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
   const int64_t c_begin = (int64_t)blockIdx.x * range_len;     // multiple of 4
   int64_t c_end = c_begin + range_len;
   if (c_end > d_c) c_end = d_c;
-  int64_t c_mid = c_begin + pp.part_a_cols;                    // part_a_cols is a multiple of the slice width
+  int64_t c_mid = c_begin + pp.part_a_cols;                    // part_a_cols is a multiple of the slice width (0: one part)
   if (c_mid > c_end) c_mid = c_end;
   const int64_t total_floats = (int64_t)P * d_c;
   const unsigned int n_bunches = (gridDim.x + kProjBunch - 1) / kProjBunch;
@@ -362,7 +362,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
   if (tid >= kPipeConsumers) {
     const int lane = tid - kPipeConsumers;
     uint32_t it = 0;
-    for (int part = 0; part < 2; ++part) {
+    for (int part = pp.part_a_cols > 0 ? 0 : 1; part < 2; ++part) {
       const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
       for (int b0 = 0; b0 < P && lo < hi; b0 += pp.batch_rows) {
         const int nb = min(pp.batch_rows, P - b0);
@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
     const int lane = tid & 31, warp = tid >> 5;
     const int dc_mod4 = (int)(d_c & 3);
     uint32_t it = 0;
-    for (int part = 0; part < 2; ++part) {
+    for (int part = pp.part_a_cols > 0 ? 0 : 1; part < 2; ++part) {
       const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
       double* mine = part_sums[part];
       if (lo >= hi) {
@@ -462,7 +462,8 @@ __global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const flo
     }
   }
   // final sums of a bunch = its part-A sums + its members' part-B sums
-  const bool done = bunch_reduce<SyncAll>(partials + (size_t)gridDim.x * n_acc, bunch_a, bunch_f, n_acc, ticket + 1, &s_flag, tid,
+  const bool done = bunch_reduce<SyncAll>(partials + (size_t)gridDim.x * n_acc, pp.part_a_cols > 0 ? bunch_a : nullptr, bunch_f, n_acc,
+                                          ticket + 1, &s_flag, tid,
                                           kPipeThreads);
   if (!done || !final_reduce) return;
   // the last bunch to finish adds the bunch sums
@@ -502,10 +503,11 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   if (range_len < slice) slice = (int)((range_len + 31) / 32 * 32);
   pp.slice_cols = slice;
   pp.slot_floats = slice + 8;
-  // part A: about an eighth of the range, whole slices, at least one
+  // part A (only when the locator kernel will work ahead on it): about an eighth of the range, whole slices, at least one
   int64_t a_slices = range_len / slice / 8;
   if (a_slices < 1) a_slices = 1;
-  pp.part_a_cols = a_slices * slice;
+  const bool two_parts = !final_reduce && uses_early_locator(plan);
+  pp.part_a_cols = two_parts ? a_slices * slice : 0;
   const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows + K) * pp.slot_floats * sizeof(float);
   SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   project_pipe_kernel<K><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->f_pitch, plan->P, plan->d_c,
@@ -516,7 +518,8 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   plan->proj_bunches = final_reduce ? 0 : n_bunches;
   plan->proj_bunch_a = plan->d_partials + 2 * (size_t)grid * n_acc;
   plan->proj_bunch_sums = plan->proj_bunch_a + (size_t)n_bunches * n_acc;
-  plan->proj_progress_target += (unsigned long long)n_bunches;     // progress[0] after this launch's part A
+  if (two_parts) plan->proj_progress_target += (unsigned long long)n_bunches;     // progress[0] after this launch's part A
+  plan->proj_two_parts = two_parts ? 1 : 0;
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }

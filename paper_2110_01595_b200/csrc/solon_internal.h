@@ -68,6 +68,7 @@ struct solon_plan {
   // projection workspace
   int proj_grid;           // CTAs of the projection kernel = number of partial sums
   double* d_partials;      // proj_grid x (K + 1) x P
+  int proj_two_parts;      // the last projection launch announced part A
   int early_locator;       // 0 never, 1 by size, 2 whenever the solver is small (solon_plan_set_early_locator)
   int proj_bunches;        // > 0: the last projection launch left this many bunch sums for the locator to add
   const double* proj_bunch_sums;   // proj_bunches x (K + 1) x P: final sums
@@ -138,6 +139,14 @@ static inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 blo
 #endif
 
 // Kernel launchers (each enqueues on plan->stream and returns a solon_status).
+// Whether solon_decode lets the locator work ahead on a partial projection (solon_plan_set_early_locator): a small
+// solver, and either mode 2 or a projection pass long enough (about 6 GB per ms) to hide the early run.
+inline bool uses_early_locator(const solon_plan* plan) {
+  const bool small_solver = plan->s > 0 && plan->max_group <= 64 && plan->s <= 5;
+  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 300e6;
+  return small_solver && (plan->early_locator == 2 || (plan->early_locator == 1 && long_pass));
+}
+
 int launch_fill_projection(solon_plan* plan);
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
 // rho_out / nu_out (and rho / nu below): device buffers, or nullptr for the plan's own
