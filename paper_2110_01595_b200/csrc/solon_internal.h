@@ -140,10 +140,11 @@ static inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 blo
 
 // Kernel launchers (each enqueues on plan->stream and returns a solon_status).
 // Whether solon_decode lets the locator work ahead on a partial projection (solon_plan_set_early_locator): a small
-// solver, and either mode 2 or a projection pass long enough (about 6 GB per ms) to hide the early run.
+// solver, and either mode 2 or a projection pass long enough to hide the early run, which takes 60-80 us beside
+// a streaming kernel (the projection kernel moves about 6 GB per ms).
 inline bool uses_early_locator(const solon_plan* plan) {
   const bool small_solver = plan->s > 0 && plan->max_group <= 64 && plan->s <= 5;
-  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 300e6;
+  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 500e6;
   return small_solver && (plan->early_locator == 2 || (plan->early_locator == 1 && long_pass));
 }
 
