@@ -156,7 +156,10 @@ int solon_encode(solon_plan* plan, const float* partition_grads, float* coded);
  *   agg_grad  device, d: receives u = sum over groups of the recovered group sums = G 1_P
  *   byz_mask  device, P bytes: 1 for every node located as Byzantine, else 0
  * Three kernels: projections rho = f R and row energies (one pass over `received`), the locator
- * (tiny, on device), the recovery (one pass over the trusted rows it needs).  If some group has
+ * (tiny, on device; see solon_plan_set_early_locator for how it overlaps the first), the recovery
+ * (one pass over the trusted rows it needs).  The projections are computed with float32
+ * products and float32 sums of eight terms at a time, float64 beyond (error at most
+ * 8 * 2^-24 of sum |f_p R_kp|, far below the locator's tolerance).  If some group has
  * no consistent set of at most s corrupt nodes the outputs hold a best guess and
  * solon_decode_status reports SOLON_ERR_UNDECODABLE. */
 int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask);

@@ -3,7 +3,9 @@
 //
 // One CTA per group; warp t of it assumes exactly t corrupt nodes, so all error counts are tried
 // concurrently.  The CTA then picks the smallest accepted count, writes the group's part of the mask and
-// builds the recovery table.
+// builds the recovery table.  The kernel is launched as a programmatic dependent of the projection kernel
+// and can do all of that ahead of time on a partial projection, leaving only a check for afterwards (see the
+// comment on the passes inside the kernel).
 #include <vector>
 
 #include "locate_core.cuh"
