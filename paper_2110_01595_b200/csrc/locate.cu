@@ -33,8 +33,8 @@ struct LocateParams {
   double* rho_w;              // with n_bunches > 0 the sums are also written here (K x P) and to nu_w (P)
   double* nu_w;
   const double* bunch_a;      // same shape as bunch_sums: the sums over part A of the projection kernel's column ranges
-  const unsigned long long* progress;   // bunches whose part-A sums are complete (cumulative over launches)
-  unsigned long long progress_target;   // its value once this decode's part A is complete
+  const unsigned long long* progress;   // bunches whose part-A sums are complete in this decode
+  unsigned long long progress_target;   // its value once part A is complete
   int* early;                 // q: outcome of the early run per group (see solon_plan_get_early_outcome)
   int spec;                   // work on part A while the projection kernel streams part B, then only check the result
   unsigned long long* tile_counter;   // work counter of the recovery kernel, zeroed here

@@ -225,7 +225,7 @@ struct ProjPipe {
   int slot_floats;    // slice_cols + 8: room for the alignment shift and the rounded-up end
   int batch_rows;     // rows per batch (<= kPipeRows), the same for all batches but the last
   int64_t part_a_cols;                // columns of part A in every CTA's range (whole slices)
-  unsigned long long* progress;       // [0] bunches whose part-A sums are complete, counted over all launches
+  unsigned long long* progress;       // [0] bunches whose part-A sums are complete (zeroed by the recovery kernel)
   int* status;
 };
 
@@ -518,7 +518,7 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   plan->proj_bunches = final_reduce ? 0 : n_bunches;
   plan->proj_bunch_a = plan->d_partials + 2 * (size_t)grid * n_acc;
   plan->proj_bunch_sums = plan->proj_bunch_a + (size_t)n_bunches * n_acc;
-  if (two_parts) plan->proj_progress_target += (unsigned long long)n_bunches;     // progress[0] after this launch's part A
+  plan->proj_progress_target = (unsigned long long)n_bunches;     // progress[0] once part A is complete (the recovery kernel zeroes it)
   plan->proj_two_parts = two_parts ? 1 : 0;
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;

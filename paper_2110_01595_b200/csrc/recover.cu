@@ -22,6 +22,7 @@ struct RecoverParams {
   const int* n_rec;      // q
   const int* rec_rows;   // P, group g's rows at [group_start[g], +n_rec[g])
   const double* coeff;   // P x m, same indexing
+  unsigned long long* proj_progress;   // the projection kernel's part-A count, zeroed here for the next decode
 };
 
 // Copy the locator's tables (group layout, rows per group, row indices, weights) into shared memory.
@@ -107,6 +108,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     pipe::fence_barrier_init();
   }
   pdl_wait();   // the locator's mask and table are complete and visible; nothing above touched global memory
+  if (blockIdx.x == 0 && tid == 0) *prm.proj_progress = 0ULL;   // every locator CTA is done with it: ready for the next decode
   const int n_rows = pack_tables(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
@@ -243,6 +245,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   int* start_s = rows_s + prm.P;
   int* n_rec_s = start_s + prm.q + 1;
   load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
+  if (blockIdx.x == 0 && threadIdx.x == 0) *prm.proj_progress = 0ULL;   // ready for the next decode
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < prm.d; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t p = e / prm.m;
     const int l = (int)(e - p * prm.m);
@@ -316,6 +319,7 @@ int launch_recover(solon_plan* plan, const float* received, float* agg) {
   prm.n_rec = plan->d_n_rec;
   prm.rec_rows = plan->d_rec_rows;
   prm.coeff = plan->d_coeff;
+  prm.proj_progress = plan->d_proj_progress;
   plan->launches += 1;
 #define SOLON_RECOVER_CASE(M_, CPT_, ACC_) \
   case M_:                                 \

@@ -73,8 +73,8 @@ struct solon_plan {
   int proj_bunches;        // > 0: the last projection launch left this many bunch sums for the locator to add
   const double* proj_bunch_sums;   // proj_bunches x (K + 1) x P: final sums
   const double* proj_bunch_a;      // same shape: sums over part A of the column ranges only
-  unsigned long long* d_proj_progress;          // [0] bunches done with part A, cumulative over launches
-  unsigned long long proj_progress_target;      // its value once the most recent launch's part A is complete
+  unsigned long long* d_proj_progress;          // [0] bunches done with part A in the current decode (the recovery kernel zeroes it)
+  unsigned long long proj_progress_target;      // its value once part A is complete
   double* d_rho;           // K x P
   double* d_nu;            // P
   unsigned int* d_proj_ticket;   // 1
