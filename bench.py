@@ -217,7 +217,7 @@ def run_ours(args, wl):
     coded = plan.encode(G)
     nodes = synth.byzantine_nodes(wl_rank)
     byz_rows = synth.byzantine_rows(wl_rank, coded, nodes)
-    nodes_dev = torch.tensor(nodes, dtype=torch.long, device="cuda")
+    nodes_dev = torch.tensor(nodes, dtype=torch.int32, device="cuda")
     agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
     mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
 
@@ -227,8 +227,7 @@ def run_ours(args, wl):
         plan.encode(G, coded)
         if events is not None:
             events[1].record()
-        if nodes:
-            coded.index_copy_(0, nodes_dev, byz_rows)         # the adversary: one device-to-device row copy
+        plan.overwrite_rows(coded, nodes_dev, byz_rows)       # the adversary: one device-to-device row copy
         if events is not None:
             events[2].record()
         if sp is not None:
@@ -356,7 +355,7 @@ def run_sweep(args):
             coded = plan.encode(G)
             nodes = synth.byzantine_nodes(wl)
             byz_rows = synth.byzantine_rows(wl, coded, nodes)
-            nodes_dev = torch.tensor(nodes, dtype=torch.long, device="cuda")
+            nodes_dev = torch.tensor(nodes, dtype=torch.int32, device="cuda")
             agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
             mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
 
@@ -366,8 +365,7 @@ def run_sweep(args):
                 plan.encode(G, coded)
                 if ev:
                     ev[1].record()
-                if nodes:
-                    coded.index_copy_(0, nodes_dev, byz_rows)
+                plan.overwrite_rows(coded, nodes_dev, byz_rows)
                 if ev:
                     ev[2].record()
                 plan.decode(coded, agg, mask)

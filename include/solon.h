@@ -208,6 +208,14 @@ int solon_lsq_grads(solon_plan* plan, const float* X, const float* y, const floa
 int solon_step_host(solon_plan* plan, const float* grads_host, int n_byz, const int* byz_nodes,
                     const float* byz_rows_host, float* agg_host, uint8_t* mask_host);
 
+/* The adversary of a device-resident simulation: overwrites rows of a P x d_c matrix in place,
+ * matrix[nodes[i]][:] = rows[i][:], on the plan's stream (what solon_step_host does from host
+ * buffers).  Not part of the method: it stands in for whatever the Byzantine nodes send.
+ *   matrix  device, P x d_c          nodes  device, n_rows ints in [0, P) (checked on the device:
+ *   rows    device, n_rows x d_c            out-of-range entries are skipped)
+ * n_rows = 0 does nothing. */
+int solon_overwrite_rows(solon_plan* plan, float* matrix, int n_rows, const int* nodes, const float* rows);
+
 /* ------------------------------------------------------------------------------------------
  * Introspection of the last decode (for parity tests and diagnostics; each synchronises).
  * ---------------------------------------------------------------------------------------- */

@@ -54,6 +54,7 @@ SIGNATURES = {
     "solon_decode_project": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_decode_finish": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_lsq_grads": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "solon_overwrite_rows": (c_int, [c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "solon_step_host": (c_int, [c_void_p, c_void_p, c_int, POINTER(c_int), c_void_p, c_void_p, c_void_p]),
     "solon_plan_get_projections": (c_int, [c_void_p, POINTER(c_double), POINTER(c_double)]),
     "solon_plan_get_recovery": (c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_double)]),
@@ -305,6 +306,17 @@ class Plan:
                                          self._dev(received, (self.P, self.d_c)), self._dev(agg_grad, (self.d,)),
                                          self._dev(byz_mask, (self.P,), torch.uint8)), "solon_decode_finish")
         return agg_grad, byz_mask
+
+    def overwrite_rows(self, matrix, nodes, rows):
+        """matrix[nodes[i]] = rows[i] on the plan's stream (the adversary of a device-resident simulation).
+        nodes: int32 CUDA tensor; rows: len(nodes) x d_c float32 CUDA tensor."""
+        torch = self._torch
+        n = int(nodes.numel())
+        if n == 0:
+            return matrix
+        _check(lib().solon_overwrite_rows(self._h, self._dev(matrix, (self.P, self.d_c)), n, self._dev(nodes, (n,), torch.int32),
+                                          self._dev(rows, (n, self.d_c))), "solon_overwrite_rows")
+        return matrix
 
     def decode_status(self) -> int:
         return lib().solon_decode_status(self._h)

@@ -43,6 +43,57 @@ extern "C" int solon_decode_finish(solon_plan* plan, const double* rho, const do
   return launch_recover(plan, received, agg_grad);
 }
 
+// Row overwrite for device-resident simulations: one streaming copy for all rows.
+__global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__ matrix, const float* __restrict__ rows,
+                                                             const int* __restrict__ nodes, int P, int64_t d_c, int vec) {
+  const int node = nodes[blockIdx.y];
+  if (node < 0 || node >= P) return;
+  float* dst = matrix + (int64_t)node * d_c;
+  const float* src = rows + (int64_t)blockIdx.y * d_c;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (vec) {   // d_c a multiple of 4 and both bases 16-byte aligned: every row starts on a 16-byte boundary
+    const int64_t n4 = d_c / 4;
+    float4* d4 = reinterpret_cast<float4*>(dst);
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    int64_t i = t0;
+    for (; i + 7 * stride < n4; i += 8 * stride) {     // eight loads in flight per thread
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = __ldcs(s4 + i + u * stride);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) d4[i + u * stride] = v[u];
+    }
+    for (; i < n4; i += stride) d4[i] = __ldcs(s4 + i);
+  } else {
+    int64_t i = t0;
+    for (; i + 7 * stride < d_c; i += 8 * stride) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + i + u * stride);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) dst[i + u * stride] = v[u];
+    }
+    for (; i < d_c; i += stride) dst[i] = __ldcs(src + i);
+  }
+}
+
+extern "C" int solon_overwrite_rows(solon_plan* plan, float* matrix, int n_rows, const int* nodes, const float* rows) {
+  if (!plan || n_rows < 0 || n_rows > plan->P) return SOLON_ERR_INVALID_ARG;
+  if (n_rows == 0) return SOLON_OK;
+  if (!matrix || !nodes || !rows) return SOLON_ERR_INVALID_ARG;
+  const int vec = (plan->d_c % 4 == 0 && !((uintptr_t)matrix & 15) && !((uintptr_t)rows & 15)) ? 1 : 0;
+  // one wave of CTAs (eight per SM) shared by the rows; every thread then has several batches of eight accesses
+  int64_t per_row = (plan->d_c / (vec ? 4 : 1) + 256 * 8 - 1) / (256 * 8);
+  int64_t cap = ((int64_t)plan->num_sms * 8 + n_rows - 1) / n_rows;
+  if (per_row > cap) per_row = cap;
+  if (per_row < 1) per_row = 1;
+  overwrite_rows_kernel<<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec);
+  SOLON_CUDA_TRY(cudaGetLastError());
+  plan->launches += 1;
+  return SOLON_OK;
+}
+
 template <typename T>
 static int stage_alloc(T** ptr, size_t count) {
   if (*ptr) return SOLON_OK;

@@ -219,6 +219,10 @@ constexpr int kPipeConsumers = 256;
 constexpr int kPipeWarps = kPipeConsumers / 32;
 constexpr int kPipeThreads = kPipeConsumers + 32;   // + one producer warp
 constexpr int kPipeStages = 2;
+#ifndef SOLON_PIPE_CTAS
+#define SOLON_PIPE_CTAS 2
+#endif
+constexpr int kPipeCtasPerSm = SOLON_PIPE_CTAS;
 
 struct ProjPipe {
   int slice_cols;     // columns per stage (multiple of 32)
@@ -323,7 +327,7 @@ __device__ __forceinline__ bool bunch_reduce(const double* __restrict__ partials
 // bunches and announced (progress[0]) on its own, so that the locator kernel can already work on a projection of
 // those columns - it is a random projection like any other - while part B streams; the final sums are A + B.
 template <int K>
-__global__ void __launch_bounds__(kPipeThreads, 2) project_pipe_kernel(const float* __restrict__ R, const float* __restrict__ f,
+__global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_kernel(const float* __restrict__ R, const float* __restrict__ f,
                                                                      int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
                                                                      ProjPipe pp, double* __restrict__ partials,
                                                                      double* __restrict__ rho_out, double* __restrict__ nu_out,
@@ -487,13 +491,13 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   pp.status = plan->d_status;
   pp.progress = plan->d_proj_progress;
   // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
-  const size_t per_cta = (size_t)227 * 1024 / 2 - 1024 - 128;
+  const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128;
   const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
   pp.batch_rows = (plan->P + n_batches - 1) / n_batches;
   int slice = (int)(per_cta / ((size_t)kPipeStages * (pp.batch_rows + K) * 4)) - 8;
   slice = slice / 32 * 32;
   if (slice > 2048) slice = 2048;
-  int grid = plan->num_sms * 2;
+  int grid = plan->num_sms * kPipeCtasPerSm;
   if (grid > plan->proj_grid) grid = plan->proj_grid;
   // leave one slot per group free: the locator's CTAs (launched as dependents) then become resident while this
   // kernel streams and use the time to stage their tables and work on part A

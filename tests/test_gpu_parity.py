@@ -286,6 +286,23 @@ def test_step_host_matches_device_path():
         assert np.abs(agg_h.numpy() - want).max() <= AGG_TOL * np.abs(want).max()
 
 
+@pytest.mark.parametrize("d", [40_000, 40_003])
+def test_overwrite_rows(d):
+    with binding.Plan(15, 2, 1, 5, d) as plan:      # m = 1: d_c = d, a multiple of 4 or not
+        g = torch.Generator(device="cuda").manual_seed(3)
+        matrix = torch.randn(15, d, device="cuda", generator=g)
+        before = matrix.clone()
+        rows = torch.randn(4, d, device="cuda", generator=g)
+        nodes = torch.tensor([14, 0, 99, 7], dtype=torch.int32, device="cuda")      # 99: out of range, skipped
+        plan.overwrite_rows(matrix, nodes, rows)
+        torch.cuda.synchronize()
+        want = before.clone()
+        want[14], want[0], want[7] = rows[0], rows[1], rows[3]
+        assert torch.equal(matrix, want)
+        plan.overwrite_rows(matrix, nodes[:0], rows[:0])                             # nothing to do
+        assert torch.equal(matrix, want)
+
+
 def test_argument_checks():
     with binding.Plan(8, 1, 2, 4, 64) as plan:
         lib = binding.lib()
