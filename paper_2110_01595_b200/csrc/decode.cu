@@ -7,7 +7,6 @@ using namespace solon;
 extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask) {
   if (!plan || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)received & 15) || ((uintptr_t)agg_grad & 15)) return SOLON_ERR_INVALID_ARG;
-  SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), plan->stream));
   int rc;
   const bool prof = plan->profiling != 0;
   auto mark = [&](int i) -> int {
@@ -37,7 +36,6 @@ extern "C" int solon_decode_finish(solon_plan* plan, const double* rho, const do
   if (!plan || !rho || !nu || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)received & 15) || ((uintptr_t)agg_grad & 15) || ((uintptr_t)rho & 7) || ((uintptr_t)nu & 7))
     return SOLON_ERR_INVALID_ARG;
-  SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), plan->stream));
   int rc;
   if ((rc = launch_locate(plan, byz_mask, rho, nu))) return rc;
   return launch_recover(plan, received, agg_grad);

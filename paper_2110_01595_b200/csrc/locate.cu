@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
       prm.early[g] = !prm.spec ? 0 : (s_ready ? 2 : 3);
-      if (!ok) atomicOr(prm.status, kStatusUndecodable);
+      (void)ok;      // an undecodable group is reported through t_acc[g] = -1
     }
   }
 }

@@ -6,6 +6,8 @@
 #include <new>
 
 #include "locate_core.cuh"
+#include <vector>
+
 #include "solon_internal.h"
 
 namespace solon {
@@ -419,11 +421,15 @@ int64_t solon_plan_kernel_launches(const solon_plan* plan) { return plan ? plan-
 
 int solon_decode_status(solon_plan* plan) {
   if (!plan) return SOLON_ERR_INVALID_ARG;
+  // the locator leaves the accepted error count of every group (-1: none); expired waits leave a sticky bit
+  std::vector<int> t_acc((size_t)plan->q, 0);
   int word[2] = {0, 0};
   SOLON_CUDA_TRY(cudaMemcpyAsync(word, plan->d_status, 2 * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaMemcpyAsync(t_acc.data(), plan->d_t_acc, (size_t)plan->q * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
   SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
   if ((word[0] | word[1]) & kStatusWaitExpired) return SOLON_ERR_INTERNAL;
-  if (word[0] & kStatusUndecodable) return SOLON_ERR_UNDECODABLE;
+  for (int g = 0; g < plan->q; ++g)
+    if (t_acc[(size_t)g] < 0) return SOLON_ERR_UNDECODABLE;
   return SOLON_OK;
 }
 
