@@ -262,9 +262,19 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       double* task = sc.tasks + (size_t)t * sc.task_stride;
       uint8_t* cand = reinterpret_cast<uint8_t*>(task);
       uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
-      if (t <= prm.s)      // warps beyond s + 1 only help with the CTA-wide steps
-        locate_task(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n,
-                    cand, bad, task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
+      if (t <= prm.s) {    // warps beyond s + 1 only help with the CTA-wide steps
+        double* tws = task + 2 * ((size_t)n / 8 + 1);
+        uint8_t* tflags = sc.flags + (size_t)t * n;
+        if (prm.s <= 2)
+          locate_task<2>(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, tflags, cand, bad, tws,
+                         &sc.recs[t]);
+        else if (prm.s <= 3)
+          locate_task<3>(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, tflags, cand, bad, tws,
+                         &sc.recs[t]);
+        else
+          locate_task<SOLON_FAST_T>(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, tflags, cand,
+                                    bad, tws, &sc.recs[t]);
+      }
     }
     __syncthreads();
     const int ok = locate_epilogue(cta, tb, n, prm.m, prm.s, sc.forced, sc.recs, sc.flags, n, sc.mask_l, &s_t_acc, sc.rows_l,
@@ -437,7 +447,7 @@ extern "C" int solon_locate_host(int n, int m, int s, int K, const double* rho, 
       double* task = sc.tasks + (size_t)t * sc.task_stride;
       uint8_t* cand = reinterpret_cast<uint8_t*>(task);
       uint8_t* bad = cand + 8 * ((size_t)n / 8 + 1);
-      locate_task(tm, tb, n, m, K, t, s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n, cand, bad,
+      locate_task<SOLON_FAST_T>(tm, tb, n, m, K, t, s, sc.rho_n, sc.forced, tau_eff, sc.flags + (size_t)t * n, cand, bad,
                   task + 2 * ((size_t)n / 8 + 1), &sc.recs[t]);
     }
   } else {

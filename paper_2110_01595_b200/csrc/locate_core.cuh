@@ -289,18 +289,21 @@ SOLON_HD inline void locate_verify(const Team& tm, const GroupTables& tb, int n,
   }
 }
 
-#define SOLON_FAST_T 5         /* error counts handled by the register-resident solver */
+#define SOLON_FAST_T 5         /* largest error count handled by the register-resident solver (locate_task<FT>, FT <= this) */
 #if defined(__CUDA_ARCH__)
 #define SOLON_FAST_RPL 2       /* rows per lane it can hold */
 #else
 #define SOLON_FAST_RPL 64
 #endif
 
-// One task: assume exactly t corrupt nodes among the n nodes of a group.
+// One task: assume exactly t corrupt nodes among the n nodes of a group.  FT: the register-resident solver is
+// compiled for error counts up to FT (the arithmetic does not depend on FT; a small FT is simply less code to
+// fetch for plans with a small s).
 //   rho_n   K x n projected values divided by the scale (0 for forced nodes)
 //   s       the plan's s (row stride of tb.Tch is s + 1);  tau  tolerance in the same normalised units
 //   flags   n bytes out: 1 for candidates that do not fit (the located nodes if accepted)
 //   cand, bad: n bytes of scratch each;  ws: locate_task_ws_doubles(n, m, K, t) doubles
+template <int FT>
 SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, int m, int K, int t, int s, const double* rho_n,
                                  const uint8_t* forced, double tau, uint8_t* flags, uint8_t* cand, uint8_t* bad,
                                  double* ws, TaskRecord* rec) {
@@ -318,34 +321,34 @@ SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, i
     const int nperp = n - m - t;               // complement of the polynomials of degree < m + t
     const int rows = K * nperp;
     double theta[SOLON_THETA_MAX];
-    if (tm.nwarps == 1 && t <= SOLON_FAST_T && rows <= SOLON_FAST_RPL * tm.nlanes) {
+    if (tm.nwarps == 1 && t <= FT && rows <= SOLON_FAST_RPL * tm.nlanes) {
       // Small system: every lane keeps its rows of [A | b] in registers.  Row (kappa, j), column i:
       //   sum_k q_{m+t+j}(w_k) rho_kappa,k T_i(w_k);  the last column carries -(...) T_t.
       // One combined lane reduction per Gram-Schmidt step yields the norm and all inner products.
-      double a[SOLON_FAST_RPL][SOLON_FAST_T + 1];
+      double a[SOLON_FAST_RPL][FT + 1];
       const int rpl = (rows + tm.nlanes - 1) / tm.nlanes;
 #pragma unroll
       for (int rr = 0; rr < SOLON_FAST_RPL; ++rr) {
         const int row = tm.lane + rr * tm.nlanes;
 #pragma unroll
-        for (int i = 0; i <= SOLON_FAST_T; ++i) a[rr][i] = 0.0;
+        for (int i = 0; i <= FT; ++i) a[rr][i] = 0.0;
         if (rr < rpl && row < rows) {
           const int kappa = row / nperp, j = row - kappa * nperp;
           const double* q = tb.Qb + (size_t)(m + t + j) * n;
           for (int k = 0; k < n; ++k) {
             const double qr = q[k] * rho_n[(size_t)kappa * n + k];
 #pragma unroll
-            for (int i = 0; i <= SOLON_FAST_T; ++i)
+            for (int i = 0; i <= FT; ++i)
               if (i <= t) a[rr][i] = fma(qr, tb.Tch[(size_t)k * ldt + i], a[rr][i]);
           }
 #pragma unroll
-          for (int i = 0; i <= SOLON_FAST_T; ++i)
+          for (int i = 0; i <= FT; ++i)
             if (i == t) a[rr][i] = -a[rr][i];
         }
       }
-      double R[SOLON_FAST_T][SOLON_FAST_T + 1], diag[SOLON_FAST_T], norm0[SOLON_FAST_T];
+      double R[FT][FT + 1], diag[FT], norm0[FT];
 #pragma unroll
-      for (int j = 0; j < SOLON_FAST_T; ++j) {
+      for (int j = 0; j < FT; ++j) {
         double v = 0.0;
 #pragma unroll
         for (int rr = 0; rr < SOLON_FAST_RPL; ++rr) v = fma(a[rr][j], a[rr][j], v);
@@ -354,22 +357,22 @@ SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, i
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) {
 #if defined(__CUDA_ARCH__)
-        double tmp[SOLON_FAST_T];
+        double tmp[FT];
 #pragma unroll
-        for (int j = 0; j < SOLON_FAST_T; ++j) tmp[j] = __shfl_xor_sync(0xffffffffu, norm0[j], off);
+        for (int j = 0; j < FT; ++j) tmp[j] = __shfl_xor_sync(0xffffffffu, norm0[j], off);
 #pragma unroll
-        for (int j = 0; j < SOLON_FAST_T; ++j) norm0[j] += tmp[j];
+        for (int j = 0; j < FT; ++j) norm0[j] += tmp[j];
 #endif
       }
 #pragma unroll
-      for (int j = 0; j < SOLON_FAST_T; ++j) {
+      for (int j = 0; j < FT; ++j) {
         diag[j] = 0.0;
 #pragma unroll
-        for (int c = 0; c <= SOLON_FAST_T; ++c) R[j][c] = 0.0;
+        for (int c = 0; c <= FT; ++c) R[j][c] = 0.0;
         if (j < t) {
-          double d[SOLON_FAST_T + 1];      // d[c] = a_j . a_c for c >= j (d[j] is the squared norm)
+          double d[FT + 1];      // d[c] = a_j . a_c for c >= j (d[j] is the squared norm)
 #pragma unroll
-          for (int c = 0; c <= SOLON_FAST_T; ++c) {
+          for (int c = 0; c <= FT; ++c) {
             double v = 0.0;
             if (c >= j && c <= t) {
 #pragma unroll
@@ -380,11 +383,11 @@ SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, i
 #if defined(__CUDA_ARCH__)
 #pragma unroll
           for (int off = 16; off > 0; off >>= 1) {
-            double tmp[SOLON_FAST_T + 1];
+            double tmp[FT + 1];
 #pragma unroll
-            for (int c = 0; c <= SOLON_FAST_T; ++c) tmp[c] = __shfl_xor_sync(0xffffffffu, d[c], off);
+            for (int c = 0; c <= FT; ++c) tmp[c] = __shfl_xor_sync(0xffffffffu, d[c], off);
 #pragma unroll
-            for (int c = 0; c <= SOLON_FAST_T; ++c) d[c] += tmp[c];
+            for (int c = 0; c <= FT; ++c) d[c] += tmp[c];
           }
 #endif
           const double nrm2 = d[j];
@@ -393,7 +396,7 @@ SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, i
           const double inv2 = dead ? 0.0 : 1.0 / nrm2;
           diag[j] = nrm;
 #pragma unroll
-          for (int c = 0; c <= SOLON_FAST_T; ++c) {
+          for (int c = 0; c <= FT; ++c) {
             if (c > j && c <= t) {
               const double coef = d[c] * inv2;
 #pragma unroll
@@ -404,14 +407,14 @@ SOLON_HD inline void locate_task(const Team& tm, const GroupTables& tb, int n, i
         }
       }
 #pragma unroll
-      for (int i = SOLON_FAST_T - 1; i >= 0; --i) {
+      for (int i = FT - 1; i >= 0; --i) {
         if (i < t) {
           double acc = 0.0;
 #pragma unroll
-          for (int c = 0; c <= SOLON_FAST_T; ++c)
+          for (int c = 0; c <= FT; ++c)
             if (c == t) acc = R[i][c];
 #pragma unroll
-          for (int c = 0; c < SOLON_FAST_T; ++c)
+          for (int c = 0; c < FT; ++c)
             if (c > i && c < t) acc = fma(-R[i][c], theta[c], acc);
           theta[i] = diag[i] > 0.0 ? acc / diag[i] : 0.0;
         }
