@@ -231,7 +231,9 @@ int solon_plan_get_recovery(solon_plan* plan, int* n_rec, int* t, int* rec_rows,
 
 /* Outcome of the early locator in the last solon_decode, one int per group (host, q entries):
  * 0 no early run, 1 the early answer was confirmed on the final projections, 2 it was not (the
- * whole locator ran), 3 the bounded wait for the partial projection expired (the whole locator ran). */
+ * whole locator ran), 3 the bounded wait for the partial projection expired (the whole locator
+ * ran), 4 the group's CTA became resident only after the projections were complete and skipped
+ * the early run. */
 int solon_plan_get_early_outcome(solon_plan* plan, int* outcome);
 
 /* Projections without any allocation.  (The paper has no counterpart: this entry point exists for

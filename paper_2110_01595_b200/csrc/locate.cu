@@ -33,7 +33,7 @@ struct LocateParams {
   double* rho_w;              // with n_bunches > 0 the sums are also written here (K x P) and to nu_w (P)
   double* nu_w;
   const double* bunch_a;      // same shape as bunch_sums: the sums over part A of the projection kernel's column ranges
-  const unsigned long long* progress;   // bunches whose part-A sums are complete in this decode
+  const unsigned long long* progress;   // bunches whose part-A sums [0] and final sums [1] are complete in this decode
   unsigned long long progress_target;   // its value once part A is complete
   int* early;                 // q: outcome of the early run per group (see solon_plan_get_early_outcome)
   int spec;                   // work on part A while the projection kernel streams part B, then only check the result
@@ -170,21 +170,26 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       // resident as a whole before this one could start and never waits for anything, so the count always comes.
       if (tid == 0) {
         int ready = 0;
-        const unsigned long long t_start = pipe_timer_ns();
-        for (;;) {
-          unsigned long long seen;
-          asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(prm.progress) : "memory");
-          if (seen >= prm.progress_target) {
-            ready = 1;
-            break;
+        unsigned long long seen;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(prm.progress + 1) : "memory");
+        if (seen >= prm.progress_target) {
+          ready = -1;      // this CTA became resident only after the projections were complete: nothing to gain
+        } else {
+          const unsigned long long t_start = pipe_timer_ns();
+          for (;;) {
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(prm.progress) : "memory");
+            if (seen >= prm.progress_target) {
+              ready = 1;
+              break;
+            }
+            if (pipe_timer_ns() - t_start > 2000000ull) break;
+            __nanosleep(200);
           }
-          if (pipe_timer_ns() - t_start > 2000000ull) break;
-          __nanosleep(200);
         }
         s_ready = ready;
       }
       __syncthreads();
-      if (!s_ready) continue;      // nothing to go on: pass 1 does all the work
+      if (s_ready <= 0) continue;      // nothing to go on: the last pass does all the work
     }
     if (prm.s == 0) {
       // pure compression code: nothing to locate, every node is trusted
@@ -292,7 +297,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
     if (tid == 0) {
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
-      prm.early[g] = !prm.spec ? 0 : (s_ready ? 2 : 3);
+      prm.early[g] = !prm.spec ? 0 : (s_ready > 0 ? 2 : (s_ready == 0 ? 3 : 4));
       (void)ok;      // an undecodable group is reported through t_acc[g] = -1
     }
   }

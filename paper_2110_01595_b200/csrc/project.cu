@@ -229,7 +229,7 @@ struct ProjPipe {
   int slot_floats;    // slice_cols + 8: room for the alignment shift and the rounded-up end
   int batch_rows;     // rows per batch (<= kPipeRows), the same for all batches but the last
   int64_t part_a_cols;                // columns of part A in every CTA's range (whole slices)
-  unsigned long long* progress;       // [0] bunches whose part-A sums are complete (zeroed by the recovery kernel)
+  unsigned long long* progress;       // bunches whose part-A sums [0] and final sums [1] are complete (zeroed by the recovery kernel)
   int* status;
 };
 
@@ -469,6 +469,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   const bool done = bunch_reduce<SyncAll>(partials + (size_t)gridDim.x * n_acc, pp.part_a_cols > 0 ? bunch_a : nullptr, bunch_f, n_acc,
                                           ticket + 1, &s_flag, tid,
                                           kPipeThreads);
+  if (done && tid == 0 && pp.part_a_cols > 0) atomicAdd(pp.progress + 1, 1ULL);   // a locator CTA that starts this late skips its early run
   if (!done || !final_reduce) return;
   // the last bunch to finish adds the bunch sums
   if (tid == 0) s_flag = atomicAdd(ticket, 1u);

@@ -108,7 +108,10 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     pipe::fence_barrier_init();
   }
   pdl_wait();   // the locator's mask and table are complete and visible; nothing above touched global memory
-  if (blockIdx.x == 0 && tid == 0) *prm.proj_progress = 0ULL;   // every locator CTA is done with it: ready for the next decode
+  if (blockIdx.x == 0 && tid == 0) {   // every locator CTA is done with them: ready for the next decode
+    prm.proj_progress[0] = 0ULL;
+    prm.proj_progress[1] = 0ULL;
+  }
   const int n_rows = pack_tables(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
@@ -245,7 +248,10 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   int* start_s = rows_s + prm.P;
   int* n_rec_s = start_s + prm.q + 1;
   load_tables(prm, coeff_s, rows_s, start_s, n_rec_s);
-  if (blockIdx.x == 0 && threadIdx.x == 0) *prm.proj_progress = 0ULL;   // ready for the next decode
+  if (blockIdx.x == 0 && threadIdx.x == 0) {   // ready for the next decode
+    prm.proj_progress[0] = 0ULL;
+    prm.proj_progress[1] = 0ULL;
+  }
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < prm.d; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t p = e / prm.m;
     const int l = (int)(e - p * prm.m);

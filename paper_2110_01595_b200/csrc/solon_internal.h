@@ -86,7 +86,7 @@ struct solon_plan {
   int* d_n_rec;            // q
   int* d_rec_rows;         // P   (global node index of the j-th recovery row of group g at start[g] + j)
   double* d_coeff;         // P x m
-  int* d_early;            // q: 0 no early run, 1 early answer confirmed, 2 not confirmed, 3 the wait for part A expired
+  int* d_early;            // q: 0 no early run, 1 early answer confirmed, 2 not confirmed, 3 the wait for part A expired, 4 started too late
   int* d_status;           // [0] status bits of the last decode, [1] sticky bits (expired waits)
   unsigned long long* d_tile_counter;   // [0] the recovery kernel's next tile (the locator kernel zeroes it);
                                         // [1], [2] the encode kernel's next tile and departed CTAs (it zeroes them itself)

@@ -14,6 +14,7 @@ from paper_2110_01595_b200 import binding, build, synth
 pytestmark = pytest.mark.gpu
 
 AGG_TOL = 1e-4
+SEEN = set()          # early outcomes observed over the module (1 confirmed, 2 rejected, 4 started too late)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -31,7 +32,8 @@ def _decode_all_modes(plan, received):
         out.append((status, agg.clone(), mask.clone(), n_rec.copy(), t_acc.copy(), rows.copy(), coeff.copy(),
                     plan.early_outcome().tolist()))
     assert set(out[0][7]) == {0}                       # mode 0 never runs early
-    assert set(out[1][7]) <= {1, 2}                    # mode 2 always does (small solvers), and the wait never expires
+    assert set(out[1][7]) <= {1, 2, 4}                 # mode 2 always tries (small solvers); the wait never expires
+    SEEN.update(out[1][7])
     return out
 
 
@@ -52,7 +54,7 @@ def test_modes_agree_on_named_workloads(name, d):
         assert res[0][0] == 0
         assert res[0][2].cpu().numpy().nonzero()[0].tolist() == nodes
         assert np.abs(res[0][1].cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
-        assert set(res[1][7]) == {1}                   # whole rows are replaced: the early run sees every attacker
+        assert set(res[1][7]) <= {1, 4}                # whole rows are replaced: an early run sees every attacker
 
 
 @pytest.mark.parametrize("P,s,m", [(15, 1, 1), (15, 3, 5), (15, 5, 2), (45, 5, 10), (105, 3, 5), (45, 1, 8)])
@@ -104,8 +106,8 @@ def test_corruption_confined_to_a_few_columns(where):
         assert np.abs(res[0][1].cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
         # groups are nodes 0-4, 5-9, 10-14; a group whose attackers the early run saw all of is confirmed
         expect = {"first": [1, 1, 1], "last": [2, 1, 1], "nan_last": [1, 1, 2], "first_and_last": [1, 2, 1]}
-        if where in expect:
-            assert res[1][7] == expect[where]
+        if where in expect:       # 4: that group's CTA became resident only after the projections and ran no early pass
+            assert all(got in (want_g, 4) for got, want_g in zip(res[1][7], expect[where]))
 
 
 def test_undecodable_and_reuse_with_the_early_locator():
@@ -126,3 +128,9 @@ def test_undecodable_and_reuse_with_the_early_locator():
         plan.decode_project(coded, rho, nu)
         agg2, mask2 = plan.decode_finish(rho, nu, coded)
         assert plan.decode_status() == 0 and torch.equal(agg, agg2) and torch.equal(mask, mask2)
+
+
+def test_both_early_outcomes_were_exercised():
+    """Runs after the cases above (same module, file order): the early answer was confirmed somewhere and rejected
+    somewhere, so both branches of the final pass are covered by the comparisons above."""
+    assert {1, 2} <= SEEN
