@@ -4,12 +4,16 @@
 // group are streamed through shared memory in batches by a producer warp that issues one bulk
 // asynchronous copy (cp.async.bulk, completion on an mbarrier) per row segment, so every gradient
 // byte is read from HBM exactly once and many kilobytes per SM are in flight without occupying
-// registers.  In the specialised kernels (m = 1, 2, 3, 5, 6, 10) each consumer thread owns whole chunks:
+// registers.  In the specialised kernels (m = 1..6, 8, 10) each consumer thread owns whole chunks:
 // it adds the r_g rows of its chunks into registers straight from the staged rows, then evaluates the
 // r_g polynomials sum_l w_k^l ybar[p m + l] by Horner's rule and stores one float32 per node (coalesced
-// along the chunk axis); no CTA-wide barrier is needed.  Arithmetic is float32 for m <= 6 and float64
-// (rounded once) for larger m, where the decoder's noise amplification leaves no room for the encoder's
-// rounding.  The generic kernel (any m) sums into a float64 ybar in shared memory first.
+// along the chunk axis); no CTA-wide barrier is needed.  The group sum ybar is accumulated in float32
+// in every specialised kernel: whatever rounding it carries is common to all nodes of the group, so the
+// coded values still lie on ONE polynomial (with coefficients ybar + delta) and the decoder returns
+// ybar + delta without amplifying delta.  Only the rounding that differs from node to node - the Horner
+// evaluation and the final rounding to float32 - is amplified by the decoder (about 2^(m-1)), so for
+// m > 6 the polynomials are evaluated in float64 and rounded once; for m <= 6 float32 is enough.  The
+// generic kernel (any m) sums into a float64 ybar in shared memory first.
 //
 // Row segments start at arbitrary 4-byte offsets (d need not be a multiple of 4): the copy starts at
 // the enclosing 16-byte boundary and consumers index from the remainder; the last few floats of the
@@ -42,11 +46,11 @@ struct EncodeParams {
 
 // Horner evaluation for all nodes of the group with the chunk held in registers.
 template <int M>
-__device__ __forceinline__ void mix_chunk(const double* __restrict__ y, const double* __restrict__ w_g, int r_g,
+__device__ __forceinline__ void mix_chunk(const float* __restrict__ y, const double* __restrict__ w_g, int r_g,
                                           float* __restrict__ out, int64_t out_stride) {
   double c[M];
 #pragma unroll
-  for (int l = 0; l < M; ++l) c[l] = y[l];
+  for (int l = 0; l < M; ++l) c[l] = (double)y[l];
   for (int k = 0; k < r_g; ++k) {
     double wk = w_g[k];
     double acc = c[M - 1];
@@ -56,12 +60,12 @@ __device__ __forceinline__ void mix_chunk(const double* __restrict__ y, const do
   }
 }
 
-__device__ __forceinline__ void mix_chunk_generic(const double* __restrict__ y, int m, const double* __restrict__ w_g,
+__device__ __forceinline__ void mix_chunk_generic(const float* __restrict__ y, int m, const double* __restrict__ w_g,
                                                   int r_g, float* __restrict__ out, int64_t out_stride) {
   for (int k = 0; k < r_g; ++k) {
     double wk = w_g[k];
-    double acc = y[m - 1];
-    for (int l = m - 2; l >= 0; --l) acc = fma(acc, wk, y[l]);
+    double acc = (double)y[m - 1];
+    for (int l = m - 2; l >= 0; --l) acc = fma(acc, wk, (double)y[l]);
     out[(int64_t)k * out_stride] = (float)acc;
   }
 }
@@ -74,14 +78,15 @@ __global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(EncodeParams prm
   const int tile_chunks = kEncConsumers * prm.chunks_per_thread;
   const int tile_floats = tile_chunks * m;
 
-  // shared memory: [barriers][w_g x 2][ybar x 2][stages x row_batch x slot]; w_g and ybar are double
-  // buffered by tile parity so that one consumer barrier per tile suffices
+  // shared memory: [barriers][w_g x 2][ybar x 2][stages x row_batch x slot]; w_g and ybar (float32, added up
+  // row by row in node order like in the specialised kernels) are double buffered by tile parity so that one
+  // consumer barrier per tile suffices
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + prm.stages;
   int* abort_flag = reinterpret_cast<int*>(empty_bar + prm.stages);
   double* w_s = reinterpret_cast<double*>(smem_raw + 256);
-  double* ybar = w_s + 2 * SOLON_MAX_GROUP;
-  float* ring = reinterpret_cast<float*>(ybar + 2 * (size_t)tile_floats);
+  float* ybar = reinterpret_cast<float*>(w_s + 2 * SOLON_MAX_GROUP);
+  float* ring = ybar + 2 * (size_t)((tile_floats + 3) & ~3);
   const size_t stage_floats = (size_t)prm.row_batch * prm.slot_floats;
 
   if (tid == 0) {
@@ -147,7 +152,7 @@ __global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(EncodeParams prm
       int64_t e1 = e0 + tile_floats;
       if (e1 > prm.d) e1 = prm.d;
       const int valid = (int)(e1 > e0 ? e1 - e0 : 0);
-      double* y = ybar + (size_t)parity * tile_floats;
+      float* y = ybar + (size_t)parity * ((tile_floats + 3) & ~3);
       double* w_g = w_s + (size_t)parity * SOLON_MAX_GROUP;
       for (int k = tid; k < r_g; k += kEncConsumers) w_g[k] = prm.w[row0 + k];
       const int d_mod4 = (int)(prm.d & 3), e0_mod4 = (int)(e0 & 3);
@@ -160,28 +165,29 @@ __global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(EncodeParams prm
         const float* base = ring + stage * stage_floats;
         // each thread owns elements tid + i * 256 of the tile, four at a time
         for (int eb = tid; eb < tile_floats; eb += 4 * kEncConsumers) {
-          double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
+          const bool i1 = eb + kEncConsumers < tile_floats, i2 = eb + 2 * kEncConsumers < tile_floats,
+                     i3 = eb + 3 * kEncConsumers < tile_floats;
+          float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+          if (b0 > 0) {   // carry on from the rows of the earlier batches
+            acc0 = y[eb];
+            if (i1) acc1 = y[eb + kEncConsumers];
+            if (i2) acc2 = y[eb + 2 * kEncConsumers];
+            if (i3) acc3 = y[eb + 3 * kEncConsumers];
+          }
           const bool v0 = eb < valid, v1 = eb + kEncConsumers < valid, v2 = eb + 2 * kEncConsumers < valid,
                      v3 = eb + 3 * kEncConsumers < valid;
           for (int j = 0; j < nb; ++j) {
             const int shift = ((((row0 + b0 + j) & 3) * d_mod4) + e0_mod4) & 3;   // (row * d + e0) mod 4
             const float* src = base + (size_t)j * prm.slot_floats + shift + eb;
-            if (v0) acc0 += (double)src[0];
-            if (v1) acc1 += (double)src[kEncConsumers];
-            if (v2) acc2 += (double)src[2 * kEncConsumers];
-            if (v3) acc3 += (double)src[3 * kEncConsumers];
+            if (v0) acc0 += src[0];
+            if (v1) acc1 += src[kEncConsumers];
+            if (v2) acc2 += src[2 * kEncConsumers];
+            if (v3) acc3 += src[3 * kEncConsumers];
           }
-          if (b0 == 0) {
-            y[eb] = acc0;
-            if (eb + kEncConsumers < tile_floats) y[eb + kEncConsumers] = acc1;
-            if (eb + 2 * kEncConsumers < tile_floats) y[eb + 2 * kEncConsumers] = acc2;
-            if (eb + 3 * kEncConsumers < tile_floats) y[eb + 3 * kEncConsumers] = acc3;
-          } else {
-            y[eb] += acc0;
-            if (eb + kEncConsumers < tile_floats) y[eb + kEncConsumers] += acc1;
-            if (eb + 2 * kEncConsumers < tile_floats) y[eb + 2 * kEncConsumers] += acc2;
-            if (eb + 3 * kEncConsumers < tile_floats) y[eb + 3 * kEncConsumers] += acc3;
-          }
+          y[eb] = acc0;
+          if (i1) y[eb + kEncConsumers] = acc1;
+          if (i2) y[eb + 2 * kEncConsumers] = acc2;
+          if (i3) y[eb + 3 * kEncConsumers] = acc3;
         }
         __syncwarp();
         if ((tid & 31) == 0) pipe::mbar_arrive(&empty_bar[stage]);
@@ -308,7 +314,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
   }
 
   const int d_mod4 = (int)(prm.d & 3);
-  Acc acc[CPT][M];
+  float acc[CPT][M];   // the group sum of this thread's chunks
   int row0 = 0, r_g = 0, valid = 0;
   int64_t e0 = 0, ct = 0;
   for (uint32_t it = 0;; ++it) {
@@ -328,7 +334,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 #pragma unroll
       for (int i = 0; i < CPT; ++i)
 #pragma unroll
-        for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
+        for (int l = 0; l < M; ++l) acc[i][l] = 0.0f;
     }
     const bool full_tile = valid == kTileFloats;
     const int nb = min(prm.row_batch, r_g - b0);
@@ -340,7 +346,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 #pragma unroll
         for (int i = 0; i < CPT; ++i)
 #pragma unroll
-          for (int l = 0; l < M; ++l) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
+          for (int l = 0; l < M; ++l) acc[i][l] += src[i * kEncConsumers * M + l];
         slot += prm.slot_floats;
         shift = (shift + d_mod4) & 3;
       }
@@ -351,7 +357,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
         for (int i = 0; i < CPT; ++i)
 #pragma unroll
           for (int l = 0; l < M; ++l)
-            if ((tid + i * kEncConsumers) * M + l < valid) acc[i][l] += (Acc)src[i * kEncConsumers * M + l];
+            if ((tid + i * kEncConsumers) * M + l < valid) acc[i][l] += src[i * kEncConsumers * M + l];
         slot += prm.slot_floats;
         shift = (shift + d_mod4) & 3;
       }
@@ -366,13 +372,18 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
     bool ok[CPT];
 #pragma unroll
     for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kEncConsumers < prm.d_c;
+    Acc c[CPT][M];   // the polynomial's coefficients in the precision of the evaluation
+#pragma unroll
+    for (int i = 0; i < CPT; ++i)
+#pragma unroll
+      for (int l = 0; l < M; ++l) c[i][l] = (Acc)acc[i][l];
     for (int k = 0; k < r_g; ++k) {
       const Acc wk = w_s[row0 + k];
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
-        Acc z = acc[i][M - 1];
+        Acc z = c[i][M - 1];
 #pragma unroll
-        for (int l = M - 2; l >= 0; --l) z = acc_fma<Acc>(z, wk, acc[i][l]);
+        for (int l = M - 2; l >= 0; --l) z = acc_fma<Acc>(z, wk, c[i][l]);
         if (ok[i]) out[i * kEncConsumers] = (float)z;
       }
       out += prm.d_c;
@@ -382,7 +393,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 
 static size_t encode_smem_bytes(int m, int cpt, int row_batch, int stages, int slot_floats) {
   size_t tile_floats = (size_t)kEncConsumers * cpt * m;
-  return 256 + 2 * SOLON_MAX_GROUP * sizeof(double) + 2 * tile_floats * sizeof(double) +
+  return 256 + 2 * SOLON_MAX_GROUP * sizeof(double) + 2 * ((tile_floats + 3) & ~(size_t)3) * sizeof(float) +
          (size_t)stages * row_batch * slot_floats * sizeof(float);
 }
 
@@ -481,9 +492,11 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
     case 1: return launch_encode_direct<1, 4, float, 3>(plan, prm);
     case 2: return launch_encode_direct<2, 2, float, 3>(plan, prm);
     case 3: return launch_encode_direct<3, 2, float, 3>(plan, prm);
+    case 4: return launch_encode_direct<4, 1, float, 3>(plan, prm);
     case 5: return launch_encode_direct<5, 1, float, 3>(plan, prm);
     case 6: return launch_encode_direct<6, 1, float, 3>(plan, prm);
-    case 10: return launch_encode_direct<10, 1, double, 2>(plan, prm);
+    case 8: return launch_encode_direct<8, 1, double, 3>(plan, prm);
+    case 10: return launch_encode_direct<10, 1, double, 3>(plan, prm);
     default: return launch_encode_generic<0>(plan, prm);
   }
 }

@@ -37,13 +37,15 @@ __device__ __forceinline__ void load_tables(const RecoverParams& prm, Acc* coeff
 }
 
 // The locator's tables, brought on chip in ONE parallel round trip (every load is independent of every other),
-// then the list of the table slots in use (all groups, in group order) built from the on-chip copies:
-//   coeff_s[slot * m + l], rows_s[slot] for slot in [group_start[g], group_start[g] + n_rec[g]); slots_s[i] = i-th
-//   slot in use.  Returns the number of slots in use.  start_s, n_rec_s: q + 1 and q ints of scratch.
-template <typename Acc>
+// then packed in order of use from the on-chip copies: the i-th row in use (all groups, in group order) has its
+// matrix row and its offset from a 16-byte boundary in rowsh_c[i] = (row << 2) | ((row * d_c) & 3) and its M
+// weights at coeff_c[i * STRIDE .. + M) (STRIDE: M rounded up so that every row of weights starts on a 16-byte
+// boundary and can be fetched with 128-bit loads).  Returns the number of rows in use.
+// coeff_s (P x M), rows_s, slots_s (P each), start_s (q + 1), n_rec_s (q): staging.
+template <typename Acc, int M, int STRIDE>
 __device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_s, Acc* coeff_s, int* slots_s, int* start_s,
-                                           int* n_rec_s, int* count_s) {
-  for (int i = threadIdx.x; i < prm.P * prm.m; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
+                                           int* n_rec_s, int* count_s, Acc* coeff_c, int* rowsh_c) {
+  for (int i = threadIdx.x; i < prm.P * M; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
   for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
   for (int i = threadIdx.x; i <= prm.q; i += blockDim.x) start_s[i] = prm.group_start[i];
   for (int i = threadIdx.x; i < prm.q; i += blockDim.x) n_rec_s[i] = prm.n_rec[i];
@@ -57,11 +59,47 @@ __device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_s
     if (g == prm.q - 1) *count_s = base + n;
   }
   __syncthreads();
-  return *count_s;
+  const int n_rows = *count_s;
+  const int dc_mod4 = (int)(prm.d_c & 3);
+  for (int i = threadIdx.x; i < n_rows; i += blockDim.x) {
+    const int row = rows_s[slots_s[i]];
+    rowsh_c[i] = (row << 2) | (((row & 3) * dc_mod4) & 3);
+  }
+  for (int i = threadIdx.x; i < n_rows * STRIDE; i += blockDim.x) {
+    const int r = i / STRIDE, l = i - r * STRIDE;
+    coeff_c[i] = l < M ? coeff_s[(size_t)slots_s[r] * M + l] : (Acc)0;
+  }
+  __syncthreads();
+  return n_rows;
 }
 
-// Bytes reserved for the P x M weight table in shared memory, rounded up to 16.
+// Bytes reserved for a P x M table of doubles in shared memory, rounded up to 16.
 __host__ __device__ inline size_t recover_coeff_bytes(int P, int M) { return ((size_t)P * M * sizeof(double) + 15) & ~(size_t)15; }
+// Weights per packed row: M rounded up to a whole number of 16-byte words.
+template <typename Acc, int M>
+struct PackedStride { static constexpr int value = (int)(((M * sizeof(Acc) + 15) / 16) * 16 / sizeof(Acc)); };
+
+// One packed row of weights from shared memory, 16 bytes per load.
+template <int STRIDE>
+__device__ __forceinline__ void load_weights(const float* __restrict__ src, float (&c)[STRIDE]) {
+#pragma unroll
+  for (int t = 0; t < STRIDE / 4; ++t) {
+    const float4 v = reinterpret_cast<const float4*>(src)[t];
+    c[4 * t] = v.x;
+    c[4 * t + 1] = v.y;
+    c[4 * t + 2] = v.z;
+    c[4 * t + 3] = v.w;
+  }
+}
+template <int STRIDE>
+__device__ __forceinline__ void load_weights(const double* __restrict__ src, double (&c)[STRIDE]) {
+#pragma unroll
+  for (int t = 0; t < STRIDE / 2; ++t) {
+    const double2 v = reinterpret_cast<const double2*>(src)[t];
+    c[2 * t] = v.x;
+    c[2 * t + 1] = v.y;
+  }
+}
 
 constexpr int kRecConsumers = 256;
 constexpr int kRecPipeThreads = kRecConsumers + 32;   // + one producer warp
@@ -90,10 +128,13 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
   int* abort_flag = b0_of + pp.stages;
   int* count_s = abort_flag + 1;
   // every region starts on a 16-byte boundary (128-bit shared loads, bulk-copy destinations)
-  Acc* coeff_p = reinterpret_cast<Acc*>(smem_raw + 256);                                  // P x M
-  int* rows_p = reinterpret_cast<int*>(smem_raw + 256 + recover_coeff_bytes(prm.P, M));   // P
+  constexpr int kStride = PackedStride<Acc, M>::value;
+  Acc* coeff_p = reinterpret_cast<Acc*>(smem_raw + 256);                                  // P x M (staging)
+  Acc* coeff_c = reinterpret_cast<Acc*>(smem_raw + 256 + recover_coeff_bytes(prm.P, M));  // P x kStride (packed)
+  int* rows_p = reinterpret_cast<int*>(smem_raw + 256 + recover_coeff_bytes(prm.P, M) + recover_coeff_bytes(prm.P, kStride));
   int* slots_p = rows_p + ((prm.P + 3) & ~3);                                             // P
-  int* start_s = slots_p + ((prm.P + 3) & ~3);                                            // q + 1
+  int* rowsh_c = slots_p + ((prm.P + 3) & ~3);                                            // P (packed)
+  int* start_s = rowsh_c + ((prm.P + 3) & ~3);                                            // q + 1
   int* n_rec_s = start_s + ((prm.q + 4) & ~3);                                            // q
   float* out_all = reinterpret_cast<float*>(n_rec_s + ((prm.q + 3) & ~3));                // 8 warps x 32 x M
   float* ring = out_all + (size_t)(kRecConsumers / 32) * 32 * M;                          // 32 M floats: 128 M bytes
@@ -112,7 +153,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     prm.proj_progress[0] = 0ULL;
     prm.proj_progress[1] = 0ULL;
   }
-  const int n_rows = pack_tables(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s);
+  const int n_rows = pack_tables<Acc, M, kStride>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
 
@@ -141,7 +182,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
           b0_of[stage] = b0;
         }
         if (lane < nb) {
-          const int64_t first = (int64_t)rows_p[slots_p[b0 + lane]] * prm.d_c + c0;
+          const int64_t first = (int64_t)(rowsh_c[b0 + lane] >> 2) * prm.d_c + c0;
           const int64_t last = first + (c1 - c0);
           const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
           int64_t a1 = (last + 3) & ~(int64_t)3;
@@ -179,9 +220,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
 
   const int lane = tid & 31, warp = tid >> 5;
   float* out_s = out_all + (size_t)warp * 32 * M;
-  const int dc_mod4 = (int)(prm.d_c & 3);
   Acc acc[CPT][M];
-  bool ok[CPT];
   for (uint32_t it = 0;; ++it) {
     const int stage = it % pp.stages;
     const uint32_t phase = (it / pp.stages) & 1;
@@ -189,32 +228,34 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     const long long tile = *(volatile long long*)&tile_of[stage];
     if (tile < 0 || *(volatile int*)abort_flag) break;
     const int b0 = *(volatile int*)&b0_of[stage];
-    const int64_t c0 = tile * kTileChunks;
+    const int64_t c0 = tile * kTileChunks;   // a multiple of 4: a row's offset from a 16-byte boundary is the same in every tile
     if (b0 == 0) {
 #pragma unroll
-      for (int i = 0; i < CPT; ++i) {
+      for (int i = 0; i < CPT; ++i)
 #pragma unroll
         for (int l = 0; l < M; ++l) acc[i][l] = (Acc)0;
-        ok[i] = c0 + tid + i * kRecConsumers < prm.d_c;
-      }
     }
+    // Chunks past the end of the matrix (last tile only) read whatever an earlier tile left in the ring: finite
+    // values, whose sums are never written back.
     const int nb = min(pp.row_batch, n_rows - b0);
     const float* slot = ring + stage * stage_floats + tid;
+    const int* rs = rowsh_c + b0;
+    const Acc* cj = coeff_c + (size_t)b0 * kStride;
+#pragma unroll 2
     for (int j = 0; j < nb; ++j) {
-      const int sl = slots_p[b0 + j];
-      const int shift = ((((rows_p[sl] & 3) * dc_mod4) + (int)(c0 & 3)) & 3);   // (row * d_c + c0) mod 4
-      const float* src = slot + shift;
+      const float* src = slot + (rs[j] & 3);
       Acc v[CPT];
 #pragma unroll
-      for (int i = 0; i < CPT; ++i) v[i] = ok[i] ? (Acc)src[i * kRecConsumers] : (Acc)0;
-      const Acc* cj = coeff_p + (size_t)sl * M;
+      for (int i = 0; i < CPT; ++i) v[i] = (Acc)src[i * kRecConsumers];
+      Acc c[kStride];
+      load_weights<kStride>(cj, c);
 #pragma unroll
       for (int l = 0; l < M; ++l) {
-        const Acc c = cj[l];
 #pragma unroll
-        for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c, v[i], acc[i][l]);
+        for (int i = 0; i < CPT; ++i) acc[i][l] = fma(c[l], v[i], acc[i][l]);
       }
       slot += pp.slot_floats;
+      cj += kStride;
     }
     __syncwarp();
     if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
@@ -272,7 +313,8 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   pp.status = plan->d_status;
   pp.slot_floats = kTileChunks + 8;
   const size_t slot_bytes = (size_t)pp.slot_floats * 4;
-  const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + 2 * (size_t)((plan->P + 3) & ~3) * sizeof(int) +
+  const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + recover_coeff_bytes(plan->P, PackedStride<Acc, M>::value) +
+                       3 * (size_t)((plan->P + 3) & ~3) * sizeof(int) +
                        (size_t)(((plan->q + 4) & ~3) + ((plan->q + 3) & ~3)) * sizeof(int) +
                        (size_t)(kRecConsumers / 32) * 32 * M * sizeof(float);
   // the locator may select up to all P rows (large m) or as few as q m; batches of about 20 KB

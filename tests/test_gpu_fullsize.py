@@ -47,7 +47,7 @@ def test_full_size(name):
         Z_s = so.encode(G_s, wl.m, sizes, w)                                       # P x len(chunks)
         got_Z = coded[:, torch.from_numpy(chunks).cuda()].cpu().numpy().astype(np.float64)
         bound = so.encode(np.abs(G_s), wl.m, sizes, np.abs(w))                     # sum of |terms|
-        ops = (max(sizes) + wl.m) if wl.m <= 6 else 1                              # float32 roundings, else one
+        ops = max(sizes) + wl.m                                                    # float32 roundings
         assert np.all(np.abs(got_Z - Z_s) <= ops * 2.0 ** -24 * bound * 1.0001 + 1e-45)
         # aggregate at the sampled coordinates against the plain float64 sum
         want_s = so.plain_sum(G_s)[in_range]

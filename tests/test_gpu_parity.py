@@ -30,19 +30,34 @@ def _oracle_plan(wl):
 
 
 def _check_encode(plan, G_cpu, coded_gpu, m, sizes, w):
-    """Coded vectors against the oracle's float64 values.  m > 6: float64 evaluation rounded once (half an ulp).
-    m <= 6: float32 sums and Horner steps, bounded by (r_g + m) roundings of the sum of absolute terms."""
-    Z = so.encode(G_cpu.numpy(), m, sizes, w)
+    """Coded vectors against the oracle's float64 values.
+
+    Every m: float32 group sums and (m <= 6) float32 Horner steps stay within (r_g + m) roundings of the sum of
+    absolute terms.  m > 6 in addition: the group sum is the float32 left-to-right sum ybar' of the group's rows
+    (its rounding is common to all nodes of the group, so the decoder returns it unamplified), and the coded
+    values are the float64 evaluation of the polynomial with coefficients ybar', rounded once: half an ulp from
+    the oracle's encoding of ybar'."""
+    G_np = G_cpu.numpy()
+    Z = so.encode(G_np, m, sizes, w)
     got = coded_gpu.cpu().numpy().astype(np.float64)
-    bound = so.encode(np.abs(G_cpu.numpy()), m, sizes, np.abs(w))          # sum of |terms| of every entry
+    bound = so.encode(np.abs(G_np), m, sizes, np.abs(w))          # sum of |terms| of every entry
     err = np.abs(got - Z)
+    ops = np.zeros((Z.shape[0], 1))
+    for start, size in zip(so.group_starts(sizes), sizes):
+        ops[start:start + size] = size + m
+    assert np.all(err <= ops * 2.0 ** -24 * bound + 1e-45), float((err / (bound + 1e-30)).max())
     if m > 6:
-        assert np.all(err <= 2.0 ** -24 * np.abs(Z) * 1.0001 + 1e-14 * bound + 1e-45), float((err / (np.abs(Z) + 1e-30)).max())
-    else:
-        ops = np.zeros((Z.shape[0], 1))
+        G_sum = np.zeros_like(G_np)                                # row `start` of each group: ybar', the others 0
         for start, size in zip(so.group_starts(sizes), sizes):
-            ops[start:start + size] = size + m
-        assert np.all(err <= ops * 2.0 ** -24 * bound + 1e-45), float((err / (bound + 1e-30)).max())
+            acc = np.zeros(G_np.shape[1], dtype=np.float32)
+            for k in range(start, start + size):
+                acc = acc + G_np[k]                                # float32 adds, rows in order
+            G_sum[start] = acc
+        Z32 = so.encode(G_sum, m, sizes, w)
+        bound32 = so.encode(np.abs(G_sum), m, sizes, np.abs(w))
+        err32 = np.abs(got - Z32)
+        assert np.all(err32 <= 2.0 ** -24 * np.abs(Z32) * 1.0001 + 1e-14 * bound32 + 1e-45), \
+            float((err32 / (np.abs(Z32) + 1e-30)).max())
     return Z
 
 
