@@ -101,8 +101,7 @@ __device__ __forceinline__ void load_weights(const double* __restrict__ src, dou
   }
 }
 
-constexpr int kRecConsumers = 256;
-constexpr int kRecPipeThreads = kRecConsumers + 32;   // + one producer warp
+constexpr int kRecConsumers = 256;   // consumer threads per CTA of the float32 kernels (template parameter NC)
 
 struct RecoverPipe {
   int row_batch;     // rows per stage
@@ -116,10 +115,10 @@ struct RecoverPipe {
 // shared-memory ring with bulk asynchronous copies; consumer threads own CPT chunks each, take one float per
 // row from the ring, apply the row's m weights, and every consumer warp writes its runs of chunks back
 // through its own shared buffer as contiguous 128-bit stores.
-template <int M, int CPT, typename Acc>
-__global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams prm, RecoverPipe pp) {
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm>
+__global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverParams prm, RecoverPipe pp) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  constexpr int kTileChunks = kRecConsumers * CPT;
+  constexpr int kTileChunks = NC * CPT;
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + pp.stages;
@@ -137,13 +136,13 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
   int* start_s = rowsh_c + ((prm.P + 3) & ~3);                                            // q + 1
   int* n_rec_s = start_s + ((prm.q + 4) & ~3);                                            // q
   float* out_all = reinterpret_cast<float*>(n_rec_s + ((prm.q + 3) & ~3));                // 8 warps x 32 x M
-  float* ring = out_all + (size_t)(kRecConsumers / 32) * 32 * M;                          // 32 M floats: 128 M bytes
+  float* ring = out_all + (size_t)(NC / 32) * 32 * M;                          // 32 M floats: 128 M bytes
   const size_t stage_floats = (size_t)pp.row_batch * pp.slot_floats;
 
   if (tid == 0) {
     for (int s = 0; s < pp.stages; ++s) {
       pipe::mbar_init(&full_bar[s], 32);
-      pipe::mbar_init(&empty_bar[s], kRecConsumers / 32);
+      pipe::mbar_init(&empty_bar[s], NC / 32);
     }
     *abort_flag = 0;
     pipe::fence_barrier_init();
@@ -161,8 +160,8 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
   // not all draw the same bandwidth (those of the fuller GPCs get about a third less), and with equal shares the
   // slow ones finish long after the rest.  The producer announces every batch's tile in tile_of[stage]; a
   // negative tile ends the stream.
-  if (tid >= kRecConsumers) {
-    const int lane = tid - kRecConsumers;
+  if (tid >= NC) {
+    const int lane = tid - NC;
     uint32_t it = 0;
     long long tile = 0;
     if (lane == 0) tile = (long long)atomicAdd(pp.tile_counter, 1ULL);
@@ -241,12 +240,12 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
     const float* slot = ring + stage * stage_floats + tid;
     const int* rs = rowsh_c + b0;
     const Acc* cj = coeff_c + (size_t)b0 * kStride;
-#pragma unroll 2
+#pragma unroll(sizeof(Acc) == 8 ? 1 : 2)
     for (int j = 0; j < nb; ++j) {
       const float* src = slot + (rs[j] & 3);
       Acc v[CPT];
 #pragma unroll
-      for (int i = 0; i < CPT; ++i) v[i] = (Acc)src[i * kRecConsumers];
+      for (int i = 0; i < CPT; ++i) v[i] = (Acc)src[i * NC];
       Acc c[kStride];
       load_weights<kStride>(cj, c);
 #pragma unroll
@@ -267,7 +266,7 @@ __global__ void __launch_bounds__(kRecPipeThreads) recover_kernel(RecoverParams 
 #pragma unroll
       for (int l = 0; l < M; ++l) out_s[lane * M + l] = (float)acc[i][l];
       __syncwarp();
-      const int64_t o0 = (c0 + (int64_t)i * kRecConsumers + warp * 32) * M;
+      const int64_t o0 = (c0 + (int64_t)i * NC + warp * 32) * M;
       int64_t o1 = o0 + 32 * M;
       if (o1 > prm.d) o1 = prm.d;
       const int count = o1 > o0 ? (int)(o1 - o0) : 0;
@@ -306,9 +305,9 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   }
 }
 
-template <int M, int CPT, typename Acc>
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm>
 static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
-  constexpr int kTileChunks = kRecConsumers * CPT;
+  constexpr int kTileChunks = NC * CPT;
   RecoverPipe pp;
   pp.status = plan->d_status;
   pp.slot_floats = kTileChunks + 8;
@@ -316,9 +315,10 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + recover_coeff_bytes(plan->P, PackedStride<Acc, M>::value) +
                        3 * (size_t)((plan->P + 3) & ~3) * sizeof(int) +
                        (size_t)(((plan->q + 4) & ~3) + ((plan->q + 3) & ~3)) * sizeof(int) +
-                       (size_t)(kRecConsumers / 32) * 32 * M * sizeof(float);
-  // the locator may select up to all P rows (large m) or as few as q m; batches of about 20 KB
-  int row_batch = (int)((size_t)20 * 1024 / slot_bytes);
+                       (size_t)(NC / 32) * 32 * M * sizeof(float);
+  // the locator may select up to all P rows (large m) or as few as q m; batches of about 20 KB (40 KB when one
+  // CTA has the SM's shared memory to itself)
+  int row_batch = (int)((size_t)(kCtasPerSm == 1 ? 40 : 20) * 1024 / slot_bytes);
   if (row_batch < 1) row_batch = 1;
   if (row_batch > 32) row_batch = 32;
   const int max_rows = M <= 6 ? plan->q * M : plan->P;
@@ -327,7 +327,7 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
     int nb = (max_rows + row_batch - 1) / row_batch;     // an even split of the expected row count
     row_batch = (max_rows + nb - 1) / nb;
   }
-  const size_t per_cta = (size_t)227 * 1024 / 2 - 1024;
+  const size_t per_cta = (size_t)227 * 1024 / kCtasPerSm - 1024;
   int stages = 4;
   while (stages > 2 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --stages;
   while (row_batch > 1 && fixed + (size_t)stages * row_batch * slot_bytes > per_cta) --row_batch;
@@ -341,17 +341,17 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   if (smem > (size_t)226 * 1024) return SOLON_ERR_INVALID_ARG;
   pp.row_batch = row_batch;
   pp.stages = stages;
-  auto kernel = recover_kernel<M, CPT, Acc>;
+  auto kernel = recover_kernel<M, CPT, Acc, NC, kCtasPerSm>;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   static_assert((32 * M * 4) % 16 == 0, "warp runs must start on a 16-byte boundary of the output");
   int64_t tiles = (plan->d_c + kTileChunks - 1) / kTileChunks;
   int per_sm = 1;
-  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kRecPipeThreads, smem));
+  SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (NC + 32), smem));
   if (per_sm < 1) per_sm = 1;
   int64_t cap = (int64_t)plan->num_sms * per_sm;
   int grid = (int)(tiles < cap ? tiles : cap);
   pp.tile_counter = plan->d_tile_counter;
-  return launch_dependent(kernel, dim3(grid), dim3(kRecPipeThreads), smem, plan->stream, prm, pp);
+  return launch_dependent(kernel, dim3(grid), dim3((NC + 32)), smem, plan->stream, prm, pp);
 }
 
 int launch_recover(solon_plan* plan, const float* received, float* agg) {
@@ -369,18 +369,18 @@ int launch_recover(solon_plan* plan, const float* received, float* agg) {
   prm.coeff = plan->d_coeff;
   prm.proj_progress = plan->d_proj_progress;
   plan->launches += 1;
-#define SOLON_RECOVER_CASE(M_, CPT_, ACC_) \
-  case M_:                                 \
-    return launch_recover_m<M_, CPT_, ACC_>(plan, prm);
+#define SOLON_RECOVER_CASE(M_, CPT_, ACC_, NC_, BLOCKS_) \
+  case M_:                                               \
+    return launch_recover_m<M_, CPT_, ACC_, NC_, BLOCKS_>(plan, prm);
   switch (plan->m) {
-    SOLON_RECOVER_CASE(1, 4, float)
-    SOLON_RECOVER_CASE(2, 4, float)
-    SOLON_RECOVER_CASE(3, 4, float)
-    SOLON_RECOVER_CASE(4, 4, float)
-    SOLON_RECOVER_CASE(5, 4, float)
-    SOLON_RECOVER_CASE(6, 2, float)
-    SOLON_RECOVER_CASE(8, 2, double)
-    SOLON_RECOVER_CASE(10, 2, double)
+    SOLON_RECOVER_CASE(1, 4, float, kRecConsumers, 2)
+    SOLON_RECOVER_CASE(2, 4, float, kRecConsumers, 2)
+    SOLON_RECOVER_CASE(3, 4, float, kRecConsumers, 2)
+    SOLON_RECOVER_CASE(4, 4, float, kRecConsumers, 2)
+    SOLON_RECOVER_CASE(5, 4, float, kRecConsumers, 2)
+    SOLON_RECOVER_CASE(6, 2, float, kRecConsumers, 2)
+    SOLON_RECOVER_CASE(8, 4, double, 480, 1)
+    SOLON_RECOVER_CASE(10, 4, double, 480, 1)
     default: break;
   }
 #undef SOLON_RECOVER_CASE
