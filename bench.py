@@ -315,7 +315,7 @@ def run_ours(args, wl):
                    "arithmetic": "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64", "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * wl.d * 4 / 1e9),
                    "parallelism": ("one problem, coordinates sharded over the GPUs, one all-reduce of (K+1) x P float64 per decode"
                                    if sp is not None else "independent problems per GPU, no collective")},
-        "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "encode_direct_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
                      "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(wl.name) if sp is None else None,
                      "algorithmic_bytes": enc_b, "ms": enc_ms},
         "path": {"encode_ms": enc_ms, "decode_ms": dec_ms, "decodes_per_s": 1e3 / dec_ms, "algorithmic_bytes": total_b,

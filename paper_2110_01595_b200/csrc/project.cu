@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(kProjThreads, 4) project_kernel(const float* _
                                                                int tile_cols, double* __restrict__ partials,
                                                                double* __restrict__ rho_out, double* __restrict__ nu_out,
                                                                unsigned int* ticket, int final_reduce) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   double* fs = reinterpret_cast<double*>(smem_raw);            // K x tile_cols
   double* sacc = fs + (size_t)K * tile_cols;                  // P x (K + 1)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -365,6 +365,8 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
 
   if (tid >= kPipeConsumers) {
     const int lane = tid - kPipeConsumers;
+    const uint64_t row_policy = pipe::policy_evict_first();   // the recovery pass re-reads only a few of these rows
+    const uint64_t f_policy = pipe::policy_evict_last();      // every decode reads the projection vectors again
     uint32_t it = 0;
     for (int part = pp.part_a_cols > 0 ? 0 : 1; part < 2; ++part) {
       const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
@@ -394,10 +396,10 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           if (lane < K) f_bytes = (uint32_t)(((cols + 3) & ~(int64_t)3) * 4);
           if (row_bytes + f_bytes) pipe::mbar_arrive_expect_tx(&full_bar[stage], row_bytes + f_bytes);
           else pipe::mbar_arrive(&full_bar[stage]);
-          if (row_bytes) pipe::bulk_load(slot, row_src, row_bytes, &full_bar[stage]);
+          if (row_bytes) pipe::bulk_load_hint(slot, row_src, row_bytes, &full_bar[stage], row_policy);
           if (f_bytes)
-            pipe::bulk_load(stage_base + (size_t)(pp.batch_rows + lane) * pp.slot_floats, f + (int64_t)lane * f_pitch + c0, f_bytes,
-                            &full_bar[stage]);
+            pipe::bulk_load_hint(stage_base + (size_t)(pp.batch_rows + lane) * pp.slot_floats, f + (int64_t)lane * f_pitch + c0,
+                                 f_bytes, &full_bar[stage], f_policy);
         }
       }
     }

@@ -162,6 +162,7 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
   // negative tile ends the stream.
   if (tid >= NC) {
     const int lane = tid - NC;
+    const uint64_t stream_policy = pipe::policy_evict_first();   // last use of the received rows
     uint32_t it = 0;
     long long tile = 0;
     if (lane == 0) tile = (long long)atomicAdd(pp.tile_counter, 1ULL);
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
           for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.R[e];   // <= 3 floats
           if (bytes) {
             pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
-            pipe::bulk_load(slot, prm.R + a0, bytes, &full_bar[stage]);
+            pipe::bulk_load_hint(slot, prm.R + a0, bytes, &full_bar[stage], stream_policy);
           } else {
             pipe::mbar_arrive(&full_bar[stage]);
           }
