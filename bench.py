@@ -415,11 +415,11 @@ def run_sweep(args):
     print(json.dumps(summary), flush=True)
 
 
-# DRAM bytes (read + write) per encode launch.  Captured with ncu on the resnet18 workload (786.7 MB for 804.5 MB of
+# DRAM bytes (read + write) per encode launch.  Captured with ncu on the resnet18 workload (785.2 MB for 804.5 MB of
 # algorithmic bytes: the input is read exactly once, part of the output is still in L2 when the kernel ends);
 # the vgg13 figure is that capture scaled by the units processed (P * d), since the kernel makes one pass.
 # Emptied (reported as null) whenever the kernel changes until it is captured again.
-TRAFFIC: dict = {"resnet18": 786.7e6, "vgg13": 786.7e6 * (45 * 28_332_000) / (15 * 11_173_962)}
+TRAFFIC: dict = {"resnet18": 785.2e6, "vgg13": 785.2e6 * (45 * 28_332_000) / (15 * 11_173_962)}
 
 
 def main():

@@ -27,7 +27,8 @@ the projected values; exact recovery of the plain sum (Definition 1) under
 0..s attackers of several kinds; the locator against brute-force subset
 enumeration (Appendix C) and against the Reed-Solomon property that the
 denominator's roots are the corrupt nodes' scalars; the fixed-s system of
-Section 3.4 against the incremental variant; Theorem 2 / its corollary and the
+Section 3.4 against the incremental variant; the r_c = 1 majority vote against
+the general decoder and the plain sum; Theorem 2 / its corollary and the
 introduction's 4-node example for feasibility; Table 2 for d_c; the
 least-squares gradient against finite differences of the loss.
 No function here is "parity unpinned".
@@ -348,6 +349,39 @@ def decode(R: np.ndarray, d: int, r_c: int, s: int, sizes: list[int], w: np.ndar
         mask[[start + k for k in V]] = 1
         u += psi(R[grp], w_g, r_c, U)
     return u[:d], mask, status
+
+
+def majority_decode(R: np.ndarray, s: int, sizes: list[int]):
+    """The r_c = 1 special case written out: repetition code and majority vote.
+
+    With r_c = 1 the encoder matrix W_j = I_d (x) [1] is the identity (Section 3.4), so every node of a group
+    sends the same vector, the group's summed gradient: Solon's code is then the repetition code, and locating
+    at most s < r / 2 corrupt nodes is a majority vote among the group's received vectors.  For each group the
+    vector held by at least r_j - s nodes is taken (rows are compared exactly), the nodes that sent anything
+    else are flagged, and the groups' vectors are added up.  Returns (u, mask, status); status is -1 if some
+    group has no such majority.
+    """
+    P, d = R.shape
+    u = np.zeros(d, dtype=np.float64)
+    mask = np.zeros(P, dtype=np.uint8)
+    status = 0
+    for start, size in zip(group_starts(sizes), sizes):
+        rows = R[start:start + size]
+        winner = None
+        for k in range(size):
+            same = [j for j in range(size) if np.array_equal(rows[j], rows[k])]
+            if len(same) >= size - s:
+                winner = (k, same)
+                break
+        if winner is None:
+            status = -1
+            continue
+        k, same = winner
+        u += rows[k].astype(np.float64)
+        for j in range(size):
+            if j not in same:
+                mask[start + j] = 1
+    return u, mask, status
 
 
 # --------------------------------------------------------------------------

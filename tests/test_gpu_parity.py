@@ -219,6 +219,29 @@ def test_all_attackers_in_one_group_and_every_count():
             assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
 
 
+@pytest.mark.parametrize("P,s,d", [(9, 2, 20_001), (45, 3, 100_003), (105, 5, 30_000)])
+def test_m1_is_the_repetition_code_with_majority_vote(P, s, d):
+    """r_c = 1: W_j = I_d, every node of a group sends the same vector (bit for bit), and the decode equals the
+    oracle's majority vote over the very same received matrix: same flagged set, the sum of the groups' majority
+    vectors within the float32 roundings of adding q terms."""
+    wl = synth.Workload("rep", P, s, 1, d, "normal", 1.0, "gaussian", s, 4242 + P)
+    sizes, w = _oracle_plan(wl)
+    G_cpu = synth.make_grads(wl, "cpu")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=3) as plan:
+        coded = plan.encode(G_cpu.cuda())
+        for start, size in zip(so.group_starts(sizes), sizes):
+            assert bool((coded[start:start + size] == coded[start]).all())
+        received, nodes = synth.apply_attack(wl, coded)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        R = received.cpu().numpy()
+        u, o_mask, o_status = so.majority_decode(R, wl.s, sizes)
+        assert o_status == 0 and o_mask.nonzero()[0].tolist() == nodes
+        assert np.array_equal(mask.cpu().numpy(), o_mask)
+        bound = 1.001 * len(sizes) * 2.0 ** -24 * np.abs(G_cpu.numpy().astype(np.float64)).sum(0)
+        assert np.all(np.abs(agg.cpu().numpy().astype(np.float64) - u) <= bound + 1e-30)
+
+
 def test_non_finite_rows_are_located():
     wl = synth.Workload("nan", 15, 2, 5, 20_000, "normal", 1.0, "none", 0, 11)
     G_cpu = synth.make_grads(wl, "cpu")

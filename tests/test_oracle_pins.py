@@ -117,6 +117,46 @@ def test_encode_m1_is_group_sum():
             assert np.array_equal(Z[k], ybar)
 
 
+@pytest.mark.parametrize("P,s", [(9, 1), (7, 3), (15, 2), (10, 0)])
+def test_majority_vote_is_the_m1_decoder(P, s):
+    """r_c = 1: the repetition code.  The majority vote returns the plain sum (Definition 1) and the exact set of
+    nodes that sent something else, and agrees with the general decoder (Algorithm 1) on the same received matrix;
+    one attacker too many in a group leaves no majority."""
+    rng = np.random.default_rng(40 + P + s)
+    m, d = 1, 29
+    sizes, w = _plan(P, s, m)
+    G = rng.normal(size=(P, d)).astype(np.float32)
+    Z = so.encode(G, m, sizes, w)
+    f = 1.0 + rng.normal(size=(2, d))
+    want = so.plain_sum(G)
+    starts = so.group_starts(sizes)
+    for n_byz in range(s + 1):
+        nodes = sorted((starts[-1] + rng.permutation(sizes[-1])[:n_byz]).tolist())
+        R = Z.copy()
+        R[nodes] = rng.normal(scale=100.0, size=(len(nodes), d))
+        u, mask, status = so.majority_decode(R, s, sizes)
+        assert status == 0
+        assert mask.nonzero()[0].tolist() == nodes
+        assert np.abs(u - want).max() <= 1e-12 * np.abs(want).max()
+        if s > 0:
+            u2, mask2, status2 = so.decode(R, d, m, s, sizes, w, f)
+            assert status2 == 0 and np.array_equal(mask2, mask)
+            assert np.abs(u2 - u).max() <= 1e-9 * np.abs(want).max()
+    if s > 0 and sizes[-1] == 2 * s + 1:
+        # s + 1 different liars in a group of 2 s + 1: only s honest copies remain, fewer than r - s
+        nodes = list(range(starts[-1], starts[-1] + s + 1))
+        R = Z.copy()
+        R[nodes] = rng.normal(scale=100.0, size=(len(nodes), d))
+        assert so.majority_decode(R, s, sizes)[2] == -1
+    # a colluding majority is believed: the vote itself cannot tell (the bound r >= 2 s + 1 is what rules it out)
+    if s > 0:
+        liars = list(range(starts[0], starts[0] + sizes[0] - s))
+        R = Z.copy()
+        R[liars] = 7.0
+        u, mask, status = so.majority_decode(R, s, sizes)
+        assert status == 0 and mask.nonzero()[0].tolist() == [k for k in range(starts[0], starts[0] + sizes[0]) if k not in liars]
+
+
 def test_encode_padding_and_chunk_order():
     """d not divisible by r_c: the last chunk is zero padded; chunk p covers coordinates p r_c .. p r_c + r_c - 1."""
     P, s, m, d = 5, 1, 3, 7
