@@ -145,9 +145,11 @@ int solon_plan_get_projection_vectors(solon_plan* plan, float* f /* host, K * d_
  *   coded            device, P x d_c: row k receives node k's coded vector,
  *                    coded[k][p] = sum_{l<m} w_k^l * ybar_g[p m + l], where ybar_g is the sum of
  *                    the gradients of k's group, zero-padded to m d_c entries.
- * Arithmetic: float32 for m <= 6; for larger m (and for m without a specialised kernel) the
- * group sum and the mix are evaluated in float64 and rounded once to float32, because the
- * decoder amplifies the encoder's rounding by a factor that grows like 2^m. */
+ * Arithmetic: ybar_g is added up in float32, the group's rows in node order (its rounding is
+ * common to all nodes of the group, so the decoder returns it unamplified).  The mix is
+ * evaluated in float32 for m <= 6; for larger m (and for m without a specialised kernel) in
+ * float64 and rounded once to float32, because the decoder amplifies rounding that differs
+ * from node to node by a factor that grows like 2^m. */
 int solon_encode(solon_plan* plan, const float* partition_grads, float* coded);
 
 /* Robust decode (Algorithm 1 with the locator phi and block decoder psi of Section 3.4).
