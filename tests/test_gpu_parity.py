@@ -203,6 +203,67 @@ def test_edge_shapes(P, s, m, r, d):
         assert np.abs(agg.cpu().numpy() - want).max() <= tol * max(np.abs(want).max(), 1e-30)
 
 
+def _random_plan(rng):
+    """A feasible (P, s, m, r, d): m up to 12, s up to 5, r anywhere from the bound 2 s + m to P, ragged d."""
+    while True:
+        P = int(rng.integers(3, 70))
+        m = int(rng.integers(1, 13))
+        if m > P:
+            continue
+        s = int(rng.integers(0, min(5, (P - m) // 2) + 1))
+        r = int(rng.integers(2 * s + m, P + 1))
+        d = int(rng.integers(1, 40_000))
+        return P, s, m, r, d
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_plans_and_placements(case):
+    """Seeded random plans (group size above the bound too, d not a multiple of m or of 4), a random number of
+    attackers (0..s) in every group, random attack kinds: mask bit-exact, aggregate within the bar of the plain
+    float64 sum and of the oracle's own decode of the same received matrix."""
+    rng = np.random.default_rng(9000 + case)
+    P, s, m, r, d = _random_plan(rng)
+    sizes = so.group_sizes(P, r)
+    w = so.node_scalars(sizes)
+    g = torch.Generator().manual_seed(9000 + case)
+    G_cpu = torch.empty((P, d), dtype=torch.float32).normal_(0.0, float(10.0 ** rng.uniform(-3, 1)), generator=g)
+    with binding.Plan(P, s, m, r, d, seed=case) as plan:
+        assert plan.group_sizes() == sizes
+        coded = plan.encode(G_cpu.cuda())
+        _check_encode(plan, G_cpu, coded, m, sizes, w)
+        Z = coded.cpu().numpy()
+        R = Z.copy()
+        nodes = []
+        scale_z = float(np.abs(Z).max()) + 1e-30
+        for start, size in zip(so.group_starts(sizes), sizes):
+            n_byz = int(rng.integers(0, s + 1))
+            for k in sorted((start + rng.permutation(size)[:n_byz]).tolist()):
+                kind = rng.integers(0, 4)
+                if kind == 0:
+                    R[k] = rng.normal(scale=100.0 * scale_z, size=Z.shape[1])
+                elif kind == 1:
+                    R[k] = -10.0 * Z[k]
+                elif kind == 2:
+                    R[k] = -Z.mean(0) + scale_z          # shifted so that it cannot coincide with the honest row
+                else:
+                    R[k, rng.integers(Z.shape[1])] += 1000.0 * scale_z
+                nodes.append(k)
+        R = R.astype(np.float32)
+        want_mask = so.true_mask(R, Z)
+        assert want_mask.nonzero()[0].tolist() == nodes
+        agg, mask = plan.decode(torch.from_numpy(R).cuda())
+        assert plan.decode_status() == 0
+        assert np.array_equal(mask.cpu().numpy(), want_mask)
+        want = so.plain_sum(G_cpu.numpy())
+        scale = np.abs(want).max()
+        got = agg.cpu().numpy().astype(np.float64)
+        assert np.abs(got - want).max() <= AGG_TOL * scale, (P, s, m, r, d, np.abs(got - want).max() / scale)
+        if s > 0:
+            u, o_mask, o_status = so.decode(R, d, m, s, sizes, w, plan.projection_vectors(), tau=TAU)
+            assert o_status == 0 and np.array_equal(o_mask, want_mask)
+            assert np.abs(got - u).max() <= AGG_TOL * scale
+
+
 def test_all_attackers_in_one_group_and_every_count():
     base = synth.Workload("placement", 45, 3, 5, 50_001, "normal", 1.0, "alie", 3, 321)
     sizes, w = _oracle_plan(base)
