@@ -60,6 +60,10 @@ struct GroupScratch {
   double* rho_n;         // K x n
   double* scratch;       // K + 2
   double* coeff_l;       // n x m
+  uint8_t* warm_trusted; // n      outputs and workspace of the recovery table's rehearsal (never read)
+  int* warm_rows;        // n
+  double* warm_coeff;    // n x m
+  double* warm_ws;       // locate_epilogue_ws_doubles
   double* tasks;         // (s + 1) x task_stride, reused by the epilogue
   size_t task_stride;
 };
@@ -72,8 +76,9 @@ SOLON_HD static inline size_t task_stride_doubles(int n, int m, int K, int s) {
 SOLON_HD static inline size_t group_ws_doubles(int n, int m, int K, int s) {
   size_t tasks = (size_t)(s + 1) * task_stride_doubles(n, m, K, s);
   size_t epi = locate_epilogue_ws_doubles(n, m, s);
+  size_t warm = ((size_t)n / 8 + 1) + ((size_t)(n + 1) / 2 + 1) + (size_t)n * m + epi;
   return ((size_t)(n + 1) / 2 + 1) + 3 * ((size_t)n / 8 + 1) + ((size_t)(s + 1) * n / 8 + 1) + 2 * (size_t)(s + 1) +
-         (size_t)(2 * K + 1) * n + K + 2 + (size_t)n * m + (tasks > epi ? tasks : epi) + 8;
+         (size_t)(2 * K + 1) * n + K + 2 + (size_t)n * m + warm + (tasks > epi ? tasks : epi) + 8;
 }
 
 SOLON_HD static inline GroupScratch carve(double* ws, int n, int m, int K, int s) {
@@ -90,6 +95,10 @@ SOLON_HD static inline GroupScratch carve(double* ws, int n, int m, int K, int s
   sc.rho_n = p;                                  p += (size_t)K * n;
   sc.scratch = p;                                p += K + 2;
   sc.coeff_l = p;                                p += (size_t)n * m;
+  sc.warm_trusted = reinterpret_cast<uint8_t*>(p); p += n / 8 + 1;
+  sc.warm_rows = reinterpret_cast<int*>(p);      p += (n + 1) / 2 + 1;
+  sc.warm_coeff = p;                             p += (size_t)n * m;
+  sc.warm_ws = p;                                p += locate_epilogue_ws_doubles(n, m, s);
   sc.tasks = p;
   sc.task_stride = task_stride_doubles(n, m, K, s);
   return sc;
@@ -279,6 +288,19 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
         else
           locate_task<SOLON_FAST_T>(Team::own_warp(), tb, n, prm.m, prm.K, t, prm.s, sc.rho_n, sc.forced, tau_eff, tflags, cand,
                                     bad, tws, &sc.recs[t]);
+      }
+      // Rehearsal of the recovery table.  The epilogue below runs that code once, after all the tasks, and between
+      // decodes gigabytes stream through L2: fetched from HBM it takes about 10 us, for a few hundred operations.  A
+      // warp with nothing else to do (else warp 0, whose task - no corrupt node - is the shortest) runs the very same
+      // code now, on a made-up trusted set and into scratch that nobody reads, so that the SM's instruction cache
+      // holds it when the epilogue comes.  Only for the subset form (m <= 6): the all-rows form takes a single warp
+      // longer than the tasks last, and the CTA would wait for it.
+      const int idle_warp = prm.s + 1 < (n_threads >> 5) ? prm.s + 1 : 0;
+      if (t == idle_warp && prm.m <= SOLON_SUBSET_MAX_M) {
+        const Team own = Team::own_warp();
+        for (int k = own.lane; k < n; k += 32) sc.warm_trusted[k] = (k == 0 && prm.s > 0) ? 0 : 1;   // one node deleted
+        __syncwarp();
+        (void)recovery_table(own, tb, n, prm.m, prm.s, sc.warm_trusted, sc.warm_rows, sc.warm_coeff, sc.warm_ws);
       }
     }
     __syncthreads();

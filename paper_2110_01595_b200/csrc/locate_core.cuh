@@ -28,8 +28,10 @@
 
 #if defined(__CUDACC__)
 #define SOLON_HD __host__ __device__
+#define SOLON_NOINLINE __noinline__   /* one copy of the code, whoever calls it: a rehearsal warms it for the real call */
 #else
 #define SOLON_HD
+#define SOLON_NOINLINE
 #endif
 
 // The threads that execute a routine together: a whole CTA, one warp of it, or (host) a single thread.
@@ -503,8 +505,8 @@ SOLON_HD inline int locate_check(const Team& tm, const GroupTables& tb, int n, i
 // i.e. the least-squares inverse of [W-hat_{m-1}]_{rows,.} (monomial basis, as the encoder used).
 // ws: locate_epilogue_ws_doubles(n, m, s).  Returns the number of rows (same value in every thread),
 // 0 if fewer than m nodes are trusted or (all-rows form) more than s are not.
-SOLON_HD inline int recovery_table(const Team& tm, const GroupTables& tb, int n, int m, int s, const uint8_t* trusted, int* rec_rows,
-                                   double* coeff, double* ws) {
+SOLON_HD SOLON_NOINLINE inline int recovery_table(const Team& tm, const GroupTables& tb, int n, int m, int s, const uint8_t* trusted,
+                                                  int* rec_rows, double* coeff, double* ws) {
   int n_u = 0;
   for (int k = 0; k < n; ++k) n_u += trusted[k] ? 1 : 0;
   if (n_u < m) return 0;
