@@ -490,7 +490,8 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   plan->launches += 1;
   switch (plan->m) {
     case 1: return launch_encode_direct<1, 4, float, 3>(plan, prm);
-    case 2: return launch_encode_direct<2, 2, float, 3>(plan, prm);
+    case 2:   // small groups: wider tiles, or the per-tile work (claim, group lookup) shows; large groups: more tiles to hand out
+      return plan->max_group <= 6 ? launch_encode_direct<2, 4, float, 3>(plan, prm) : launch_encode_direct<2, 2, float, 3>(plan, prm);
     case 3: return launch_encode_direct<3, 2, float, 3>(plan, prm);
     case 4: return launch_encode_direct<4, 1, float, 3>(plan, prm);
     case 5: return launch_encode_direct<5, 1, float, 3>(plan, prm);
