@@ -119,3 +119,35 @@ def test_config_lsq_full_size():
         scale = float(G.sum(dim=0, dtype=torch.float64).abs().max())
         got = agg[ct].cpu().numpy().astype(np.float64)
         assert np.abs(got - want_G.sum(0)).max() <= AGG_TOL * scale
+
+
+def test_gradient_longer_than_two_to_the_31():
+    """d beyond 2^31 coordinates (every index is 64-bit): P=5, s=1, m=3, d = 2^31 + 5 (ragged: d is neither a multiple
+    of m nor of 4), one node sends -3 z.  Mask exact, aggregate against a float64 device-side sum, slice by slice."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100e9:
+        pytest.skip("needs about 80 GB of free device memory")
+    P, s, m, d = 5, 1, 3, 2 ** 31 + 5
+    G = torch.empty((P, d), dtype=torch.float32, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(31)
+    for i in range(P):
+        G[i].normal_(0.0, 1.0, generator=gen)
+    with binding.Plan(P, s, m, 2 * s + m, d, seed=5) as plan:
+        coded = plan.encode(G)
+        received = coded.clone()
+        received[1].mul_(-3.0)
+        agg, mask = plan.decode(received)
+        assert plan.decode_status() == 0
+        assert mask.nonzero().flatten().tolist() == [1]
+        worst, scale = 0.0, 0.0
+        for lo in range(0, d, 1 << 28):
+            hi = min(d, lo + (1 << 28))
+            ref = G[:, lo:hi].sum(dim=0, dtype=torch.float64)
+            worst = max(worst, float((agg[lo:hi].double() - ref).abs().max()))
+            scale = max(scale, float(ref.abs().max()))
+        assert worst <= AGG_TOL * scale
+        # the last chunk is padded (d = 2 mod 3): its two real coordinates against the oracle
+        tail = G[:, d - 2:].cpu().numpy()
+        assert np.abs(agg[d - 2:].cpu().numpy() - so.plain_sum(tail)).max() <= AGG_TOL * scale
+    del G, coded, received, agg
+    torch.cuda.empty_cache()
