@@ -195,7 +195,12 @@ int solon_decode_finish(solon_plan* plan, const double* rho, const double* nu, c
  *   X      device, (P * rows) x d; partition i owns rows [i rows, (i+1) rows)
  *   y      device, P * rows
  *   w      device, d
- *   grads  device, P x d (output) */
+ *   grads  device, P x d (output)
+ * Two streaming passes over X (residuals, then gradients), sums in float64.  When d is a multiple
+ * of 4 and X, w and grads are 16-byte aligned the passes use 128-bit loads and float32 products
+ * (one rounding per term); any other layout takes scalar loads and float64 products.  Allocates
+ * the residual buffer (P * rows floats) on first use or when rows grows: returns SOLON_ERR_NOMEM
+ * if that fails. */
 int solon_lsq_grads(solon_plan* plan, const float* X, const float* y, const float* w, float* grads);
 
 /* One whole step with HOST buffers: copies the gradients to the device, encodes, overwrites the

@@ -142,20 +142,26 @@ def test_config_sweep_small(P, s, m):
     _run_case(wl)
 
 
-def test_config_lsq_small():
-    wl = dataclasses.replace(synth.WORKLOADS["lsq"], d=5_003, lsq_rows=64)
+@pytest.mark.parametrize("d", [5_003, 5_004])          # rows off and on 16-byte boundaries: scalar and 128-bit-load kernels
+@pytest.mark.parametrize("iterate", ["zero", "random"])
+def test_config_lsq_small(d, iterate):
+    wl = dataclasses.replace(synth.WORKLOADS["lsq"], d=d, lsq_rows=64)
     sizes, w = _oracle_plan(wl)
     X, y, wvec = synth.make_lsq_problem(wl, "cpu")
+    if iterate == "random":
+        wvec = torch.empty(d, dtype=torch.float32).normal_(0.0, 1.0, generator=torch.Generator().manual_seed(77))
     want_G = so.lsq_grads(X.numpy(), y.numpy(), wvec.numpy(), wl.lsq_rows)
     with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
         G = plan.lsq_grads(X.cuda(), y.cuda(), wvec.cuda(), rows=wl.lsq_rows)
         got_G = G.cpu().numpy().astype(np.float64)
         Xa = np.abs(X.numpy()).astype(np.float64)
         e = np.abs(X.numpy().astype(np.float64) @ wvec.numpy().astype(np.float64) - y.numpy())
+        # residuals: float32 products summed in float64 and one rounding to float32; gradients likewise
+        e_err = 2.0 ** -24 * (Xa @ np.abs(wvec.numpy()).astype(np.float64)) + 2.0 ** -24 * e
         for i in range(wl.P):
             rows = slice(i * wl.lsq_rows, (i + 1) * wl.lsq_rows)
             bound = Xa[rows].T @ e[rows]                      # sum of |terms|
-            assert np.all(np.abs(got_G[i] - want_G[i]) <= 3e-7 * bound + 1e-30)
+            assert np.all(np.abs(got_G[i] - want_G[i]) <= 3e-7 * bound + 1.01 * Xa[rows].T @ e_err[rows] + 1e-30)
         coded = plan.encode(G)
         received, nodes = synth.apply_attack(wl, coded)
         agg, mask = plan.decode(received)
