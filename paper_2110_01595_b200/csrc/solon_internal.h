@@ -144,7 +144,7 @@ static inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 blo
 // a streaming kernel (the projection kernel moves about 6 GB per ms).
 inline bool uses_early_locator(const solon_plan* plan) {
   const bool small_solver = plan->s > 0 && plan->max_group <= 64 && plan->s <= 5;
-  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 500e6;
+  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 350e6;
   return small_solver && (plan->early_locator == 2 || (plan->early_locator == 1 && long_pass));
 }
 
