@@ -142,6 +142,71 @@ __global__ void __launch_bounds__(kLsqThreads, 4) lsq_gradient_vec_kernel(const 
   }
 }
 
+// Finer-grained form of the gradient pass: a work item is (partition, block of 64 x four columns); the CTA's four
+// groups of 64 threads each take a quarter of the partition's rows for those columns and their sums are added up
+// through shared memory.  About ten items per CTA instead of two or three, so no CTA is left with half the kernel
+// to do alone.  All residuals (P * rows floats) are staged in shared memory once.
+constexpr int kLsqItemCols4 = 64;
+__global__ void __launch_bounds__(kLsqThreads, 4) lsq_gradient_items_kernel(const float4* __restrict__ X4, const float* __restrict__ resid,
+                                                                        int64_t d4, int rows, int P, float4* __restrict__ grads4) {
+  extern __shared__ __align__(16) unsigned char lsq_smem[];
+  double* part_s = reinterpret_cast<double*>(lsq_smem);                    // 3 x 64 x 4 partial sums (quarters 1..3)
+  float* e_s = reinterpret_cast<float*>(part_s + 3 * kLsqItemCols4 * 4);   // P x rows residuals
+  for (int i = threadIdx.x; i < P * rows; i += kLsqThreads) e_s[i] = resid[i];
+  __syncthreads();
+  const int cq = threadIdx.x & (kLsqItemCols4 - 1), rq = threadIdx.x / kLsqItemCols4;
+  const int quarter = (rows + 3) / 4;
+  const int r_begin = rq * quarter < rows ? rq * quarter : rows;
+  const int r_end = r_begin + quarter < rows ? r_begin + quarter : rows;
+  const int64_t blocks = (d4 + kLsqItemCols4 - 1) / kLsqItemCols4;
+  const int64_t items = blocks * P;
+  for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+    const int part = (int)(item / blocks);
+    const int64_t c = (item - (int64_t)part * blocks) * kLsqItemCols4 + cq;
+    const float4* Xi = X4 + (int64_t)part * rows * d4;
+    const float* e = e_s + (size_t)part * rows;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    if (c < d4) {
+      int r = r_begin;
+      for (; r + 8 <= r_end; r += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = load_stream_pinned(Xi + (int64_t)(r + u) * d4 + c);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float ev = e[r + u];
+          a0 += (double)(v[u].x * ev);
+          a1 += (double)(v[u].y * ev);
+          a2 += (double)(v[u].z * ev);
+          a3 += (double)(v[u].w * ev);
+        }
+      }
+      for (; r < r_end; ++r) {
+        const float4 v = __ldcs(Xi + (int64_t)r * d4 + c);
+        const float ev = e[r];
+        a0 += (double)(v.x * ev);
+        a1 += (double)(v.y * ev);
+        a2 += (double)(v.z * ev);
+        a3 += (double)(v.w * ev);
+      }
+    }
+    if (rq > 0) {
+      double* dst = part_s + ((size_t)(rq - 1) * kLsqItemCols4 + cq) * 4;
+      dst[0] = a0; dst[1] = a1; dst[2] = a2; dst[3] = a3;
+    }
+    __syncthreads();
+    if (rq == 0 && c < d4) {
+#pragma unroll
+      for (int o = 0; o < 3; ++o) {      // quarters in row order: the sum does not depend on which CTA ran the item
+        const double* src = part_s + ((size_t)o * kLsqItemCols4 + cq) * 4;
+        a0 += src[0]; a1 += src[1]; a2 += src[2]; a3 += src[3];
+      }
+      grads4[(int64_t)part * d4 + c] = make_float4((float)a0, (float)a1, (float)a2, (float)a3);
+    }
+    __syncthreads();
+  }
+}
+
 int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w, float* grads) {
   const int64_t n_rows = (int64_t)plan->P * plan->lsq_rows;
   if (plan->resid_capacity < n_rows) {
@@ -165,11 +230,19 @@ int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w,
     lsq_residual_vec_kernel<<<grid1, kLsqThreads, 0, plan->stream>>>(reinterpret_cast<const float4*>(X), y,
                                                                       reinterpret_cast<const float4*>(w), d4, n_rows, plan->d_resid);
     SOLON_CUDA_TRY(cudaGetLastError());
-    int64_t col_blocks = (d4 + kLsqThreads - 1) / kLsqThreads;
-    int64_t cap = (resident + plan->P - 1) / plan->P;
-    dim3 grid2((unsigned)(col_blocks < cap ? col_blocks : cap), plan->P);
-    lsq_gradient_vec_kernel<<<grid2, kLsqThreads, smem, plan->stream>>>(reinterpret_cast<const float4*>(X), plan->d_resid, d4,
-                                                                        plan->lsq_rows, reinterpret_cast<float4*>(grads));
+    const size_t smem_items = 3 * kLsqItemCols4 * 4 * sizeof(double) + (size_t)n_rows * sizeof(float);
+    if (smem_items <= 40 * 1024) {
+      const int64_t items = ((d4 + kLsqItemCols4 - 1) / kLsqItemCols4) * plan->P;
+      const int grid2 = (int)(items < resident ? items : resident);
+      lsq_gradient_items_kernel<<<grid2, kLsqThreads, smem_items, plan->stream>>>(
+          reinterpret_cast<const float4*>(X), plan->d_resid, d4, plan->lsq_rows, plan->P, reinterpret_cast<float4*>(grads));
+    } else {
+      int64_t col_blocks = (d4 + kLsqThreads - 1) / kLsqThreads;
+      int64_t cap = (resident + plan->P - 1) / plan->P;
+      dim3 grid2((unsigned)(col_blocks < cap ? col_blocks : cap), plan->P);
+      lsq_gradient_vec_kernel<<<grid2, kLsqThreads, smem, plan->stream>>>(reinterpret_cast<const float4*>(X), plan->d_resid, d4,
+                                                                          plan->lsq_rows, reinterpret_cast<float4*>(grads));
+    }
     SOLON_CUDA_TRY(cudaGetLastError());
   } else {
     lsq_residual_kernel<<<grid1, kLsqThreads, 0, plan->stream>>>(X, y, w, plan->d, n_rows, plan->d_resid);
