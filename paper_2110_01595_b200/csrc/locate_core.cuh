@@ -515,14 +515,17 @@ SOLON_HD SOLON_NOINLINE inline int recovery_table(const Team& tm, const GroupTab
   const int n_rec = subset ? m : n_u;
   {
     // every thread derives the same list; thread 0 stores it
+    // the j-th of the n_rec rows is the trusted node number want(j) (in node order): all of them in the all-rows
+    // form, m of them spread evenly over the trusted nodes in the subset form; want is only recomputed (an integer
+    // division) when j moves on
     int seen = 0, next = 0;
+    int want = !subset ? 0 : (m == 1 ? (n_u - 1) / 2 : ((m - 1) / 2) / (m - 1));
     for (int k = 0; k < n && next < n_rec; ++k) {
       if (!trusted[k]) continue;
-      const int want = !subset ? next
-                       : (m == 1 ? (n_u - 1) / 2 : (next * (n_u - 1) + (m - 1) / 2) / (m - 1));
       if (seen == want) {
         if (SOLON_TID == 0) rec_rows[next] = k;
         ++next;
+        want = !subset ? next : (m == 1 ? n : (next * (n_u - 1) + (m - 1) / 2) / (m - 1));
       }
       ++seen;
     }
