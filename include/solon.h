@@ -271,6 +271,8 @@ int solon_project_noalloc(const float* received, const float* f, int64_t f_pitch
  * solon_decode record an event before and after each of their kernels; solon_plan_get_timings
  * synchronises the stream and returns the durations of the most recent calls in milliseconds:
  * ms[0] encode, ms[1] projections, ms[2] locator, ms[3] recovery (0 for a kernel not yet run).
+ * While it is on, the two calls also open NVTX ranges on the calling thread ("solon_encode";
+ * "solon_decode" with "project", "locate", "recover" inside) for timeline tools.
  * Off by default (the events cost a few microseconds per call). */
 int solon_plan_set_profiling(solon_plan* plan, int on);
 int solon_plan_get_timings(solon_plan* plan, float* ms /* host, 4 */);

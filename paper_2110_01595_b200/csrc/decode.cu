@@ -15,12 +15,22 @@ extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_
     plan->ev_valid[i] = 1;
     return SOLON_OK;
   };
+  TraceRange range(prof, "solon_decode");
   if ((rc = mark(2))) return rc;
-  if (plan->s > 0 && (rc = launch_project(plan, received))) return rc;   // s = 0: nothing to locate
+  {
+    TraceRange step(prof, "project");
+    if (plan->s > 0 && (rc = launch_project(plan, received))) return rc;   // s = 0: nothing to locate
+  }
   if ((rc = mark(3))) return rc;
-  if ((rc = launch_locate(plan, byz_mask))) return rc;
+  {
+    TraceRange step(prof, "locate");
+    if ((rc = launch_locate(plan, byz_mask))) return rc;
+  }
   if ((rc = mark(4))) return rc;
-  if ((rc = launch_recover(plan, received, agg_grad))) return rc;
+  {
+    TraceRange step(prof, "recover");
+    if ((rc = launch_recover(plan, received, agg_grad))) return rc;
+  }
   return mark(5);
 }
 

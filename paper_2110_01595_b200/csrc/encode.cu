@@ -507,6 +507,7 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
 extern "C" int solon_encode(solon_plan* plan, const float* partition_grads, float* coded) {
   if (!plan || !partition_grads || !coded) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)partition_grads & 15) || ((uintptr_t)coded & 3)) return SOLON_ERR_INVALID_ARG;
+  solon::TraceRange range(plan->profiling != 0, "solon_encode");
   if (plan->profiling) {
     SOLON_CUDA_TRY(cudaEventRecord(plan->ev[0], plan->stream));
     plan->ev_valid[0] = 1;

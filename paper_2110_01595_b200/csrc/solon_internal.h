@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include <vector>
@@ -137,6 +138,21 @@ static inline int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 blo
   return SOLON_OK;
 }
 #endif
+
+// A named range on the calling host thread while `on` (plans with profiling switched on): timeline tools show the
+// library's calls and, inside solon_decode, its three launches under their names.  Header-only NVTX: costs nothing
+// measurable when no tool is attached.
+struct TraceRange {
+  bool on;
+  TraceRange(bool on_, const char* name) : on(on_) {
+    if (on) nvtxRangePushA(name);
+  }
+  ~TraceRange() {
+    if (on) nvtxRangePop();
+  }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 // Kernel launchers (each enqueues on plan->stream and returns a solon_status).
 // Whether solon_decode lets the locator work ahead on a partial projection (solon_plan_set_early_locator): a small
