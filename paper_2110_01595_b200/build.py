@@ -31,18 +31,33 @@ def build(verbose: bool = False, force: bool = False) -> str:
     """Compile every CUDA source for sm_100a into one shared library next to this file."""
     if not force and not needs_build():
         return LIB
-    cmd = [
-        _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-        "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
-    ]
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
-    proc = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or proc.returncode != 0:
-        sys.stderr.write(proc.stdout + proc.stderr)
-    if proc.returncode != 0:
-        raise RuntimeError("nvcc failed building libsolon.so")
+    # several processes (one rank per GPU) may get here at once: one builds, the others wait for the lock and find
+    # the library fresh; the compiler writes to a temporary name that is renamed into place when complete
+    import fcntl
+
+    with open(os.path.join(HERE, ".build.lock"), "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if not force and not needs_build():
+                return LIB
+            tmp = f"{LIB}.{os.getpid()}.tmp"
+            cmd = [
+                _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+                "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+            ]
+            if verbose:
+                cmd += ["-Xptxas", "-v"]
+            cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", tmp]
+            proc = subprocess.run(cmd, capture_output=True, text=True)
+            if verbose or proc.returncode != 0:
+                sys.stderr.write(proc.stdout + proc.stderr)
+            if proc.returncode != 0:
+                if os.path.exists(tmp):
+                    os.remove(tmp)
+                raise RuntimeError("nvcc failed building libsolon.so")
+            os.replace(tmp, LIB)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB
 
 
