@@ -30,7 +30,10 @@ denominator's roots are the corrupt nodes' scalars; the fixed-s system of
 Section 3.4 against the incremental variant; the r_c = 1 majority vote against
 the general decoder and the plain sum; Theorem 2 / its corollary and the
 introduction's 4-node example for feasibility; Table 2 for d_c; the
-least-squares gradient against finite differences of the loss.
+least-squares gradient against finite differences of the loss; the row
+energies against an entry-by-entry sum on a hand-made matrix and the
+floating-point tolerance by its value and by a deviation of half and of twice
+the tolerance sent through Algorithm 1.
 No function here is "parity unpinned".
 """
 

@@ -383,6 +383,53 @@ def test_fp32_rounded_coded_vectors_still_decode():
                 assert np.abs(u - want).max() <= 1e-4 * np.abs(want).max(), (P, s, m, kind)
 
 
+def test_row_energy_is_the_sum_of_squares_along_a_row():
+    """nu[k] = sum_p R[k, p]^2, added up entry by entry on a 3 x 4 matrix whose rows, columns and signs all differ
+    (a sum of absolute values, a sum down the columns or a squared sum would each give other numbers)."""
+    R = np.array([[1.0, -2.0, 3.0, 0.5], [0.0, 4.0, -1.0, 2.0], [-3.0, 0.25, 0.0, 1.0]], dtype=np.float32)
+    want = []
+    for k in range(3):
+        acc = 0.0
+        for p in range(4):
+            acc += float(R[k, p]) * float(R[k, p])
+        want.append(acc)
+    assert want == [14.25, 21.0, 10.0625]
+    assert np.array_equal(so.row_energy(R), np.array(want))
+
+
+def test_detection_tolerance_value_and_threshold():
+    """The floating-point reading of the locator's "!=" (Section 3.4): a node is off the fitted polynomial when its
+    projected value misses it by more than tau * sqrt(2 * median row energy).  The number itself on a hand-made
+    energy vector, then the decision through Algorithm 1: one coordinate of one honest coded vector is moved so that
+    the node's projected value moves by half the tolerance (not located, nothing to locate: Lemma 3's set is about
+    exact inequality, the floating-point test cannot see it) and by twice the tolerance (located)."""
+    assert so.detection_tolerance(np.array([8.0, 2.0, 18.0]), 0.5) == 2.0          # median 8: 0.5 * sqrt(16)
+    assert so.detection_tolerance(np.array([50.0, 2.0, 2.0, 50.0]), 1e-3) == pytest.approx(1e-3 * math.sqrt(52.0))
+    rng = np.random.default_rng(29)
+    P, s, m, d = 8, 1, 2, 64
+    sizes, w = _plan(P, s, m, r=8)                       # one group of eight: leverage of a node about m / 8
+    G = 300.0 * rng.normal(size=(P, d))                  # far from 1, so that sum R^2 and sum |R| differ by orders
+    Z = so.encode(G, m, sizes, w)
+    f = 1.0 + rng.normal(size=(1, Z.shape[1]))
+    tau = 1e-6
+    nu = [sum(float(v) * float(v) for v in Z[k]) for k in range(P)]
+    tol = tau * math.sqrt(2.0 * sorted(nu)[3] / 2.0 + 2.0 * sorted(nu)[4] / 2.0)   # median of eight: mean of the middle two
+    k, p0 = 5, 17
+    for factor, located in ((0.5, False), (2.0, True)):
+        R = Z.copy()
+        R[k, p0] += factor * tol / f[0, p0]
+        u, mask, status = so.decode(R, d, m, s, sizes, w, f, tau=tau)
+        assert status == 0
+        assert mask.nonzero()[0].tolist() == ([k] if located else []), factor
+    # the same two deviations straight through the locator with an explicit tolerance
+    rho = so.project(Z, f)
+    for factor, want_V in ((0.5, []), (2.0, [k])):
+        moved = rho.copy()
+        moved[0, k] += factor * tol
+        V, t = so.phi_incremental(moved, w, m, s, tol)
+        assert V == want_V and t == len(want_V)
+
+
 # ---------------------------------------------------------------- least-squares gradients
 
 
