@@ -119,7 +119,9 @@ int solon_plan_set_tolerance(solon_plan* plan, double tau);
  * fails (an attacker who spared those columns) the whole locator runs as it would have anyway.
  * Results do not depend on the mode.  mode 0: never; 1 (default): when the projection pass is long
  * enough to hide the early run (P * d_c * 4 bytes >= 350 MB) and the solver is small (groups of at
- * most 64 nodes, s <= 5); 2: whenever the solver is small. */
+ * most 64 nodes, s <= 5); 2: whenever the solver is small; 3: diagnostic - as 2, but the projection
+ * kernel announces no partial sums, so the locator's bounded wait for them (2 ms) runs out and it
+ * takes its ordinary path afterwards (outcome 3 of solon_plan_get_early_outcome; results unchanged). */
 int solon_plan_set_early_locator(solon_plan* plan, int mode);
 
 /* Rows per partition for solon_lsq_grads (default 256). */
@@ -169,6 +171,11 @@ int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8
 /* Status of the most recent solon_decode: synchronises the plan's stream, then returns SOLON_OK,
  * SOLON_ERR_UNDECODABLE, SOLON_ERR_INTERNAL or SOLON_ERR_CUDA. */
 int solon_decode_status(solon_plan* plan);
+
+/* Health of the plan's kernels so far, for callers that encode without decoding: synchronises the
+ * plan's stream, then returns SOLON_OK, SOLON_ERR_INTERNAL (a bounded wait inside one of the plan's
+ * kernels - solon_encode's included - ran out at some point; the bit is sticky) or SOLON_ERR_CUDA. */
+int solon_plan_status(solon_plan* plan);
 
 /* The decode in two halves, for a coded matrix whose COLUMNS are spread over several devices.
  * Equation (1)'s locator needs only the projected values rho = f R, and f R is a sum over
@@ -257,9 +264,13 @@ int solon_plan_get_early_outcome(solon_plan* plan, int* outcome);
  * The kernel's scratch (per-block partial sums and completion counters, about 1.3 MB) is a fixed
  * array inside the library's device image, so every GPU that loads the library holds it until the
  * process exits.  Limits: (K + 1) * P <= 512 and K <= 4; larger problems get SOLON_ERR_INVALID_ARG.
- * Nothing is allocated or freed, here or in any routine this calls.
- * The first call on each device looks up the array's device address (with that device current);
- * make that first call outside any stream capture.  All calls on a device share the one array: two
+ * No allocation routine is called, here or in anything this calls.  One thing is outside the library's
+ * hands: the CUDA runtime places the library's device code, this array included, on a device the first
+ * time anything of the library runs there.  A caller about to hand all device memory to its own pool
+ * should therefore make one call of this entry point (or create and destroy a plan) on each device at
+ * start-up, before the memory is given away.
+ * That first call on each device also looks up the array's device address (with that device current);
+ * make it outside any stream capture.  All calls on a device share the one array: two
  * calls whose kernels may overlap on the GPU (different streams, no ordering) race on it and
  * corrupt each other's sums; calls on one stream, or otherwise ordered, are fine.  The counters are
  * cleared at the start of every call; the partial sums are fully rewritten by every call.

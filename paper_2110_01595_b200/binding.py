@@ -51,6 +51,7 @@ SIGNATURES = {
     "solon_encode": (c_int, [c_void_p, c_void_p, c_void_p]),
     "solon_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_decode_status": (c_int, [c_void_p]),
+    "solon_plan_status": (c_int, [c_void_p]),
     "solon_decode_project": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_decode_finish": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "solon_lsq_grads": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -200,6 +201,7 @@ class Plan:
     def set_stream(self, stream) -> None:
         raw = stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
         _check(lib().solon_plan_set_stream(self._h, c_void_p(raw)), "solon_plan_set_stream")
+        self.stream_handle = int(raw)      # the cudaStream_t the plan's calls enqueue on
 
     def set_num_projections(self, K: int) -> None:
         _check(lib().solon_plan_set_num_projections(self._h, K), "solon_plan_set_num_projections")
@@ -211,7 +213,8 @@ class Plan:
         _check(lib().solon_plan_set_tolerance(self._h, tau), "solon_plan_set_tolerance")
 
     def set_early_locator(self, mode: int) -> None:
-        """0: never start the locator on a partial projection; 1 (default): when the projection pass is long; 2: always."""
+        """0: never start the locator on a partial projection; 1 (default): when the projection pass is long; 2: always;
+        3: diagnostic, the locator's wait for the partial sums runs out (outcome 3), results unchanged."""
         _check(lib().solon_plan_set_early_locator(self._h, mode), "solon_plan_set_early_locator")
 
     def early_outcome(self) -> np.ndarray:
@@ -320,6 +323,10 @@ class Plan:
 
     def decode_status(self) -> int:
         return lib().solon_decode_status(self._h)
+
+    def status(self) -> int:
+        """solon_plan_status: OK, or ERR_INTERNAL once a bounded wait inside one of the plan's kernels has run out."""
+        return lib().solon_plan_status(self._h)
 
     def lsq_grads(self, X, y, w, grads=None, rows: int | None = None):
         torch = self._torch

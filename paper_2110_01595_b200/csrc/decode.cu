@@ -21,15 +21,22 @@ extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_
     TraceRange step(prof, "project");
     if (plan->s > 0 && (rc = launch_project(plan, received))) return rc;   // s = 0: nothing to locate
   }
-  if ((rc = mark(3))) return rc;
+  // from here on the projection kernel may have announced partial sums on the progress counters, which only the
+  // recovery kernel puts back to zero: a failure before that kernel is enqueued clears them here instead
+  auto fail = [&](int code) -> int {
+    if (plan->s > 0) (void)cudaMemsetAsync(plan->d_proj_progress, 0, 2 * sizeof(unsigned long long), plan->stream);
+    (void)cudaGetLastError();
+    return code;
+  };
+  if ((rc = mark(3))) return fail(rc);
   {
     TraceRange step(prof, "locate");
-    if ((rc = launch_locate(plan, byz_mask))) return rc;
+    if ((rc = launch_locate(plan, byz_mask))) return fail(rc);
   }
-  if ((rc = mark(4))) return rc;
+  if ((rc = mark(4))) return fail(rc);
   {
     TraceRange step(prof, "recover");
-    if ((rc = launch_recover(plan, received, agg_grad))) return rc;
+    if ((rc = launch_recover(plan, received, agg_grad))) return fail(rc);
   }
   return mark(5);
 }

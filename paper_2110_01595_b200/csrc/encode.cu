@@ -13,7 +13,8 @@
 // ybar + delta without amplifying delta.  Only the rounding that differs from node to node - the Horner
 // evaluation and the final rounding to float32 - is amplified by the decoder (about 2^(m-1)), so for
 // m > 6 the polynomials are evaluated in float64 and rounded once; for m <= 6 float32 is enough.  The
-// generic kernel (any m) sums into a float64 ybar in shared memory first.
+// generic kernel (any m) sums into a float32 ybar tile in shared memory first (rows in node order, like the
+// specialised kernels) and evaluates in float64.
 //
 // Row segments start at arbitrary 4-byte offsets (d need not be a multiple of 4): the copy starts at
 // the enclosing 16-byte boundary and consumers index from the remainder; the last few floats of the

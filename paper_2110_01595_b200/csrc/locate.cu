@@ -429,7 +429,7 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   prm.use_smem = need <= 128 * 1024 ? 1 : 0;
   // working ahead on part A pays for a small solver beside a long projection pass (about 6 GB per ms); otherwise it
   // would still be at it when the projections end
-  prm.spec = (fused && plan->proj_two_parts) ? 1 : 0;
+  prm.spec = (fused && (plan->proj_two_parts || (early_locator_starved(plan) && uses_early_locator(plan)))) ? 1 : 0;
   size_t smem = prm.use_smem ? need : 0;
   const size_t tables = (2 * (size_t)plan->max_group * plan->max_group + (size_t)plan->max_group * (plan->s + 2)) * sizeof(double);
   prm.stage_tables = (prm.use_smem && smem + tables <= 200 * 1024) ? 1 : 0;

@@ -316,7 +316,7 @@ int solon_plan_reseed(solon_plan* plan, uint64_t seed) {
 }
 
 int solon_plan_set_early_locator(solon_plan* plan, int mode) {
-  if (!plan || mode < 0 || mode > 2) return SOLON_ERR_INVALID_ARG;
+  if (!plan || mode < 0 || mode > 3) return SOLON_ERR_INVALID_ARG;
   plan->early_locator = mode;
   return SOLON_OK;
 }
@@ -418,6 +418,14 @@ int solon_plan_get_timings(solon_plan* plan, float* ms) {
 }
 
 int64_t solon_plan_kernel_launches(const solon_plan* plan) { return plan ? plan->launches : SOLON_ERR_INVALID_ARG; }
+
+int solon_plan_status(solon_plan* plan) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  int word[2] = {0, 0};
+  SOLON_CUDA_TRY(cudaMemcpyAsync(word, plan->d_status, 2 * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  return ((word[0] | word[1]) & kStatusWaitExpired) ? SOLON_ERR_INTERNAL : SOLON_OK;
+}
 
 int solon_decode_status(solon_plan* plan) {
   if (!plan) return SOLON_ERR_INVALID_ARG;

@@ -5,7 +5,8 @@
 // Two forms: the plan's decode uses the streaming kernel (rows and f brought through a shared-memory ring by
 // bulk copies, float32 products in short runs, float64 sums: see project_pipe_kernel); the entry point that
 // allocates nothing uses the direct kernel (each warp loads its own rows, the tile of f in shared memory as
-// float64, every product and sum in float64).  Per-CTA partial sums go to global memory and are added in a
+// float64, every product and sum of rho in float64; nu is added in float32 inside a lane for one tile at a time
+// and in float64 beyond).  Per-CTA partial sums go to global memory and are added in a
 // fixed order by the last CTAs to finish (atomic tickets, no waiting), so results are bit-reproducible.
 #include <mutex>
 
@@ -513,7 +514,7 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   // part A (only when the locator kernel will work ahead on it): about an eighth of the range, whole slices, at least one
   int64_t a_slices = range_len / slice / 8;
   if (a_slices < 1) a_slices = 1;
-  const bool two_parts = !final_reduce && uses_early_locator(plan);
+  const bool two_parts = !final_reduce && uses_early_locator(plan) && !early_locator_starved(plan);
   pp.part_a_cols = two_parts ? a_slices * slice : 0;
   const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows + K) * pp.slot_floats * sizeof(float);
   SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -70,7 +70,7 @@ struct solon_plan {
   int proj_grid;           // CTAs of the projection kernel = number of partial sums
   double* d_partials;      // proj_grid x (K + 1) x P
   int proj_two_parts;      // the last projection launch announced part A
-  int early_locator;       // 0 never, 1 by size, 2 whenever the solver is small (solon_plan_set_early_locator)
+  int early_locator;       // 0 never, 1 by size, 2 whenever the solver is small, 3 diagnostic (solon_plan_set_early_locator)
   int proj_bunches;        // > 0: the last projection launch left this many bunch sums for the locator to add
   const double* proj_bunch_sums;   // proj_bunches x (K + 1) x P: final sums
   const double* proj_bunch_a;      // same shape: sums over part A of the column ranges only
@@ -161,8 +161,11 @@ struct TraceRange {
 inline bool uses_early_locator(const solon_plan* plan) {
   const bool small_solver = plan->s > 0 && plan->max_group <= 64 && plan->s <= 5;
   const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 350e6;
-  return small_solver && (plan->early_locator == 2 || (plan->early_locator == 1 && long_pass));
+  return small_solver && (plan->early_locator >= 2 || (plan->early_locator == 1 && long_pass));
 }
+// Mode 3 (diagnostic): the locator works ahead as in mode 2 but the projection kernel announces no partial sums,
+// so the locator's bounded wait for them runs out and it falls back to its ordinary path.
+inline bool early_locator_starved(const solon_plan* plan) { return plan->early_locator == 3; }
 
 int launch_fill_projection(solon_plan* plan);
 int launch_encode(solon_plan* plan, const float* grads, float* coded);

@@ -76,6 +76,9 @@ class ShardedPlan:
         """
         sums = self._buffer(received_local)
         rho, nu = sums[: self.K], sums[self.K]
+        if received_local.is_cuda and self.plan.stream_handle != torch.cuda.current_stream().cuda_stream:
+            raise RuntimeError("ShardedPlan.decode: the plan's stream is not torch's current stream, so the all-reduce "
+                               "would not be ordered between the two halves of the decode (use plan.set_stream)")
         if self.s > 0:
             self.plan.decode_project(received_local, rho, nu)
             if all_reduce is not None:

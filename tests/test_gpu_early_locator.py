@@ -130,6 +130,32 @@ def test_undecodable_and_reuse_with_the_early_locator():
         assert plan.decode_status() == 0 and torch.equal(agg, agg2) and torch.equal(mask, mask2)
 
 
+def test_the_bounded_wait_for_partial_sums_runs_out_and_the_decode_is_unchanged():
+    """Mode 3 lets the locator wait for partial sums that the projection kernel never announces: the wait (2 ms) gives
+    up, the locator takes its ordinary path after the projections, reports outcome 3, and every output equals what
+    mode 0 gives; the next decode in an ordinary mode is unaffected."""
+    wl = synth.small_variant(synth.WORKLOADS["resnet18"], 150_003)
+    G_cpu = synth.make_grads(wl, "cpu")
+    want = so.plain_sum(G_cpu.numpy())
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        received, nodes = synth.apply_attack(wl, plan.encode(G_cpu.cuda()))
+        out = []
+        for mode in (0, 3, 3, 2):
+            plan.set_early_locator(mode)
+            agg, mask = plan.decode(received)
+            status = plan.decode_status()
+            n_rec, t_acc, rows, coeff = plan.recovery()
+            out.append((status, agg.clone(), mask.clone(), n_rec.copy(), t_acc.copy(), rows.copy(), coeff.copy(),
+                        plan.early_outcome().tolist()))
+        assert set(out[0][7]) == {0}
+        assert set(out[1][7]) == {3} and set(out[2][7]) == {3}          # the wait expired, twice in a row
+        assert set(out[3][7]) <= {1, 4}                                 # and the counters were left clean
+        for other in out[1:]:
+            assert _same(out[0], other)
+        assert out[0][0] == 0 and out[0][2].cpu().numpy().nonzero()[0].tolist() == nodes
+        assert np.abs(out[0][1].cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+
+
 def test_both_early_outcomes_were_exercised():
     """Runs after the cases above (same module, file order): the early answer was confirmed somewhere and rejected
     somewhere, so both branches of the final pass are covered by the comparisons above."""

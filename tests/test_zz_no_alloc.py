@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import solon_oracle as so
 from paper_2110_01595_b200 import binding, build, synth
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +45,36 @@ def test_project_noalloc_matches_plan_path_twice_in_a_row():
             # nu is summed in float32 inside a lane before float64 takes over, so it depends on how the
             # columns are split among blocks: the parity tests' bound for nu applies
             assert np.allclose(got_nu, want_nu, rtol=1e-4), attempt
+            # and against the oracle's float64 projections and row energies of the same matrix: this kernel keeps
+            # exact float64 products and float64 sums for rho (only the order of the additions differs), and adds
+            # nu in float32 inside a lane for a tile at a time
+            R = received.cpu().numpy()
+            o_rho, o_nu = so.project(R, f[:, :d_c].cpu().numpy()), so.row_energy(R)
+            assert np.all(np.abs(got_rho - o_rho) <= 1e-12 * fn[:, None] * np.sqrt(o_nu)[None, :]), attempt
+            assert np.allclose(got_nu, o_nu, rtol=1e-5), attempt
+
+
+@pytest.mark.parametrize("K,P,d_c,pad", [(1, 7, 5, 3), (3, 15, 4099, 1), (4, 33, 70_001, 7), (2, 9, 1, 3), (4, 102, 2048, 0)])
+def test_project_noalloc_against_the_oracle_on_odd_shapes(K, P, d_c, pad):
+    """Every K, fewer columns than blocks (most blocks own no column), rows that start off 16-byte boundaries, and a
+    row pitch of f larger than d_c with junk in the padding, which the kernel must ignore."""
+    build.build()
+    gen = torch.Generator(device="cuda").manual_seed(1234 + K + P)
+    received = torch.randn((P, d_c), generator=gen, device="cuda", dtype=torch.float32)
+    pitch = (d_c + pad + 3) // 4 * 4
+    f = torch.full((K, pitch), 1.0e30, dtype=torch.float32, device="cuda")          # junk beyond d_c
+    f[:, :d_c] = 1.0 + torch.randn((K, d_c), generator=gen, device="cuda", dtype=torch.float32)
+    rho = torch.full((K, P), float("nan"), dtype=torch.float64, device="cuda")
+    nu = torch.full((P,), float("nan"), dtype=torch.float64, device="cuda")
+    for _ in range(2):
+        status = binding.solon_project_noalloc(received, f, rho, nu)
+        assert status == 0, binding.strerror(status)
+    torch.cuda.synchronize()
+    R, F = received.cpu().numpy(), f[:, :d_c].cpu().numpy()
+    o_rho, o_nu = so.project(R, F), so.row_energy(R)
+    lim = np.sqrt((F.astype(np.float64) ** 2).sum(1))[:, None] * np.sqrt(o_nu)[None, :]
+    assert np.all(np.abs(rho.cpu().numpy() - o_rho) <= 1e-12 * lim)
+    assert np.allclose(nu.cpu().numpy(), o_nu, rtol=1e-5)
 
 
 def test_project_noalloc_rejects_oversized_problems():
