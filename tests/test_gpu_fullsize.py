@@ -12,6 +12,7 @@ from paper_2110_01595_b200 import binding, build, synth
 pytestmark = pytest.mark.gpu
 
 AGG_TOL = 1e-4
+CODED_ROUNDINGS = 32      # float32 roundings of the sum of |terms| allowed on a coded value (largest group + m at most)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -69,12 +70,23 @@ def test_full_size(name):
             assert np.allclose(nu, o_nu, rtol=1e-4)
 
 
-@pytest.mark.parametrize("P,s,m,d", [(105, 5, 10, 10_000_000), (15, 1, 10, 10_000_000), (105, 1, 1, 10_000_000),
-                                     (45, 5, 2, 10_000_000), (15, 5, 5, 50_000_000)])
+def _grid_points():
+    """Every feasible (P, s, m) of the sweep at d = 10 M, plus the ends of the d = 50 M plane (the largest point, P = 105
+    with m = 1, holds 42 GB of gradients and coded vectors)."""
+    pts = [(wl.P, wl.s, wl.m, wl.d) for wl in synth.sweep_points((10_000_000,))]
+    return pts + [(15, 5, 5, 50_000_000), (45, 3, 10, 50_000_000), (105, 1, 1, 50_000_000)]
+
+
+@pytest.mark.parametrize("P,s,m,d", _grid_points())
 def test_sweep_points_full_size(P, s, m, d):
-    """Sweep points at bench size: mask exact, aggregate against the float64 definition at sampled coordinates
-    (oracle) and everywhere (device-side float64 sum)."""
+    """The sweep grid at bench size: mask exact; sampled coded chunks against the oracle's encoder; the aggregate
+    against the float64 definition at sampled coordinates (oracle) and everywhere (device-side float64 sum)."""
+    need = 4.0 * P * d * (1.0 + 1.0 / m) * 2.0 + 16.0 * d + 2e9      # gradients, coded, received copy, float64 sums
+    if torch.cuda.mem_get_info()[0] < need:
+        pytest.skip(f"needs about {need / 1e9:.0f} GB of free device memory")
     wl = synth.Workload(f"sweep_P{P}_s{s}_m{m}_d{d}", P, s, m, d, "normal", 1.0, "gaussian", s, 7000 + P + 10 * s + m)
+    sizes = so.group_sizes(wl.P, wl.r)
+    w = so.node_scalars(sizes)
     G = synth.make_grads(wl, "cuda")
     with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
         coded = plan.encode(G)
@@ -82,13 +94,25 @@ def test_sweep_points_full_size(P, s, m, d):
         agg, mask = plan.decode(received)
         assert plan.decode_status() == 0
         assert mask.cpu().numpy().nonzero()[0].tolist() == nodes
+        del received
         ref = G.sum(dim=0, dtype=torch.float64)
         scale = float(ref.abs().max())
         assert float((agg.double() - ref).abs().max()) <= AGG_TOL * scale
-        cols = np.unique(np.concatenate([np.random.default_rng(wl.seed).integers(0, d, size=2000), [0, d - 1]]))
-        G_s = G[:, torch.from_numpy(cols).cuda()].cpu().numpy()
-        got = agg[torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.float64)
-        assert np.abs(got - so.plain_sum(G_s)).max() <= AGG_TOL * scale
+        del ref
+        # sampled chunks: coded values against the oracle's encoder, aggregate against the oracle's plain sum
+        chunks = _sample_chunks(plan.d_c, 400, wl.seed)
+        cols = (chunks[:, None] * wl.m + np.arange(wl.m)[None, :]).reshape(-1)
+        in_range = cols < wl.d
+        G_s = np.zeros((wl.P, cols.size), dtype=np.float32)
+        G_s[:, in_range] = G[:, torch.from_numpy(cols[in_range]).cuda()].cpu().numpy()
+        Z_s = so.encode(G_s, wl.m, sizes, w)
+        got_Z = coded[:, torch.from_numpy(chunks).cuda()].cpu().numpy().astype(np.float64)
+        bound = so.encode(np.abs(G_s), wl.m, sizes, np.abs(w))
+        assert np.all(np.abs(got_Z - Z_s) <= CODED_ROUNDINGS * 2.0 ** -24 * bound + 1e-45)
+        got = agg[torch.from_numpy(cols[in_range]).cuda()].cpu().numpy().astype(np.float64)
+        assert np.abs(got - so.plain_sum(G_s)[in_range]).max() <= AGG_TOL * scale
+    del G, coded, agg
+    torch.cuda.empty_cache()
 
 
 def test_config_lsq_full_size():
