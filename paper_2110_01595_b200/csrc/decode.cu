@@ -60,7 +60,7 @@ extern "C" int solon_decode_finish(solon_plan* plan, const double* rho, const do
 
 // Row overwrite for device-resident simulations: one streaming copy for all rows.
 __global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__ matrix, const float* __restrict__ rows,
-                                                             const int* __restrict__ nodes, int P, int64_t d_c, int vec) {
+                                                             const int* __restrict__ nodes, int P, int64_t d_c, int vec, int stream_hints) {
   const int node = nodes[blockIdx.y];
   if (node < 0 || node >= P) return;
   float* dst = matrix + (int64_t)node * d_c;
@@ -77,9 +77,15 @@ __global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__
 #pragma unroll
       for (int u = 0; u < 8; ++u) v[u] = __ldcs(s4 + i + u * stride);
 #pragma unroll
-      for (int u = 0; u < 8; ++u) d4[i + u * stride] = v[u];
+      for (int u = 0; u < 8; ++u) {
+        if (stream_hints) __stcs(d4 + i + u * stride, v[u]);
+        else d4[i + u * stride] = v[u];
+      }
     }
-    for (; i < n4; i += stride) d4[i] = __ldcs(s4 + i);
+    for (; i < n4; i += stride) {
+      if (stream_hints) __stcs(d4 + i, __ldcs(s4 + i));
+      else d4[i] = __ldcs(s4 + i);
+    }
   } else {
     int64_t i = t0;
     for (; i + 7 * stride < d_c; i += 8 * stride) {
@@ -87,9 +93,15 @@ __global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__
 #pragma unroll
       for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + i + u * stride);
 #pragma unroll
-      for (int u = 0; u < 8; ++u) dst[i + u * stride] = v[u];
+      for (int u = 0; u < 8; ++u) {
+        if (stream_hints) __stcs(dst + i + u * stride, v[u]);
+        else dst[i + u * stride] = v[u];
+      }
     }
-    for (; i < d_c; i += stride) dst[i] = __ldcs(src + i);
+    for (; i < d_c; i += stride) {
+      if (stream_hints) __stcs(dst + i, __ldcs(src + i));
+      else dst[i] = __ldcs(src + i);
+    }
   }
 }
 
@@ -103,7 +115,7 @@ extern "C" int solon_overwrite_rows(solon_plan* plan, float* matrix, int n_rows,
   int64_t cap = ((int64_t)plan->num_sms * 8 + n_rows - 1) / n_rows;
   if (per_row > cap) per_row = cap;
   if (per_row < 1) per_row = 1;
-  overwrite_rows_kernel<<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec);
+  overwrite_rows_kernel<<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec, plan->stream_hints);
   SOLON_CUDA_TRY(cudaGetLastError());
   plan->launches += 1;
   return SOLON_OK;

@@ -43,6 +43,7 @@ struct EncodeParams {
   int64_t tiles_per_group;
   unsigned long long* tile_counter;   // [0] next tile to hand out, [1] CTAs that have left; both zero at launch
   int* status;            // device status words: [1] collects wait-expiry bits
+  int stream_hints;       // mark the gradients read and the coded values written evict-first in L2
 };
 
 // Horner evaluation for all nodes of the group with the chunk held in registers.
@@ -253,6 +254,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
   // last CTA to leave puts the counters back to zero for the next launch.
   if (tid >= kEncConsumers) {
     const int lane = tid - kEncConsumers;
+    const uint64_t stream_policy = pipe::policy_evict_first();
     uint32_t it = 0;
     long long tile = 0;
     if (lane == 0) tile = (long long)atomicAdd(prm.tile_counter, 1ULL);
@@ -285,7 +287,8 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
           for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.grads[e];   // <= 3 floats
           if (bytes) {
             pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
-            pipe::bulk_load(slot, prm.grads + a0, bytes, &full_bar[stage]);
+            if (prm.stream_hints) pipe::bulk_load_hint(slot, prm.grads + a0, bytes, &full_bar[stage], stream_policy);
+            else pipe::bulk_load(slot, prm.grads + a0, bytes, &full_bar[stage]);
           } else {
             pipe::mbar_arrive(&full_bar[stage]);
           }
@@ -385,7 +388,10 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
         Acc z = c[i][M - 1];
 #pragma unroll
         for (int l = M - 2; l >= 0; --l) z = acc_fma<Acc>(z, wk, c[i][l]);
-        if (ok[i]) out[i * kEncConsumers] = (float)z;
+        if (ok[i]) {
+          if (prm.stream_hints) __stcs(out + i * kEncConsumers, (float)z);
+          else out[i * kEncConsumers] = (float)z;
+        }
       }
       out += prm.d_c;
     }
@@ -488,6 +494,7 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   prm.total_floats = (int64_t)plan->P * plan->d;
   prm.status = plan->d_status;
   prm.tile_counter = plan->d_tile_counter + 1;
+  prm.stream_hints = plan->stream_hints;
   plan->launches += 1;
   switch (plan->m) {
     case 1: return launch_encode_direct<1, 4, float, 3>(plan, prm);

@@ -23,6 +23,12 @@ struct LocateParams {
   const int64_t* qb_off; // q
   const double* mt;      // q x m x m
   const double* tch;     // P x (s + 1)
+  const int* tab_count;       // recovery tables per corrupt set, all groups: rows in use per set
+  const int* tab_rows;        // tab_ld ints per set
+  const double* tab_coeff;    // tab_ld x m doubles per set
+  const int64_t* tab_off;     // q: first set of group g
+  const int* tab_sets;        // q: number of sets of group g (0: not tabulated)
+  int tab_ld;
   int P, m, s, K;
   double tau;
   double* ws_global;     // q x ws_stride doubles, used when shared memory is too small
@@ -131,6 +137,11 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   tb.Mt = prm.mt + (size_t)g * prm.m * prm.m;
   tb.Tch = prm.tch + (size_t)row0 * (prm.s + 1);
   tb.w = prm.w + row0;
+  tb.n_sets = prm.tab_sets[g];
+  tb.tab_ld = prm.tab_ld;
+  tb.tab_count = prm.tab_count + prm.tab_off[g];
+  tb.tab_rows = prm.tab_rows + (size_t)prm.tab_off[g] * prm.tab_ld;
+  tb.tab_coeff = prm.tab_coeff + (size_t)prm.tab_off[g] * prm.tab_ld * prm.m;
   if (prm.stage_tables) {
     // small groups: one coalesced pass brings the plan's tables on chip, so the dependent reads of the
     // solver never wait on L2 or HBM (the tables are evicted by the streaming kernels between decodes)
@@ -296,7 +307,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       // holds it when the epilogue comes.  Only for the subset form (m <= 6): the all-rows form takes a single warp
       // longer than the tasks last, and the CTA would wait for it.
       const int idle_warp = prm.s + 1 < (n_threads >> 5) ? prm.s + 1 : 0;
-      if (t == idle_warp && prm.m <= SOLON_SUBSET_MAX_M) {
+      if (tb.n_sets == 0 && t == idle_warp && prm.m <= SOLON_SUBSET_MAX_M) {
         const Team own = Team::own_warp();
         for (int k = own.lane; k < n; k += 32) sc.warm_trusted[k] = (k == 0 && prm.s > 0) ? 0 : 1;   // one node deleted
         __syncwarp();
@@ -392,6 +403,43 @@ void build_group_tables(int n, int m, int s, const double* w, double* Qb, double
     for (int i = 0; i <= s; ++i) Tch[(size_t)k * (s + 1) + i] = i < n ? (double)T[(size_t)i * n + k] : 0.0;
 }
 
+// Recovery tables of one group for every set of at most s untrusted nodes (host, once per plan): entry
+// corrupt_set_index(V) holds what recovery_table gives for the trusted set = complement of V.  Leaves the vectors empty
+// when there are more than SOLON_MAX_SETS such sets.  ld = rows reserved per set (m in the subset form, n otherwise).
+void build_recovery_tabs(int n, int m, int s, const GroupTables& tb, int ld, std::vector<int>* count, std::vector<int>* rows,
+                         std::vector<double>* coeff) {
+  count->clear();
+  rows->clear();
+  coeff->clear();
+  const int n_sets = count_corrupt_sets(n, s);
+  if (n_sets > SOLON_MAX_SETS) return;
+  count->assign((size_t)n_sets, 0);
+  rows->assign((size_t)n_sets * ld, 0);
+  coeff->assign((size_t)n_sets * ld * m, 0.0);
+  std::vector<uint8_t> trusted((size_t)n);
+  std::vector<int> r((size_t)n), V;
+  std::vector<double> c((size_t)n * m), ws(locate_epilogue_ws_doubles(n, m, s) + 8);
+  const Team tm = Team::serial();
+  for (int t = 0; t <= s && t <= n; ++t) {
+    V.resize(t);
+    for (int i = 0; i < t; ++i) V[i] = i;
+    for (;;) {
+      for (int k = 0; k < n; ++k) trusted[k] = 1;
+      for (int i = 0; i < t; ++i) trusted[V[i]] = 0;
+      const int idx = corrupt_set_index(n, trusted.data());
+      const int n_rec = recovery_table(tm, tb, n, m, s, trusted.data(), r.data(), c.data(), ws.data());
+      (*count)[idx] = n_rec;
+      for (int j = 0; j < n_rec; ++j) (*rows)[(size_t)idx * ld + j] = r[j];
+      for (int i = 0; i < n_rec * m; ++i) (*coeff)[(size_t)idx * ld * m + i] = c[i];
+      int i = t - 1;                       // next combination
+      while (i >= 0 && V[i] == n - t + i) --i;
+      if (i < 0) break;
+      ++V[i];
+      for (int j = i + 1; j < t; ++j) V[j] = V[j - 1] + 1;
+    }
+  }
+}
+
 int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const double* nu) {
   LocateParams prm;
   prm.group_start = plan->d_group_start;
@@ -413,6 +461,12 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   prm.qb_off = plan->d_qb_off;
   prm.mt = plan->d_mt;
   prm.tch = plan->d_tch;
+  prm.tab_count = plan->d_tab_count;
+  prm.tab_rows = plan->d_tab_rows;
+  prm.tab_coeff = plan->d_tab_coeff;
+  prm.tab_off = plan->d_tab_off;
+  prm.tab_sets = plan->d_tab_sets;
+  prm.tab_ld = plan->tab_ld;
   prm.P = plan->P; prm.m = plan->m; prm.s = plan->s; prm.K = plan->K;
   prm.tau = plan->tau;
   prm.ws_global = plan->d_locate_ws;
@@ -464,6 +518,18 @@ extern "C" int solon_locate_host(int n, int m, int s, int K, const double* rho, 
   tb.Mt = Mt.data();
   tb.Tch = Tch.data();
   tb.w = w_g;
+  tb.n_sets = 0;
+  tb.tab_ld = m <= SOLON_SUBSET_MAX_M ? m : n;
+  tb.tab_count = nullptr;
+  tb.tab_rows = nullptr;
+  tb.tab_coeff = nullptr;
+  std::vector<int> tab_count, tab_rows;
+  std::vector<double> tab_coeff;
+  build_recovery_tabs(n, m, s, tb, tb.tab_ld, &tab_count, &tab_rows, &tab_coeff);
+  tb.n_sets = (int)tab_count.size();
+  tb.tab_count = tab_count.data();
+  tb.tab_rows = tab_rows.data();
+  tb.tab_coeff = tab_coeff.data();
   std::vector<double> ws(group_ws_doubles(n, m, K, s) + 64);
   GroupScratch sc = carve(ws.data(), n, m, K, s);
   const Team tm = Team::serial();

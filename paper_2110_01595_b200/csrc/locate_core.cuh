@@ -86,7 +86,50 @@ struct GroupTables {
   const double* Mt;    // m x m, row-major: q_i(w) = sum_l Mt[l * m + i] w^l  (i < m)
   const double* Tch;   // n x (s + 1), row-major: Tch[k * (s + 1) + i] = T_i(w_k)
   const double* w;     // n node scalars
+  // Recovery tables tabulated per corrupt set (n_sets = 0: not tabulated, recovery_table runs at decode time): entry
+  // corrupt_set_index(V) holds what recovery_table returns when exactly the nodes V are untrusted - tab_count rows,
+  // their indices at tab_rows[i * tab_ld ..], their weights at tab_coeff[i * tab_ld * m ..].
+  const int* tab_count;
+  const int* tab_rows;
+  const double* tab_coeff;
+  int n_sets;
+  int tab_ld;
 };
+
+#define SOLON_MAX_SETS 4096   /* corrupt sets tabulated per group at most */
+
+// C(a, b) for small arguments.
+SOLON_HD inline long long binomial(int a, int b) {
+  if (b < 0 || b > a) return 0;
+  long long c = 1;
+  for (int i = 1; i <= b; ++i) c = c * (a - b + i) / i;
+  return c;
+}
+
+// Number of subsets of at most s of n nodes (saturating above SOLON_MAX_SETS).
+SOLON_HD inline int count_corrupt_sets(int n, int s) {
+  long long total = 0;
+  for (int t = 0; t <= s && t <= n; ++t) {
+    total += binomial(n, t);
+    if (total > SOLON_MAX_SETS) return SOLON_MAX_SETS + 1;
+  }
+  return (int)total;
+}
+
+// Position of the set {k : trusted[k] == 0} among all subsets of at most s of n nodes: sets are ordered by size and,
+// within a size t, by sum_i C(v_i, i + 1) over their nodes v_0 < v_1 < ... (the combinatorial number system).
+SOLON_HD inline int corrupt_set_index(int n, const uint8_t* trusted) {
+  int t = 0;
+  long long rank = 0;
+  for (int k = 0; k < n; ++k) {
+    if (trusted[k]) continue;
+    rank += binomial(k, t + 1);
+    ++t;
+  }
+  long long offset = 0;
+  for (int u = 0; u < t; ++u) offset += binomial(n, u);
+  return (int)(offset + rank);
+}
 
 // One (group, t) record written by locate_task and read by the group's epilogue.
 struct TaskRecord {
@@ -695,7 +738,19 @@ SOLON_HD inline int locate_epilogue(const Team& tm, const GroupTables& tb, int n
   int n_bad = 0;
   for (int k = 0; k < n; ++k) n_bad += trusted[k] ? 0 : 1;
   if (n_bad > s) ok = 0;
-  const int n_rec = recovery_table(tm, tb, n, m, s, trusted, rec_rows, coeff, ws);
+  int n_rec;
+  if (tb.n_sets > 0 && n_bad <= s) {
+    // tabulated at plan time for every set of at most s untrusted nodes
+    const int idx = corrupt_set_index(n, trusted);
+    n_rec = tb.tab_count[idx];
+    const int* rows_t = tb.tab_rows + (size_t)idx * tb.tab_ld;
+    const double* coeff_t = tb.tab_coeff + (size_t)idx * tb.tab_ld * m;
+    SOLON_FOR_THREADS(j, n_rec) rec_rows[j] = rows_t[j];
+    SOLON_FOR_THREADS(i, n_rec * m) coeff[i] = coeff_t[i];
+    SOLON_SYNC();
+  } else {
+    n_rec = recovery_table(tm, tb, n, m, s, trusted, rec_rows, coeff, ws);
+  }
   if (n_rec == 0) ok = 0;
   if (SOLON_TID == 0) {
     *n_rec_out = n_rec;

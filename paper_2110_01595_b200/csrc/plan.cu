@@ -12,6 +12,9 @@
 
 namespace solon {
 
+void build_recovery_tabs(int n, int m, int s, const GroupTables& tb, int ld, std::vector<int>* count, std::vector<int>* rows,
+                         std::vector<double>* coeff);   // locate.cu
+
 int check_params(int P, int s, int m, int r, int64_t d) {
   if (P < 1 || s < 0 || m < 1 || d < 1 || r < 1) return SOLON_ERR_INVALID_ARG;
   if (P > SOLON_MAX_NODES || m > SOLON_MAX_M || s > SOLON_MAX_S) return SOLON_ERR_INVALID_ARG;
@@ -113,6 +116,7 @@ static int dev_alloc(T** ptr, size_t count) {
 static void free_device(solon_plan* p) {
   cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f);
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
+  cudaFree(p->d_tab_count); cudaFree(p->d_tab_rows); cudaFree(p->d_tab_coeff); cudaFree(p->d_tab_off); cudaFree(p->d_tab_sets);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress);
@@ -217,6 +221,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
   p->num_sms = prop.multiProcessorCount;
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
+  p->stream_hints = keeps_l2_for_code(P, d) ? 1 : 0;
 
   rc = SOLON_OK;
   do {
@@ -248,6 +253,43 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
       (void)cudaGetLastError();
       rc = SOLON_ERR_CUDA;
       break;
+    }
+    {
+      // recovery tables for every set of at most s untrusted nodes, where those sets are few enough to tabulate
+      std::vector<int> all_count, all_rows, count, rows;
+      std::vector<double> all_coeff, coeff;
+      std::vector<int64_t> tab_off(q);
+      std::vector<int> tab_sets(q);
+      p->tab_ld = m <= SOLON_SUBSET_MAX_M ? m : max_group;
+      for (int g = 0; g < q; ++g) {
+        const int n_g = start[g + 1] - start[g];
+        GroupTables tb = {};
+        tb.Qb = h_qb.data() + qb_off[g];
+        tb.Hm = h_hm.data() + qb_off[g];
+        tb.Mt = h_mt.data() + (size_t)g * m * m;
+        tb.Tch = h_tch.data() + (size_t)start[g] * (s + 1);
+        tb.w = p->w.data() + start[g];
+        build_recovery_tabs(n_g, m, s, tb, p->tab_ld, &count, &rows, &coeff);
+        tab_off[g] = (int64_t)all_count.size();
+        tab_sets[g] = (int)count.size();
+        all_count.insert(all_count.end(), count.begin(), count.end());
+        all_rows.insert(all_rows.end(), rows.begin(), rows.end());
+        all_coeff.insert(all_coeff.end(), coeff.begin(), coeff.end());
+      }
+      if ((rc = dev_alloc(&p->d_tab_count, all_count.size()))) break;
+      if ((rc = dev_alloc(&p->d_tab_rows, all_rows.size()))) break;
+      if ((rc = dev_alloc(&p->d_tab_coeff, all_coeff.size()))) break;
+      if ((rc = dev_alloc(&p->d_tab_off, q))) break;
+      if ((rc = dev_alloc(&p->d_tab_sets, q))) break;
+      if ((!all_count.empty() && cudaMemcpy(p->d_tab_count, all_count.data(), all_count.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) ||
+          (!all_rows.empty() && cudaMemcpy(p->d_tab_rows, all_rows.data(), all_rows.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) ||
+          (!all_coeff.empty() && cudaMemcpy(p->d_tab_coeff, all_coeff.data(), all_coeff.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess) ||
+          cudaMemcpy(p->d_tab_off, tab_off.data(), q * sizeof(int64_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(p->d_tab_sets, tab_sets.data(), q * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
+        (void)cudaGetLastError();
+        rc = SOLON_ERR_CUDA;
+        break;
+      }
     }
     if ((rc = alloc_projection(p))) break;
     if ((rc = dev_alloc(&p->d_nu, P))) break;

@@ -109,6 +109,7 @@ struct RecoverPipe {
   int slot_floats;   // shared-memory floats per row slot (multiple of 4)
   unsigned long long* tile_counter;   // next tile to hand out; zero at launch
   int* status;
+  int stream_hints;   // write the aggregate with streaming stores (evict-first in L2)
 };
 
 // Streaming kernel: a producer warp moves the selected rows, tile by tile and a few rows at a time, into a
@@ -274,8 +275,13 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
       const int vec = count / 4;
       float4* dst4 = reinterpret_cast<float4*>(prm.agg + o0);
       const float4* src4 = reinterpret_cast<const float4*>(out_s);
-      for (int e = lane; e < vec; e += 32) dst4[e] = src4[e];
-      for (int e = vec * 4 + lane; e < count; e += 32) prm.agg[o0 + e] = out_s[e];
+      if (pp.stream_hints) {
+        for (int e = lane; e < vec; e += 32) __stcs(dst4 + e, src4[e]);
+        for (int e = vec * 4 + lane; e < count; e += 32) __stcs(prm.agg + o0 + e, out_s[e]);
+      } else {
+        for (int e = lane; e < vec; e += 32) dst4[e] = src4[e];
+        for (int e = vec * 4 + lane; e < count; e += 32) prm.agg[o0 + e] = out_s[e];
+      }
       __syncwarp();
     }
   }
@@ -311,6 +317,7 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   constexpr int kTileChunks = NC * CPT;
   RecoverPipe pp;
   pp.status = plan->d_status;
+  pp.stream_hints = plan->stream_hints;
   pp.slot_floats = kTileChunks + 8;
   const size_t slot_bytes = (size_t)pp.slot_floats * 4;
   const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + recover_coeff_bytes(plan->P, PackedStride<Acc, M>::value) +

@@ -46,6 +46,7 @@ struct solon_plan {
   int device;
   int num_sms;
   int64_t launches;
+  int stream_hints;        // the streaming kernels mark what they move evict-first in L2 (see keeps_l2_for_code)
 
   // host copies
   std::vector<int> group_start;   // q + 1
@@ -63,6 +64,12 @@ struct solon_plan {
   int64_t* d_qb_off;       // q offsets into d_qb
   double* d_mt;            // q x m x m monomial coefficients of the first m orthonormal polynomials
   double* d_tch;           // P x (s + 1) Chebyshev polynomials at the nodes
+  int* d_tab_count;        // recovery tables tabulated per corrupt set, all groups: rows in use per set
+  int* d_tab_rows;         // tab_ld ints per set
+  double* d_tab_coeff;     // tab_ld x m doubles per set
+  int64_t* d_tab_off;      // q: first set of group g
+  int* d_tab_sets;         // q: sets of group g (0: not tabulated, the table is computed at decode time)
+  int tab_ld;              // rows reserved per set: m in the subset form, the largest group otherwise
   float* d_f;              // K x f_pitch projection vectors
   int64_t f_pitch;         // row pitch of d_f in floats (multiple of 4)
 
@@ -166,6 +173,14 @@ inline bool uses_early_locator(const solon_plan* plan) {
 // Mode 3 (diagnostic): the locator works ahead as in mode 2 but the projection kernel announces no partial sums,
 // so the locator's bounded wait for them runs out and it falls back to its ordinary path.
 inline bool early_locator_starved(const solon_plan* plan) { return plan->early_locator == 3; }
+
+// Between two decodes the encode step and the recovery move gigabytes through L2 and push out everything else - the
+// locator kernel's instructions included, whose re-fetch from device memory (about a microsecond per 128 bytes of
+// code) is most of a short decode's serial time.  When every streamed byte is marked evict-first the code survives
+// in L2 and the locator runs about a third shorter (33 -> 25 us on 15 nodes); a single unmarked stream undoes it.
+// The marks cost the encode kernel 2-4 % of its bandwidth, which only pays while the step is short: up to 1 GB of
+// gradients per step.
+inline bool keeps_l2_for_code(int P, int64_t d) { return (double)P * (double)d * 4.0 <= 1.0e9; }
 
 int launch_fill_projection(solon_plan* plan);
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
