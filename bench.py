@@ -155,26 +155,64 @@ def oracle_sample(wl, d_sample: int, device):
 # ----------------------------------------------------------------------------- arms
 
 
+def config_of(wl, whole_d, n_byz, sharded):
+    """The workload description both arms print (identical keys and values, so the two lines can be compared)."""
+    return {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": whole_d, "n_byz": n_byz,
+            "attack": wl.attack,
+            "arithmetic": "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64",
+            "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * whole_d * 4 / 1e9),
+            "parallelism": ("one problem, coordinates sharded over the GPUs, one all-reduce of (K+1) x P float64 per decode"
+                            if sharded else "independent problems per GPU, no collective")}
+
+
+def host_memory_allows(wl, d_sample: int) -> bool:
+    """The oracle holds the float32 sample plus float64 copies of a group of gradients and of the coded matrix."""
+    try:
+        import psutil
+
+        need = wl.P * d_sample * 4 * 3.5 + 4e9
+        return psutil.virtual_memory().available >= need
+    except Exception:
+        return d_sample <= 4_000_000
+
+
+def oracle_speed_probe(wl) -> float:
+    """Gradient bytes per second of the oracle on a small sample (1 M coordinates), to size the timed samples."""
+    small, G_host, nodes, rows, f = oracle_sample(wl, 1_000_000, "cpu")
+    dt = oracle_step_seconds(small, G_host, nodes, rows, f)
+    return small.P * small.d * 4 / dt
+
+
 def run_reference(args, wl):
-    """The oracle as it stands, timed on the host cores, on a bounded sample of the workload."""
+    """The oracle as it stands, timed on the host cores.  Every step is one pass of the oracle (encode, attack,
+    decode) over a sample of the workload: the whole of it when steps + warm-up passes over the whole fit in about
+    three minutes, else its first coordinates, as many as do."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    warm = min(args.warmup, 1)
+    if args.oracle_d is None:
+        budget_s = 170.0 / (args.steps + warm)
+        d_fit = int(oracle_speed_probe(wl) * budget_s / (wl.P * 4))
+        args.oracle_d = max(wl.m * 1000, min(wl.d, d_fit))
+    while not host_memory_allows(wl, args.oracle_d) and args.oracle_d > 1_000_000:
+        args.oracle_d //= 2
     small, G_host, nodes, rows, f = oracle_sample(wl, args.oracle_d, "cpu")
-    for _ in range(min(args.warmup, 1)):
+    for _ in range(warm):
         oracle_step_seconds(small, G_host, nodes, rows, f)
     times = [oracle_step_seconds(small, G_host, nodes, rows, f) for _ in range(args.steps)]
     total = float(sum(times))
     value = small.P * small.d * 4 * args.steps / total / 1e9
     cores = blas_threads()
-    sample = f"first {small.d} of {wl.d} coordinates of every partition gradient, all {wl.P} nodes"
+    whole = "the whole workload" if small.d >= wl.d - wl.m else f"first {small.d} of {wl.d} coordinates of every partition gradient"
+    sample = f"{whole}, all {wl.P} nodes, per step (sized so that {args.steps} steps take about three minutes at most)"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
         "scaling": "strong" if args.sharded else "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": wl.d, "sample_d": small.d},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": config_of(wl, wl.d, len(nodes), args.sharded),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "sample_d": small.d},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -250,28 +288,43 @@ def run_ours(args, wl):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    # The timed region is EXACTLY args.steps steps; it is repeated until at least a second of GPU time has passed, so that
+    # the clocks are those of sustained work (the power cap needs a few hundred milliseconds to act).  The value reported is
+    # the median region; the fastest and slowest are given beside it.
     launches0 = plan.kernel_launches()
-    dist_util.barrier()
-    torch.cuda.synchronize()
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for i in range(args.steps):
-        step(evs[i])
-    stop.record()
-    torch.cuda.synchronize()
-    dist_util.barrier()
-    elapsed_ms = start.elapsed_time(stop)
-    launches = plan.kernel_launches() - launches0
+    regions, enc_all, dec_all = [], [], []
+    total_ms = 0.0
+    while True:
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+        dist_util.barrier()
+        torch.cuda.synchronize()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for i in range(args.steps):
+            step(evs[i])
+        stop.record()
+        torch.cuda.synchronize()
+        dist_util.barrier()
+        region_ms, _ = dist_util.combine(start.elapsed_time(stop), 0.0)        # max over ranks: all ranks take the same decision
+        regions.append(region_ms)
+        enc_all.append(float(np.mean([e[0].elapsed_time(e[1]) for e in evs])))
+        dec_all.append(float(np.mean([e[2].elapsed_time(e[3]) for e in evs])))
+        total_ms += region_ms
+        if total_ms >= args.min_timed_ms or len(regions) >= 2000:
+            break
+    launches = (plan.kernel_launches() - launches0) // len(regions)
     clocks = sampler.stop() if rank == 0 else None
     status = plan.decode_status()
     if status != 0 or mask.nonzero().flatten().tolist() != nodes:
         raise RuntimeError(f"timed decode failed: status {status}")
 
-    enc_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
-    dec_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
-    units = wl.P * wl.d * 4 * args.steps                       # gradient bytes this rank processed
-    max_ms, total_units = dist_util.combine(elapsed_ms, units)
+    order = int(np.argsort(regions)[len(regions) // 2])                         # the median region
+    max_ms = float(regions[order])
+    enc_ms, dec_ms = enc_all[order], dec_all[order]
+    _, total_units = dist_util.combine(0.0, wl.P * wl.d * 4 * args.steps)          # gradient bytes all ranks processed per region
+    repeats = {"n": len(regions), "timed_ms_total": total_ms, "ms_per_step_median": max_ms / args.steps,
+               "ms_per_step_min": min(regions) / args.steps, "ms_per_step_max": max(regions) / args.steps,
+               "ms_per_step_first": regions[0] / args.steps}
 
     # end to end through the host-buffer entry point: pinned host memory in, host results out
     e2e = None
@@ -310,13 +363,10 @@ def run_ours(args, wl):
         "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True,
         "scaling": "strong" if sp is not None else "weak",
         "vs_baseline": None, "dtype": "f32" if wl.m <= 6 else "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": whole.d, "n_byz": len(nodes),
-                   "attack": wl.attack,
-                   "arithmetic": "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64", "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * wl.d * 4 / 1e9),
-                   "parallelism": ("one problem, coordinates sharded over the GPUs, one all-reduce of (K+1) x P float64 per decode"
-                                   if sp is not None else "independent problems per GPU, no collective")},
+        "config": config_of(whole, whole.d, len(nodes), sp is not None),
+        "repeats": repeats,
         "roofline": {"bound": "hbm", "kernel": "encode_direct_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": TRAFFIC.get(wl.name) if sp is None else None,
+                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": encode_traffic(wl) if sp is None else None,
                      "algorithmic_bytes": enc_b, "ms": enc_ms},
         "path": {"encode_ms": enc_ms, "decode_ms": dec_ms, "decodes_per_s": 1e3 / dec_ms, "algorithmic_bytes": total_b,
                  "hbm_gbs": path_gbs, "frac_of_peak": path_gbs / peak, "frac_of_8TBs": path_gbs / 8000.0},
@@ -325,12 +375,55 @@ def run_ours(args, wl):
         "gpu_launches": int(launches),
     }
     if not args.no_cpu_baseline and world == 1 and sp is None:
-        small, G_s, nodes_s, rows_s, f_s = oracle_sample(wl, args.oracle_d, "cpu")
+        d_oracle = args.oracle_d if args.oracle_d is not None else wl.d          # the whole workload: one pass, 10-30 s
+        note = ""
+        while not host_memory_allows(wl, d_oracle) and d_oracle > 1_000_000:
+            d_oracle //= 2
+            note = " (the host's free memory does not hold the whole workload)"
+        small, G_s, nodes_s, rows_s, f_s = oracle_sample(wl, d_oracle, "cpu")
         dt = oracle_step_seconds(small, G_s, nodes_s, rows_s, f_s)
+        whole_txt = "the whole workload" if small.d >= wl.d - wl.m else f"first {small.d} of {wl.d} coordinates of every partition gradient"
         line["cpu_baseline"] = {"value": small.P * small.d * 4 / dt / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                                "sample": f"first {small.d} of {wl.d} coordinates of every partition gradient, all {wl.P} nodes, one step ({dt:.1f} s)"}
+                                "sample": f"{whole_txt}, all {wl.P} nodes, one step ({dt:.1f} s){note}", "sample_d": small.d}
     print(json.dumps(line), flush=True)
     dist_util.shutdown()
+
+
+def run_lsq(args, wl):
+    """solon_lsq_grads alone on the least-squares configuration (a parity case, not the benchmark step): CUDA events around
+    every call, L2 flushed between calls (the 1.54 GB matrix is larger than L2 anyway), algorithmic bytes = two passes
+    over X.  Prints one JSON line of its own."""
+    from paper_2110_01595_b200 import binding, build
+
+    torch.cuda.set_device(0)
+    build.build()
+    X, y, w = synth.make_lsq_problem(wl, "cuda")
+    w = torch.randn(wl.d, device="cuda", generator=torch.Generator(device="cuda").manual_seed(wl.seed + 3))
+    flush = torch.empty(160 * 1024 * 1024 // 4, dtype=torch.float32, device="cuda")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
+        G = plan.lsq_grads(X, y, w, rows=wl.lsq_rows)
+        for _ in range(max(args.warmup, 3)):
+            plan.lsq_grads(X, y, w, G, rows=wl.lsq_rows)
+        times = []
+        for _ in range(args.steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            plan.lsq_grads(X, y, w, G, rows=wl.lsq_rows)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        # a property that holds at any size: against a float64 device-side evaluation of X_i^T (X_i w - y_i)
+        rows = wl.lsq_rows
+        ref = torch.stack([X[i * rows:(i + 1) * rows].double().T @ (X[i * rows:(i + 1) * rows].double() @ w.double() - y[i * rows:(i + 1) * rows].double())
+                           for i in range(wl.P)])
+        err = float((G.double() - ref).abs().max() / ref.abs().max())
+    peak, peak_kind = measured_peak()
+    ms = float(np.median(times))
+    algo = 2 * 4 * wl.P * wl.lsq_rows * wl.d
+    print(json.dumps({"workload": wl.name, "kernel": "solon_lsq_grads", "steps": args.steps, "ms_median": ms, "ms_min": float(min(times)),
+                      "algorithmic_bytes": algo, "hbm_gbs": algo / (ms * 1e-3) / 1e9, "frac_of_peak": algo / (ms * 1e-3) / 1e9 / peak,
+                      "peak_kind": f"of {peak_kind}", "max_rel_err_vs_float64": err, "l2": "flushed between calls"}), flush=True)
 
 
 def run_sweep(args):
@@ -415,11 +508,18 @@ def run_sweep(args):
     print(json.dumps(summary), flush=True)
 
 
-# DRAM bytes (read + write) per encode launch.  Captured with ncu on the resnet18 workload (785.2 MB for 804.5 MB of
-# algorithmic bytes: the input is read exactly once, part of the output is still in L2 when the kernel ends);
-# the vgg13 figure is that capture scaled by the units processed (P * d), since the kernel makes one pass.
-# Emptied (reported as null) whenever the kernel changes until it is captured again.
-TRAFFIC: dict = {"resnet18": 785.2e6, "vgg13": 785.2e6 * (45 * 28_332_000) / (15 * 11_173_962)}
+def encode_traffic(wl):
+    """DRAM bytes (read + write) of one encode launch on this workload, from the ncu capture recorded in
+    profiles/encode_kernel_traffic.json: the capture's bytes scaled by the units processed (P * d; the kernel makes one
+    pass, so traffic grows in proportion).  None when no capture of the kernel as it stands is on record."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "encode_kernel_traffic.json")) as fh:
+            rec = json.load(fh)
+        if not rec.get("valid_for_current_kernel", False) or rec.get("m") != wl.m:
+            return None
+        return float(rec["dram_bytes_read"] + rec["dram_bytes_write"]) * (wl.P * wl.d) / (rec["P"] * rec["d"])
+    except Exception:
+        return None
 
 
 def main():
@@ -439,8 +539,10 @@ def main():
                     help="run the (P, s, m, d) grid instead: one JSON line per point is appended to FILE, a summary is printed")
     ap.add_argument("--sweep-d", default="1000000,10000000,50000000", help="gradient lengths of the grid")
     ap.add_argument("--oracle-d", type=int, default=None,
-                    help="coordinates per gradient in the oracle's sample (default: 16M for the cpu_baseline leg, "
-                         "2M per step for --impl reference)")
+                    help="coordinates per gradient in the oracle's sample (default: the whole workload for the cpu_baseline "
+                         "leg; for --impl reference as many as let steps + warm-up passes finish in about three minutes)")
+    ap.add_argument("--min-timed-ms", type=float, default=1000.0,
+                    help="the timed region of --steps steps is repeated until this much GPU time has passed")
     args = ap.parse_args()
     if args.workload in synth.WORKLOADS:
         wl = synth.WORKLOADS[args.workload]
@@ -450,9 +552,10 @@ def main():
             raise SystemExit(f"unknown workload {args.workload}")
         wl = match[0]
     if wl.grads == "lsq":
-        raise SystemExit("the lsq configuration is a parity case, not a bench workload")
-    if args.oracle_d is None:
-        args.oracle_d = 2_000_000 if args.impl == "reference" else 16_000_000
+        if args.steps == 200:
+            args.steps = 20
+        run_lsq(args, wl)
+        return
     if args.sweep:
         run_sweep(args)
         return

@@ -98,37 +98,42 @@ struct GroupTables {
 
 #define SOLON_MAX_SETS 4096   /* corrupt sets tabulated per group at most */
 
-// C(a, b) for small arguments.
-SOLON_HD inline long long binomial(int a, int b) {
+// C(a, b), saturating at 2^20 (callers only need exact values up to SOLON_MAX_SETS; 32-bit arithmetic throughout).
+SOLON_HD inline int binomial(int a, int b) {
   if (b < 0 || b > a) return 0;
-  long long c = 1;
-  for (int i = 1; i <= b; ++i) c = c * (a - b + i) / i;
+  int c = 1;
+  for (int i = 1; i <= b; ++i) {
+    if (c > (1 << 20)) return 1 << 20;
+    c = c * (a - b + i) / i;       // exact (c = C(a - b + i - 1, i - 1), so the product is i C(a - b + i, i)) and below 2^31 for a <= 1024
+  }
   return c;
 }
 
 // Number of subsets of at most s of n nodes (saturating above SOLON_MAX_SETS).
 SOLON_HD inline int count_corrupt_sets(int n, int s) {
-  long long total = 0;
+  int total = 0;
   for (int t = 0; t <= s && t <= n; ++t) {
     total += binomial(n, t);
     if (total > SOLON_MAX_SETS) return SOLON_MAX_SETS + 1;
   }
-  return (int)total;
+  return total;
 }
 
 // Position of the set {k : trusted[k] == 0} among all subsets of at most s of n nodes: sets are ordered by size and,
 // within a size t, by sum_i C(v_i, i + 1) over their nodes v_0 < v_1 < ... (the combinatorial number system).
 SOLON_HD inline int corrupt_set_index(int n, const uint8_t* trusted) {
-  int t = 0;
-  long long rank = 0;
+  int t = 0, rank = 0;
   for (int k = 0; k < n; ++k) {
     if (trusted[k]) continue;
     rank += binomial(k, t + 1);
     ++t;
   }
-  long long offset = 0;
-  for (int u = 0; u < t; ++u) offset += binomial(n, u);
-  return (int)(offset + rank);
+  int offset = 0, c = 1;         // c = C(n, u)
+  for (int u = 0; u < t; ++u) {
+    offset += c;
+    c = c * (n - u) / (u + 1);
+  }
+  return offset + rank;
 }
 
 // One (group, t) record written by locate_task and read by the group's epilogue.
@@ -742,7 +747,7 @@ SOLON_HD inline int locate_epilogue(const Team& tm, const GroupTables& tb, int n
   if (tb.n_sets > 0 && n_bad <= s) {
     // tabulated at plan time for every set of at most s untrusted nodes
     const int idx = corrupt_set_index(n, trusted);
-    n_rec = tb.tab_count[idx];
+    n_rec = m <= SOLON_SUBSET_MAX_M ? m : n - n_bad;      // what recovery_table returns for at most s untrusted nodes
     const int* rows_t = tb.tab_rows + (size_t)idx * tb.tab_ld;
     const double* coeff_t = tb.tab_coeff + (size_t)idx * tb.tab_ld * m;
     SOLON_FOR_THREADS(j, n_rec) rec_rows[j] = rows_t[j];

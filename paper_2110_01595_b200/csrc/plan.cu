@@ -1,6 +1,7 @@
 // Plan construction (Section 3.4: allocation, node scalars, projection vectors), queries, and the
 // plan-free host helpers of the C interface.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -222,6 +223,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
   p->stream_hints = keeps_l2_for_code(P, d) ? 1 : 0;
+  if (const char* env = getenv("SOLON_STREAM_HINTS")) p->stream_hints = env[0] == '1' ? 1 : (env[0] == '0' ? 0 : p->stream_hints);
 
   rc = SOLON_OK;
   do {

@@ -12,7 +12,7 @@ from paper_2110_01595_b200 import binding, build, synth
 pytestmark = pytest.mark.gpu
 
 AGG_TOL = 1e-4
-CODED_ROUNDINGS = 32      # float32 roundings of the sum of |terms| allowed on a coded value (largest group + m at most)
+CODED_ROUNDINGS = 8.0     # float32 roundings of the sum of |terms| allowed on a coded value: twice the largest error observed (3.8)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -48,8 +48,7 @@ def test_full_size(name):
         Z_s = so.encode(G_s, wl.m, sizes, w)                                       # P x len(chunks)
         got_Z = coded[:, torch.from_numpy(chunks).cuda()].cpu().numpy().astype(np.float64)
         bound = so.encode(np.abs(G_s), wl.m, sizes, np.abs(w))                     # sum of |terms|
-        ops = max(sizes) + wl.m                                                    # float32 roundings
-        assert np.all(np.abs(got_Z - Z_s) <= ops * 2.0 ** -24 * bound * 1.0001 + 1e-45)
+        assert np.all(np.abs(got_Z - Z_s) <= CODED_ROUNDINGS * 2.0 ** -24 * bound + 1e-45)
         # aggregate at the sampled coordinates against the plain float64 sum
         want_s = so.plain_sum(G_s)[in_range]
         got_s = agg[torch.from_numpy(cols[in_range]).cuda()].cpu().numpy().astype(np.float64)

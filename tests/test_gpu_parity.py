@@ -16,6 +16,11 @@ pytestmark = pytest.mark.gpu
 AGG_TOL = 1e-4          # max |agg_gpu - agg*| / ||agg*||_inf
 TAU = 1e-5              # the library's default detection tolerance, also given to the oracle
 RHO_TOL = 8 * 2.0 ** -24 * 1.01   # projections: worst case of the kernel's float32 runs, relative to ||f|| ||R_k||
+# Coded values against the oracle's float64 encoding, in float32 roundings (2^-24) of the sum of |terms|.  The largest
+# error seen over this suite's shapes is 3.8 roundings (m <= 6: float32 group sum and Horner steps), 3.0 (m = 8, 10) and
+# 3.1 (other m: float32 group sum, float64 evaluation); the bar is about twice that, far below the worst case (r_g + m).
+CODED_ROUNDINGS = 8.0
+OBSERVED = {"coded_roundings": 0.0}
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -32,8 +37,8 @@ def _oracle_plan(wl):
 def _check_encode(plan, G_cpu, coded_gpu, m, sizes, w):
     """Coded vectors against the oracle's float64 values.
 
-    Every m: float32 group sums and (m <= 6) float32 Horner steps stay within (r_g + m) roundings of the sum of
-    absolute terms.  m > 6 in addition: the group sum is the float32 left-to-right sum ybar' of the group's rows
+    Every m: float32 group sums and (m <= 6) float32 Horner steps stay within CODED_ROUNDINGS roundings of the sum of
+    absolute terms (about twice the largest error observed; the worst case would be r_g + m).  m > 6 in addition: the group sum is the float32 left-to-right sum ybar' of the group's rows
     (its rounding is common to all nodes of the group, so the decoder returns it unamplified), and the coded
     values are the float64 evaluation of the polynomial with coefficients ybar', rounded once: half an ulp from
     the oracle's encoding of ybar'."""
@@ -42,10 +47,9 @@ def _check_encode(plan, G_cpu, coded_gpu, m, sizes, w):
     got = coded_gpu.cpu().numpy().astype(np.float64)
     bound = so.encode(np.abs(G_np), m, sizes, np.abs(w))          # sum of |terms| of every entry
     err = np.abs(got - Z)
-    ops = np.zeros((Z.shape[0], 1))
-    for start, size in zip(so.group_starts(sizes), sizes):
-        ops[start:start + size] = size + m
-    assert np.all(err <= ops * 2.0 ** -24 * bound + 1e-45), float((err / (bound + 1e-30)).max())
+    worst = float((err / (2.0 ** -24 * bound + 1e-300)).max())
+    OBSERVED["coded_roundings"] = max(OBSERVED["coded_roundings"], worst)
+    assert np.all(err <= CODED_ROUNDINGS * 2.0 ** -24 * bound + 1e-45), worst
     if m > 6:
         G_sum = np.zeros_like(G_np)                                # row `start` of each group: ybar', the others 0
         for start, size in zip(so.group_starts(sizes), sizes):
@@ -102,6 +106,13 @@ def _run_case(wl, n_byz=None, check_intermediates=True):
             # and sum |f_p R_kp| <= ||f|| ||R_k||
             assert np.all(np.abs(rho - o_rho) <= RHO_TOL * lim + 1e-300)
             assert np.allclose(nu, o_nu, rtol=1e-4)
+            # what matters to the locator: on rows of ordinary size (honest ones) the error stays below a tenth of the
+            # detection tolerance tau * sqrt(2 median nu) of the row's group, so it cannot flip a decision
+            for start, size in zip(so.group_starts(sizes), sizes):
+                grp = slice(start, start + size)
+                tol = so.detection_tolerance(o_nu[grp], TAU)
+                ordinary = o_nu[grp] <= 4.0 * np.median(o_nu[grp])
+                assert np.all(np.abs(rho - o_rho)[:, grp][:, ordinary] <= 0.1 * tol + 1e-300)
             n_rec, t_acc, rows, coeff = plan.recovery()
             starts = so.group_starts(sizes)
             off = 0
