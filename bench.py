@@ -35,13 +35,13 @@ FALLBACK_HBM_GBS = 6650.0
 # ----------------------------------------------------------------------------- helpers
 
 
-def algorithmic_bytes(wl, n_rec_rows: int):
-    """Bytes each kernel must move (float32): encode 4 P d + 4 P d_c; projections 4 P d_c + 4 K d_c;
-    recovery 4 n_rows d_c + 4 d with n_rows the trusted rows the locator selected."""
+def algorithmic_bytes(wl, n_rec_rows: int, eb: int = 4):
+    """Bytes each kernel must move (eb bytes per element: 4 or 8): encode eb P d + eb P d_c; projections eb P d_c + 4 K d_c
+    (the vectors f are float32); recovery eb n_rows d_c + eb d with n_rows the trusted rows the locator selected."""
     d_c = wl.d_c
-    enc = 4 * wl.P * wl.d + 4 * wl.P * d_c
-    proj = 4 * wl.P * d_c + 4 * 2 * d_c
-    rec = 4 * n_rec_rows * d_c + 4 * wl.d
+    enc = eb * wl.P * wl.d + eb * wl.P * d_c
+    proj = eb * wl.P * d_c + 4 * 2 * d_c
+    rec = eb * n_rec_rows * d_c + eb * wl.d
     return enc, proj, rec
 
 
@@ -155,12 +155,13 @@ def oracle_sample(wl, d_sample: int, device):
 # ----------------------------------------------------------------------------- arms
 
 
-def config_of(wl, whole_d, n_byz, sharded):
+def config_of(wl, whole_d, n_byz, sharded, eb=4):
     """The workload description both arms print (identical keys and values, so the two lines can be compared)."""
     return {"workload": wl.name, "P": wl.P, "s": wl.s, "m": wl.m, "r": wl.r, "d": whole_d, "n_byz": n_byz,
-            "attack": wl.attack,
-            "arithmetic": "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64",
-            "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * whole_d * 4 / 1e9),
+            "attack": wl.attack, "element_bytes": eb,
+            "arithmetic": ("float64 elements at the boundary, float64 throughout" if eb == 8 else
+                           "encode and recovery in f32 for m <= 6 (f64 above), projections and locator in f64"),
+            "l2": "inputs (%.2f GB of gradients per step) are larger than L2" % (wl.P * whole_d * eb / 1e9),
             "parallelism": ("one problem, coordinates sharded over the GPUs, one all-reduce of (K+1) x P float64 per decode"
                             if sharded else "independent problems per GPU, no collective")}
 
@@ -202,7 +203,8 @@ def run_reference(args, wl):
         oracle_step_seconds(small, G_host, nodes, rows, f)
     times = [oracle_step_seconds(small, G_host, nodes, rows, f) for _ in range(args.steps)]
     total = float(sum(times))
-    value = small.P * small.d * 4 * args.steps / total / 1e9
+    eb = 8 if args.dtype == "f64" else 4
+    value = small.P * small.d * eb * args.steps / total / 1e9
     cores = blas_threads()
     whole = "the whole workload" if small.d >= wl.d - wl.m else f"first {small.d} of {wl.d} coordinates of every partition gradient"
     sample = f"{whole}, all {wl.P} nodes, per step (sized so that {args.steps} steps take about three minutes at most)"
@@ -211,7 +213,7 @@ def run_reference(args, wl):
         "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
         "scaling": "strong" if args.sharded else "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": config_of(wl, wl.d, len(nodes), args.sharded),
+        "config": config_of(wl, wl.d, len(nodes), args.sharded, 8 if args.dtype == "f64" else 4),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "sample_d": small.d},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -251,12 +253,15 @@ def run_ours(args, wl):
         whole = wl
         wl_rank = dataclasses.replace(wl, seed=wl.seed + 17 * rank)      # every rank its own problem
         G = synth.make_grads(wl_rank, "cuda")
-        plan = binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl_rank.seed)
+        if args.dtype == "f64":
+            G = G.double()
+        plan = binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl_rank.seed, dtype=args.dtype)
     coded = plan.encode(G)
     nodes = synth.byzantine_nodes(wl_rank)
     byz_rows = synth.byzantine_rows(wl_rank, coded, nodes)
     nodes_dev = torch.tensor(nodes, dtype=torch.int32, device="cuda")
-    agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+    eb = 8 if args.dtype == "f64" else 4
+    agg = torch.empty(wl.d, dtype=G.dtype, device="cuda")
     mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
 
     def step(events=None):
@@ -282,7 +287,7 @@ def run_ours(args, wl):
     if status != 0 or mask.nonzero().flatten().tolist() != nodes:
         raise RuntimeError(f"warm-up decode failed: status {status}")
     n_rec, _, _, _ = plan.recovery()
-    enc_b, proj_b, rec_b = algorithmic_bytes(wl, int(n_rec.sum()))
+    enc_b, proj_b, rec_b = algorithmic_bytes(wl, int(n_rec.sum()), eb)
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -321,7 +326,7 @@ def run_ours(args, wl):
     order = int(np.argsort(regions)[len(regions) // 2])                         # the median region
     max_ms = float(regions[order])
     enc_ms, dec_ms = enc_all[order], dec_all[order]
-    _, total_units = dist_util.combine(0.0, wl.P * wl.d * 4 * args.steps)          # gradient bytes all ranks processed per region
+    _, total_units = dist_util.combine(0.0, wl.P * wl.d * eb * args.steps)          # gradient bytes all ranks processed per region
     repeats = {"n": len(regions), "timed_ms_total": total_ms, "ms_per_step_median": max_ms / args.steps,
                "ms_per_step_min": min(regions) / args.steps, "ms_per_step_max": max(regions) / args.steps,
                "ms_per_step_first": regions[0] / args.steps}
@@ -329,10 +334,10 @@ def run_ours(args, wl):
     # end to end through the host-buffer entry point: pinned host memory in, host results out
     e2e = None
     if not args.no_e2e and sp is None:
-        G_host = torch.empty((wl.P, wl.d), dtype=torch.float32).pin_memory()
+        G_host = torch.empty((wl.P, wl.d), dtype=G.dtype).pin_memory()
         G_host.copy_(G)
         rows_host = byz_rows.cpu().pin_memory() if nodes else torch.empty((0, wl.d_c))
-        agg_host = torch.empty(wl.d, dtype=torch.float32).pin_memory()
+        agg_host = torch.empty(wl.d, dtype=G.dtype).pin_memory()
         mask_host = torch.empty(wl.P, dtype=torch.uint8).pin_memory()
         plan.step_host(G_host, nodes, rows_host, agg_host, mask_host)             # allocates staging, warms up
         dist_util.barrier()
@@ -344,9 +349,9 @@ def run_ours(args, wl):
         e2e_ms = (time.perf_counter() - t0) * 1e3
         if st != 0 or mask_host.nonzero().flatten().tolist() != nodes:
             raise RuntimeError("host-buffer step failed")
-        e2e_max_ms, e2e_units = dist_util.combine(e2e_ms, wl.P * wl.d * 4 * args.e2e_steps)
+        e2e_max_ms, e2e_units = dist_util.combine(e2e_ms, wl.P * wl.d * eb * args.e2e_steps)
         e2e = {"value": e2e_units / (e2e_max_ms * 1e-3) / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": wl.P * wl.d * 4 + len(nodes) * wl.d_c * 4, "d2h_bytes_per_step": wl.d * 4 + wl.P,
+               "h2d_bytes_per_step": wl.P * wl.d * eb + len(nodes) * wl.d_c * eb, "d2h_bytes_per_step": wl.d * eb + wl.P,
                "steps": args.e2e_steps}
         del G_host, agg_host
 
@@ -362,11 +367,11 @@ def run_ours(args, wl):
         "metric": METRIC, "value": total_units / (max_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True,
         "scaling": "strong" if sp is not None else "weak",
-        "vs_baseline": None, "dtype": "f32" if wl.m <= 6 else "f64", "data": "synthetic",
-        "config": config_of(whole, whole.d, len(nodes), sp is not None),
+        "vs_baseline": None, "dtype": "f64" if (args.dtype == "f64" or wl.m > 6) else "f32", "data": "synthetic",
+        "config": config_of(whole, whole.d, len(nodes), sp is not None, eb),
         "repeats": repeats,
         "roofline": {"bound": "hbm", "kernel": "encode_direct_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": encode_traffic(wl) if sp is None else None,
+                     "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": encode_traffic(wl) if (sp is None and eb == 4) else None,
                      "algorithmic_bytes": enc_b, "ms": enc_ms},
         "path": {"encode_ms": enc_ms, "decode_ms": dec_ms, "decodes_per_s": 1e3 / dec_ms, "algorithmic_bytes": total_b,
                  "hbm_gbs": path_gbs, "frac_of_peak": path_gbs / peak, "frac_of_8TBs": path_gbs / 8000.0},
@@ -383,7 +388,7 @@ def run_ours(args, wl):
         small, G_s, nodes_s, rows_s, f_s = oracle_sample(wl, d_oracle, "cpu")
         dt = oracle_step_seconds(small, G_s, nodes_s, rows_s, f_s)
         whole_txt = "the whole workload" if small.d >= wl.d - wl.m else f"first {small.d} of {wl.d} coordinates of every partition gradient"
-        line["cpu_baseline"] = {"value": small.P * small.d * 4 / dt / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+        line["cpu_baseline"] = {"value": small.P * small.d * eb / dt / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                 "sample": f"{whole_txt}, all {wl.P} nodes, one step ({dt:.1f} s){note}", "sample_d": small.d}
     print(json.dumps(line), flush=True)
     dist_util.shutdown()
@@ -529,6 +534,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vgg13")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "f64"],
+                    help="element type of gradients, coded vectors and aggregate (f64: the paper's 8-byte wire format)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -44,6 +44,12 @@ typedef enum solon_status {
 #define SOLON_MAX_S 16            /* adversaries per group                                    */
 #define SOLON_MAX_PROJECTIONS 4   /* random projections K                                     */
 
+/* Element type of partition gradients, coded vectors and aggregate (a property of the plan). */
+typedef enum solon_dtype {
+  SOLON_F32 = 0, /* float32 at the boundary (solon_encode, solon_decode, ...)                                   */
+  SOLON_F64 = 1  /* float64 at the boundary, the paper's wire format (Table 2): the calls with the suffix _f64 */
+} solon_dtype;
+
 typedef struct solon_plan solon_plan;
 
 /* ------------------------------------------------------------------------------------------
@@ -95,6 +101,18 @@ const char* solon_strerror(int status);
  * Synchronises the device once.  *out receives the plan, to be released by solon_plan_destroy. */
 int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solon_plan** out);
 int solon_plan_destroy(solon_plan* plan);
+
+/* The same with the element type chosen (solon_plan_create is dtype = SOLON_F32).  A SOLON_F64 plan moves 8-byte
+ * gradients, coded vectors and aggregates - what the paper's implementation sent (Table 2: 89.6 MB for ResNet-18's
+ * 11,173k parameters) and the precision for which it reports decoding trouble only "when r_c > 14" (appendix on
+ * limitations) - through solon_encode_f64, solon_decode_f64, solon_overwrite_rows_f64 and solon_step_host_f64; the
+ * float32 calls, solon_lsq_grads and the two-call decode return SOLON_ERR_INVALID_ARG on such a plan, and the _f64 calls
+ * on a float32 plan.  Group sums, polynomial evaluation, projections and recovery are all float64 then; the locator's
+ * default tolerance is 1e-10.  Compression ratios with a float64 kernel: m = 1..6, 8, 10, 12, 14
+ * (solon_float64_m_supported); any other m gives SOLON_ERR_INVALID_ARG. */
+int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, int dtype, solon_plan** out);
+int solon_float64_m_supported(int m);
+int solon_plan_dtype(const solon_plan* plan);          /* SOLON_F32 or SOLON_F64 */
 
 /* Stream on which later calls enqueue (a cudaStream_t passed as void*). */
 int solon_plan_set_stream(solon_plan* plan, void* cuda_stream);
@@ -168,6 +186,12 @@ int solon_encode(solon_plan* plan, const float* partition_grads, float* coded);
  * solon_decode_status reports SOLON_ERR_UNDECODABLE. */
 int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask);
 
+/* Encode and decode of a SOLON_F64 plan: as solon_encode / solon_decode with float64 buffers of the same shapes (bases
+ * 16-byte aligned).  The group sum, the mix and the recovery are float64 throughout, the projections exact float64
+ * products of the (float32-valued) vectors f with the received values. */
+int solon_encode_f64(solon_plan* plan, const double* partition_grads, double* coded);
+int solon_decode_f64(solon_plan* plan, const double* received, double* agg_grad, uint8_t* byz_mask);
+
 /* Status of the most recent solon_decode: synchronises the plan's stream, then returns SOLON_OK,
  * SOLON_ERR_UNDECODABLE, SOLON_ERR_INTERNAL or SOLON_ERR_CUDA. */
 int solon_decode_status(solon_plan* plan);
@@ -229,6 +253,11 @@ int solon_step_host(solon_plan* plan, const float* grads_host, int n_byz, const 
  *   rows    device, n_rows x d_c            out-of-range entries are skipped)
  * n_rows = 0 does nothing. */
 int solon_overwrite_rows(solon_plan* plan, float* matrix, int n_rows, const int* nodes, const float* rows);
+
+/* solon_step_host and solon_overwrite_rows for a SOLON_F64 plan (float64 buffers, same shapes and rules). */
+int solon_step_host_f64(solon_plan* plan, const double* grads_host, int n_byz, const int* byz_nodes,
+                        const double* byz_rows_host, double* agg_host, uint8_t* mask_host);
+int solon_overwrite_rows_f64(solon_plan* plan, double* matrix, int n_rows, const int* nodes, const double* rows);
 
 /* ------------------------------------------------------------------------------------------
  * Introspection of the last decode (for parity tests and diagnostics; each synchronises).

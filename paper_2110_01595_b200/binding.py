@@ -22,6 +22,8 @@ ERR_CUDA = -3
 ERR_UNDECODABLE = -4
 ERR_INTERNAL = -5
 ERR_NOMEM = -6
+F32 = 0
+F64 = 1
 
 # name -> (restype, argtypes); every symbol the header declares
 SIGNATURES = {
@@ -33,6 +35,9 @@ SIGNATURES = {
                                   POINTER(c_double)]),
     "solon_strerror": (c_char_p, [c_int]),
     "solon_plan_create": (c_int, [c_int, c_int, c_int, c_int, c_int64, c_uint64, POINTER(c_void_p)]),
+    "solon_plan_create_ex": (c_int, [c_int, c_int, c_int, c_int, c_int64, c_uint64, c_int, POINTER(c_void_p)]),
+    "solon_float64_m_supported": (c_int, [c_int]),
+    "solon_plan_dtype": (c_int, [c_void_p]),
     "solon_plan_destroy": (c_int, [c_void_p]),
     "solon_plan_set_stream": (c_int, [c_void_p, c_void_p]),
     "solon_plan_set_num_projections": (c_int, [c_void_p, c_int]),
@@ -50,6 +55,10 @@ SIGNATURES = {
     "solon_plan_get_projection_vectors": (c_int, [c_void_p, POINTER(c_float)]),
     "solon_encode": (c_int, [c_void_p, c_void_p, c_void_p]),
     "solon_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
+    "solon_encode_f64": (c_int, [c_void_p, c_void_p, c_void_p]),
+    "solon_decode_f64": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
+    "solon_overwrite_rows_f64": (c_int, [c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
+    "solon_step_host_f64": (c_int, [c_void_p, c_void_p, c_int, POINTER(c_int), c_void_p, c_void_p, c_void_p]),
     "solon_decode_status": (c_int, [c_void_p]),
     "solon_plan_status": (c_int, [c_void_p]),
     "solon_decode_project": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -168,12 +177,16 @@ def solon_project_noalloc(received, f, rho, nu, stream=None) -> int:
 class Plan:
     """Owner of a solon_plan*.  Methods mirror the C calls; tensors are torch CUDA tensors (float32, contiguous)."""
 
-    def __init__(self, P: int, s: int, m: int, r: int, d: int, seed: int = 0, stream=None):
+    def __init__(self, P: int, s: int, m: int, r: int, d: int, seed: int = 0, stream=None, dtype: str = "f32"):
         import torch
 
         self._torch = torch
+        if dtype not in ("f32", "f64"):
+            raise ValueError("dtype must be 'f32' or 'f64'")
+        self.dtype = dtype
+        self.tdtype = torch.float64 if dtype == "f64" else torch.float32     # element type of gradients, coded vectors, aggregate
         handle = c_void_p()
-        _check(lib().solon_plan_create(P, s, m, r, d, seed, byref(handle)), "solon_plan_create")
+        _check(lib().solon_plan_create_ex(P, s, m, r, d, seed, F64 if dtype == "f64" else F32, byref(handle)), "solon_plan_create_ex")
         self._h = handle
         self.P, self.s, self.m, self.r, self.d = P, s, m, r, d
         self.d_c = int(lib().solon_plan_dc(self._h))
@@ -265,8 +278,7 @@ class Plan:
 
     # -- hot path
     def _dev(self, t, shape, dtype=None):
-        torch = self._torch
-        dtype = dtype or torch.float32
+        dtype = dtype or self.tdtype
         if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype and tuple(t.shape) == tuple(shape)):
             raise ValueError(f"expected a contiguous CUDA {dtype} tensor of shape {tuple(shape)}, got {tuple(t.shape)} {t.dtype}")
         return c_void_p(t.data_ptr())
@@ -274,18 +286,20 @@ class Plan:
     def encode(self, partition_grads, coded=None):
         torch = self._torch
         if coded is None:
-            coded = torch.empty((self.P, self.d_c), dtype=torch.float32, device=partition_grads.device)
-        _check(lib().solon_encode(self._h, self._dev(partition_grads, (self.P, self.d)), self._dev(coded, (self.P, self.d_c))),
+            coded = torch.empty((self.P, self.d_c), dtype=self.tdtype, device=partition_grads.device)
+        fn = lib().solon_encode_f64 if self.dtype == "f64" else lib().solon_encode
+        _check(fn(self._h, self._dev(partition_grads, (self.P, self.d)), self._dev(coded, (self.P, self.d_c))),
                "solon_encode")
         return coded
 
     def decode(self, received, agg_grad=None, byz_mask=None):
         torch = self._torch
         if agg_grad is None:
-            agg_grad = torch.empty(self.d, dtype=torch.float32, device=received.device)
+            agg_grad = torch.empty(self.d, dtype=self.tdtype, device=received.device)
         if byz_mask is None:
             byz_mask = torch.empty(self.P, dtype=torch.uint8, device=received.device)
-        _check(lib().solon_decode(self._h, self._dev(received, (self.P, self.d_c)), self._dev(agg_grad, (self.d,)),
+        fn = lib().solon_decode_f64 if self.dtype == "f64" else lib().solon_decode
+        _check(fn(self._h, self._dev(received, (self.P, self.d_c)), self._dev(agg_grad, (self.d,)),
                                   self._dev(byz_mask, (self.P,), torch.uint8)), "solon_decode")
         return agg_grad, byz_mask
 
@@ -317,7 +331,8 @@ class Plan:
         n = int(nodes.numel())
         if n == 0:
             return matrix
-        _check(lib().solon_overwrite_rows(self._h, self._dev(matrix, (self.P, self.d_c)), n, self._dev(nodes, (n,), torch.int32),
+        fn = lib().solon_overwrite_rows_f64 if self.dtype == "f64" else lib().solon_overwrite_rows
+        _check(fn(self._h, self._dev(matrix, (self.P, self.d_c)), n, self._dev(nodes, (n,), torch.int32),
                                           self._dev(rows, (n, self.d_c))), "solon_overwrite_rows")
         return matrix
 
@@ -348,7 +363,8 @@ class Plan:
         n_byz = len(byz_nodes)
         nodes = np.asarray(byz_nodes, dtype=np.int32)
         rows_ptr = c_void_p(byz_rows_host.data_ptr()) if n_byz else c_void_p(0)
-        return lib().solon_step_host(self._h, c_void_p(grads_host.data_ptr()), n_byz,
+        fn = lib().solon_step_host_f64 if self.dtype == "f64" else lib().solon_step_host
+        return fn(self._h, c_void_p(grads_host.data_ptr()), n_byz,
                                      _dptr(nodes, c_int) if n_byz else None, rows_ptr,
                                      c_void_p(agg_host.data_ptr()), c_void_p(mask_host.data_ptr()))
 

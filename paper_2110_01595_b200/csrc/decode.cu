@@ -4,8 +4,10 @@
 
 using namespace solon;
 
-extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask) {
+template <typename T>
+static int decode_t(solon_plan* plan, const T* received, T* agg_grad, uint8_t* byz_mask) {
   if (!plan || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
+  if (plan->dtype != (sizeof(T) == 8 ? SOLON_F64 : SOLON_F32)) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)received & 15) || ((uintptr_t)agg_grad & 15)) return SOLON_ERR_INVALID_ARG;
   int rc;
   const bool prof = plan->profiling != 0;
@@ -15,11 +17,19 @@ extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_
     plan->ev_valid[i] = 1;
     return SOLON_OK;
   };
+  auto project = [&]() -> int {
+    if constexpr (sizeof(T) == 8) return launch_project_f64(plan, received);
+    else return launch_project(plan, received);
+  };
+  auto recover = [&]() -> int {
+    if constexpr (sizeof(T) == 8) return launch_recover_f64(plan, received, agg_grad);
+    else return launch_recover(plan, received, agg_grad);
+  };
   TraceRange range(prof, "solon_decode");
   if ((rc = mark(2))) return rc;
   {
     TraceRange step(prof, "project");
-    if (plan->s > 0 && (rc = launch_project(plan, received))) return rc;   // s = 0: nothing to locate
+    if (plan->s > 0 && (rc = project())) return rc;   // s = 0: nothing to locate
   }
   // from here on the projection kernel may have announced partial sums on the progress counters, which only the
   // recovery kernel puts back to zero: a failure before that kernel is enqueued clears them here instead
@@ -36,13 +46,21 @@ extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_
   if ((rc = mark(4))) return fail(rc);
   {
     TraceRange step(prof, "recover");
-    if ((rc = launch_recover(plan, received, agg_grad))) return fail(rc);
+    if ((rc = recover())) return fail(rc);
   }
   return mark(5);
 }
 
+extern "C" int solon_decode(solon_plan* plan, const float* received, float* agg_grad, uint8_t* byz_mask) {
+  return decode_t<float>(plan, received, agg_grad, byz_mask);
+}
+
+extern "C" int solon_decode_f64(solon_plan* plan, const double* received, double* agg_grad, uint8_t* byz_mask) {
+  return decode_t<double>(plan, received, agg_grad, byz_mask);
+}
+
 extern "C" int solon_decode_project(solon_plan* plan, const float* received, double* rho, double* nu) {
-  if (!plan || !received || !rho || !nu) return SOLON_ERR_INVALID_ARG;
+  if (!plan || !received || !rho || !nu || plan->dtype != SOLON_F32) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)received & 15) || ((uintptr_t)rho & 7) || ((uintptr_t)nu & 7)) return SOLON_ERR_INVALID_ARG;
   if (plan->s == 0) return SOLON_OK;
   return launch_project(plan, received, rho, nu);
@@ -50,7 +68,7 @@ extern "C" int solon_decode_project(solon_plan* plan, const float* received, dou
 
 extern "C" int solon_decode_finish(solon_plan* plan, const double* rho, const double* nu, const float* received,
                                    float* agg_grad, uint8_t* byz_mask) {
-  if (!plan || !rho || !nu || !received || !agg_grad || !byz_mask) return SOLON_ERR_INVALID_ARG;
+  if (!plan || !rho || !nu || !received || !agg_grad || !byz_mask || plan->dtype != SOLON_F32) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)received & 15) || ((uintptr_t)agg_grad & 15) || ((uintptr_t)rho & 7) || ((uintptr_t)nu & 7))
     return SOLON_ERR_INVALID_ARG;
   int rc;
@@ -59,16 +77,18 @@ extern "C" int solon_decode_finish(solon_plan* plan, const double* rho, const do
 }
 
 // Row overwrite for device-resident simulations: one streaming copy for all rows.
-__global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__ matrix, const float* __restrict__ rows,
+template <typename T>
+__global__ void __launch_bounds__(256) overwrite_rows_kernel(T* __restrict__ matrix, const T* __restrict__ rows,
                                                              const int* __restrict__ nodes, int P, int64_t d_c, int vec, int stream_hints) {
+  constexpr int kVec = 16 / sizeof(T);     // elements per 16 bytes
   const int node = nodes[blockIdx.y];
   if (node < 0 || node >= P) return;
-  float* dst = matrix + (int64_t)node * d_c;
-  const float* src = rows + (int64_t)blockIdx.y * d_c;
+  T* dst = matrix + (int64_t)node * d_c;
+  const T* src = rows + (int64_t)blockIdx.y * d_c;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (vec) {   // d_c a multiple of 4 and both bases 16-byte aligned: every row starts on a 16-byte boundary
-    const int64_t n4 = d_c / 4;
+  if (vec) {   // d_c a multiple of 16 bytes and both bases 16-byte aligned: every row starts on a 16-byte boundary
+    const int64_t n4 = d_c / kVec;
     float4* d4 = reinterpret_cast<float4*>(dst);
     const float4* s4 = reinterpret_cast<const float4*>(src);
     int64_t i = t0;
@@ -89,7 +109,7 @@ __global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__
   } else {
     int64_t i = t0;
     for (; i + 7 * stride < d_c; i += 8 * stride) {
-      float v[8];
+      T v[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + i + u * stride);
 #pragma unroll
@@ -105,20 +125,32 @@ __global__ void __launch_bounds__(256) overwrite_rows_kernel(float* __restrict__
   }
 }
 
-extern "C" int solon_overwrite_rows(solon_plan* plan, float* matrix, int n_rows, const int* nodes, const float* rows) {
+template <typename T>
+static int overwrite_rows_t(solon_plan* plan, T* matrix, int n_rows, const int* nodes, const T* rows) {
   if (!plan || n_rows < 0 || n_rows > plan->P) return SOLON_ERR_INVALID_ARG;
+  if (plan->dtype != (sizeof(T) == 8 ? SOLON_F64 : SOLON_F32)) return SOLON_ERR_INVALID_ARG;
   if (n_rows == 0) return SOLON_OK;
   if (!matrix || !nodes || !rows) return SOLON_ERR_INVALID_ARG;
-  const int vec = (plan->d_c % 4 == 0 && !((uintptr_t)matrix & 15) && !((uintptr_t)rows & 15)) ? 1 : 0;
+  constexpr int kVec = 16 / sizeof(T);
+  const int vec = (plan->d_c % kVec == 0 && !((uintptr_t)matrix & 15) && !((uintptr_t)rows & 15)) ? 1 : 0;
   // one wave of CTAs (eight per SM) shared by the rows; every thread then has several batches of eight accesses
-  int64_t per_row = (plan->d_c / (vec ? 4 : 1) + 256 * 8 - 1) / (256 * 8);
+  int64_t per_row = (plan->d_c / (vec ? kVec : 1) + 256 * 8 - 1) / (256 * 8);
   int64_t cap = ((int64_t)plan->num_sms * 8 + n_rows - 1) / n_rows;
   if (per_row > cap) per_row = cap;
   if (per_row < 1) per_row = 1;
-  overwrite_rows_kernel<<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec, plan->stream_hints);
+  overwrite_rows_kernel<T><<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec,
+                                                                                               plan->stream_hints);
   SOLON_CUDA_TRY(cudaGetLastError());
   plan->launches += 1;
   return SOLON_OK;
+}
+
+extern "C" int solon_overwrite_rows(solon_plan* plan, float* matrix, int n_rows, const int* nodes, const float* rows) {
+  return overwrite_rows_t<float>(plan, matrix, n_rows, nodes, rows);
+}
+
+extern "C" int solon_overwrite_rows_f64(solon_plan* plan, double* matrix, int n_rows, const int* nodes, const double* rows) {
+  return overwrite_rows_t<double>(plan, matrix, n_rows, nodes, rows);
 }
 
 template <typename T>
@@ -133,28 +165,45 @@ static int stage_alloc(T** ptr, size_t count) {
   return SOLON_OK;
 }
 
-extern "C" int solon_step_host(solon_plan* plan, const float* grads_host, int n_byz, const int* byz_nodes,
-                               const float* byz_rows_host, float* agg_host, uint8_t* mask_host) {
+template <typename T>
+static int step_host_t(solon_plan* plan, const T* grads_host, int n_byz, const int* byz_nodes, const T* byz_rows_host, T* agg_host,
+                       uint8_t* mask_host) {
   if (!plan || !grads_host || !agg_host || !mask_host || n_byz < 0) return SOLON_ERR_INVALID_ARG;
+  if (plan->dtype != (sizeof(T) == 8 ? SOLON_F64 : SOLON_F32)) return SOLON_ERR_INVALID_ARG;
   if (n_byz > 0 && (!byz_nodes || !byz_rows_host)) return SOLON_ERR_INVALID_ARG;
   for (int i = 0; i < n_byz; ++i)
     if (byz_nodes[i] < 0 || byz_nodes[i] >= plan->P) return SOLON_ERR_INVALID_ARG;
   int rc;
   const size_t n_grad = (size_t)plan->P * plan->d, n_coded = (size_t)plan->P * plan->d_c;
-  if ((rc = stage_alloc(&plan->d_stage_grads, n_grad))) return rc;
-  if ((rc = stage_alloc(&plan->d_stage_coded, n_coded))) return rc;
-  if ((rc = stage_alloc(&plan->d_stage_agg, (size_t)plan->d))) return rc;
+  // the staging buffers are typed by the plan's element type (allocated in bytes)
+  T** grads_dev = reinterpret_cast<T**>(&plan->d_stage_grads);
+  T** coded_dev = reinterpret_cast<T**>(&plan->d_stage_coded);
+  T** agg_dev = reinterpret_cast<T**>(&plan->d_stage_agg);
+  if ((rc = stage_alloc(grads_dev, n_grad))) return rc;
+  if ((rc = stage_alloc(coded_dev, n_coded))) return rc;
+  if ((rc = stage_alloc(agg_dev, (size_t)plan->d))) return rc;
   if ((rc = stage_alloc(&plan->d_stage_mask, (size_t)plan->P))) return rc;
   cudaStream_t st = plan->stream;
-  SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_stage_grads, grads_host, n_grad * sizeof(float), cudaMemcpyHostToDevice, st));
-  if ((rc = solon_encode(plan, plan->d_stage_grads, plan->d_stage_coded))) return rc;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(*grads_dev, grads_host, n_grad * sizeof(T), cudaMemcpyHostToDevice, st));
+  if constexpr (sizeof(T) == 8) rc = solon_encode_f64(plan, *grads_dev, *coded_dev);
+  else rc = solon_encode(plan, *grads_dev, *coded_dev);
+  if (rc) return rc;
   for (int i = 0; i < n_byz; ++i) {
-    SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_stage_coded + (size_t)byz_nodes[i] * plan->d_c,
-                                   byz_rows_host + (size_t)i * plan->d_c, (size_t)plan->d_c * sizeof(float),
-                                   cudaMemcpyHostToDevice, st));
+    SOLON_CUDA_TRY(cudaMemcpyAsync(*coded_dev + (size_t)byz_nodes[i] * plan->d_c, byz_rows_host + (size_t)i * plan->d_c,
+                                   (size_t)plan->d_c * sizeof(T), cudaMemcpyHostToDevice, st));
   }
-  if ((rc = solon_decode(plan, plan->d_stage_coded, plan->d_stage_agg, plan->d_stage_mask))) return rc;
-  SOLON_CUDA_TRY(cudaMemcpyAsync(agg_host, plan->d_stage_agg, (size_t)plan->d * sizeof(float), cudaMemcpyDeviceToHost, st));
+  if ((rc = decode_t<T>(plan, *coded_dev, *agg_dev, plan->d_stage_mask))) return rc;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(agg_host, *agg_dev, (size_t)plan->d * sizeof(T), cudaMemcpyDeviceToHost, st));
   SOLON_CUDA_TRY(cudaMemcpyAsync(mask_host, plan->d_stage_mask, (size_t)plan->P, cudaMemcpyDeviceToHost, st));
   return solon_decode_status(plan);
+}
+
+extern "C" int solon_step_host(solon_plan* plan, const float* grads_host, int n_byz, const int* byz_nodes,
+                               const float* byz_rows_host, float* agg_host, uint8_t* mask_host) {
+  return step_host_t<float>(plan, grads_host, n_byz, byz_nodes, byz_rows_host, agg_host, mask_host);
+}
+
+extern "C" int solon_step_host_f64(solon_plan* plan, const double* grads_host, int n_byz, const int* byz_nodes,
+                                   const double* byz_rows_host, double* agg_host, uint8_t* mask_host) {
+  return step_host_t<double>(plan, grads_host, n_byz, byz_nodes, byz_rows_host, agg_host, mask_host);
 }

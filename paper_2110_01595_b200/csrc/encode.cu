@@ -28,14 +28,15 @@ constexpr int kEncConsumers = 256;                 // consumer threads per CTA
 constexpr int kEncThreads = kEncConsumers + 32;    // + one producer warp
 constexpr int kEncMaxBatch = 32;                   // rows per pipeline stage (one per producer lane)
 
-struct EncodeParams {
-  const float* grads;
-  float* coded;
+template <typename T>
+struct EncodeParamsT {
+  const T* grads;
+  T* coded;
   const int* group_start;
   const double* w;
   int q, m, P;
   int64_t d, d_c;
-  int64_t total_floats;   // P * d
+  int64_t total_floats;   // P * d (elements)
   int chunks_per_thread;  // tile = kEncConsumers * chunks_per_thread chunks
   int row_batch;          // rows per stage
   int stages;
@@ -45,6 +46,11 @@ struct EncodeParams {
   int* status;            // device status words: [1] collects wait-expiry bits
   int stream_hints;       // mark the gradients read and the coded values written evict-first in L2
 };
+typedef EncodeParamsT<float> EncodeParams;
+
+// Elements per 16 bytes (the granularity of bulk copies): 4 floats or 2 doubles.
+template <typename T>
+struct Vec16 { static constexpr int64_t n = 16 / sizeof(T); };
 
 // Horner evaluation for all nodes of the group with the chunk held in registers.
 template <int M>
@@ -219,8 +225,9 @@ __device__ __forceinline__ float acc_fma<float>(float a, float b, float c) { ret
 template <>
 __device__ __forceinline__ double acc_fma<double>(double a, double b, double c) { return fma(a, b, c); }
 
-template <int M, int CPT, typename Acc, int kMinBlocks>
-__global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(EncodeParams prm) {
+template <int M, int CPT, typename Acc, int kMinBlocks, typename T>
+__global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(EncodeParamsT<T> prm) {
+  constexpr int64_t kVec = Vec16<T>::n;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x;
   constexpr int kTileChunks = kEncConsumers * CPT;
@@ -232,7 +239,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
   int* b0_of = reinterpret_cast<int*>(tile_of + prm.stages);                  // per stage: first row of that batch
   int* abort_flag = b0_of + prm.stages;
   Acc* w_s = reinterpret_cast<Acc*>(smem_raw + 256);                       // all P node scalars
-  float* ring = reinterpret_cast<float*>(smem_raw + 256 + (((size_t)prm.P * sizeof(Acc) + 15) & ~(size_t)15));
+  T* ring = reinterpret_cast<T*>(smem_raw + 256 + (((size_t)prm.P * sizeof(Acc) + 15) & ~(size_t)15));
   const size_t stage_floats = (size_t)prm.row_batch * prm.slot_floats;
 
   if (tid == 0) {
@@ -278,13 +285,13 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
         if (lane < nb) {
           const int64_t first = (int64_t)(row0 + b0 + lane) * prm.d + e0;
           const int64_t last = first + (e1 - e0);
-          const int64_t a0 = first & ~(int64_t)3;
-          int64_t a1 = (last + 3) & ~(int64_t)3;
-          const int64_t safe_end = prm.total_floats & ~(int64_t)3;
+          const int64_t a0 = first & ~(kVec - 1);
+          int64_t a1 = (last + kVec - 1) & ~(kVec - 1);
+          const int64_t safe_end = prm.total_floats & ~(kVec - 1);
           if (a1 > safe_end) a1 = safe_end;
-          float* slot = ring + stage * stage_floats + (size_t)lane * prm.slot_floats;
-          const uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
-          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.grads[e];   // <= 3 floats
+          T* slot = ring + stage * stage_floats + (size_t)lane * prm.slot_floats;
+          const uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * sizeof(T)) : 0u;
+          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.grads[e];   // fewer than 16 bytes
           if (bytes) {
             pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
             if (prm.stream_hints) pipe::bulk_load_hint(slot, prm.grads + a0, bytes, &full_bar[stage], stream_policy);
@@ -317,8 +324,8 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
     return;
   }
 
-  const int d_mod4 = (int)(prm.d & 3);
-  float acc[CPT][M];   // the group sum of this thread's chunks
+  const int d_mod4 = (int)(prm.d & (kVec - 1));
+  T acc[CPT][M];   // the group sum of this thread's chunks (in the element type)
   int row0 = 0, r_g = 0, valid = 0;
   int64_t e0 = 0, ct = 0;
   for (uint32_t it = 0;; ++it) {
@@ -338,32 +345,32 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 #pragma unroll
       for (int i = 0; i < CPT; ++i)
 #pragma unroll
-        for (int l = 0; l < M; ++l) acc[i][l] = 0.0f;
+        for (int l = 0; l < M; ++l) acc[i][l] = (T)0;
     }
     const bool full_tile = valid == kTileFloats;
     const int nb = min(prm.row_batch, r_g - b0);
-    const float* slot = ring + stage * stage_floats + tid * M;
-    int shift = ((((row0 + b0) & 3) * d_mod4) + (int)(e0 & 3)) & 3;        // (row * d + e0) mod 4
+    const T* slot = ring + stage * stage_floats + tid * M;
+    int shift = (int)(((((row0 + b0) & (kVec - 1)) * d_mod4) + (e0 & (kVec - 1))) & (kVec - 1));   // (row * d + e0) mod (elements per 16 bytes)
     if (full_tile) {
       for (int j = 0; j < nb; ++j) {
-        const float* src = slot + shift;
+        const T* src = slot + shift;
 #pragma unroll
         for (int i = 0; i < CPT; ++i)
 #pragma unroll
           for (int l = 0; l < M; ++l) acc[i][l] += src[i * kEncConsumers * M + l];
         slot += prm.slot_floats;
-        shift = (shift + d_mod4) & 3;
+        shift = (int)((shift + d_mod4) & (kVec - 1));
       }
     } else {
       for (int j = 0; j < nb; ++j) {
-        const float* src = slot + shift;
+        const T* src = slot + shift;
 #pragma unroll
         for (int i = 0; i < CPT; ++i)
 #pragma unroll
           for (int l = 0; l < M; ++l)
             if ((tid + i * kEncConsumers) * M + l < valid) acc[i][l] += src[i * kEncConsumers * M + l];
         slot += prm.slot_floats;
-        shift = (shift + d_mod4) & 3;
+        shift = (int)((shift + d_mod4) & (kVec - 1));
       }
     }
     __syncwarp();
@@ -372,7 +379,7 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 
     // last batch of the tile: one Horner evaluation per node of the group, coalesced stores
     const int64_t c0 = ct * kTileChunks;
-    float* out = prm.coded + (int64_t)row0 * prm.d_c + c0 + tid;
+    T* out = prm.coded + (int64_t)row0 * prm.d_c + c0 + tid;
     bool ok[CPT];
 #pragma unroll
     for (int i = 0; i < CPT; ++i) ok[i] = c0 + tid + i * kEncConsumers < prm.d_c;
@@ -389,8 +396,8 @@ __global__ void __launch_bounds__(kEncThreads, kMinBlocks) encode_direct_kernel(
 #pragma unroll
         for (int l = M - 2; l >= 0; --l) z = acc_fma<Acc>(z, wk, c[i][l]);
         if (ok[i]) {
-          if (prm.stream_hints) __stcs(out + i * kEncConsumers, (float)z);
-          else out[i * kEncConsumers] = (float)z;
+          if (prm.stream_hints) __stcs(out + i * kEncConsumers, (T)z);
+          else out[i * kEncConsumers] = (T)z;
         }
       }
       out += prm.d_c;
@@ -442,12 +449,13 @@ static int launch_encode_generic(solon_plan* plan, EncodeParams& prm) {
   return SOLON_OK;
 }
 
-template <int M, int CPT, typename Acc, int kMinBlocks>
-static int launch_encode_direct(solon_plan* plan, EncodeParams& prm) {
+template <int M, int CPT, typename Acc, int kMinBlocks, typename T>
+static int launch_encode_direct(solon_plan* plan, EncodeParamsT<T>& prm) {
   constexpr int kTileFloats = kEncConsumers * CPT * M;
+  constexpr int kVec = (int)Vec16<T>::n;
   prm.chunks_per_thread = CPT;
-  prm.slot_floats = ((kTileFloats + 3) / 4) * 4 + 8;
-  const size_t slot_bytes = (size_t)prm.slot_floats * 4;
+  prm.slot_floats = ((kTileFloats + kVec - 1) / kVec) * kVec + 2 * kVec;   // elements: room for the alignment shift and the rounded-up end
+  const size_t slot_bytes = (size_t)prm.slot_floats * sizeof(T);
   const size_t fixed = 256 + (((size_t)plan->P * sizeof(Acc) + 15) & ~(size_t)15);
   const size_t per_cta = (size_t)227 * 1024 / kMinBlocks - 1024;      // shared memory one CTA may take
   // rows per stage: about 20 KB per stage, an even split of the largest group
@@ -473,28 +481,33 @@ static int launch_encode_direct(solon_plan* plan, EncodeParams& prm) {
   if (per_sm < 1) per_sm = 1;
   const int64_t resident = (int64_t)plan->num_sms * per_sm;
   const int grid = (int)(total_tiles < resident ? total_tiles : resident);
-  auto kernel = encode_direct_kernel<M, CPT, Acc, kMinBlocks>;
+  auto kernel = encode_direct_kernel<M, CPT, Acc, kMinBlocks, T>;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kernel<<<grid, kEncThreads, smem, plan->stream>>>(prm);
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }
 
+template <typename T>
+static void fill_encode_params(solon_plan* plan, const T* grads, T* coded, EncodeParamsT<T>* prm) {
+  prm->grads = grads;
+  prm->coded = coded;
+  prm->group_start = plan->d_group_start;
+  prm->w = plan->d_w;
+  prm->q = plan->q;
+  prm->m = plan->m;
+  prm->P = plan->P;
+  prm->d = plan->d;
+  prm->d_c = plan->d_c;
+  prm->total_floats = (int64_t)plan->P * plan->d;
+  prm->status = plan->d_status;
+  prm->tile_counter = plan->d_tile_counter + 1;
+  prm->stream_hints = plan->stream_hints;
+}
+
 int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   EncodeParams prm;
-  prm.grads = grads;
-  prm.coded = coded;
-  prm.group_start = plan->d_group_start;
-  prm.w = plan->d_w;
-  prm.q = plan->q;
-  prm.m = plan->m;
-  prm.P = plan->P;
-  prm.d = plan->d;
-  prm.d_c = plan->d_c;
-  prm.total_floats = (int64_t)plan->P * plan->d;
-  prm.status = plan->d_status;
-  prm.tile_counter = plan->d_tile_counter + 1;
-  prm.stream_hints = plan->stream_hints;
+  fill_encode_params(plan, grads, coded, &prm);
   plan->launches += 1;
   switch (plan->m) {
     case 1: return launch_encode_direct<1, 4, float, 3>(plan, prm);
@@ -510,10 +523,31 @@ int launch_encode(solon_plan* plan, const float* grads, float* coded) {
   }
 }
 
+// float64 gradients (the paper's wire format, Table 2): group sums and polynomial evaluation in float64 throughout.
+// Compression ratios with a kernel of their own only (solon_float64_m_supported).
+int launch_encode_f64(solon_plan* plan, const double* grads, double* coded) {
+  EncodeParamsT<double> prm;
+  fill_encode_params(plan, grads, coded, &prm);
+  plan->launches += 1;
+  switch (plan->m) {
+    case 1: return launch_encode_direct<1, 2, double, 3>(plan, prm);
+    case 2: return launch_encode_direct<2, 2, double, 3>(plan, prm);
+    case 3: return launch_encode_direct<3, 1, double, 3>(plan, prm);
+    case 4: return launch_encode_direct<4, 1, double, 3>(plan, prm);
+    case 5: return launch_encode_direct<5, 1, double, 3>(plan, prm);
+    case 6: return launch_encode_direct<6, 1, double, 3>(plan, prm);
+    case 8: return launch_encode_direct<8, 1, double, 2>(plan, prm);
+    case 10: return launch_encode_direct<10, 1, double, 2>(plan, prm);
+    case 12: return launch_encode_direct<12, 1, double, 2>(plan, prm);
+    case 14: return launch_encode_direct<14, 1, double, 2>(plan, prm);
+    default: return SOLON_ERR_INVALID_ARG;
+  }
+}
+
 }  // namespace solon
 
 extern "C" int solon_encode(solon_plan* plan, const float* partition_grads, float* coded) {
-  if (!plan || !partition_grads || !coded) return SOLON_ERR_INVALID_ARG;
+  if (!plan || !partition_grads || !coded || plan->dtype != SOLON_F32) return SOLON_ERR_INVALID_ARG;
   if (((uintptr_t)partition_grads & 15) || ((uintptr_t)coded & 3)) return SOLON_ERR_INVALID_ARG;
   solon::TraceRange range(plan->profiling != 0, "solon_encode");
   if (plan->profiling) {
@@ -521,6 +555,22 @@ extern "C" int solon_encode(solon_plan* plan, const float* partition_grads, floa
     plan->ev_valid[0] = 1;
   }
   int rc = solon::launch_encode(plan, partition_grads, coded);
+  if (rc == SOLON_OK && plan->profiling) {
+    SOLON_CUDA_TRY(cudaEventRecord(plan->ev[1], plan->stream));
+    plan->ev_valid[1] = 1;
+  }
+  return rc;
+}
+
+extern "C" int solon_encode_f64(solon_plan* plan, const double* partition_grads, double* coded) {
+  if (!plan || !partition_grads || !coded || plan->dtype != SOLON_F64) return SOLON_ERR_INVALID_ARG;
+  if (((uintptr_t)partition_grads & 15) || ((uintptr_t)coded & 7)) return SOLON_ERR_INVALID_ARG;
+  solon::TraceRange range(plan->profiling != 0, "solon_encode");
+  if (plan->profiling) {
+    SOLON_CUDA_TRY(cudaEventRecord(plan->ev[0], plan->stream));
+    plan->ev_valid[0] = 1;
+  }
+  int rc = solon::launch_encode_f64(plan, partition_grads, coded);
   if (rc == SOLON_OK && plan->profiling) {
     SOLON_CUDA_TRY(cudaEventRecord(plan->ev[1], plan->stream));
     plan->ev_valid[1] = 1;

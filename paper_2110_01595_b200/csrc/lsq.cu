@@ -260,6 +260,7 @@ int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w,
 }  // namespace solon
 
 extern "C" int solon_lsq_grads(solon_plan* plan, const float* X, const float* y, const float* w, float* grads) {
+  if (plan && plan->dtype != SOLON_F32) return SOLON_ERR_INVALID_ARG;
   if (!plan || !X || !y || !w || !grads) return SOLON_ERR_INVALID_ARG;
   return solon::launch_lsq(plan, X, y, w, grads);
 }

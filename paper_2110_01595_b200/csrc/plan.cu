@@ -184,11 +184,21 @@ const char* solon_strerror(int status) {
   }
 }
 
+int solon_float64_m_supported(int m) { return (m >= 1 && m <= 6) || m == 8 || m == 10 || m == 12 || m == 14; }
+
 int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solon_plan** out) {
+  return solon_plan_create_ex(P, s, m, r, d, seed, SOLON_F32, out);
+}
+
+int solon_plan_dtype(const solon_plan* plan) { return plan ? plan->dtype : SOLON_ERR_INVALID_ARG; }
+
+int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, int dtype, solon_plan** out) {
   if (!out) return SOLON_ERR_INVALID_ARG;
   *out = nullptr;
+  if (dtype != SOLON_F32 && dtype != SOLON_F64) return SOLON_ERR_INVALID_ARG;
   int rc = check_params(P, s, m, r, d);
   if (rc) return rc;
+  if (dtype == SOLON_F64 && !solon_float64_m_supported(m)) return SOLON_ERR_INVALID_ARG;
   std::vector<int> start;
   group_layout(P, r, &start);
   int q = (int)start.size() - 1;
@@ -205,7 +215,8 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
   solon_plan* p = new (std::nothrow) solon_plan();
   if (!p) return SOLON_ERR_NOMEM;
   p->P = P; p->s = s; p->m = m; p->r = r; p->K = 2; p->d = d; p->d_c = (d + m - 1) / m;
-  p->seed = seed; p->tau = 1e-5; p->lsq_rows = 256; p->stream = 0; p->launches = 0;
+  p->dtype = dtype;
+  p->seed = seed; p->tau = dtype == SOLON_F64 ? 1e-10 : 1e-5; p->lsq_rows = 256; p->stream = 0; p->launches = 0;
   p->group_start = start; p->q = q; p->max_group = max_group;
   p->group_of.assign(P, 0);
   for (int g = 0; g < q; ++g)
@@ -222,7 +233,7 @@ int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solo
   p->num_sms = prop.multiProcessorCount;
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
-  p->stream_hints = keeps_l2_for_code(P, d) ? 1 : 0;
+  p->stream_hints = keeps_l2_for_code(P, dtype == SOLON_F64 ? 2 * d : d) ? 1 : 0;
   if (const char* env = getenv("SOLON_STREAM_HINTS")) p->stream_hints = env[0] == '1' ? 1 : (env[0] == '0' ? 0 : p->stream_hints);
 
   rc = SOLON_OK;

@@ -285,6 +285,25 @@ __device__ __forceinline__ void pipe_consume(const float* const* rows, const flo
   }
 }
 
+// The same for float64 rows: exact products and sums in float64 (f is widened), four independent steps in flight.
+template <int K, int NR>
+__device__ __forceinline__ void pipe_consume(const double* const* rows, const float* fs, int slot_floats, int cols, int lane,
+                                             double (*rho)[K], double* nu) {
+#pragma unroll 4
+  for (int c = lane; c < cols; c += 32) {
+    double fv[K];
+#pragma unroll
+    for (int kappa = 0; kappa < K; ++kappa) fv[kappa] = (double)fs[(size_t)kappa * slot_floats + c];
+#pragma unroll
+    for (int j = 0; j < NR; ++j) {
+      const double v = rows[j][c];
+#pragma unroll
+      for (int kappa = 0; kappa < K; ++kappa) rho[j][kappa] = fma(fv[kappa], v, rho[j][kappa]);
+      nu[j] = fma(v, v, nu[j]);
+    }
+  }
+}
+
 // Sums of one bunch of kProjBunch CTAs, added in a fixed order by the last of them to arrive (atomic ticket, nobody
 // waits).  Called by n_threads threads of the CTA that synchronise through Sync; every one of them gets the same
 // answer: whether this CTA was the one that completed the bunch.  bunch_out[i] = add_in[i] + sum over members.
@@ -327,8 +346,8 @@ __device__ __forceinline__ bool bunch_reduce(const double* __restrict__ partials
 // The CTA's column range is walked in two parts.  Part A (the first eighth or so) is summed, reduced over the
 // bunches and announced (progress[0]) on its own, so that the locator kernel can already work on a projection of
 // those columns - it is a random projection like any other - while part B streams; the final sums are A + B.
-template <int K>
-__global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_kernel(const float* __restrict__ R, const float* __restrict__ f,
+template <int K, typename T>
+__global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_kernel(const T* __restrict__ R, const float* __restrict__ f,
                                                                      int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
                                                                      ProjPipe pp, double* __restrict__ partials,
                                                                      double* __restrict__ rho_out, double* __restrict__ nu_out,
@@ -339,8 +358,10 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + kPipeStages;
   int* abort_flag = reinterpret_cast<int*>(empty_bar + kPipeStages);
-  float* ring = reinterpret_cast<float*>(smem_raw + 128);
-  const size_t stage_floats = (size_t)(pp.batch_rows + K) * pp.slot_floats;   // the rows of a batch, then f
+  constexpr int64_t kVec = 16 / sizeof(T);                    // elements per 16 bytes
+  unsigned char* ring = smem_raw + 128;
+  const size_t rows_bytes = (size_t)pp.batch_rows * pp.slot_floats * sizeof(T);
+  const size_t stage_bytes = rows_bytes + (size_t)K * pp.slot_floats * sizeof(float);   // the rows of a batch, then f
   const int n_acc = (K + 1) * P;
   pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading the final sums
   if (tid == 0) {
@@ -378,20 +399,20 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           const uint32_t phase = (it / kPipeStages) & 1;
           if (it >= (uint32_t)kPipeStages) pipe::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, pp.status + 1);
           const int64_t cols = (hi - c0) < pp.slice_cols ? (hi - c0) : pp.slice_cols;
-          float* stage_base = ring + stage * stage_floats;
+          unsigned char* stage_base = ring + stage * stage_bytes;
           uint32_t row_bytes = 0, f_bytes = 0;
-          const float* row_src = nullptr;
-          float* slot = stage_base + (size_t)lane * pp.slot_floats;
+          const T* row_src = nullptr;
+          T* slot = reinterpret_cast<T*>(stage_base) + (size_t)lane * pp.slot_floats;
           if (lane < nb) {
             const int64_t first = (int64_t)(b0 + lane) * d_c + c0;
             const int64_t last = first + cols;
-            const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
-            int64_t a1 = (last + 3) & ~(int64_t)3;
-            const int64_t safe_end = total_floats & ~(int64_t)3;      // bulk copies stay inside the matrix
+            const int64_t a0 = first & ~(kVec - 1);                   // enclosing 16-byte boundary
+            int64_t a1 = (last + kVec - 1) & ~(kVec - 1);
+            const int64_t safe_end = total_floats & ~(kVec - 1);      // bulk copies stay inside the matrix
             if (a1 > safe_end) a1 = safe_end;
-            row_bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
+            row_bytes = a1 > a0 ? (uint32_t)((a1 - a0) * sizeof(T)) : 0u;
             row_src = R + a0;
-            for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = R[e];   // <= 3 floats
+            for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = R[e];   // fewer than 16 bytes
           }
           // the first K lanes also bring the slice of f (16-byte aligned rows padded to a multiple of 4 floats)
           if (lane < K) f_bytes = (uint32_t)(((cols + 3) & ~(int64_t)3) * 4);
@@ -399,15 +420,15 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           else pipe::mbar_arrive(&full_bar[stage]);
           if (row_bytes) pipe::bulk_load_hint(slot, row_src, row_bytes, &full_bar[stage], row_policy);
           if (f_bytes)
-            pipe::bulk_load_hint(stage_base + (size_t)(pp.batch_rows + lane) * pp.slot_floats, f + (int64_t)lane * f_pitch + c0,
-                                 f_bytes, &full_bar[stage], f_policy);
+            pipe::bulk_load_hint(reinterpret_cast<float*>(stage_base + rows_bytes) + (size_t)lane * pp.slot_floats,
+                                 f + (int64_t)lane * f_pitch + c0, f_bytes, &full_bar[stage], f_policy);
         }
       }
     }
     if (*(volatile int*)abort_flag) pipe::drain_delay();
   } else {
     const int lane = tid & 31, warp = tid >> 5;
-    const int dc_mod4 = (int)(d_c & 3);
+    const int dc_mod4 = (int)(d_c & (kVec - 1));
     uint32_t it = 0;
     for (int part = pp.part_a_cols > 0 ? 0 : 1; part < 2; ++part) {
       const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
@@ -420,7 +441,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
         const int nr = warp < nb ? (nb - warp + kPipeWarps - 1) / kPipeWarps : 0;    // rows warp, warp + 8, ... below nb
         int shift[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) shift[j] = (((b0 + warp + 8 * j) & 3) * dc_mod4) & 3;   // (row * d_c + c0) mod 4
+        for (int j = 0; j < 4; ++j) shift[j] = (int)((((b0 + warp + 8 * j) & (kVec - 1)) * dc_mod4) & (kVec - 1));   // (row * d_c + c0) mod (elements per 16 bytes)
         double rho[4][K], nu[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -433,11 +454,11 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           const uint32_t phase = (it / kPipeStages) & 1;
           pipe::mbar_wait(&full_bar[stage], phase, abort_flag, pp.status + 1);
           const int cols = (int)((hi - c0) < pp.slice_cols ? (hi - c0) : pp.slice_cols);
-          const float* base = ring + stage * stage_floats;
-          const float* fs = base + (size_t)pp.batch_rows * pp.slot_floats;
-          const float* rows[4];
+          const unsigned char* base = ring + stage * stage_bytes;
+          const float* fs = reinterpret_cast<const float*>(base + rows_bytes);
+          const T* rows[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) rows[j] = base + (size_t)(warp + 8 * j) * pp.slot_floats + shift[j];
+          for (int j = 0; j < 4; ++j) rows[j] = reinterpret_cast<const T*>(base) + (size_t)(warp + 8 * j) * pp.slot_floats + shift[j];
           if (nr == 4) pipe_consume<K, 4>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 3) pipe_consume<K, 3>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
@@ -489,8 +510,8 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   if (tid == 0) *ticket = 0u;
 }
 
-template <int K>
-static int launch_project_pipe_k(solon_plan* plan, const float* received, double* rho_out, double* nu_out, int final_reduce) {
+template <int K, typename T>
+static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rho_out, double* nu_out, int final_reduce) {
   ProjPipe pp;
   pp.status = plan->d_status;
   pp.progress = plan->d_proj_progress;
@@ -498,7 +519,7 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128;
   const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
   pp.batch_rows = (plan->P + n_batches - 1) / n_batches;
-  int slice = (int)(per_cta / ((size_t)kPipeStages * (pp.batch_rows + K) * 4)) - 8;
+  int slice = (int)(per_cta / ((size_t)kPipeStages * (pp.batch_rows * sizeof(T) + K * sizeof(float)))) - 8;
   slice = slice / 32 * 32;
   if (slice > 2048) slice = 2048;
   int grid = plan->num_sms * kPipeCtasPerSm;
@@ -516,9 +537,9 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   if (a_slices < 1) a_slices = 1;
   const bool two_parts = !final_reduce && uses_early_locator(plan) && !early_locator_starved(plan);
   pp.part_a_cols = two_parts ? a_slices * slice : 0;
-  const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows + K) * pp.slot_floats * sizeof(float);
-  SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  project_pipe_kernel<K><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->f_pitch, plan->P, plan->d_c,
+  const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows * sizeof(T) + K * sizeof(float)) * pp.slot_floats;
+  SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  project_pipe_kernel<K, T><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->f_pitch, plan->P, plan->d_c,
                                                                      range_len, pp, plan->d_partials, rho_out, nu_out,
                                                                      plan->d_proj_ticket, final_reduce);
   const int n_bunches = (grid + kProjBunch - 1) / kProjBunch;
@@ -532,19 +553,27 @@ static int launch_project_pipe_k(solon_plan* plan, const float* received, double
   return SOLON_OK;
 }
 
-int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
+template <typename T>
+static int launch_project_t(solon_plan* plan, const T* received, double* rho_out, double* nu_out) {
   // no output buffers: the decode proper, whose locator kernel adds the last level of partial sums itself
   const int final_reduce = (rho_out || nu_out) ? 1 : 0;
   if (!rho_out) rho_out = plan->d_rho;
   if (!nu_out) nu_out = plan->d_nu;
   plan->launches += 1;
   switch (plan->K) {
-    case 1: return launch_project_pipe_k<1>(plan, received, rho_out, nu_out, final_reduce);
-    case 2: return launch_project_pipe_k<2>(plan, received, rho_out, nu_out, final_reduce);
-    case 3: return launch_project_pipe_k<3>(plan, received, rho_out, nu_out, final_reduce);
-    case 4: return launch_project_pipe_k<4>(plan, received, rho_out, nu_out, final_reduce);
+    case 1: return launch_project_pipe_k<1, T>(plan, received, rho_out, nu_out, final_reduce);
+    case 2: return launch_project_pipe_k<2, T>(plan, received, rho_out, nu_out, final_reduce);
+    case 3: return launch_project_pipe_k<3, T>(plan, received, rho_out, nu_out, final_reduce);
+    case 4: return launch_project_pipe_k<4, T>(plan, received, rho_out, nu_out, final_reduce);
     default: return SOLON_ERR_INVALID_ARG;
   }
+}
+
+int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
+  return launch_project_t<float>(plan, received, rho_out, nu_out);
+}
+int launch_project_f64(solon_plan* plan, const double* received, double* rho_out, double* nu_out) {
+  return launch_project_t<double>(plan, received, rho_out, nu_out);
 }
 
 // ---- projections without any allocation ------------------------------------------------------------

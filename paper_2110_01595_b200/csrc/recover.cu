@@ -13,9 +13,10 @@ namespace solon {
 
 constexpr int kRecThreads = 256;
 
-struct RecoverParams {
-  const float* R;
-  float* agg;
+template <typename T>
+struct RecoverParamsT {
+  const T* R;
+  T* agg;
   int64_t d, d_c;
   int q, m, P;
   const int* group_start;
@@ -24,10 +25,11 @@ struct RecoverParams {
   const double* coeff;   // P x m, same indexing
   unsigned long long* proj_progress;   // the projection kernel's part-A count, zeroed here for the next decode
 };
+typedef RecoverParamsT<float> RecoverParams;
 
 // Copy the locator's tables (group layout, rows per group, row indices, weights) into shared memory.
-template <typename Acc>
-__device__ __forceinline__ void load_tables(const RecoverParams& prm, Acc* coeff_s, int* rows_s, int* start_s,
+template <typename Acc, typename Prm>
+__device__ __forceinline__ void load_tables(const Prm& prm, Acc* coeff_s, int* rows_s, int* start_s,
                                             int* n_rec_s) {
   for (int i = threadIdx.x; i < prm.P * prm.m; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
   for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
@@ -42,8 +44,8 @@ __device__ __forceinline__ void load_tables(const RecoverParams& prm, Acc* coeff
 // weights at coeff_c[i * STRIDE .. + M) (STRIDE: M rounded up so that every row of weights starts on a 16-byte
 // boundary and can be fetched with 128-bit loads).  Returns the number of rows in use.
 // coeff_s (P x M), rows_s, slots_s (P each), start_s (q + 1), n_rec_s (q): staging.
-template <typename Acc, int M, int STRIDE>
-__device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_s, Acc* coeff_s, int* slots_s, int* start_s,
+template <typename Acc, int M, int STRIDE, int VEC, typename Prm>
+__device__ __forceinline__ int pack_tables(const Prm& prm, int* rows_s, Acc* coeff_s, int* slots_s, int* start_s,
                                            int* n_rec_s, int* count_s, Acc* coeff_c, int* rowsh_c) {
   for (int i = threadIdx.x; i < prm.P * M; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
   for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
@@ -60,10 +62,10 @@ __device__ __forceinline__ int pack_tables(const RecoverParams& prm, int* rows_s
   }
   __syncthreads();
   const int n_rows = *count_s;
-  const int dc_mod4 = (int)(prm.d_c & 3);
+  const int dc_mod4 = (int)(prm.d_c & (VEC - 1));       // VEC: elements per 16 bytes
   for (int i = threadIdx.x; i < n_rows; i += blockDim.x) {
     const int row = rows_s[slots_s[i]];
-    rowsh_c[i] = (row << 2) | (((row & 3) * dc_mod4) & 3);
+    rowsh_c[i] = (row << 2) | (((row & (VEC - 1)) * dc_mod4) & (VEC - 1));
   }
   for (int i = threadIdx.x; i < n_rows * STRIDE; i += blockDim.x) {
     const int r = i / STRIDE, l = i - r * STRIDE;
@@ -116,10 +118,11 @@ struct RecoverPipe {
 // shared-memory ring with bulk asynchronous copies; consumer threads own CPT chunks each, take one float per
 // row from the ring, apply the row's m weights, and every consumer warp writes its runs of chunks back
 // through its own shared buffer as contiguous 128-bit stores.
-template <int M, int CPT, typename Acc, int NC, int kCtasPerSm>
-__global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverParams prm, RecoverPipe pp) {
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T>
+__global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverParamsT<T> prm, RecoverPipe pp) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int kTileChunks = NC * CPT;
+  constexpr int64_t kVec = 16 / sizeof(T);     // elements per 16 bytes
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + pp.stages;
@@ -136,8 +139,8 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
   int* rowsh_c = slots_p + ((prm.P + 3) & ~3);                                            // P (packed)
   int* start_s = rowsh_c + ((prm.P + 3) & ~3);                                            // q + 1
   int* n_rec_s = start_s + ((prm.q + 4) & ~3);                                            // q
-  float* out_all = reinterpret_cast<float*>(n_rec_s + ((prm.q + 3) & ~3));                // 8 warps x 32 x M
-  float* ring = out_all + (size_t)(NC / 32) * 32 * M;                          // 32 M floats: 128 M bytes
+  T* out_all = reinterpret_cast<T*>(n_rec_s + ((prm.q + 3) & ~3));                        // one buffer of 32 x M per consumer warp
+  T* ring = out_all + (size_t)(NC / 32) * 32 * M;                              // 32 M elements: a multiple of 16 bytes
   const size_t stage_floats = (size_t)pp.row_batch * pp.slot_floats;
 
   if (tid == 0) {
@@ -153,7 +156,7 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
     prm.proj_progress[0] = 0ULL;
     prm.proj_progress[1] = 0ULL;
   }
-  const int n_rows = pack_tables<Acc, M, kStride>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c);
+  const int n_rows = pack_tables<Acc, M, kStride, (int)kVec>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
 
@@ -185,13 +188,13 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
         if (lane < nb) {
           const int64_t first = (int64_t)(rowsh_c[b0 + lane] >> 2) * prm.d_c + c0;
           const int64_t last = first + (c1 - c0);
-          const int64_t a0 = first & ~(int64_t)3;                   // enclosing 16-byte boundary
-          int64_t a1 = (last + 3) & ~(int64_t)3;
-          const int64_t safe_end = total_floats & ~(int64_t)3;      // bulk copies stay inside the matrix
+          const int64_t a0 = first & ~(kVec - 1);                   // enclosing 16-byte boundary
+          int64_t a1 = (last + kVec - 1) & ~(kVec - 1);
+          const int64_t safe_end = total_floats & ~(kVec - 1);      // bulk copies stay inside the matrix
           if (a1 > safe_end) a1 = safe_end;
-          float* slot = ring + stage * stage_floats + (size_t)lane * pp.slot_floats;
-          const uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * 4) : 0u;
-          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.R[e];   // <= 3 floats
+          T* slot = ring + stage * stage_floats + (size_t)lane * pp.slot_floats;
+          const uint32_t bytes = a1 > a0 ? (uint32_t)((a1 - a0) * sizeof(T)) : 0u;
+          for (int64_t e = (a1 > a0 ? a1 : a0); e < last; ++e) slot[e - a0] = prm.R[e];   // fewer than 16 bytes
           if (bytes) {
             pipe::mbar_arrive_expect_tx(&full_bar[stage], bytes);
             pipe::bulk_load_hint(slot, prm.R + a0, bytes, &full_bar[stage], stream_policy);
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
   }
 
   const int lane = tid & 31, warp = tid >> 5;
-  float* out_s = out_all + (size_t)warp * 32 * M;
+  T* out_s = out_all + (size_t)warp * 32 * M;
   Acc acc[CPT][M];
   for (uint32_t it = 0;; ++it) {
     const int stage = it % pp.stages;
@@ -239,12 +242,12 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
     // Chunks past the end of the matrix (last tile only) read whatever an earlier tile left in the ring: finite
     // values, whose sums are never written back.
     const int nb = min(pp.row_batch, n_rows - b0);
-    const float* slot = ring + stage * stage_floats + tid;
+    const T* slot = ring + stage * stage_floats + tid;
     const int* rs = rowsh_c + b0;
     const Acc* cj = coeff_c + (size_t)b0 * kStride;
 #pragma unroll(sizeof(Acc) == 8 ? 1 : 2)
     for (int j = 0; j < nb; ++j) {
-      const float* src = slot + (rs[j] & 3);
+      const T* src = slot + (rs[j] & 3);
       Acc v[CPT];
 #pragma unroll
       for (int i = 0; i < CPT; ++i) v[i] = (Acc)src[i * NC];
@@ -266,21 +269,21 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
 #pragma unroll
     for (int i = 0; i < CPT; ++i) {
 #pragma unroll
-      for (int l = 0; l < M; ++l) out_s[lane * M + l] = (float)acc[i][l];
+      for (int l = 0; l < M; ++l) out_s[lane * M + l] = (T)acc[i][l];
       __syncwarp();
       const int64_t o0 = (c0 + (int64_t)i * NC + warp * 32) * M;
       int64_t o1 = o0 + 32 * M;
       if (o1 > prm.d) o1 = prm.d;
       const int count = o1 > o0 ? (int)(o1 - o0) : 0;
-      const int vec = count / 4;
+      const int vec = count / (int)kVec;                          // whole 16-byte words
       float4* dst4 = reinterpret_cast<float4*>(prm.agg + o0);
       const float4* src4 = reinterpret_cast<const float4*>(out_s);
       if (pp.stream_hints) {
         for (int e = lane; e < vec; e += 32) __stcs(dst4 + e, src4[e]);
-        for (int e = vec * 4 + lane; e < count; e += 32) __stcs(prm.agg + o0 + e, out_s[e]);
+        for (int e = vec * (int)kVec + lane; e < count; e += 32) __stcs(prm.agg + o0 + e, out_s[e]);
       } else {
         for (int e = lane; e < vec; e += 32) dst4[e] = src4[e];
-        for (int e = vec * 4 + lane; e < count; e += 32) prm.agg[o0 + e] = out_s[e];
+        for (int e = vec * (int)kVec + lane; e < count; e += 32) prm.agg[o0 + e] = out_s[e];
       }
       __syncwarp();
     }
@@ -312,18 +315,18 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   }
 }
 
-template <int M, int CPT, typename Acc, int NC, int kCtasPerSm>
-static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T>
+static int launch_recover_m(solon_plan* plan, RecoverParamsT<T>& prm) {
   constexpr int kTileChunks = NC * CPT;
   RecoverPipe pp;
   pp.status = plan->d_status;
   pp.stream_hints = plan->stream_hints;
   pp.slot_floats = kTileChunks + 8;
-  const size_t slot_bytes = (size_t)pp.slot_floats * 4;
+  const size_t slot_bytes = (size_t)pp.slot_floats * sizeof(T);
   const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + recover_coeff_bytes(plan->P, PackedStride<Acc, M>::value) +
                        3 * (size_t)((plan->P + 3) & ~3) * sizeof(int) +
                        (size_t)(((plan->q + 4) & ~3) + ((plan->q + 3) & ~3)) * sizeof(int) +
-                       (size_t)(NC / 32) * 32 * M * sizeof(float);
+                       (size_t)(NC / 32) * 32 * M * sizeof(T);
   // the locator may select up to all P rows (large m) or as few as q m; batches of about 20 KB (40 KB when one
   // CTA has the SM's shared memory to itself)
   int row_batch = (int)((size_t)(kCtasPerSm == 1 ? 40 : 20) * 1024 / slot_bytes);
@@ -349,9 +352,9 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   if (smem > (size_t)226 * 1024) return SOLON_ERR_INVALID_ARG;
   pp.row_batch = row_batch;
   pp.stages = stages;
-  auto kernel = recover_kernel<M, CPT, Acc, NC, kCtasPerSm>;
+  auto kernel = recover_kernel<M, CPT, Acc, NC, kCtasPerSm, T>;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  static_assert((32 * M * 4) % 16 == 0, "warp runs must start on a 16-byte boundary of the output");
+  static_assert((32 * M * sizeof(T)) % 16 == 0, "warp runs must start on a 16-byte boundary of the output");
   int64_t tiles = (plan->d_c + kTileChunks - 1) / kTileChunks;
   int per_sm = 1;
   SOLON_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (NC + 32), smem));
@@ -362,20 +365,45 @@ static int launch_recover_m(solon_plan* plan, RecoverParams& prm) {
   return launch_dependent(kernel, dim3(grid), dim3((NC + 32)), smem, plan->stream, prm, pp);
 }
 
+template <typename T>
+static void fill_recover_params(solon_plan* plan, const T* received, T* agg, RecoverParamsT<T>* prm) {
+  prm->R = received;
+  prm->agg = agg;
+  prm->d = plan->d;
+  prm->d_c = plan->d_c;
+  prm->q = plan->q;
+  prm->m = plan->m;
+  prm->P = plan->P;
+  prm->group_start = plan->d_group_start;
+  prm->n_rec = plan->d_n_rec;
+  prm->rec_rows = plan->d_rec_rows;
+  prm->coeff = plan->d_coeff;
+  prm->proj_progress = plan->d_proj_progress;
+}
+
+// float64 received vectors and aggregate: weights and sums in float64 for every compression ratio.
+int launch_recover_f64(solon_plan* plan, const double* received, double* agg) {
+  RecoverParamsT<double> prm;
+  fill_recover_params(plan, received, agg, &prm);
+  plan->launches += 1;
+  switch (plan->m) {
+    case 1: return launch_recover_m<1, 4, double, kRecConsumers, 2>(plan, prm);
+    case 2: return launch_recover_m<2, 4, double, kRecConsumers, 2>(plan, prm);
+    case 3: return launch_recover_m<3, 4, double, kRecConsumers, 2>(plan, prm);
+    case 4: return launch_recover_m<4, 2, double, kRecConsumers, 2>(plan, prm);
+    case 5: return launch_recover_m<5, 2, double, kRecConsumers, 2>(plan, prm);
+    case 6: return launch_recover_m<6, 2, double, kRecConsumers, 2>(plan, prm);
+    case 8: return launch_recover_m<8, 4, double, 480, 1>(plan, prm);
+    case 10: return launch_recover_m<10, 4, double, 480, 1>(plan, prm);
+    case 12: return launch_recover_m<12, 2, double, 480, 1>(plan, prm);
+    case 14: return launch_recover_m<14, 2, double, 480, 1>(plan, prm);
+    default: return SOLON_ERR_INVALID_ARG;
+  }
+}
+
 int launch_recover(solon_plan* plan, const float* received, float* agg) {
   RecoverParams prm;
-  prm.R = received;
-  prm.agg = agg;
-  prm.d = plan->d;
-  prm.d_c = plan->d_c;
-  prm.q = plan->q;
-  prm.m = plan->m;
-  prm.P = plan->P;
-  prm.group_start = plan->d_group_start;
-  prm.n_rec = plan->d_n_rec;
-  prm.rec_rows = plan->d_rec_rows;
-  prm.coeff = plan->d_coeff;
-  prm.proj_progress = plan->d_proj_progress;
+  fill_recover_params(plan, received, agg, &prm);
   plan->launches += 1;
 #define SOLON_RECOVER_CASE(M_, CPT_, ACC_, NC_, BLOCKS_) \
   case M_:                                               \

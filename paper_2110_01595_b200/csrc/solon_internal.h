@@ -38,6 +38,7 @@ enum : int {
 
 struct solon_plan {
   int P, s, m, r, K;
+  int dtype;               // SOLON_F32 or SOLON_F64: element type of gradients, coded vectors and aggregate
   int64_t d, d_c;
   uint64_t seed;
   double tau;
@@ -184,10 +185,13 @@ inline bool keeps_l2_for_code(int P, int64_t d) { return (double)P * (double)d *
 
 int launch_fill_projection(solon_plan* plan);
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
+int launch_encode_f64(solon_plan* plan, const double* grads, double* coded);
 // rho_out / nu_out (and rho / nu below): device buffers, or nullptr for the plan's own
 int launch_project(solon_plan* plan, const float* received, double* rho_out = nullptr, double* nu_out = nullptr);
+int launch_project_f64(solon_plan* plan, const double* received, double* rho_out = nullptr, double* nu_out = nullptr);
 int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho = nullptr, const double* nu = nullptr);
 int launch_recover(solon_plan* plan, const float* received, float* agg);
+int launch_recover_f64(solon_plan* plan, const double* received, double* agg);
 int launch_lsq(solon_plan* plan, const float* X, const float* y, const float* w, float* grads);
 
 // Doubles of workspace one locator CTA needs for a group of n nodes.
