@@ -97,7 +97,8 @@ const char* solon_strerror(int status);
 /* Build the mechanism (A, E, D) of Section 3.4 for P nodes, s adversaries per group,
  * compression ratio m, minimum group size r (>= 2 s + m) and gradient length d: group layout,
  * node scalars, K = 2 projection vectors f_kappa[p] = 1 + N(0,1) drawn on the device from
- * `seed` (f ~ N(1, I) in Section 3.4), and all device workspace.  Uses the current CUDA device.
+ * `seed` (f ~ N(1, I) in Section 3.4; redrawn by every decode, see solon_plan_set_fresh_projections),
+ * and all device workspace.  Uses the current CUDA device.
  * Synchronises the device once.  *out receives the plan, to be released by solon_plan_destroy. */
 int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solon_plan** out);
 int solon_plan_destroy(solon_plan* plan);
@@ -121,9 +122,21 @@ int solon_plan_set_stream(solon_plan* plan, void* cuda_stream);
  * single f).  All projections share one error-locator polynomial.  Redraws f; synchronises. */
 int solon_plan_set_num_projections(solon_plan* plan, int K);
 
-/* Redraw the projection vectors from a new seed (the paper draws a fresh f for every decode).
+/* Restart the sequence of draws from a new seed: the vectors in memory become draw 0 of that seed.
  * Enqueued on the plan's stream. */
 int solon_plan_reseed(solon_plan* plan, uint64_t seed);
+
+/* Algorithm 1 draws its random vector inside the decoder, and the proof that every corrupt node is located with
+ * probability 1 (Lemma 3) needs f independent of what the adversary sent.  on = 1 (default): every decode projects
+ * with vectors no earlier decode used - draw n of the plan's seed, n counted on the device, so that a replayed CUDA
+ * graph of a decode moves on as well.  The next decode's vectors are written, into a second buffer, by spare CTAs of
+ * the locator kernel (solon_decode, solon_decode_finish) while the locator's few CTAs work and the rest of the GPU is
+ * idle: no kernel is added and, unless K d_c is large against the locator's time, no time.  They are drawn before
+ * the adversary's next vectors exist and stay on the device.  on = 0: the vectors in memory are reused by every decode
+ * until solon_plan_reseed; that is only sound against an adversary that can neither read nor infer them, since
+ * one that knows f can send a deviation orthogonal to all K vectors and stay unseen.
+ * solon_plan_get_projection_vectors returns the vectors the most recent decode used. */
+int solon_plan_set_fresh_projections(solon_plan* plan, int on);
 
 /* tau of the floating-point "!=" test of the locator: node k is inconsistent with a fitted
  * polynomial Q when |rho_k - Q(w_k)| > tau * sqrt(2 * median_k nu_k).  Default 1e-5, about

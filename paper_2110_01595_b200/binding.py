@@ -42,6 +42,7 @@ SIGNATURES = {
     "solon_plan_set_stream": (c_int, [c_void_p, c_void_p]),
     "solon_plan_set_num_projections": (c_int, [c_void_p, c_int]),
     "solon_plan_reseed": (c_int, [c_void_p, c_uint64]),
+    "solon_plan_set_fresh_projections": (c_int, [c_void_p, c_int]),
     "solon_plan_set_tolerance": (c_int, [c_void_p, c_double]),
     "solon_plan_set_early_locator": (c_int, [c_void_p, c_int]),
     "solon_plan_set_lsq_rows": (c_int, [c_void_p, c_int]),
@@ -221,6 +222,10 @@ class Plan:
 
     def reseed(self, seed: int) -> None:
         _check(lib().solon_plan_reseed(self._h, seed), "solon_plan_reseed")
+
+    def set_fresh_projections(self, on: bool) -> None:
+        """True (default): every decode draws new projection vectors first; False: the ones in memory are reused."""
+        _check(lib().solon_plan_set_fresh_projections(self._h, 1 if on else 0), "solon_plan_set_fresh_projections")
 
     def set_tolerance(self, tau: float) -> None:
         _check(lib().solon_plan_set_tolerance(self._h, tau), "solon_plan_set_tolerance")

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "locate_core.cuh"
+#include "projection_draw.cuh"
 #include "solon_internal.h"
 
 namespace solon {
@@ -51,7 +52,11 @@ struct LocateParams {
   int* rec_rows;         // P
   double* coeff;         // P x m
   int* status;
+  DrawParams draw;       // the vectors f of the next decode, written by the CTAs beyond the q locator CTAs (n_draw_ctas of them)
+  int n_draw_ctas;
 };
+
+DrawParams draw_params(const solon_plan* plan);   // plan.cu
 
 // Workspace of one group, shared by the device kernel and the host mirror.
 struct GroupScratch {
@@ -126,6 +131,15 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   extern __shared__ __align__(16) double smem_ws[];
   const int g = blockIdx.x;
   const int tid = threadIdx.x, n_threads = blockDim.x;
+  if (g >= (int)gridDim.x - prm.n_draw_ctas) {
+    // Not a locator CTA: these draw the vectors f of the NEXT decode (Algorithm 1 draws its random vector anew in every
+    // decode) into the buffer the projection kernel just before this one did not read, while the locator's few CTAs
+    // work and the rest of the GPU would be idle.  The projection kernel must be done with the draw count first.
+    pdl_trigger();
+    pdl_wait();
+    draw_projection_vectors(prm.draw, 1, g - ((int)gridDim.x - prm.n_draw_ctas), prm.n_draw_ctas, tid, n_threads);
+    return;
+  }
   const int row0 = prm.group_start[g];
   const int n = prm.group_start[g + 1] - row0;
   double* ws = prm.use_smem ? smem_ws : prm.ws_global + (size_t)g * prm.ws_stride;
@@ -493,11 +507,21 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   }
   if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  // CTAs that draw the next decode's vectors beside the locator's: a few per SM, a thread per several quads
+  prm.draw = draw_params(plan);
+  prm.n_draw_ctas = 0;
+  if (plan->fresh_f && plan->s > 0) {
+    const int64_t quads = ((plan->d_c + 3) / 4) * plan->K;
+    int64_t want = (quads + 127) / 128;
+    const int64_t cap = (int64_t)plan->num_sms * 8;      // more CTAs per SM than eight bought nothing
+    prm.n_draw_ctas = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+  }
+  plan->last_decode_advanced = prm.n_draw_ctas > 0 ? 1 : 0;
   plan->launches += 1;
   // one warp per error count, at least four for the CTA-wide steps (four still fit, at 128 registers a thread, in the
   // slot the projection kernel leaves free, so the CTA is resident early)
   const int warps = plan->s + 1 < 4 ? 4 : plan->s + 1;
-  return launch_dependent(locate_kernel, dim3(plan->q), dim3(32 * warps), smem, plan->stream, prm);
+  return launch_dependent(locate_kernel, dim3(plan->q + prm.n_draw_ctas), dim3(32 * warps), smem, plan->stream, prm);
 }
 
 }  // namespace solon

@@ -9,6 +9,7 @@
 #include "locate_core.cuh"
 #include <vector>
 
+#include "projection_draw.cuh"
 #include "solon_internal.h"
 
 namespace solon {
@@ -48,56 +49,32 @@ void node_scalars(const std::vector<int>& start, std::vector<double>* w) {
   }
 }
 
-// ---- projection vectors: f[kappa][p] = 1 + N(0,1), Philox4x32-10 counters + Box-Muller -------------
+// ---- projection vectors: see projection_draw.cuh ------------------------------------------------------
 
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
-                                              uint32_t k1, uint32_t out[4]) {
-  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
-#pragma unroll
-  for (int round = 0; round < 10; ++round) {
-    uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-    uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-    uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
-    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
-    k0 += W0;
-    k1 += W1;
-  }
-  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+__global__ void __launch_bounds__(256) fill_projection_kernel(DrawParams dp, int advance) {
+  draw_projection_vectors(dp, advance, blockIdx.x, gridDim.x, threadIdx.x, blockDim.x);
 }
 
-__global__ void fill_projection_kernel(float* __restrict__ f, int64_t d_c, int64_t pitch, int K, uint64_t seed) {
-  int64_t quads = (d_c + 3) / 4;
-  int64_t total = quads * K;
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    int kappa = (int)(i / quads);
-    int64_t quad = i - (int64_t)kappa * quads;
-    uint32_t x[4];
-    philox4x32_10((uint32_t)quad, (uint32_t)(quad >> 32), (uint32_t)kappa, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
-    float v[4];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      float u1 = ((float)x[2 * h] + 0.5f) * 2.3283064365386963e-10f;       // (0, 1]
-      float u2 = ((float)x[2 * h + 1] + 0.5f) * 2.3283064365386963e-10f;
-      u1 = fminf(fmaxf(u1, 1.0e-12f), 1.0f);
-      float rad = sqrtf(-2.0f * logf(u1));
-      float sn, cs;
-      sincospif(2.0f * u2, &sn, &cs);
-      v[2 * h] = 1.0f + rad * cs;
-      v[2 * h + 1] = 1.0f + rad * sn;
-    }
-    float* row = f + (int64_t)kappa * pitch + quad * 4;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) row[e] = (quad * 4 + e < d_c) ? v[e] : 0.0f;   // pitch is a multiple of 4
-  }
+DrawParams draw_params(const solon_plan* plan) {
+  DrawParams dp;
+  dp.f[0] = plan->d_f;
+  dp.f[1] = plan->d_f2;
+  dp.d_c = plan->d_c;
+  dp.pitch = plan->f_pitch;
+  dp.K = plan->K;
+  dp.seed = plan->seed;
+  dp.draw = plan->d_draw;
+  return dp;
 }
 
-int launch_fill_projection(solon_plan* plan) {
+int launch_fill_projection(solon_plan* plan, int advance) {
   int64_t total = ((plan->d_c + 3) / 4) * plan->K;
   int threads = 256;
   int64_t want = (total + threads - 1) / threads;
   int blocks = (int)(want < (int64_t)plan->num_sms * 8 ? (want < 1 ? 1 : want) : (int64_t)plan->num_sms * 8);
-  fill_projection_kernel<<<blocks, threads, 0, plan->stream>>>(plan->d_f, plan->d_c, plan->f_pitch, plan->K, plan->seed);
+  fill_projection_kernel<<<blocks, threads, 0, plan->stream>>>(draw_params(plan), advance);
   plan->launches += 1;
+  plan->last_decode_advanced = 0;
   SOLON_CUDA_TRY(cudaGetLastError());
   return SOLON_OK;
 }
@@ -115,12 +92,12 @@ static int dev_alloc(T** ptr, size_t count) {
 }
 
 static void free_device(solon_plan* p) {
-  cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f);
+  cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f); cudaFree(p->d_f2);
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_tab_count); cudaFree(p->d_tab_rows); cudaFree(p->d_tab_coeff); cudaFree(p->d_tab_off); cudaFree(p->d_tab_sets);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_locate_ws);
-  cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress);
+  cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress); cudaFree(p->d_draw);
   cudaFree(p->d_resid);
   for (int i = 0; i < 6; ++i)
     if (p->ev[i]) cudaEventDestroy(p->ev[i]);
@@ -130,11 +107,13 @@ static void free_device(solon_plan* p) {
 
 static int alloc_projection(solon_plan* p) {
   int rc;
-  cudaFree(p->d_f); cudaFree(p->d_partials); cudaFree(p->d_rho);
+  cudaFree(p->d_f); cudaFree(p->d_f2); cudaFree(p->d_partials); cudaFree(p->d_rho);
   cudaFree(p->d_locate_ws);
   (void)cudaGetLastError();
+  p->d_f2 = nullptr;
   p->d_f = nullptr; p->d_partials = nullptr; p->d_rho = nullptr; p->d_locate_ws = nullptr;
   if ((rc = dev_alloc(&p->d_f, (size_t)p->K * p->f_pitch))) return rc;
+  if ((rc = dev_alloc(&p->d_f2, (size_t)p->K * p->f_pitch))) return rc;
   // per-CTA partial sums of the two parts of every column range, then the per-bunch sums of part A and of the whole
   if ((rc = dev_alloc(&p->d_partials, 2 * (size_t)(p->proj_grid + p->proj_grid / 16 + 1) * (p->K + 1) * p->P))) return rc;
   if ((rc = dev_alloc(&p->d_rho, (size_t)p->K * p->P))) return rc;
@@ -233,6 +212,7 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
   p->num_sms = prop.multiProcessorCount;
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
+  p->fresh_f = 1;
   p->stream_hints = keeps_l2_for_code(P, dtype == SOLON_F64 ? 2 * d : d) ? 1 : 0;
   if (const char* env = getenv("SOLON_STREAM_HINTS")) p->stream_hints = env[0] == '1' ? 1 : (env[0] == '0' ? 0 : p->stream_hints);
 
@@ -315,6 +295,7 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
     if ((rc = dev_alloc(&p->d_tile_counter, 4))) break;
     if ((rc = dev_alloc(&p->d_early, (size_t)q))) break;
     if ((rc = dev_alloc(&p->d_proj_progress, 2))) break;
+    if ((rc = dev_alloc(&p->d_draw, 2))) break;
     cudaError_t e = cudaSuccess;
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_start, start.data(), (q + 1) * sizeof(int), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_group_of, p->group_of.data(), P * sizeof(int), cudaMemcpyHostToDevice);
@@ -324,10 +305,11 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
     if (e == cudaSuccess) e = cudaMemset(p->d_tile_counter, 0, 4 * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(p->d_early, 0, q * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_proj_progress, 0, 2 * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(p->d_draw, 0, 2 * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(p->d_n_rec, 0, q * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_t_acc, 0, q * sizeof(int));
     if (e != cudaSuccess) { (void)cudaGetLastError(); rc = SOLON_ERR_CUDA; break; }
-    if ((rc = launch_fill_projection(p))) break;
+    if ((rc = launch_fill_projection(p, 0))) break;
     if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); rc = SOLON_ERR_CUDA; break; }
   } while (0);
   if (rc) {
@@ -359,7 +341,8 @@ int solon_plan_set_num_projections(solon_plan* plan, int K) {
   plan->K = K;
   int rc = alloc_projection(plan);
   if (rc) return rc;
-  if ((rc = launch_fill_projection(plan))) return rc;
+  SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_draw, 0, 2 * sizeof(unsigned long long), plan->stream));
+  if ((rc = launch_fill_projection(plan, 0))) return rc;
   SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
   return SOLON_OK;
 }
@@ -367,7 +350,14 @@ int solon_plan_set_num_projections(solon_plan* plan, int K) {
 int solon_plan_reseed(solon_plan* plan, uint64_t seed) {
   if (!plan) return SOLON_ERR_INVALID_ARG;
   plan->seed = seed;
-  return launch_fill_projection(plan);
+  SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_draw, 0, 2 * sizeof(unsigned long long), plan->stream));   // draw 0 of the new seed
+  return launch_fill_projection(plan, 0);
+}
+
+int solon_plan_set_fresh_projections(solon_plan* plan, int on) {
+  if (!plan) return SOLON_ERR_INVALID_ARG;
+  plan->fresh_f = on ? 1 : 0;
+  return SOLON_OK;
 }
 
 int solon_plan_set_early_locator(solon_plan* plan, int mode) {
@@ -417,7 +407,13 @@ int solon_plan_get_node_scalars(const solon_plan* plan, double* w) {
 }
 int solon_plan_get_projection_vectors(solon_plan* plan, float* f) {
   if (!plan || !f) return SOLON_ERR_INVALID_ARG;
-  SOLON_CUDA_TRY(cudaMemcpy2DAsync(f, plan->d_c * sizeof(float), plan->d_f, plan->f_pitch * sizeof(float),
+  // draw n lives in buffer n & 1; a decode that drew anew has already advanced the count past the draw it used
+  unsigned long long n = 0;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(&n, plan->d_draw, sizeof(n), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  if (plan->last_decode_advanced && n > 0) n -= 1;
+  const float* src = (n & 1ULL) ? plan->d_f2 : plan->d_f;
+  SOLON_CUDA_TRY(cudaMemcpy2DAsync(f, plan->d_c * sizeof(float), src, plan->f_pitch * sizeof(float),
                                    plan->d_c * sizeof(float), plan->K, cudaMemcpyDeviceToHost, plan->stream));
   SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
   return SOLON_OK;

@@ -347,7 +347,9 @@ __device__ __forceinline__ bool bunch_reduce(const double* __restrict__ partials
 // bunches and announced (progress[0]) on its own, so that the locator kernel can already work on a projection of
 // those columns - it is a random projection like any other - while part B streams; the final sums are A + B.
 template <int K, typename T>
-__global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_kernel(const T* __restrict__ R, const float* __restrict__ f,
+__global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_kernel(const T* __restrict__ R, const float* __restrict__ f_even,
+                                                                     const float* __restrict__ f_odd,
+                                                                     const unsigned long long* __restrict__ draw,
                                                                      int64_t f_pitch, int P, int64_t d_c, int64_t range_len,
                                                                      ProjPipe pp, double* __restrict__ partials,
                                                                      double* __restrict__ rho_out, double* __restrict__ nu_out,
@@ -364,6 +366,8 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   const size_t stage_bytes = rows_bytes + (size_t)K * pp.slot_floats * sizeof(float);   // the rows of a batch, then f
   const int n_acc = (K + 1) * P;
   pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading the final sums
+  // the vectors of draw n live in the buffer n & 1; the count moves on only after this kernel has completed
+  const float* __restrict__ f = (draw[0] & 1ULL) ? f_odd : f_even;
   if (tid == 0) {
     for (int s = 0; s < kPipeStages; ++s) {
       pipe::mbar_init(&full_bar[s], 32);
@@ -539,7 +543,7 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   pp.part_a_cols = two_parts ? a_slices * slice : 0;
   const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows * sizeof(T) + K * sizeof(float)) * pp.slot_floats;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  project_pipe_kernel<K, T><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->f_pitch, plan->P, plan->d_c,
+  project_pipe_kernel<K, T><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->d_f2, plan->d_draw, plan->f_pitch, plan->P, plan->d_c,
                                                                      range_len, pp, plan->d_partials, rho_out, nu_out,
                                                                      plan->d_proj_ticket, final_reduce);
   const int n_bunches = (grid + kProjBunch - 1) / kProjBunch;

@@ -71,8 +71,12 @@ struct solon_plan {
   int64_t* d_tab_off;      // q: first set of group g
   int* d_tab_sets;         // q: sets of group g (0: not tabulated, the table is computed at decode time)
   int tab_ld;              // rows reserved per set: m in the subset form, the largest group otherwise
-  float* d_f;              // K x f_pitch projection vectors
+  float* d_f;              // K x f_pitch projection vectors: the draws with an even index
+  float* d_f2;             // the draws with an odd index
+  int last_decode_advanced;    // the most recent decode drew new vectors for the next one (the count is one ahead of what it used)
   int64_t f_pitch;         // row pitch of d_f in floats (multiple of 4)
+  int fresh_f;             // every decode draws new vectors first (solon_plan_set_fresh_projections)
+  unsigned long long* d_draw;   // [0] index of the draw now in d_f, [1] ticket of the fill kernel
 
   // projection workspace
   int proj_grid;           // CTAs of the projection kernel = number of partial sums
@@ -183,7 +187,7 @@ inline bool early_locator_starved(const solon_plan* plan) { return plan->early_l
 // gradients per step.
 inline bool keeps_l2_for_code(int P, int64_t d) { return (double)P * (double)d * 4.0 <= 1.0e9; }
 
-int launch_fill_projection(solon_plan* plan);
+int launch_fill_projection(solon_plan* plan, int advance);   // advance = 1: the next draw (device-side count), 0: redo the current one
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
 int launch_encode_f64(solon_plan* plan, const double* grads, double* coded);
 // rho_out / nu_out (and rho / nu below): device buffers, or nullptr for the plan's own

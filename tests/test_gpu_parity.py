@@ -354,14 +354,62 @@ def test_decode_is_bit_reproducible_and_reusable():
     with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
         coded = plan.encode(G)
         received, nodes = synth.apply_attack(wl, coded)
+        # by default every decode draws new vectors f: different projections, the same results
+        a0, m0 = plan.decode(received)
+        a0, m0 = a0.clone(), m0.clone()
+        f0, r0 = plan.projection_vectors(), plan.projections()
         a1, m1 = plan.decode(received)
-        r1 = plan.projections()
+        a1, m1 = a1.clone(), m1.clone()
+        f1, r1 = plan.projection_vectors(), plan.projections()
+        assert not np.array_equal(f0, f1) and not np.array_equal(r0[0], r1[0])
+        assert abs(f1.mean() - 1.0) < 0.02 and abs(f1.std() - 1.0) < 0.02 and abs(np.corrcoef(f0[0], f1[0])[0, 1]) < 0.02
+        assert torch.equal(a0, a1) and torch.equal(m0, m1) and np.array_equal(r0[1], r1[1])
+        # with the draw switched off the vectors stay and everything is bit-reproducible run to run
+        plan.set_fresh_projections(False)
+        a1, m1 = plan.decode(received)
+        a1, m1 = a1.clone(), m1.clone()
+        r1, f_kept = plan.projections(), plan.projection_vectors()
         a2, m2 = plan.decode(received)
         r2 = plan.projections()
-        assert torch.equal(a1, a2) and torch.equal(m1, m2)
+        assert np.array_equal(plan.projection_vectors(), f_kept) and not np.array_equal(f_kept, f1)
+        assert torch.equal(a1, a2) and torch.equal(m1, m2) and torch.equal(a0, a2)
         assert np.array_equal(r1[0], r2[0]) and np.array_equal(r1[1], r2[1])
         c2 = plan.encode(G)
         assert torch.equal(coded, c2)
+
+
+def test_a_replayed_graph_of_a_decode_draws_new_vectors_each_time():
+    """The count of the draws lives on the device: every replay of a captured decode projects with vectors of its own."""
+    wl = synth.small_variant(synth.WORKLOADS["resnet18"], 90_001)
+    G = synth.make_grads(wl, "cuda")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=5) as plan:
+        coded = plan.encode(G)
+        received, nodes = synth.apply_attack(wl, coded)
+        agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+        mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            plan.set_stream(side)
+            for _ in range(2):
+                plan.decode(received, agg, mask)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            plan.set_stream(torch.cuda.current_stream())
+            plan.decode(received, agg, mask)
+        plan.set_stream(torch.cuda.current_stream())
+        seen = []
+        for _ in range(3):
+            graph.replay()
+            torch.cuda.synchronize()
+            assert plan.decode_status() == 0 and mask.nonzero().flatten().tolist() == nodes
+            f = plan.projection_vectors()
+            rho, _ = plan.projections()
+            assert np.allclose(rho, so.project(received.cpu().numpy(), f), rtol=0, atol=1e-5 * np.abs(rho).max())   # these are the vectors it used
+            seen.append(f)
+        assert not np.array_equal(seen[0], seen[1]) and not np.array_equal(seen[1], seen[2]) and not np.array_equal(seen[0], seen[2])
 
 
 def test_projection_settings():

@@ -18,6 +18,7 @@ def test_project_noalloc_matches_plan_path_twice_in_a_row():
     G = synth.make_grads(wl, "cuda")
     with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=wl.seed) as plan:
         coded = plan.encode(G)
+        plan.set_fresh_projections(False)        # both paths must see the same vectors f: the plan's stay as they are
         K, d_c = plan.K, plan.d_c
         # a row pitch that is a multiple of 4 floats, as the entry point requires
         pitch = (d_c + 3) // 4 * 4
