@@ -155,6 +155,19 @@ int solon_plan_set_tolerance(solon_plan* plan, double tau);
  * takes its ordinary path afterwards (outcome 3 of solon_plan_get_early_outcome; results unchanged). */
 int solon_plan_set_early_locator(solon_plan* plan, int mode);
 
+/* Optimistic decode (Algorithm 1 with the block decoder's work done ahead of the locator's verdict).  When no node is
+ * corrupt the recovery reads a fixed set of rows, m per group.  The projection kernel, which has every row on chip
+ * anyway, can apply the inverse for those rows to each column slice as it passes and write the aggregate itself; if the
+ * locator then finds every group free of corrupt nodes, the recovery kernel returns at once and the decode has read the
+ * received matrix once instead of 1 + q m / P times.  If a node is corrupt the recovery kernel runs as usual and
+ * overwrites the aggregate: results never depend on the mode (the optimistic aggregate is computed in the recovery
+ * kernel's arithmetic and order, bit for bit).  mode 0: never; 1 (default): for the decode after one that found every
+ * node honest (decided on the device, no host round trip); 2: always.  Eligible plans: float32, s > 0, m <= 6 and
+ * q m rows fitting in the projection kernel's first batch of rows (at most 32); other plans ignore the mode. */
+int solon_plan_set_optimistic(solon_plan* plan, int mode);
+/* *skipped = 1 if the recovery kernel of the most recent solon_decode had nothing to do.  Synchronises. */
+int solon_plan_get_optimistic_outcome(solon_plan* plan, int* skipped);
+
 /* Rows per partition for solon_lsq_grads (default 256). */
 int solon_plan_set_lsq_rows(solon_plan* plan, int rows_per_partition);
 

@@ -45,6 +45,8 @@ SIGNATURES = {
     "solon_plan_set_fresh_projections": (c_int, [c_void_p, c_int]),
     "solon_plan_set_tolerance": (c_int, [c_void_p, c_double]),
     "solon_plan_set_early_locator": (c_int, [c_void_p, c_int]),
+    "solon_plan_set_optimistic": (c_int, [c_void_p, c_int]),
+    "solon_plan_get_optimistic_outcome": (c_int, [c_void_p, POINTER(c_int)]),
     "solon_plan_set_lsq_rows": (c_int, [c_void_p, c_int]),
     "solon_plan_dc": (c_int64, [c_void_p]),
     "solon_plan_num_groups": (c_int, [c_void_p]),
@@ -234,6 +236,17 @@ class Plan:
         """0: never start the locator on a partial projection; 1 (default): when the projection pass is long; 2: always;
         3: diagnostic, the locator's wait for the partial sums runs out (outcome 3), results unchanged."""
         _check(lib().solon_plan_set_early_locator(self._h, mode), "solon_plan_set_early_locator")
+
+    def set_optimistic(self, mode: int) -> None:
+        """0: the projection pass never recovers the aggregate itself; 1 (default): after a decode that found every node
+        honest; 2: always.  The recovery kernel is skipped when the locator confirms that no node is corrupt."""
+        _check(lib().solon_plan_set_optimistic(self._h, mode), "solon_plan_set_optimistic")
+
+    def optimistic_outcome(self) -> bool:
+        """True if the recovery kernel of the most recent decode had nothing to do."""
+        out = c_int(0)
+        _check(lib().solon_plan_get_optimistic_outcome(self._h, byref(out)), "solon_plan_get_optimistic_outcome")
+        return bool(out.value)
 
     def early_outcome(self) -> np.ndarray:
         """Per group: 0 no early run, 1 early answer confirmed, 2 not confirmed, 3 wait expired (last decode)."""

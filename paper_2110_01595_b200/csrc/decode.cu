@@ -19,7 +19,7 @@ static int decode_t(solon_plan* plan, const T* received, T* agg_grad, uint8_t* b
   };
   auto project = [&]() -> int {
     if constexpr (sizeof(T) == 8) return launch_project_f64(plan, received);
-    else return launch_project(plan, received);
+    else return launch_project(plan, received, nullptr, nullptr, agg_grad);
   };
   auto recover = [&]() -> int {
     if constexpr (sizeof(T) == 8) return launch_recover_f64(plan, received, agg_grad);

@@ -52,6 +52,8 @@ struct LocateParams {
   int* rec_rows;         // P
   double* coeff;         // P x m
   int* status;
+  int* opt;              // optimistic decode: [0] on for the next projection pass, [1] recovery may skip, [2] clean groups, [3] ticket, [4] mode
+  int opt_eligible;      // the plan has default rows in the projection kernel's first batch and this is a whole decode
   DrawParams draw;       // the vectors f of the next decode, written by the CTAs beyond the q locator CTAs (n_draw_ctas of them)
   int n_draw_ctas;
 };
@@ -123,6 +125,25 @@ __device__ __forceinline__ unsigned long long pipe_timer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+}
+
+// Optimistic decode, once per group at the end of its locator CTA (thread 0): count the groups without a corrupt node; the
+// last group to report decides whether the recovery kernel may skip - every group clean AND the projection pass of this
+// decode did recover from the default rows - and whether the next projection pass shall recover too (mode 2: always; mode
+// 1: when this decode found every node honest).  Nobody waits: an atomic ticket.
+__device__ __forceinline__ void optimistic_report(int* opt, int eligible, int q, bool group_clean) {
+  if (group_clean) atomicAdd(opt + 2, 1);
+  __threadfence();
+  if (atomicAdd(opt + 3, 1) != q - 1) return;
+  __threadfence();
+  const int clean = *(volatile int*)(opt + 2);
+  const int mode = *(volatile int*)(opt + 4);
+  const int was_on = *(volatile int*)(opt + 0);
+  const bool all_clean = clean == q;
+  opt[1] = (eligible && was_on && all_clean) ? 1 : 0;
+  opt[0] = (eligible && (mode == 2 || (mode == 1 && all_clean))) ? 1 : 0;
+  opt[2] = 0;
+  opt[3] = 0;
 }
 
 constexpr int kGatherBatch = 20;   // bunch sums fetched at once per column (the projection kernel leaves 37 on 148 SMs: two rounds)
@@ -294,6 +315,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
           prm.n_rec[g] = n_rec;
           prm.t_acc[g] = s_t_acc;
           prm.early[g] = 1;
+          optimistic_report(prm.opt, prm.opt_eligible, (int)gridDim.x - prm.n_draw_ctas, s_t_acc == 0);
         }
         return;
       }
@@ -345,6 +367,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
       prm.early[g] = !prm.spec ? 0 : (s_ready > 0 ? 2 : (s_ready == 0 ? 3 : 4));
+      optimistic_report(prm.opt, prm.opt_eligible, (int)gridDim.x - prm.n_draw_ctas, s_t_acc == 0);
       (void)ok;      // an undecodable group is reported through t_acc[g] = -1
     }
   }
@@ -507,6 +530,8 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   }
   if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  prm.opt = plan->d_opt;
+  prm.opt_eligible = (fused && plan->opt_rows > 0 && plan->optimistic != 0) ? 1 : 0;
   // CTAs that draw the next decode's vectors beside the locator's: a few per SM, a thread per several quads
   prm.draw = draw_params(plan);
   prm.n_draw_ctas = 0;

@@ -95,6 +95,7 @@ static void free_device(solon_plan* p) {
   cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f); cudaFree(p->d_f2);
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_tab_count); cudaFree(p->d_tab_rows); cudaFree(p->d_tab_coeff); cudaFree(p->d_tab_off); cudaFree(p->d_tab_sets);
+  cudaFree(p->d_row_order); cudaFree(p->d_opt_row); cudaFree(p->d_opt_coeff); cudaFree(p->d_opt);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress); cudaFree(p->d_draw);
@@ -269,6 +270,50 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
         all_rows.insert(all_rows.end(), rows.begin(), rows.end());
         all_coeff.insert(all_coeff.end(), coeff.begin(), coeff.end());
       }
+      {
+        // Optimistic decode: the rows the recovery reads when no node is corrupt (subset form), group by group, with
+        // their weights rounded as the recovery kernel rounds them; eligible when they all fit in the projection
+        // kernel's first batch of rows, which then takes them first.
+        std::vector<int> order, opt_row;
+        std::vector<float> opt_coeff;
+        std::vector<uint8_t> is_default((size_t)P, 0);
+        const int n_batches = (P + 31) / 32;
+        const int batch_rows = (P + n_batches - 1) / n_batches;
+        bool eligible = dtype == SOLON_F32 && s > 0 && m <= SOLON_SUBSET_MAX_M && q * m <= batch_rows;
+        for (int g = 0; g < q && eligible; ++g) {
+          if (tab_sets[g] == 0) { eligible = false; break; }
+          const size_t first = (size_t)tab_off[g];             // the empty corrupt set is entry 0 of the group
+          for (int j = 0; j < m; ++j) {
+            const int node = start[g] + all_rows[first * p->tab_ld + j];
+            opt_row.push_back(node);
+            is_default[(size_t)node] = 1;
+            for (int l = 0; l < m; ++l) opt_coeff.push_back((float)all_coeff[(first * p->tab_ld + j) * m + l]);
+          }
+        }
+        if (!eligible) {
+          opt_row.clear();
+          opt_coeff.clear();
+          is_default.assign((size_t)P, 0);
+        }
+        order = opt_row;
+        for (int k = 0; k < P; ++k)
+          if (!is_default[(size_t)k]) order.push_back(k);
+        p->opt_rows = (int)opt_row.size();
+        p->optimistic = 1;
+        if ((rc = dev_alloc(&p->d_row_order, (size_t)P))) break;
+        if ((rc = dev_alloc(&p->d_opt_row, opt_row.size()))) break;
+        if ((rc = dev_alloc(&p->d_opt_coeff, opt_coeff.size()))) break;
+        if ((rc = dev_alloc(&p->d_opt, 8))) break;
+        const int opt_init[8] = {0, 0, 0, 0, p->optimistic, 0, 0, 0};
+        if (cudaMemcpy(p->d_row_order, order.data(), (size_t)P * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess ||
+            (!opt_row.empty() && cudaMemcpy(p->d_opt_row, opt_row.data(), opt_row.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) ||
+            (!opt_coeff.empty() && cudaMemcpy(p->d_opt_coeff, opt_coeff.data(), opt_coeff.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) ||
+            cudaMemcpy(p->d_opt, opt_init, sizeof(opt_init), cudaMemcpyHostToDevice) != cudaSuccess) {
+          (void)cudaGetLastError();
+          rc = SOLON_ERR_CUDA;
+          break;
+        }
+      }
       if ((rc = dev_alloc(&p->d_tab_count, all_count.size()))) break;
       if ((rc = dev_alloc(&p->d_tab_rows, all_rows.size()))) break;
       if ((rc = dev_alloc(&p->d_tab_coeff, all_coeff.size()))) break;
@@ -357,6 +402,25 @@ int solon_plan_reseed(solon_plan* plan, uint64_t seed) {
 int solon_plan_set_fresh_projections(solon_plan* plan, int on) {
   if (!plan) return SOLON_ERR_INVALID_ARG;
   plan->fresh_f = on ? 1 : 0;
+  return SOLON_OK;
+}
+
+int solon_plan_set_optimistic(solon_plan* plan, int mode) {
+  if (!plan || mode < 0 || mode > 2) return SOLON_ERR_INVALID_ARG;
+  plan->optimistic = mode;
+  // the mode is read on the device by the locator kernel; a change also forgets what the last decode found
+  const int init[5] = {mode == 2 ? 1 : 0, 0, 0, 0, mode};
+  SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_opt, init, sizeof(init), cudaMemcpyHostToDevice, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  return SOLON_OK;
+}
+
+int solon_plan_get_optimistic_outcome(solon_plan* plan, int* skipped) {
+  if (!plan || !skipped) return SOLON_ERR_INVALID_ARG;
+  int word[2] = {0, 0};
+  SOLON_CUDA_TRY(cudaMemcpyAsync(word, plan->d_opt, sizeof(word), cudaMemcpyDeviceToHost, plan->stream));
+  SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+  *skipped = word[1];
   return SOLON_OK;
 }
 

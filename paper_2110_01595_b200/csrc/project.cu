@@ -232,7 +232,57 @@ struct ProjPipe {
   int64_t part_a_cols;                // columns of part A in every CTA's range (whole slices)
   unsigned long long* progress;       // bunches whose part-A sums [0] and final sums [1] are complete (zeroed by the recovery kernel)
   int* status;
+  const int* row_order;               // P: the rows in the order the kernel takes them (the default recovery rows first)
+  // optimistic decode: the default recovery rows are the first opt_rows rows of the first batch; when opt_flags[0] is set the
+  // consumers also recover the aggregate of every column slice from them, exactly as the recovery kernel would
+  int opt_rows;                       // 0: never
+  const int* opt_row;                 // opt_rows: global node index of the default rows
+  const float* opt_coeff;             // opt_rows x m weights
+  const int* opt_flags;               // device flags of the optimistic decode
+  float* agg;                         // d: the aggregate (written only when the flag is set)
+  int m;
+  int64_t d;
 };
+
+// Aggregate of one column slice from the default recovery rows (the first n_def row slots of the stage), in the recovery
+// kernel's arithmetic and order: acc = fma(weight, value, acc) over the rows, group by group.  A thread owns chunks
+// tid, tid + 256, tid + 512, tid + 768 of each 1024 and shares a row's weights (eight floats per row in shared memory,
+// fetched with two 128-bit loads) between them.
+constexpr int kOptChunks = 4;
+template <int M>
+__device__ __forceinline__ void opt_recover_slice(const float* base, int slot_floats, const int* s_shift, const float* s_coeff, int n_def,
+                                                  int cols, int64_t c0, float* __restrict__ agg, int64_t d, int tid) {
+  for (int c = tid; c < cols; c += kOptChunks * kPipeConsumers) {
+    float acc[kOptChunks][M];
+#pragma unroll
+    for (int i = 0; i < kOptChunks; ++i)
+#pragma unroll
+      for (int l = 0; l < M; ++l) acc[i][l] = 0.0f;
+    for (int j = 0; j < n_def; ++j) {
+      const float* row = base + (size_t)j * slot_floats + s_shift[j];
+      float v[kOptChunks];
+#pragma unroll
+      for (int i = 0; i < kOptChunks; ++i) v[i] = c + i * kPipeConsumers < cols ? row[c + i * kPipeConsumers] : 0.0f;
+      const float4 w0 = *reinterpret_cast<const float4*>(s_coeff + j * 8);
+      const float4 w1 = *reinterpret_cast<const float4*>(s_coeff + j * 8 + 4);
+      const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+      for (int l = 0; l < M; ++l)
+#pragma unroll
+        for (int i = 0; i < kOptChunks; ++i) acc[i][l] = fmaf(w[l], v[i], acc[i][l]);
+    }
+#pragma unroll
+    for (int i = 0; i < kOptChunks; ++i) {
+      const int ci = c + i * kPipeConsumers;
+      if (ci < cols) {
+        const int64_t o = (c0 + ci) * M;
+#pragma unroll
+        for (int l = 0; l < M; ++l)
+          if (o + l < d) __stcs(agg + o + l, acc[i][l]);
+      }
+    }
+  }
+}
 
 // One slice for the NR rows of this warp: rows[j] point at column 0 of the slice in the warp's j-th row.
 template <int K, int NR>
@@ -356,6 +406,8 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
                                                                      unsigned int* ticket, int final_reduce) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ unsigned int s_flag;
+  __shared__ __align__(16) float s_opt_coeff[kPipeRows * 8];     // eight floats per default row: m weights, then zeros
+  __shared__ int s_opt_shift[kPipeRows];
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + kPipeStages;
@@ -375,6 +427,15 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
     }
     *abort_flag = 0;
     pipe::fence_barrier_init();
+  }
+  // optimistic decode (float32 plans): this pass also recovers the aggregate from the default rows
+  bool opt = false;
+  if constexpr (sizeof(T) == 4) {
+    opt = pp.opt_rows > 0 && pp.opt_flags[0] != 0;
+    if (opt) {
+      for (int i = tid; i < pp.opt_rows * 8; i += kPipeThreads) s_opt_coeff[i] = (i & 7) < pp.m ? pp.opt_coeff[(i >> 3) * pp.m + (i & 7)] : 0.0f;
+      for (int j = tid; j < pp.opt_rows; j += kPipeThreads) s_opt_shift[j] = (int)((((int64_t)pp.opt_row[j] & 3) * (d_c & 3)) & 3);
+    }
   }
   __syncthreads();
 
@@ -408,7 +469,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           const T* row_src = nullptr;
           T* slot = reinterpret_cast<T*>(stage_base) + (size_t)lane * pp.slot_floats;
           if (lane < nb) {
-            const int64_t first = (int64_t)(b0 + lane) * d_c + c0;
+            const int64_t first = (int64_t)pp.row_order[b0 + lane] * d_c + c0;
             const int64_t last = first + cols;
             const int64_t a0 = first & ~(kVec - 1);                   // enclosing 16-byte boundary
             int64_t a1 = (last + kVec - 1) & ~(kVec - 1);
@@ -443,9 +504,12 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
       for (int b0 = 0; b0 < P && lo < hi; b0 += pp.batch_rows) {
         const int nb = min(pp.batch_rows, P - b0);
         const int nr = warp < nb ? (nb - warp + kPipeWarps - 1) / kPipeWarps : 0;    // rows warp, warp + 8, ... below nb
-        int shift[4];
+        int shift[4], row_of[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) shift[j] = (int)((((b0 + warp + 8 * j) & (kVec - 1)) * dc_mod4) & (kVec - 1));   // (row * d_c + c0) mod (elements per 16 bytes)
+        for (int j = 0; j < 4; ++j) {
+          row_of[j] = j < nr ? pp.row_order[b0 + warp + 8 * j] : 0;
+          shift[j] = (int)(((row_of[j] & (kVec - 1)) * dc_mod4) & (kVec - 1));   // (row * d_c + c0) mod (elements per 16 bytes)
+        }
         double rho[4][K], nu[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -467,13 +531,26 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           else if (nr == 3) pipe_consume<K, 3>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
+          if constexpr (sizeof(T) == 4) {
+            if (opt && b0 == 0) {
+              const float* rows0 = reinterpret_cast<const float*>(base);
+              switch (pp.m) {
+                case 1: opt_recover_slice<1>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+                case 2: opt_recover_slice<2>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+                case 3: opt_recover_slice<3>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+                case 4: opt_recover_slice<4>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+                case 5: opt_recover_slice<5>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+                default: opt_recover_slice<6>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+              }
+            }
+          }
           __syncwarp();
           if (lane == 0) pipe::mbar_arrive(&empty_bar[stage]);
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           if (j < nr) {
-            const int row = b0 + warp + 8 * j;
+            const int row = row_of[j];
 #pragma unroll
             for (int kappa = 0; kappa < K; ++kappa) {
               const double t = warp_sum(rho[j][kappa]);
@@ -515,10 +592,19 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
 }
 
 template <int K, typename T>
-static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rho_out, double* nu_out, int final_reduce) {
+static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rho_out, double* nu_out, int final_reduce, T* agg) {
   ProjPipe pp;
   pp.status = plan->d_status;
   pp.progress = plan->d_proj_progress;
+  pp.row_order = plan->d_row_order;
+  // optimistic decode: only in the whole decode (the aggregate's buffer is known) of a float32 plan that is eligible
+  pp.opt_rows = (!final_reduce && agg && sizeof(T) == 4 && plan->optimistic != 0) ? plan->opt_rows : 0;
+  pp.opt_row = plan->d_opt_row;
+  pp.opt_coeff = plan->d_opt_coeff;
+  pp.opt_flags = plan->d_opt;
+  pp.agg = reinterpret_cast<float*>(agg);
+  pp.m = plan->m;
+  pp.d = plan->d;
   // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
   const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128;
   const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
@@ -558,26 +644,26 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
 }
 
 template <typename T>
-static int launch_project_t(solon_plan* plan, const T* received, double* rho_out, double* nu_out) {
+static int launch_project_t(solon_plan* plan, const T* received, double* rho_out, double* nu_out, T* agg) {
   // no output buffers: the decode proper, whose locator kernel adds the last level of partial sums itself
   const int final_reduce = (rho_out || nu_out) ? 1 : 0;
   if (!rho_out) rho_out = plan->d_rho;
   if (!nu_out) nu_out = plan->d_nu;
   plan->launches += 1;
   switch (plan->K) {
-    case 1: return launch_project_pipe_k<1, T>(plan, received, rho_out, nu_out, final_reduce);
-    case 2: return launch_project_pipe_k<2, T>(plan, received, rho_out, nu_out, final_reduce);
-    case 3: return launch_project_pipe_k<3, T>(plan, received, rho_out, nu_out, final_reduce);
-    case 4: return launch_project_pipe_k<4, T>(plan, received, rho_out, nu_out, final_reduce);
+    case 1: return launch_project_pipe_k<1, T>(plan, received, rho_out, nu_out, final_reduce, agg);
+    case 2: return launch_project_pipe_k<2, T>(plan, received, rho_out, nu_out, final_reduce, agg);
+    case 3: return launch_project_pipe_k<3, T>(plan, received, rho_out, nu_out, final_reduce, agg);
+    case 4: return launch_project_pipe_k<4, T>(plan, received, rho_out, nu_out, final_reduce, agg);
     default: return SOLON_ERR_INVALID_ARG;
   }
 }
 
-int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out) {
-  return launch_project_t<float>(plan, received, rho_out, nu_out);
+int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out, float* agg) {
+  return launch_project_t<float>(plan, received, rho_out, nu_out, agg);
 }
 int launch_project_f64(solon_plan* plan, const double* received, double* rho_out, double* nu_out) {
-  return launch_project_t<double>(plan, received, rho_out, nu_out);
+  return launch_project_t<double>(plan, received, rho_out, nu_out, nullptr);
 }
 
 // ---- projections without any allocation ------------------------------------------------------------

@@ -24,6 +24,7 @@ struct RecoverParamsT {
   const int* rec_rows;   // P, group g's rows at [group_start[g], +n_rec[g])
   const double* coeff;   // P x m, same indexing
   unsigned long long* proj_progress;   // the projection kernel's part-A count, zeroed here for the next decode
+  const int* opt;        // optimistic decode: opt[1] != 0 - the projection pass has already written the aggregate
 };
 typedef RecoverParamsT<float> RecoverParams;
 
@@ -156,6 +157,7 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
     prm.proj_progress[0] = 0ULL;
     prm.proj_progress[1] = 0ULL;
   }
+  if (prm.opt[1] != 0) return;   // every group's default rows were confirmed and the projection pass recovered from them
   const int n_rows = pack_tables<Acc, M, kStride, (int)kVec>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c);
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
@@ -379,6 +381,7 @@ static void fill_recover_params(solon_plan* plan, const T* received, T* agg, Rec
   prm->rec_rows = plan->d_rec_rows;
   prm->coeff = plan->d_coeff;
   prm->proj_progress = plan->d_proj_progress;
+  prm->opt = plan->d_opt;
 }
 
 // float64 received vectors and aggregate: weights and sums in float64 for every compression ratio.

@@ -71,6 +71,16 @@ struct solon_plan {
   int64_t* d_tab_off;      // q: first set of group g
   int* d_tab_sets;         // q: sets of group g (0: not tabulated, the table is computed at decode time)
   int tab_ld;              // rows reserved per set: m in the subset form, the largest group otherwise
+
+  // optimistic decode (solon_plan_set_optimistic): the projection pass also writes the aggregate recovered from the
+  // rows that are read when no node is corrupt, and the recovery kernel is skipped when the locator confirms them
+  int optimistic;          // 0 never, 1 after a decode that found every node honest (default), 2 always
+  int opt_rows;            // number of default rows over all groups (0: the plan is not eligible)
+  int* d_row_order;        // P: order in which the projection kernel takes the rows (default rows first)
+  int* d_opt_row;          // opt_rows: the default rows (global node index), group by group
+  float* d_opt_coeff;      // opt_rows x m: their weights, as the recovery kernel would use them
+  int* d_opt;              // [0] next projection pass recovers too, [1] the recovery kernel may skip, [2] clean groups, [3] ticket,
+                           // [4] mode (copied from `optimistic`)
   float* d_f;              // K x f_pitch projection vectors: the draws with an even index
   float* d_f2;             // the draws with an odd index
   int last_decode_advanced;    // the most recent decode drew new vectors for the next one (the count is one ahead of what it used)
@@ -191,7 +201,8 @@ int launch_fill_projection(solon_plan* plan, int advance);   // advance = 1: the
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
 int launch_encode_f64(solon_plan* plan, const double* grads, double* coded);
 // rho_out / nu_out (and rho / nu below): device buffers, or nullptr for the plan's own
-int launch_project(solon_plan* plan, const float* received, double* rho_out = nullptr, double* nu_out = nullptr);
+// agg: where the optimistic decode may write the aggregate (the whole decode only; nullptr: never)
+int launch_project(solon_plan* plan, const float* received, double* rho_out = nullptr, double* nu_out = nullptr, float* agg = nullptr);
 int launch_project_f64(solon_plan* plan, const double* received, double* rho_out = nullptr, double* nu_out = nullptr);
 int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho = nullptr, const double* nu = nullptr);
 int launch_recover(solon_plan* plan, const float* received, float* agg);
