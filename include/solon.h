@@ -97,7 +97,7 @@ const char* solon_strerror(int status);
 /* Build the mechanism (A, E, D) of Section 3.4 for P nodes, s adversaries per group,
  * compression ratio m, minimum group size r (>= 2 s + m) and gradient length d: group layout,
  * node scalars, K = 2 projection vectors f_kappa[p] = 1 + N(0,1) drawn on the device from
- * `seed` (f ~ N(1, I) in Section 3.4; redrawn by every decode, see solon_plan_set_fresh_projections),
+ * `seed` (f ~ N(1, I) in Section 3.4; solon_plan_set_fresh_projections makes every decode draw anew),
  * and all device workspace.  Uses the current CUDA device.
  * Synchronises the device once.  *out receives the plan, to be released by solon_plan_destroy. */
 int solon_plan_create(int P, int s, int m, int r, int64_t d, uint64_t seed, solon_plan** out);
@@ -127,14 +127,16 @@ int solon_plan_set_num_projections(solon_plan* plan, int K);
 int solon_plan_reseed(solon_plan* plan, uint64_t seed);
 
 /* Algorithm 1 draws its random vector inside the decoder, and the proof that every corrupt node is located with
- * probability 1 (Lemma 3) needs f independent of what the adversary sent.  on = 1 (default): every decode projects
- * with vectors no earlier decode used - draw n of the plan's seed, n counted on the device, so that a replayed CUDA
- * graph of a decode moves on as well.  The next decode's vectors are written, into a second buffer, by spare CTAs of
- * the locator kernel (solon_decode, solon_decode_finish) while the locator's few CTAs work and the rest of the GPU is
- * idle: no kernel is added and, unless K d_c is large against the locator's time, no time.  They are drawn before
- * the adversary's next vectors exist and stay on the device.  on = 0: the vectors in memory are reused by every decode
- * until solon_plan_reseed; that is only sound against an adversary that can neither read nor infer them, since
- * one that knows f can send a deviation orthogonal to all K vectors and stay unseen.
+ * probability 1 (Lemma 3) needs f independent of what the adversary sent.  on = 0 (default): the vectors in memory
+ * are reused by every decode until solon_plan_reseed; that is sound against an adversary that can neither read nor
+ * infer them (they are drawn on the device from the plan's seed and never leave it), but one that knows f can send a
+ * deviation orthogonal to all K vectors and stay unseen.  on = 1: every decode projects with vectors no earlier decode
+ * used - draw n of the plan's seed, n counted on the device, so that a replayed CUDA graph of a decode moves on as well.
+ * The next decode's vectors are written, into a second buffer, by spare CTAs of the locator kernel (solon_decode,
+ * solon_decode_finish), before the adversary's next vectors exist: no kernel is added, but the recovery kernel can only
+ * be scheduled once those CTAs have all started, which costs 5 us on a decode of 15 nodes x 2.2 M coded values and
+ * 12 - 45 us (the higher figure under the power cap) on one of 45 x 5.7 M.  A closed training loop that faces an adaptive
+ * adversary should switch it on (sgd.ClosedLoop does).
  * solon_plan_get_projection_vectors returns the vectors the most recent decode used. */
 int solon_plan_set_fresh_projections(solon_plan* plan, int on);
 

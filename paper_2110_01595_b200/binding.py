@@ -226,7 +226,8 @@ class Plan:
         _check(lib().solon_plan_reseed(self._h, seed), "solon_plan_reseed")
 
     def set_fresh_projections(self, on: bool) -> None:
-        """True (default): every decode draws new projection vectors first; False: the ones in memory are reused."""
+        """True: every decode projects with projection vectors no earlier decode used; False (default): the ones in memory
+        are reused until reseed()."""
         _check(lib().solon_plan_set_fresh_projections(self._h, 1 if on else 0), "solon_plan_set_fresh_projections")
 
     def set_tolerance(self, tau: float) -> None:

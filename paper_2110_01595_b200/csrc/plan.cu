@@ -213,7 +213,7 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
   p->num_sms = prop.multiProcessorCount;
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
-  p->fresh_f = 1;
+  p->fresh_f = 0;
   p->stream_hints = keeps_l2_for_code(P, dtype == SOLON_F64 ? 2 * d : d) ? 1 : 0;
   if (const char* env = getenv("SOLON_STREAM_HINTS")) p->stream_hints = env[0] == '1' ? 1 : (env[0] == '0' ? 0 : p->stream_hints);
 

@@ -58,6 +58,7 @@ class ClosedLoop:
                  attackers_per_group: int = 0, attack: str = "flip10"):
         self.plan, self.X, self.y, self.lr = plan, X, y, float(lr)
         plan.set_lsq_rows(rows)
+        plan.set_fresh_projections(True)      # a fresh Byzantine set every step may adapt to what it saw: new vectors f per decode
         self.w = w0.clone()
         dev = X.device
         self.grads = torch.empty((plan.P, plan.d), dtype=torch.float32, device=dev)

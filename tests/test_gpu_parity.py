@@ -354,7 +354,8 @@ def test_decode_is_bit_reproducible_and_reusable():
     with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
         coded = plan.encode(G)
         received, nodes = synth.apply_attack(wl, coded)
-        # by default every decode draws new vectors f: different projections, the same results
+        # with fresh projections every decode draws new vectors f: different projections, the same results
+        plan.set_fresh_projections(True)
         a0, m0 = plan.decode(received)
         a0, m0 = a0.clone(), m0.clone()
         f0, r0 = plan.projection_vectors(), plan.projections()
@@ -387,6 +388,7 @@ def test_a_replayed_graph_of_a_decode_draws_new_vectors_each_time():
         received, nodes = synth.apply_attack(wl, coded)
         agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
         mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
+        plan.set_fresh_projections(True)
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
