@@ -30,6 +30,7 @@ struct LocateParams {
   const int64_t* tab_off;     // q: first set of group g
   const int* tab_sets;        // q: number of sets of group g (0: not tabulated)
   int tab_ld;
+  int use_tabs;               // look recovery tables up (else compute them): pays when the tables survive in L2 between decodes
   int P, m, s, K;
   double tau;
   double* ws_global;     // q x ws_stride doubles, used when shared memory is too small
@@ -52,8 +53,7 @@ struct LocateParams {
   int* rec_rows;         // P
   double* coeff;         // P x m
   int* status;
-  int* opt;              // optimistic decode: [0] on for the next projection pass, [1] recovery may skip, [2] clean groups, [3] ticket, [4] mode
-  int opt_eligible;      // the plan has default rows in the projection kernel's first batch and this is a whole decode
+  int* opt;              // optimistic decode: opt[8 + g] receives whether group g had no corrupt node
   DrawParams draw;       // the vectors f of the next decode, written by the CTAs beyond the q locator CTAs (n_draw_ctas of them)
   int n_draw_ctas;
 };
@@ -127,25 +127,6 @@ __device__ __forceinline__ unsigned long long pipe_timer_ns() {
   return t;
 }
 
-// Optimistic decode, once per group at the end of its locator CTA (thread 0): count the groups without a corrupt node; the
-// last group to report decides whether the recovery kernel may skip - every group clean AND the projection pass of this
-// decode did recover from the default rows - and whether the next projection pass shall recover too (mode 2: always; mode
-// 1: when this decode found every node honest).  Nobody waits: an atomic ticket.
-__device__ __forceinline__ void optimistic_report(int* opt, int eligible, int q, bool group_clean) {
-  if (group_clean) atomicAdd(opt + 2, 1);
-  __threadfence();
-  if (atomicAdd(opt + 3, 1) != q - 1) return;
-  __threadfence();
-  const int clean = *(volatile int*)(opt + 2);
-  const int mode = *(volatile int*)(opt + 4);
-  const int was_on = *(volatile int*)(opt + 0);
-  const bool all_clean = clean == q;
-  opt[1] = (eligible && was_on && all_clean) ? 1 : 0;
-  opt[0] = (eligible && (mode == 2 || (mode == 1 && all_clean))) ? 1 : 0;
-  opt[2] = 0;
-  opt[3] = 0;
-}
-
 constexpr int kGatherBatch = 20;   // bunch sums fetched at once per column (the projection kernel leaves 37 on 148 SMs: two rounds)
 
 __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocateParams prm) {
@@ -172,7 +153,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   tb.Mt = prm.mt + (size_t)g * prm.m * prm.m;
   tb.Tch = prm.tch + (size_t)row0 * (prm.s + 1);
   tb.w = prm.w + row0;
-  tb.n_sets = prm.tab_sets[g];
+  tb.n_sets = prm.use_tabs ? prm.tab_sets[g] : 0;
   tb.tab_ld = prm.tab_ld;
   tb.tab_count = prm.tab_count + prm.tab_off[g];
   tb.tab_rows = prm.tab_rows + (size_t)prm.tab_off[g] * prm.tab_ld;
@@ -315,7 +296,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
           prm.n_rec[g] = n_rec;
           prm.t_acc[g] = s_t_acc;
           prm.early[g] = 1;
-          optimistic_report(prm.opt, prm.opt_eligible, (int)gridDim.x - prm.n_draw_ctas, s_t_acc == 0);
+          prm.opt[8 + g] = s_t_acc == 0 ? 1 : 0;      // optimistic decode: this group had no corrupt node
         }
         return;
       }
@@ -367,7 +348,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
       prm.early[g] = !prm.spec ? 0 : (s_ready > 0 ? 2 : (s_ready == 0 ? 3 : 4));
-      optimistic_report(prm.opt, prm.opt_eligible, (int)gridDim.x - prm.n_draw_ctas, s_t_acc == 0);
+      prm.opt[8 + g] = s_t_acc == 0 ? 1 : 0;      // optimistic decode: this group had no corrupt node
       (void)ok;      // an undecodable group is reported through t_acc[g] = -1
     }
   }
@@ -504,6 +485,7 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   prm.tab_off = plan->d_tab_off;
   prm.tab_sets = plan->d_tab_sets;
   prm.tab_ld = plan->tab_ld;
+  prm.use_tabs = plan->stream_hints;
   prm.P = plan->P; prm.m = plan->m; prm.s = plan->s; prm.K = plan->K;
   prm.tau = plan->tau;
   prm.ws_global = plan->d_locate_ws;
@@ -531,7 +513,6 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prm.opt = plan->d_opt;
-  prm.opt_eligible = (fused && plan->opt_rows > 0 && plan->optimistic != 0) ? 1 : 0;
   // CTAs that draw the next decode's vectors beside the locator's: a few per SM, a thread per several quads
   prm.draw = draw_params(plan);
   prm.n_draw_ctas = 0;
@@ -542,6 +523,7 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
     prm.n_draw_ctas = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
   }
   plan->last_decode_advanced = prm.n_draw_ctas > 0 ? 1 : 0;
+  if (prm.n_draw_ctas > 0) plan->draw_parity = -1;      // the count moves on the device from here on
   plan->launches += 1;
   // one warp per error count, at least four for the CTA-wide steps (four still fit, at 128 registers a thread, in the
   // slot the projection kernel leaves free, so the CTA is resident early)

@@ -95,7 +95,7 @@ static void free_device(solon_plan* p) {
   cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f); cudaFree(p->d_f2);
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_tab_count); cudaFree(p->d_tab_rows); cudaFree(p->d_tab_coeff); cudaFree(p->d_tab_off); cudaFree(p->d_tab_sets);
-  cudaFree(p->d_row_order); cudaFree(p->d_opt_row); cudaFree(p->d_opt_coeff); cudaFree(p->d_opt);
+  cudaFree(p->d_opt_coeff); cudaFree(p->d_opt);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress); cudaFree(p->d_draw);
@@ -214,7 +214,8 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
   p->fresh_f = 0;
-  p->stream_hints = keeps_l2_for_code(P, dtype == SOLON_F64 ? 2 * d : d) ? 1 : 0;
+  p->draw_parity = 0;
+  p->stream_hints = keeps_l2_for_code(P, m, dtype == SOLON_F64 ? 2 * d : d) ? 1 : 0;
   if (const char* env = getenv("SOLON_STREAM_HINTS")) p->stream_hints = env[0] == '1' ? 1 : (env[0] == '0' ? 0 : p->stream_hints);
 
   rc = SOLON_OK;
@@ -274,7 +275,7 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
         // Optimistic decode: the rows the recovery reads when no node is corrupt (subset form), group by group, with
         // their weights rounded as the recovery kernel rounds them; eligible when they all fit in the projection
         // kernel's first batch of rows, which then takes them first.
-        std::vector<int> order, opt_row;
+        std::vector<int> opt_row;
         std::vector<float> opt_coeff;
         std::vector<uint8_t> is_default((size_t)P, 0);
         const int n_batches = (P + 31) / 32;
@@ -295,20 +296,15 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
           opt_coeff.clear();
           is_default.assign((size_t)P, 0);
         }
-        order = opt_row;
-        for (int k = 0; k < P; ++k)
-          if (!is_default[(size_t)k]) order.push_back(k);
         p->opt_rows = (int)opt_row.size();
+        p->opt_row_host = opt_row;
         p->optimistic = 1;
-        if ((rc = dev_alloc(&p->d_row_order, (size_t)P))) break;
-        if ((rc = dev_alloc(&p->d_opt_row, opt_row.size()))) break;
         if ((rc = dev_alloc(&p->d_opt_coeff, opt_coeff.size()))) break;
-        if ((rc = dev_alloc(&p->d_opt, 8))) break;
-        const int opt_init[8] = {0, 0, 0, 0, p->optimistic, 0, 0, 0};
-        if (cudaMemcpy(p->d_row_order, order.data(), (size_t)P * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess ||
-            (!opt_row.empty() && cudaMemcpy(p->d_opt_row, opt_row.data(), opt_row.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) ||
-            (!opt_coeff.empty() && cudaMemcpy(p->d_opt_coeff, opt_coeff.data(), opt_coeff.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) ||
-            cudaMemcpy(p->d_opt, opt_init, sizeof(opt_init), cudaMemcpyHostToDevice) != cudaSuccess) {
+        if ((rc = dev_alloc(&p->d_opt, (size_t)8 + q))) break;
+        std::vector<int> opt_init((size_t)8 + q, 0);
+        opt_init[4] = p->optimistic;
+        if ((!opt_coeff.empty() && cudaMemcpy(p->d_opt_coeff, opt_coeff.data(), opt_coeff.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) ||
+            cudaMemcpy(p->d_opt, opt_init.data(), opt_init.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
           (void)cudaGetLastError();
           rc = SOLON_ERR_CUDA;
           break;
@@ -387,6 +383,7 @@ int solon_plan_set_num_projections(solon_plan* plan, int K) {
   int rc = alloc_projection(plan);
   if (rc) return rc;
   SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_draw, 0, 2 * sizeof(unsigned long long), plan->stream));
+  plan->draw_parity = 0;
   if ((rc = launch_fill_projection(plan, 0))) return rc;
   SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
   return SOLON_OK;
@@ -396,31 +393,42 @@ int solon_plan_reseed(solon_plan* plan, uint64_t seed) {
   if (!plan) return SOLON_ERR_INVALID_ARG;
   plan->seed = seed;
   SOLON_CUDA_TRY(cudaMemsetAsync(plan->d_draw, 0, 2 * sizeof(unsigned long long), plan->stream));   // draw 0 of the new seed
+  plan->draw_parity = 0;
   return launch_fill_projection(plan, 0);
 }
 
 int solon_plan_set_fresh_projections(solon_plan* plan, int on) {
   if (!plan) return SOLON_ERR_INVALID_ARG;
   plan->fresh_f = on ? 1 : 0;
+  if (!on && plan->draw_parity < 0) {
+    // decodes stop drawing: the count now stands still, so the host may know which buffer holds the current draw
+    unsigned long long n = 0;
+    SOLON_CUDA_TRY(cudaMemcpyAsync(&n, plan->d_draw, sizeof(n), cudaMemcpyDeviceToHost, plan->stream));
+    SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
+    plan->draw_parity = (int)(n & 1ULL);
+  }
   return SOLON_OK;
 }
 
 int solon_plan_set_optimistic(solon_plan* plan, int mode) {
   if (!plan || mode < 0 || mode > 2) return SOLON_ERR_INVALID_ARG;
   plan->optimistic = mode;
-  // the mode is read on the device by the locator kernel; a change also forgets what the last decode found
-  const int init[5] = {mode == 2 ? 1 : 0, 0, 0, 0, mode};
-  SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_opt, init, sizeof(init), cudaMemcpyHostToDevice, plan->stream));
+  // the mode is read on the device by the projection kernel; a change also forgets what the last decode found
+  std::vector<int> init((size_t)8 + plan->q, 0);
+  init[4] = mode;
+  SOLON_CUDA_TRY(cudaMemcpyAsync(plan->d_opt, init.data(), init.size() * sizeof(int), cudaMemcpyHostToDevice, plan->stream));
   SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
   return SOLON_OK;
 }
 
 int solon_plan_get_optimistic_outcome(solon_plan* plan, int* skipped) {
   if (!plan || !skipped) return SOLON_ERR_INVALID_ARG;
-  int word[2] = {0, 0};
-  SOLON_CUDA_TRY(cudaMemcpyAsync(word, plan->d_opt, sizeof(word), cudaMemcpyDeviceToHost, plan->stream));
+  std::vector<int> word((size_t)8 + plan->q, 0);
+  SOLON_CUDA_TRY(cudaMemcpyAsync(word.data(), plan->d_opt, word.size() * sizeof(int), cudaMemcpyDeviceToHost, plan->stream));
   SOLON_CUDA_TRY(cudaStreamSynchronize(plan->stream));
-  *skipped = word[1];
+  int all_clean = 1;
+  for (int g = 0; g < plan->q; ++g) all_clean &= word[(size_t)8 + g] != 0 ? 1 : 0;
+  *skipped = (word[1] != 0 && all_clean) ? 1 : 0;      // what the recovery kernel itself evaluates
   return SOLON_OK;
 }
 

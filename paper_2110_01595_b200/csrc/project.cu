@@ -232,16 +232,28 @@ struct ProjPipe {
   int64_t part_a_cols;                // columns of part A in every CTA's range (whole slices)
   unsigned long long* progress;       // bunches whose part-A sums [0] and final sums [1] are complete (zeroed by the recovery kernel)
   int* status;
-  const int* row_order;               // P: the rows in the order the kernel takes them (the default recovery rows first)
-  // optimistic decode: the default recovery rows are the first opt_rows rows of the first batch; when opt_flags[0] is set the
-  // consumers also recover the aggregate of every column slice from them, exactly as the recovery kernel would
-  int opt_rows;                       // 0: never
-  const int* opt_row;                 // opt_rows: global node index of the default rows
+  // Optimistic decode.  The default recovery rows (those read when no node is corrupt: opt_rows of them, ascending) are
+  // taken first, so that they all lie in the first batch of rows; the other rows follow in ascending order.  When the
+  // device flags say so (mode 2, or mode 1 and every group of the previous decode was clean) the consumers also recover
+  // the aggregate of every column slice from them, exactly as the recovery kernel would.  The row list travels in the
+  // kernel's parameters: nothing has to come from device memory before the first loads can be issued.
+  int opt_rows;                       // 0: rows in natural order, never optimistic
+  uint16_t def_rows[kPipeRows];       // the default rows, ascending
+  int q;                              // groups (their clean flags are opt_flags[8 + g])
   const float* opt_coeff;             // opt_rows x m weights
-  const int* opt_flags;               // device flags of the optimistic decode
-  float* agg;                         // d: the aggregate (written only when the flag is set)
+  int* opt_flags;                     // [1] this pass recovered (written here), [4] mode, [8 + g] group g was clean in the last decode
+  float* agg;                         // d: the aggregate (written only when this pass recovers)
   int m;
   int64_t d;
+
+  // The row taken at position pos of the kernel's order.
+  __device__ __forceinline__ int row_at(int pos) const {
+    if (pos < opt_rows) return def_rows[pos];
+    int r = pos - opt_rows;
+    for (int j = 0; j < opt_rows; ++j)
+      if ((int)def_rows[j] <= r) ++r;
+    return r;
+  }
 };
 
 // Aggregate of one column slice from the default recovery rows (the first n_def row slots of the stage), in the recovery
@@ -408,6 +420,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   __shared__ unsigned int s_flag;
   __shared__ __align__(16) float s_opt_coeff[kPipeRows * 8];     // eight floats per default row: m weights, then zeros
   __shared__ int s_opt_shift[kPipeRows];
+  __shared__ int s_opt_on;
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + kPipeStages;
@@ -418,8 +431,10 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   const size_t stage_bytes = rows_bytes + (size_t)K * pp.slot_floats * sizeof(float);   // the rows of a batch, then f
   const int n_acc = (K + 1) * P;
   pdl_trigger();   // the locator may be scheduled early; it waits for this grid before reading the final sums
-  // the vectors of draw n live in the buffer n & 1; the count moves on only after this kernel has completed
-  const float* __restrict__ f = (draw[0] & 1ULL) ? f_odd : f_even;
+  // the vectors of draw n live in the buffer n & 1 (the count moves on only after this kernel has completed); when the
+  // host knows which buffer that is it passes it as f_even and no count
+  const float* __restrict__ f = f_even;
+  if (draw != nullptr) f = (draw[0] & 1ULL) ? f_odd : f_even;
   if (tid == 0) {
     for (int s = 0; s < kPipeStages; ++s) {
       pipe::mbar_init(&full_bar[s], 32);
@@ -428,16 +443,20 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
     *abort_flag = 0;
     pipe::fence_barrier_init();
   }
-  // optimistic decode (float32 plans): this pass also recovers the aggregate from the default rows
-  bool opt = false;
+  __syncthreads();
+  // Optimistic decode (float32 plans): does this pass also recover the aggregate from the default rows?  Mode 2, or mode
+  // 1 and every group clean in the previous decode.  The flags are fetched here by the first consumer warp and looked at
+  // only when the first stage's projection work is done (see below), so that their round trip to device memory hides
+  // behind it.  CTA 0 records the answer for this decode's recovery kernel (0 until it is known).
+  int opt_mode = 0, opt_clean = 1;
   if constexpr (sizeof(T) == 4) {
-    opt = pp.opt_rows > 0 && pp.opt_flags[0] != 0;
-    if (opt) {
-      for (int i = tid; i < pp.opt_rows * 8; i += kPipeThreads) s_opt_coeff[i] = (i & 7) < pp.m ? pp.opt_coeff[(i >> 3) * pp.m + (i & 7)] : 0.0f;
-      for (int j = tid; j < pp.opt_rows; j += kPipeThreads) s_opt_shift[j] = (int)((((int64_t)pp.opt_row[j] & 3) * (d_c & 3)) & 3);
+    if (tid < 32 && pp.opt_rows > 0) {
+      opt_mode = pp.opt_flags[4];
+      opt_clean = tid < pp.q ? pp.opt_flags[8 + tid] : 1;            // q <= 32 for plans with default rows
     }
   }
-  __syncthreads();
+  if (blockIdx.x == 0 && tid == 0) pp.opt_flags[1] = 0;
+  bool opt = false, opt_resolved = false;
 
   const int64_t c_begin = (int64_t)blockIdx.x * range_len;     // multiple of 4
   int64_t c_end = c_begin + range_len;
@@ -459,6 +478,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
       const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
       for (int b0 = 0; b0 < P && lo < hi; b0 += pp.batch_rows) {
         const int nb = min(pp.batch_rows, P - b0);
+        const int lane_row = lane < nb ? pp.row_at(b0 + lane) : 0;
         for (int64_t c0 = lo; c0 < hi; c0 += pp.slice_cols, ++it) {
           const int stage = it % kPipeStages;
           const uint32_t phase = (it / kPipeStages) & 1;
@@ -469,7 +489,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           const T* row_src = nullptr;
           T* slot = reinterpret_cast<T*>(stage_base) + (size_t)lane * pp.slot_floats;
           if (lane < nb) {
-            const int64_t first = (int64_t)pp.row_order[b0 + lane] * d_c + c0;
+            const int64_t first = (int64_t)lane_row * d_c + c0;
             const int64_t last = first + cols;
             const int64_t a0 = first & ~(kVec - 1);                   // enclosing 16-byte boundary
             int64_t a1 = (last + kVec - 1) & ~(kVec - 1);
@@ -507,7 +527,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
         int shift[4], row_of[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          row_of[j] = j < nr ? pp.row_order[b0 + warp + 8 * j] : 0;
+          row_of[j] = j < nr ? pp.row_at(b0 + warp + 8 * j) : 0;
           shift[j] = (int)(((row_of[j] & (kVec - 1)) * dc_mod4) & (kVec - 1));   // (row * d_c + c0) mod (elements per 16 bytes)
         }
         double rho[4][K], nu[4];
@@ -532,6 +552,26 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           if constexpr (sizeof(T) == 4) {
+            if (pp.opt_rows > 0 && b0 == 0 && !opt_resolved) {
+              // first stage of this CTA: the flags have long arrived; all consumer warps pass here together
+              if (tid < 32) {
+                const bool all_clean = __all_sync(0xffffffffu, opt_clean != 0);
+                if (tid == 0) {
+                  s_opt_on = (opt_mode == 2 || (opt_mode == 1 && all_clean)) ? 1 : 0;
+                  if (blockIdx.x == 0) pp.opt_flags[1] = s_opt_on;
+                }
+              }
+              pipe::named_barrier_sync(1, kPipeConsumers);
+              opt = s_opt_on != 0;
+              if (opt) {
+                for (int i = tid; i < pp.opt_rows * 8; i += kPipeConsumers)
+                  s_opt_coeff[i] = (i & 7) < pp.m ? pp.opt_coeff[(i >> 3) * pp.m + (i & 7)] : 0.0f;
+                for (int j = tid; j < pp.opt_rows; j += kPipeConsumers)
+                  s_opt_shift[j] = (int)((((int64_t)pp.def_rows[j] & 3) * (d_c & 3)) & 3);
+                pipe::named_barrier_sync(1, kPipeConsumers);
+              }
+              opt_resolved = true;
+            }
             if (opt && b0 == 0) {
               const float* rows0 = reinterpret_cast<const float*>(base);
               switch (pp.m) {
@@ -596,17 +636,18 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   ProjPipe pp;
   pp.status = plan->d_status;
   pp.progress = plan->d_proj_progress;
-  pp.row_order = plan->d_row_order;
   // optimistic decode: only in the whole decode (the aggregate's buffer is known) of a float32 plan that is eligible
   pp.opt_rows = (!final_reduce && agg && sizeof(T) == 4 && plan->optimistic != 0) ? plan->opt_rows : 0;
-  pp.opt_row = plan->d_opt_row;
+  for (int j = 0; j < kPipeRows; ++j) pp.def_rows[j] = j < pp.opt_rows ? (uint16_t)plan->opt_row_host[(size_t)j] : 0;
+  pp.q = plan->q;
   pp.opt_coeff = plan->d_opt_coeff;
   pp.opt_flags = plan->d_opt;
   pp.agg = reinterpret_cast<float*>(agg);
   pp.m = plan->m;
   pp.d = plan->d;
   // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
-  const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128;
+  // (the kernel's static shared memory - the optimistic decode's weights - is 1.2 KB)
+  const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128 - 1536;
   const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
   pp.batch_rows = (plan->P + n_batches - 1) / n_batches;
   int slice = (int)(per_cta / ((size_t)kPipeStages * (pp.batch_rows * sizeof(T) + K * sizeof(float)))) - 8;
@@ -628,8 +669,12 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   const bool two_parts = !final_reduce && uses_early_locator(plan) && !early_locator_starved(plan);
   pp.part_a_cols = two_parts ? a_slices * slice : 0;
   const size_t smem = 128 + (size_t)kPipeStages * (pp.batch_rows * sizeof(T) + K * sizeof(float)) * pp.slot_floats;
+  // which buffer holds the current draw: known on the host while decodes do not draw (the count then stands still)
+  const bool host_knows = !plan->fresh_f && plan->draw_parity >= 0;
+  const float* f_first = host_knows ? (plan->draw_parity ? plan->d_f2 : plan->d_f) : plan->d_f;
+  const unsigned long long* draw_count = host_knows ? nullptr : plan->d_draw;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(project_pipe_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  project_pipe_kernel<K, T><<<grid, kPipeThreads, smem, plan->stream>>>(received, plan->d_f, plan->d_f2, plan->d_draw, plan->f_pitch, plan->P, plan->d_c,
+  project_pipe_kernel<K, T><<<grid, kPipeThreads, smem, plan->stream>>>(received, f_first, plan->d_f2, draw_count, plan->f_pitch, plan->P, plan->d_c,
                                                                      range_len, pp, plan->d_partials, rho_out, nu_out,
                                                                      plan->d_proj_ticket, final_reduce);
   const int n_bunches = (grid + kProjBunch - 1) / kProjBunch;

@@ -24,7 +24,7 @@ struct RecoverParamsT {
   const int* rec_rows;   // P, group g's rows at [group_start[g], +n_rec[g])
   const double* coeff;   // P x m, same indexing
   unsigned long long* proj_progress;   // the projection kernel's part-A count, zeroed here for the next decode
-  const int* opt;        // optimistic decode: opt[1] != 0 - the projection pass has already written the aggregate
+  const int* opt;        // optimistic decode: opt[1] - the projection pass of this decode recovered too; opt[8 + g] - group g is clean
 };
 typedef RecoverParamsT<float> RecoverParams;
 
@@ -112,14 +112,15 @@ struct RecoverPipe {
   int slot_floats;   // shared-memory floats per row slot (multiple of 4)
   unsigned long long* tile_counter;   // next tile to hand out; zero at launch
   int* status;
-  int stream_hints;   // write the aggregate with streaming stores (evict-first in L2)
 };
 
 // Streaming kernel: a producer warp moves the selected rows, tile by tile and a few rows at a time, into a
 // shared-memory ring with bulk asynchronous copies; consumer threads own CPT chunks each, take one float per
 // row from the ring, apply the row's m weights, and every consumer warp writes its runs of chunks back
 // through its own shared buffer as contiguous 128-bit stores.
-template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T>
+// kStreamStores: write the aggregate with streaming stores (evict-first in L2; a template parameter, not a run-time
+// branch: with both forms in one kernel the compiler kept 94 registers instead of 72 and the kernel ran 7 - 40 % longer).
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T, bool kStreamStores>
 __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverParamsT<T> prm, RecoverPipe pp) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int kTileChunks = NC * CPT;
@@ -157,8 +158,12 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
     prm.proj_progress[0] = 0ULL;
     prm.proj_progress[1] = 0ULL;
   }
-  if (prm.opt[1] != 0) return;   // every group's default rows were confirmed and the projection pass recovered from them
+  // optimistic decode: the projection pass has already written the aggregate, and it stands if every group is clean
+  // (no branch on the first word before the other loads: they all go out together with the table loads below)
+  int clean = prm.opt[1] != 0 ? 1 : 0;
+  for (int g = tid; g < prm.q; g += blockDim.x) clean &= prm.opt[8 + g] != 0 ? 1 : 0;
   const int n_rows = pack_tables<Acc, M, kStride, (int)kVec>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c);
+  if (__syncthreads_and(clean)) return;   // every group's default rows were confirmed and the projection pass recovered from them
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
 
@@ -280,7 +285,7 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
       const int vec = count / (int)kVec;                          // whole 16-byte words
       float4* dst4 = reinterpret_cast<float4*>(prm.agg + o0);
       const float4* src4 = reinterpret_cast<const float4*>(out_s);
-      if (pp.stream_hints) {
+      if constexpr (kStreamStores) {
         for (int e = lane; e < vec; e += 32) __stcs(dst4 + e, src4[e]);
         for (int e = vec * (int)kVec + lane; e < count; e += 32) __stcs(prm.agg + o0 + e, out_s[e]);
       } else {
@@ -317,12 +322,11 @@ __global__ void __launch_bounds__(kRecThreads) recover_generic_kernel(RecoverPar
   }
 }
 
-template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T>
-static int launch_recover_m(solon_plan* plan, RecoverParamsT<T>& prm) {
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T, bool kStreamStores>
+static int launch_recover_hint(solon_plan* plan, RecoverParamsT<T>& prm) {
   constexpr int kTileChunks = NC * CPT;
   RecoverPipe pp;
   pp.status = plan->d_status;
-  pp.stream_hints = plan->stream_hints;
   pp.slot_floats = kTileChunks + 8;
   const size_t slot_bytes = (size_t)pp.slot_floats * sizeof(T);
   const size_t fixed = 256 + recover_coeff_bytes(plan->P, M) + recover_coeff_bytes(plan->P, PackedStride<Acc, M>::value) +
@@ -354,7 +358,7 @@ static int launch_recover_m(solon_plan* plan, RecoverParamsT<T>& prm) {
   if (smem > (size_t)226 * 1024) return SOLON_ERR_INVALID_ARG;
   pp.row_batch = row_batch;
   pp.stages = stages;
-  auto kernel = recover_kernel<M, CPT, Acc, NC, kCtasPerSm, T>;
+  auto kernel = recover_kernel<M, CPT, Acc, NC, kCtasPerSm, T, kStreamStores>;
   SOLON_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   static_assert((32 * M * sizeof(T)) % 16 == 0, "warp runs must start on a 16-byte boundary of the output");
   int64_t tiles = (plan->d_c + kTileChunks - 1) / kTileChunks;
@@ -365,6 +369,12 @@ static int launch_recover_m(solon_plan* plan, RecoverParamsT<T>& prm) {
   int grid = (int)(tiles < cap ? tiles : cap);
   pp.tile_counter = plan->d_tile_counter;
   return launch_dependent(kernel, dim3(grid), dim3((NC + 32)), smem, plan->stream, prm, pp);
+}
+
+template <int M, int CPT, typename Acc, int NC, int kCtasPerSm, typename T>
+static int launch_recover_m(solon_plan* plan, RecoverParamsT<T>& prm) {
+  if (plan->stream_hints) return launch_recover_hint<M, CPT, Acc, NC, kCtasPerSm, T, true>(plan, prm);
+  return launch_recover_hint<M, CPT, Acc, NC, kCtasPerSm, T, false>(plan, prm);
 }
 
 template <typename T>

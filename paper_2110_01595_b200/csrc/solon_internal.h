@@ -76,11 +76,11 @@ struct solon_plan {
   // rows that are read when no node is corrupt, and the recovery kernel is skipped when the locator confirms them
   int optimistic;          // 0 never, 1 after a decode that found every node honest (default), 2 always
   int opt_rows;            // number of default rows over all groups (0: the plan is not eligible)
-  int* d_row_order;        // P: order in which the projection kernel takes the rows (default rows first)
-  int* d_opt_row;          // opt_rows: the default rows (global node index), group by group
+  std::vector<int> opt_row_host;   // the default rows (global node index), ascending
   float* d_opt_coeff;      // opt_rows x m: their weights, as the recovery kernel would use them
-  int* d_opt;              // [0] next projection pass recovers too, [1] the recovery kernel may skip, [2] clean groups, [3] ticket,
-                           // [4] mode (copied from `optimistic`)
+  int* d_opt;              // [1] the projection pass of this decode recovered too, [4] mode (copied from `optimistic`),
+                           // [8 + g] group g had no corrupt node in the last decode
+  int draw_parity;         // which buffer holds the current draw of f (0, 1), or -1: only the device knows (decodes draw anew)
   float* d_f;              // K x f_pitch projection vectors: the draws with an even index
   float* d_f2;             // the draws with an odd index
   int last_decode_advanced;    // the most recent decode drew new vectors for the next one (the count is one ahead of what it used)
@@ -190,12 +190,15 @@ inline bool uses_early_locator(const solon_plan* plan) {
 inline bool early_locator_starved(const solon_plan* plan) { return plan->early_locator == 3; }
 
 // Between two decodes the encode step and the recovery move gigabytes through L2 and push out everything else - the
-// locator kernel's instructions included, whose re-fetch from device memory (about a microsecond per 128 bytes of
-// code) is most of a short decode's serial time.  When every streamed byte is marked evict-first the code survives
-// in L2 and the locator runs about a third shorter (33 -> 25 us on 15 nodes); a single unmarked stream undoes it.
-// The marks cost the encode kernel 2-4 % of its bandwidth, which only pays while the step is short: up to 1 GB of
-// gradients per step.
-inline bool keeps_l2_for_code(int P, int64_t d) { return (double)P * (double)d * 4.0 <= 1.0e9; }
+// locator kernel's instructions and tables included, whose re-fetch from device memory (about a microsecond per 128
+// bytes of code) is most of a short decode's serial time.  When every streamed byte is marked evict-first the code
+// survives in L2; a single unmarked stream undoes it.  The marks have a price: the encode kernel loses 2-4 % of its
+// bandwidth, the recovery kernel's streaming stores are slower than plain ones (33 -> 41 us at m = 2, 49 -> 70 us at
+// m = 1 on 15 nodes x 10 M), and the coded matrix no longer lingers in L2 for the projection pass of a decode that
+// follows an encode.  Measured per case (same box, switch in the environment): worth it where the locator is long
+// and the streams are short - m > 6 (all-rows recovery tables, 89 -> 67 us per decode on 15 nodes x 10 M at m = 10) -
+// and a wash or a loss for m <= 6.  So: m > 6 and at most 1 GB of gradients per step.
+inline bool keeps_l2_for_code(int P, int m, int64_t d) { return m > 6 && (double)P * (double)d * 4.0 <= 1.0e9; }
 
 int launch_fill_projection(solon_plan* plan, int advance);   // advance = 1: the next draw (device-side count), 0: redo the current one
 int launch_encode(solon_plan* plan, const float* grads, float* coded);

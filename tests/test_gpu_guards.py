@@ -41,17 +41,22 @@ def _built():
     (33, 2, 4, 8, 65_537),      # four groups, one of nine
     (40, 2, 12, 20, 3_001),     # m = 12 (generic kernels)
 ])
-def test_outputs_stay_inside_their_buffers_and_inputs_are_not_written(P, s, m, r, d):
+@pytest.mark.parametrize("dtype", ["f32", "f64"])
+def test_outputs_stay_inside_their_buffers_and_inputs_are_not_written(P, s, m, r, d, dtype):
+    if dtype == "f64" and m == 7:
+        pytest.skip("no float64 kernel for m = 7")
     wl = synth.Workload("guard", P, s, m, d, "normal", 1.0, "gaussian", s, 60 + P + m)
     G = synth.make_grads(wl, "cuda")
+    tdtype, eb = (torch.float64, 8) if dtype == "f64" else (torch.float32, 4)
+    G = G.to(tdtype)
     G_before = G.clone()
-    with binding.Plan(P, s, m, r, d, seed=9) as plan:
+    with binding.Plan(P, s, m, r, d, seed=9, dtype=dtype) as plan:
         d_c = plan.d_c
-        coded_whole, coded_bytes = _guarded(P * d_c * 4)
-        coded = coded_bytes.view(torch.float32).view(P, d_c)
+        coded_whole, coded_bytes = _guarded(P * d_c * eb)
+        coded = coded_bytes.view(tdtype).view(P, d_c)
         plan.encode(G, coded)
         torch.cuda.synchronize()
-        assert _guards_intact(coded_whole, P * d_c * 4)
+        assert _guards_intact(coded_whole, P * d_c * eb)
         assert torch.equal(G, G_before)
         fresh = plan.encode(G)                                            # every entry was written: equal to an encode into an ordinary buffer
         assert torch.equal(coded, fresh)
@@ -61,13 +66,13 @@ def test_outputs_stay_inside_their_buffers_and_inputs_are_not_written(P, s, m, r
         if nodes:
             received[nodes] = synth.byzantine_rows(wl, coded, nodes)
         received_before = received.clone()
-        agg_whole, agg_bytes = _guarded(d * 4)
+        agg_whole, agg_bytes = _guarded(d * eb)
         mask_whole, mask_bytes = _guarded(P)
-        agg = agg_bytes.view(torch.float32)
+        agg = agg_bytes.view(tdtype)
         plan.decode(received, agg, mask_bytes)
         status = plan.decode_status()
         assert status == 0, binding.strerror(status)
-        assert _guards_intact(agg_whole, d * 4) and _guards_intact(mask_whole, P)
+        assert _guards_intact(agg_whole, d * eb) and _guards_intact(mask_whole, P)
         assert torch.equal(received, received_before)
         assert mask_bytes.nonzero().flatten().tolist() == nodes
         agg2, mask2 = plan.decode(received)

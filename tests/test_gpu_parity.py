@@ -414,6 +414,29 @@ def test_a_replayed_graph_of_a_decode_draws_new_vectors_each_time():
         assert not np.array_equal(seen[0], seen[1]) and not np.array_equal(seen[1], seen[2]) and not np.array_equal(seen[0], seen[2])
 
 
+def test_plan_status_after_encode_and_argument_errors_leave_the_plan_usable():
+    """solon_plan_status reports the sticky wait-expired bit without a decode (OK here: no wait ever runs out), and calls
+    refused for their arguments enqueue nothing: the next decode is unaffected."""
+    wl = synth.small_variant(synth.WORKLOADS["vgg13"], 120_000)
+    G = synth.make_grads(wl, "cuda")
+    want = so.plain_sum(G.cpu().numpy())
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d) as plan:
+        coded = plan.encode(G)
+        assert plan.status() == binding.OK
+        received, nodes = synth.apply_attack(wl, coded)
+        from ctypes import c_void_p
+        lib = binding.lib()
+        agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+        mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
+        assert lib.solon_decode(plan._h, c_void_p(received.data_ptr()), c_void_p(agg.data_ptr()), c_void_p(0)) == binding.ERR_INVALID_ARG
+        assert lib.solon_decode(plan._h, c_void_p(received.data_ptr() + 4), c_void_p(agg.data_ptr()), c_void_p(mask.data_ptr())) == binding.ERR_INVALID_ARG
+        for _ in range(2):
+            plan.decode(received, agg, mask)
+            assert plan.decode_status() == 0 and plan.status() == binding.OK
+            assert mask.nonzero().flatten().tolist() == nodes
+            assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * np.abs(want).max()
+
+
 def test_projection_settings():
     wl = synth.small_variant(synth.WORKLOADS["resnet18"], 60_000)
     G = synth.make_grads(wl, "cuda")
