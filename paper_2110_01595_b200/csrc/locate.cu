@@ -53,7 +53,8 @@ struct LocateParams {
   int* rec_rows;         // P
   double* coeff;         // P x m
   int* status;
-  int* opt;              // optimistic decode: opt[8 + g] receives whether group g had no corrupt node
+  int* opt;              // optimistic decode: opt[8 + g] receives whether the rows of group g's previous recovery table are trusted now
+  int opt_track;         // the plan can decode optimistically (m <= 6): keep opt[8 + g] (else it is written as 0)
   DrawParams draw;       // the vectors f of the next decode, written by the CTAs beyond the q locator CTAs (n_draw_ctas of them)
   int n_draw_ctas;
 };
@@ -127,6 +128,18 @@ __device__ __forceinline__ unsigned long long pipe_timer_ns() {
   return t;
 }
 
+// Optimistic decode: 1 if the m rows of the group's previous recovery table are all trusted by this decode's mask (then an
+// aggregate recovered from them is this decode's aggregate, and the table would have served this decode too).
+__device__ __forceinline__ int old_rows_trusted(const LocateParams& prm, const int* old_row, int old_n, int t_acc, const uint8_t* mask_l,
+                                                int row0, int n) {
+  if (!prm.opt_track || t_acc < 0 || old_n != prm.m) return 0;
+  for (int j = 0; j < prm.m; ++j) {
+    const int k = old_row[j] - row0;
+    if (k < 0 || k >= n || mask_l[k]) return 0;
+  }
+  return 1;
+}
+
 constexpr int kGatherBatch = 20;   // bunch sums fetched at once per column (the projection kernel leaves 37 on 148 SMs: two rounds)
 
 __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocateParams prm) {
@@ -147,6 +160,13 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   double* ws = prm.use_smem ? smem_ws : prm.ws_global + (size_t)g * prm.ws_stride;
   GroupScratch sc = carve(ws, n, prm.m, prm.K, prm.s);
   __shared__ int s_n_rec, s_t_acc;
+  // Optimistic decode: the rows of this group's recovery table as the previous decode left it - the rows the projection
+  // kernel of THIS decode may have recovered from - are read before anything here overwrites them.
+  __shared__ int s_old_row[SOLON_SUBSET_MAX_M], s_old_n;
+  if (prm.opt_track) {
+    if (tid < prm.m) s_old_row[tid] = prm.rec_rows[row0 + tid];
+    if (tid == 0) s_old_n = prm.n_rec[g];
+  }
   GroupTables tb;
   tb.Qb = prm.qb + prm.qb_off[g];
   tb.Hm = prm.hm + prm.qb_off[g];
@@ -296,7 +316,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
           prm.n_rec[g] = n_rec;
           prm.t_acc[g] = s_t_acc;
           prm.early[g] = 1;
-          prm.opt[8 + g] = s_t_acc == 0 ? 1 : 0;      // optimistic decode: this group had no corrupt node
+          prm.opt[8 + g] = old_rows_trusted(prm, s_old_row, s_old_n, s_t_acc, sc.mask_l, row0, n);
         }
         return;
       }
@@ -348,7 +368,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
       prm.early[g] = !prm.spec ? 0 : (s_ready > 0 ? 2 : (s_ready == 0 ? 3 : 4));
-      prm.opt[8 + g] = s_t_acc == 0 ? 1 : 0;      // optimistic decode: this group had no corrupt node
+      prm.opt[8 + g] = old_rows_trusted(prm, s_old_row, s_old_n, s_t_acc, sc.mask_l, row0, n);
       (void)ok;      // an undecodable group is reported through t_acc[g] = -1
     }
   }
@@ -419,6 +439,14 @@ void build_group_tables(int n, int m, int s, const double* w, double* Qb, double
     }
   for (int k = 0; k < n; ++k)
     for (int i = 0; i <= s; ++i) Tch[(size_t)k * (s + 1) + i] = i < n ? (double)T[(size_t)i * n + k] : 0.0;
+}
+
+// Recovery table of one group when every node is trusted (host, once per plan): what the locator writes after a decode
+// that found no corrupt node.  rows: n ints, coeff: n x m doubles; returns the rows in use.
+int clean_recovery_table(int n, int m, int s, const GroupTables& tb, int* rows, double* coeff) {
+  std::vector<uint8_t> trusted((size_t)n, 1);
+  std::vector<double> ws(locate_epilogue_ws_doubles(n, m, s) + 8);
+  return recovery_table(Team::serial(), tb, n, m, s, trusted.data(), rows, coeff, ws.data());
 }
 
 // Recovery tables of one group for every set of at most s untrusted nodes (host, once per plan): entry
@@ -513,6 +541,7 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
   if (smem > 48 * 1024)
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prm.opt = plan->d_opt;
+  prm.opt_track = plan->opt_rows > 0 ? 1 : 0;
   // CTAs that draw the next decode's vectors beside the locator's: a few per SM, a thread per several quads
   prm.draw = draw_params(plan);
   prm.n_draw_ctas = 0;

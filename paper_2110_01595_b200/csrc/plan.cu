@@ -16,6 +16,7 @@ namespace solon {
 
 void build_recovery_tabs(int n, int m, int s, const GroupTables& tb, int ld, std::vector<int>* count, std::vector<int>* rows,
                          std::vector<double>* coeff);   // locate.cu
+int clean_recovery_table(int n, int m, int s, const GroupTables& tb, int* rows, double* coeff);   // locate.cu
 
 int check_params(int P, int s, int m, int r, int64_t d) {
   if (P < 1 || s < 0 || m < 1 || d < 1 || r < 1) return SOLON_ERR_INVALID_ARG;
@@ -95,7 +96,7 @@ static void free_device(solon_plan* p) {
   cudaFree(p->d_group_start); cudaFree(p->d_group_of); cudaFree(p->d_w); cudaFree(p->d_f); cudaFree(p->d_f2);
   cudaFree(p->d_qb); cudaFree(p->d_hm); cudaFree(p->d_qb_off); cudaFree(p->d_mt); cudaFree(p->d_tch);
   cudaFree(p->d_tab_count); cudaFree(p->d_tab_rows); cudaFree(p->d_tab_coeff); cudaFree(p->d_tab_off); cudaFree(p->d_tab_sets);
-  cudaFree(p->d_opt_coeff); cudaFree(p->d_opt);
+  cudaFree(p->d_opt);
   cudaFree(p->d_partials); cudaFree(p->d_rho); cudaFree(p->d_nu); cudaFree(p->d_proj_ticket);
   cudaFree(p->d_locate_ws);
   cudaFree(p->d_t_acc); cudaFree(p->d_n_rec); cudaFree(p->d_rec_rows); cudaFree(p->d_coeff); cudaFree(p->d_status); cudaFree(p->d_early); cudaFree(p->d_tile_counter); cudaFree(p->d_proj_progress); cudaFree(p->d_draw);
@@ -249,6 +250,8 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
       rc = SOLON_ERR_CUDA;
       break;
     }
+    std::vector<int> rec_rows_init((size_t)P, 0), n_rec_init((size_t)q, 0);
+    std::vector<double> coeff_init((size_t)P * m, 0.0);
     {
       // recovery tables for every set of at most s untrusted nodes, where those sets are few enough to tabulate
       std::vector<int> all_count, all_rows, count, rows;
@@ -272,39 +275,40 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
         all_coeff.insert(all_coeff.end(), coeff.begin(), coeff.end());
       }
       {
-        // Optimistic decode: the rows the recovery reads when no node is corrupt (subset form), group by group, with
-        // their weights rounded as the recovery kernel rounds them; eligible when they all fit in the projection
-        // kernel's first batch of rows, which then takes them first.
-        std::vector<int> opt_row;
-        std::vector<float> opt_coeff;
-        std::vector<uint8_t> is_default((size_t)P, 0);
+        // Optimistic decode: the projection pass may recover the aggregate from the rows the previous decode's recovery
+        // read (subset form: m per group), i.e. from the locator's last recovery table; eligible when those rows all fit
+        // in the projection kernel's first batch of rows, which then takes them first.  Before the first decode that
+        // table is the one for no corrupt node.
+        std::vector<int> opt_src;
         const int n_batches = (P + 31) / 32;
         const int batch_rows = (P + n_batches - 1) / n_batches;
         bool eligible = dtype == SOLON_F32 && s > 0 && m <= SOLON_SUBSET_MAX_M && q * m <= batch_rows;
+        std::vector<int> rows_g((size_t)max_group);
+        std::vector<double> coeff_g((size_t)max_group * m);
         for (int g = 0; g < q && eligible; ++g) {
-          if (tab_sets[g] == 0) { eligible = false; break; }
-          const size_t first = (size_t)tab_off[g];             // the empty corrupt set is entry 0 of the group
+          const int n_g = start[g + 1] - start[g];
+          GroupTables tb = {};
+          tb.Qb = h_qb.data() + qb_off[g];
+          tb.Hm = h_hm.data() + qb_off[g];
+          tb.Mt = h_mt.data() + (size_t)g * m * m;
+          tb.Tch = h_tch.data() + (size_t)start[g] * (s + 1);
+          tb.w = p->w.data() + start[g];
+          if (clean_recovery_table(n_g, m, s, tb, rows_g.data(), coeff_g.data()) != m) { eligible = false; break; }
+          n_rec_init[(size_t)g] = m;
           for (int j = 0; j < m; ++j) {
-            const int node = start[g] + all_rows[first * p->tab_ld + j];
-            opt_row.push_back(node);
-            is_default[(size_t)node] = 1;
-            for (int l = 0; l < m; ++l) opt_coeff.push_back((float)all_coeff[(first * p->tab_ld + j) * m + l]);
+            opt_src.push_back(start[g] + j);
+            rec_rows_init[(size_t)start[g] + j] = start[g] + rows_g[(size_t)j];
+            for (int l = 0; l < m; ++l) coeff_init[((size_t)start[g] + j) * m + l] = coeff_g[(size_t)j * m + l];
           }
         }
-        if (!eligible) {
-          opt_row.clear();
-          opt_coeff.clear();
-          is_default.assign((size_t)P, 0);
-        }
-        p->opt_rows = (int)opt_row.size();
-        p->opt_row_host = opt_row;
+        if (!eligible) opt_src.clear();
+        p->opt_rows = (int)opt_src.size();
+        p->opt_src_host = opt_src;
         p->optimistic = 1;
-        if ((rc = dev_alloc(&p->d_opt_coeff, opt_coeff.size()))) break;
         if ((rc = dev_alloc(&p->d_opt, (size_t)8 + q))) break;
         std::vector<int> opt_init((size_t)8 + q, 0);
         opt_init[4] = p->optimistic;
-        if ((!opt_coeff.empty() && cudaMemcpy(p->d_opt_coeff, opt_coeff.data(), opt_coeff.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) ||
-            cudaMemcpy(p->d_opt, opt_init.data(), opt_init.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
+        if (cudaMemcpy(p->d_opt, opt_init.data(), opt_init.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
           (void)cudaGetLastError();
           rc = SOLON_ERR_CUDA;
           break;
@@ -332,6 +336,13 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
     if ((rc = dev_alloc(&p->d_n_rec, q))) break;
     if ((rc = dev_alloc(&p->d_rec_rows, P))) break;
     if ((rc = dev_alloc(&p->d_coeff, (size_t)P * m))) break;
+    if (cudaMemcpy(p->d_n_rec, n_rec_init.data(), (size_t)q * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(p->d_rec_rows, rec_rows_init.data(), (size_t)P * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(p->d_coeff, coeff_init.data(), coeff_init.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess) {
+      (void)cudaGetLastError();
+      rc = SOLON_ERR_CUDA;
+      break;
+    }
     if ((rc = dev_alloc(&p->d_status, 2))) break;
     if ((rc = dev_alloc(&p->d_tile_counter, 4))) break;
     if ((rc = dev_alloc(&p->d_early, (size_t)q))) break;

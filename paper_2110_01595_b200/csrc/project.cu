@@ -232,65 +232,103 @@ struct ProjPipe {
   int64_t part_a_cols;                // columns of part A in every CTA's range (whole slices)
   unsigned long long* progress;       // bunches whose part-A sums [0] and final sums [1] are complete (zeroed by the recovery kernel)
   int* status;
-  // Optimistic decode.  The default recovery rows (those read when no node is corrupt: opt_rows of them, ascending) are
-  // taken first, so that they all lie in the first batch of rows; the other rows follow in ascending order.  When the
-  // device flags say so (mode 2, or mode 1 and every group of the previous decode was clean) the consumers also recover
-  // the aggregate of every column slice from them, exactly as the recovery kernel would.  The row list travels in the
-  // kernel's parameters: nothing has to come from device memory before the first loads can be issued.
+  // Optimistic decode.  The rows of the locator's last recovery table (m per group: what the previous decode's recovery
+  // read; opt_rows of them over all groups, ascending) are the ones this decode speculates on.  When the device flags say
+  // so (mode 2, or mode 1 and the previous decode's flags all set) the consumers also recover the aggregate of every
+  // column slice from them, exactly as the recovery kernel would with that table.  They must all lie in one stage of the
+  // ring: with a single batch of rows the order stays the natural one and nothing has to come from device memory before
+  // the first loads are issued; with several batches they are taken first (the other rows follow in ascending order),
+  // and the kernel starts by fetching the list.
   int opt_rows;                       // 0: rows in natural order, never optimistic
-  uint16_t def_rows[kPipeRows];       // the default rows, ascending
-  int q;                              // groups (their clean flags are opt_flags[8 + g])
-  const float* opt_coeff;             // opt_rows x m weights
-  int* opt_flags;                     // [1] this pass recovered (written here), [4] mode, [8 + g] group g was clean in the last decode
+  int multi_batch;                    // more than one batch of rows
+  int opt_ch;                         // chunks per consumer thread and pass of the recovery (1..4): slice_cols is a multiple of 256 opt_ch
+  uint16_t spec_src[kPipeRows];       // positions of those rows in rec_rows and rec_coeff: group_start[g] + j, j < m
+  int q;                              // groups (their flags are opt_flags[8 + g])
+  const int* rec_rows;                // P: the locator's last recovery table (rows as node indices, per group from group_start[g])
+  const double* rec_coeff;            // P x m: its weights
+  const int* n_rec;                   // q: rows in use per group (m after a decode that succeeded)
+  int* opt_flags;                     // [1] this pass recovered (written here), [4] mode, [8 + g] see the locator kernel
   float* agg;                         // d: the aggregate (written only when this pass recovers)
   int m;
   int64_t d;
-
-  // The row taken at position pos of the kernel's order.
-  __device__ __forceinline__ int row_at(int pos) const {
-    if (pos < opt_rows) return def_rows[pos];
-    int r = pos - opt_rows;
-    for (int j = 0; j < opt_rows; ++j)
-      if ((int)def_rows[j] <= r) ++r;
-    return r;
-  }
 };
 
-// Aggregate of one column slice from the default recovery rows (the first n_def row slots of the stage), in the recovery
-// kernel's arithmetic and order: acc = fma(weight, value, acc) over the rows, group by group.  A thread owns chunks
-// tid, tid + 256, tid + 512, tid + 768 of each 1024 and shares a row's weights (eight floats per row in shared memory,
-// fetched with two 128-bit loads) between them.
+// The row taken at position pos of the kernel's order: the n_first rows of first_rows (ascending), then all others in
+// ascending order.
+__device__ __forceinline__ int pipe_row_at(int pos, int n_first, const int* first_rows) {
+  if (pos < n_first) return first_rows[pos];
+  int r = pos - n_first;
+  for (int j = 0; j < n_first; ++j)
+    if (first_rows[j] <= r) ++r;
+  return r;
+}
+
+// Two float32 values in one 64-bit register, and the packed fused multiply-add of sm_100 (fma.rn.f32x2: each half is an
+// ordinary IEEE fma.rn, so results equal those of two scalar instructions bit for bit, in one issue slot).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+
+// Aggregate of one column slice from the n_def rows speculated on (row j starts s_off[j] floats into the stage), in the
+// recovery kernel's arithmetic and order: acc = fma(weight, value, acc) over the rows, group by group.  A lane owns the
+// chunks c + i * 256, i < ch, of each 256 ch, two chunks to a packed multiply-add, and shares a row's weights (eight
+// pairs (w_l, w_l) per row in shared memory, fetched with 128-bit loads) between them; it writes each chunk's m floats
+// itself (routing them through shared memory into 128-bit stores, as the recovery kernel does, made this kernel 20 %
+// slower: its consumer warps are bound by instruction issue).
 constexpr int kOptChunks = 4;
 template <int M>
-__device__ __forceinline__ void opt_recover_slice(const float* base, int slot_floats, const int* s_shift, const float* s_coeff, int n_def,
-                                                  int cols, int64_t c0, float* __restrict__ agg, int64_t d, int tid) {
-  for (int c = tid; c < cols; c += kOptChunks * kPipeConsumers) {
-    float acc[kOptChunks][M];
+__device__ __forceinline__ void opt_recover_slice(const float* base, const int* s_off, const f32x2* s_coeff2, int n_def,
+                                                  int cols, int ch, int64_t c0, float* __restrict__ agg, int64_t d, int warp, int lane) {
+  // ch (1..4): chunks per lane and pass; the slice width is a multiple of 256 ch, so that every pass but the one at the
+  // ragged end of a range keeps all lanes busy
+  for (int cb = warp * 32; cb < cols; cb += ch * kPipeConsumers) {
+    const int c = cb + lane;
+    f32x2 acc[kOptChunks / 2][M];
 #pragma unroll
-    for (int i = 0; i < kOptChunks; ++i)
+    for (int h = 0; h < kOptChunks / 2; ++h)
 #pragma unroll
-      for (int l = 0; l < M; ++l) acc[i][l] = 0.0f;
+      for (int l = 0; l < M; ++l) acc[h][l] = 0ULL;          // (+0.0f, +0.0f)
     for (int j = 0; j < n_def; ++j) {
-      const float* row = base + (size_t)j * slot_floats + s_shift[j];
+      const float* row = base + s_off[j];
+      f32x2 w[(M + 1) / 2 * 2];
+#pragma unroll
+      for (int t = 0; t < (M + 1) / 2; ++t) {
+        const ulonglong2 ww = *reinterpret_cast<const ulonglong2*>(s_coeff2 + j * 8 + 2 * t);
+        w[2 * t] = ww.x;
+        w[2 * t + 1] = ww.y;
+      }
       float v[kOptChunks];
 #pragma unroll
-      for (int i = 0; i < kOptChunks; ++i) v[i] = c + i * kPipeConsumers < cols ? row[c + i * kPipeConsumers] : 0.0f;
-      const float4 w0 = *reinterpret_cast<const float4*>(s_coeff + j * 8);
-      const float4 w1 = *reinterpret_cast<const float4*>(s_coeff + j * 8 + 4);
-      const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+      for (int i = 0; i < kOptChunks; ++i) v[i] = (i < ch && c + i * kPipeConsumers < cols) ? row[c + i * kPipeConsumers] : 0.0f;
 #pragma unroll
-      for (int l = 0; l < M; ++l)
+      for (int h = 0; h < kOptChunks / 2; ++h) {
+        if (2 * h < ch) {
+          const f32x2 vv = pack2(v[2 * h], v[2 * h + 1]);
 #pragma unroll
-        for (int i = 0; i < kOptChunks; ++i) acc[i][l] = fmaf(w[l], v[i], acc[i][l]);
+          for (int l = 0; l < M; ++l) acc[h][l] = fma2(w[l], vv, acc[h][l]);
+        }
+      }
     }
 #pragma unroll
     for (int i = 0; i < kOptChunks; ++i) {
-      const int ci = c + i * kPipeConsumers;
-      if (ci < cols) {
+      const int ci = cb + i * kPipeConsumers + lane;
+      if (i < ch && ci < cols) {
         const int64_t o = (c0 + ci) * M;
 #pragma unroll
-        for (int l = 0; l < M; ++l)
-          if (o + l < d) __stcs(agg + o + l, acc[i][l]);
+        for (int l = 0; l < M; ++l) {
+          float lo, hi;
+          unpack2(acc[i / 2][l], lo, hi);
+          if (o + l < d) __stcs(agg + o + l, (i & 1) ? hi : lo);
+        }
       }
     }
   }
@@ -418,9 +456,10 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
                                                                      unsigned int* ticket, int final_reduce) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ unsigned int s_flag;
-  __shared__ __align__(16) float s_opt_coeff[kPipeRows * 8];     // eight floats per default row: m weights, then zeros
-  __shared__ int s_opt_shift[kPipeRows];
-  __shared__ int s_opt_on;
+  __shared__ __align__(16) f32x2 s_opt_coeff[kPipeRows * 8];     // eight pairs per speculated row: (w_l, w_l) for l < m, then zeros
+  __shared__ int s_opt_off[kPipeRows];                           // where that row starts in a stage of the first batch
+  __shared__ int s_first_row[kPipeRows];                         // rows taken first (several batches of rows only)
+  __shared__ int s_n_first, s_opt_on;
   const int tid = threadIdx.x;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw);
   uint64_t* empty_bar = full_bar + kPipeStages;
@@ -443,19 +482,40 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
     *abort_flag = 0;
     pipe::fence_barrier_init();
   }
-  __syncthreads();
-  // Optimistic decode (float32 plans): does this pass also recover the aggregate from the default rows?  Mode 2, or mode
-  // 1 and every group clean in the previous decode.  The flags are fetched here by the first consumer warp and looked at
-  // only when the first stage's projection work is done (see below), so that their round trip to device memory hides
-  // behind it.  CTA 0 records the answer for this decode's recovery kernel (0 until it is known).
-  int opt_mode = 0, opt_clean = 1;
+  // Optimistic decode (float32 plans): does this pass also recover the aggregate, from the rows of the last recovery table?
+  // Mode 2, or mode 1 and every flag of the previous decode set; and only if that table is whole (m rows in every group,
+  // ascending node indices).  Flags, rows and weights are fetched here - one load per thread - and looked at only when the
+  // first stage's projection work is done (see below), so that their round trip to device memory hides behind it; with
+  // several batches of rows the row order depends on the list, and the kernel waits for it here.  CTA 0 records the
+  // answer for this decode's recovery kernel (0 until it is known).
+  int opt_mode = 0, opt_flag = 1, spec_row = 0;      // raw values: nothing is computed from them before they are needed
+  bool spec_whole = false;
+  double spec_coeff = 0.0;
   if constexpr (sizeof(T) == 4) {
-    if (tid < 32 && pp.opt_rows > 0) {
-      opt_mode = pp.opt_flags[4];
-      opt_clean = tid < pp.q ? pp.opt_flags[8 + tid] : 1;            // q <= 32 for plans with default rows
+    if (pp.opt_rows > 0) {
+      if (tid < 32) {
+        opt_mode = pp.opt_flags[4];
+        if (tid < pp.q) opt_flag = pp.opt_flags[8 + tid];                           // q <= 32 when opt_rows > 0
+        const int rows_g = tid < pp.q ? pp.n_rec[tid] : pp.m;
+        spec_row = tid < pp.opt_rows ? pp.rec_rows[pp.spec_src[tid]] : 0x7fffffff;  // opt_rows <= 32
+        if (pp.multi_batch) {
+          const int below = __shfl_up_sync(0xffffffffu, spec_row, 1);
+          const bool lane_ok = rows_g == pp.m && (tid >= pp.opt_rows || (spec_row >= 0 && spec_row < P && (tid == 0 || spec_row > below)));
+          spec_whole = __all_sync(0xffffffffu, lane_ok);
+          s_first_row[tid] = spec_row;
+          if (tid == 0) s_n_first = spec_whole ? pp.opt_rows : 0;
+        } else {
+          spec_whole = rows_g == pp.m;      // this lane's part; completed when the flags are looked at
+        }
+      }
+      if (tid < pp.opt_rows * 8 && (tid & 7) < pp.m)                                // opt_rows * 8 <= 256 consumer threads
+        spec_coeff = pp.rec_coeff[(size_t)pp.spec_src[tid >> 3] * pp.m + (tid & 7)];
     }
   }
+  if (tid == 0 && !(sizeof(T) == 4 && pp.opt_rows > 0 && pp.multi_batch)) s_n_first = 0;
   if (blockIdx.x == 0 && tid == 0) pp.opt_flags[1] = 0;
+  __syncthreads();
+  const int n_first = s_n_first;
   bool opt = false, opt_resolved = false;
 
   const int64_t c_begin = (int64_t)blockIdx.x * range_len;     // multiple of 4
@@ -478,7 +538,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
       const int64_t lo = part ? c_mid : c_begin, hi = part ? c_end : c_mid;
       for (int b0 = 0; b0 < P && lo < hi; b0 += pp.batch_rows) {
         const int nb = min(pp.batch_rows, P - b0);
-        const int lane_row = lane < nb ? pp.row_at(b0 + lane) : 0;
+        const int lane_row = lane < nb ? pipe_row_at(b0 + lane, n_first, s_first_row) : 0;
         for (int64_t c0 = lo; c0 < hi; c0 += pp.slice_cols, ++it) {
           const int stage = it % kPipeStages;
           const uint32_t phase = (it / kPipeStages) & 1;
@@ -527,7 +587,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
         int shift[4], row_of[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          row_of[j] = j < nr ? pp.row_at(b0 + warp + 8 * j) : 0;
+          row_of[j] = j < nr ? pipe_row_at(b0 + warp + 8 * j, n_first, s_first_row) : 0;
           shift[j] = (int)(((row_of[j] & (kVec - 1)) * dc_mod4) & (kVec - 1));   // (row * d_c + c0) mod (elements per 16 bytes)
         }
         double rho[4][K], nu[4];
@@ -553,34 +613,38 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           if constexpr (sizeof(T) == 4) {
             if (pp.opt_rows > 0 && b0 == 0 && !opt_resolved) {
-              // first stage of this CTA: the flags have long arrived; all consumer warps pass here together
+              // first stage of this CTA: flags, rows and weights have long arrived; all consumer warps pass here together
               if (tid < 32) {
-                const bool all_clean = __all_sync(0xffffffffu, opt_clean != 0);
+                if (!pp.multi_batch) {
+                  const int below = __shfl_up_sync(0xffffffffu, spec_row, 1);
+                  const bool lane_ok = spec_whole && (tid >= pp.opt_rows || (spec_row >= 0 && spec_row < P && (tid == 0 || spec_row > below)));
+                  spec_whole = __all_sync(0xffffffffu, lane_ok);
+                }
+                const bool all_clean = __all_sync(0xffffffffu, opt_flag != 0);
                 if (tid == 0) {
-                  s_opt_on = (opt_mode == 2 || (opt_mode == 1 && all_clean)) ? 1 : 0;
+                  s_opt_on = (spec_whole && (opt_mode == 2 || (opt_mode == 1 && all_clean))) ? 1 : 0;
                   if (blockIdx.x == 0) pp.opt_flags[1] = s_opt_on;
                 }
+                if (tid < pp.opt_rows && spec_whole) {
+                  // slot of the row in a stage of the first batch: its position in the kernel's order
+                  const int slot = pp.multi_batch ? tid : spec_row;
+                  s_opt_off[tid] = slot * pp.slot_floats + (int)((((int64_t)spec_row & 3) * (d_c & 3)) & 3);
+                }
               }
+              if (tid < pp.opt_rows * 8) s_opt_coeff[tid] = pack2((float)spec_coeff, (float)spec_coeff);   // rounded as the recovery kernel rounds it
               pipe::named_barrier_sync(1, kPipeConsumers);
               opt = s_opt_on != 0;
-              if (opt) {
-                for (int i = tid; i < pp.opt_rows * 8; i += kPipeConsumers)
-                  s_opt_coeff[i] = (i & 7) < pp.m ? pp.opt_coeff[(i >> 3) * pp.m + (i & 7)] : 0.0f;
-                for (int j = tid; j < pp.opt_rows; j += kPipeConsumers)
-                  s_opt_shift[j] = (int)((((int64_t)pp.def_rows[j] & 3) * (d_c & 3)) & 3);
-                pipe::named_barrier_sync(1, kPipeConsumers);
-              }
               opt_resolved = true;
             }
             if (opt && b0 == 0) {
               const float* rows0 = reinterpret_cast<const float*>(base);
               switch (pp.m) {
-                case 1: opt_recover_slice<1>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
-                case 2: opt_recover_slice<2>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
-                case 3: opt_recover_slice<3>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
-                case 4: opt_recover_slice<4>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
-                case 5: opt_recover_slice<5>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
-                default: opt_recover_slice<6>(rows0, pp.slot_floats, s_opt_shift, s_opt_coeff, pp.opt_rows, cols, c0, pp.agg, pp.d, tid); break;
+                case 1: opt_recover_slice<1>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 2: opt_recover_slice<2>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 3: opt_recover_slice<3>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 4: opt_recover_slice<4>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 5: opt_recover_slice<5>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                default: opt_recover_slice<6>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
               }
             }
           }
@@ -638,18 +702,21 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   pp.progress = plan->d_proj_progress;
   // optimistic decode: only in the whole decode (the aggregate's buffer is known) of a float32 plan that is eligible
   pp.opt_rows = (!final_reduce && agg && sizeof(T) == 4 && plan->optimistic != 0) ? plan->opt_rows : 0;
-  for (int j = 0; j < kPipeRows; ++j) pp.def_rows[j] = j < pp.opt_rows ? (uint16_t)plan->opt_row_host[(size_t)j] : 0;
+  for (int j = 0; j < kPipeRows; ++j) pp.spec_src[j] = j < pp.opt_rows ? (uint16_t)plan->opt_src_host[(size_t)j] : 0;
   pp.q = plan->q;
-  pp.opt_coeff = plan->d_opt_coeff;
+  pp.rec_rows = plan->d_rec_rows;
+  pp.rec_coeff = plan->d_coeff;
+  pp.n_rec = plan->d_n_rec;
   pp.opt_flags = plan->d_opt;
   pp.agg = reinterpret_cast<float*>(agg);
   pp.m = plan->m;
   pp.d = plan->d;
   // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
-  // (the kernel's static shared memory - the optimistic decode's weights - is 1.2 KB)
-  const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128 - 1536;
+  // (the kernel's static shared memory - the optimistic decode's weights above all - is 2.4 KB)
+  const size_t per_cta = (size_t)227 * 1024 / kPipeCtasPerSm - 1024 - 128 - 2560;
   const int n_batches = (plan->P + kPipeRows - 1) / kPipeRows;
   pp.batch_rows = (plan->P + n_batches - 1) / n_batches;
+  pp.multi_batch = n_batches > 1 ? 1 : 0;
   int slice = (int)(per_cta / ((size_t)kPipeStages * (pp.batch_rows * sizeof(T) + K * sizeof(float)))) - 8;
   slice = slice / 32 * 32;
   if (slice > 2048) slice = 2048;
@@ -661,6 +728,12 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   int64_t range_len = (plan->d_c + grid - 1) / grid;
   range_len = (range_len + 3) / 4 * 4;
   if (range_len < slice) slice = (int)((range_len + 31) / 32 * 32);
+  // the optimistic recovery hands a slice out in passes of 256 opt_ch columns: a width that is a multiple of that
+  pp.opt_ch = kOptChunks;
+  if (pp.opt_rows > 0 && slice >= kPipeConsumers) {
+    pp.opt_ch = slice / kPipeConsumers < kOptChunks ? slice / kPipeConsumers : kOptChunks;
+    slice = slice / (kPipeConsumers * pp.opt_ch) * (kPipeConsumers * pp.opt_ch);
+  }
   pp.slice_cols = slice;
   pp.slot_floats = slice + 8;
   // part A (only when the locator kernel will work ahead on it): about an eighth of the range, whole slices, at least one

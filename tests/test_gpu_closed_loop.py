@@ -38,12 +38,14 @@ def _oracle_descent(X, y, w0, lr):
     return out
 
 
-def _run(per_group, attack, graph, early=1):
+def _run(per_group, attack, graph, early=1, optimistic=None):
     X, y, w0, lr = _problem()
     rng = np.random.default_rng(99)
     iterates, masks, sets = [], [], []
     with binding.Plan(P, S, M, R, D, seed=5) as plan:
         plan.set_early_locator(early)
+        if optimistic is not None:
+            plan.set_optimistic(optimistic)
         loop = sgd.ClosedLoop(plan, X.cuda(), y.cuda(), w0.cuda(), lr, ROWS, attackers_per_group=per_group, attack=attack)
         if graph:
             loop.set_attackers(sgd.draw_attackers(plan, np.random.default_rng(1), per_group))
@@ -79,8 +81,15 @@ def test_iterates_equal_the_attack_free_run(attack):
 
 @pytest.mark.parametrize("early", [0, 2])
 def test_graph_replay_equals_eager_steps(early):
-    eager, masks_e, sets_e = _run(S, "alie", graph=False)
-    replay, masks_g, sets_g = _run(S, "alie", graph=True, early=early)
+    # bit for bit with the optimistic decode off: with it on, an aggregate may come from the previous decode's recovery
+    # table (other trusted rows, the same sum up to rounding), and the captured run has one more decode behind it
+    eager, masks_e, sets_e = _run(S, "alie", graph=False, optimistic=0)
+    replay, masks_g, sets_g = _run(S, "alie", graph=True, early=early, optimistic=0)
     assert sets_e == sets_g and masks_e == masks_g == sets_e
     for a, b in zip(eager, replay):
         assert np.array_equal(a, b)
+    # default mode: the same iterates up to that rounding
+    replay_d, masks_d, sets_d = _run(S, "alie", graph=True, early=early)
+    assert sets_d == sets_e and masks_d == sets_e
+    for a, b in zip(eager, replay_d):
+        assert np.abs(a - b).max() <= 2e-5 * np.abs(a).max()

@@ -1,6 +1,7 @@
-"""Optimistic decode (solon_plan_set_optimistic): the projection pass recovers the aggregate from the rows that are read
-when no node is corrupt, and the recovery kernel is skipped when the locator confirms them.  Results must not depend on
-the mode: bit for bit the same aggregate, the same mask, with and without attackers, and against the oracle."""
+"""Optimistic decode (solon_plan_set_optimistic): the projection pass recovers the aggregate from the rows of the previous
+decode's recovery table, and the recovery kernel is skipped when the locator finds all of them trusted.  Results must not
+depend on the mode: the same mask, the same aggregate (bit for bit whenever the same table is used, within the tolerance
+otherwise), with and without attackers, with attackers that stay and attackers that move, and against the oracle."""
 
 import dataclasses
 
@@ -46,29 +47,57 @@ def test_modes_agree_with_and_without_attackers(name, d, early):
         assert np.abs(ref_clean[1].cpu().numpy() - want).max() <= AGG_TOL * scale
         assert np.abs(ref_attacked[1].cpu().numpy() - want).max() <= AGG_TOL * scale
 
+        # attackers that move onto a row the table for `nodes` reads: in group 0 the first trusted node (m >= 2: the rows are
+        # spread over the trusted nodes from the first to the last), the middle one for m = 1
+        n0 = so.group_sizes(wl.P, wl.r)[0]
+        trusted0 = [k for k in range(n0) if k not in nodes]
+        moved_to = [trusted0[0] if wl.m >= 2 else trusted0[(len(trusted0) - 1) // 2]]
+        attacked_b = coded.clone()
+        attacked_b[moved_to] = synth.byzantine_rows(dataclasses.replace(wl, attack="gaussian", n_byz=1), coded, moved_to)
+        ref_moved = _decode(plan, attacked_b)
+        assert ref_moved[0] == 0 and ref_moved[2].nonzero().flatten().tolist() == moved_to
+
         def same(got, ref):
             return got[0] == ref[0] and torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
 
-        # mode 1: optimistic only after a decode that found every node honest
+        def agrees(got, ref):
+            # another table (other trusted rows) gives the same sum up to rounding; the recovery kernel itself always uses
+            # the table of its own decode
+            ok = got[0] == ref[0] and torch.equal(got[2], ref[2]) and np.abs(got[1].cpu().numpy() - want).max() <= AGG_TOL * scale
+            return ok and (got[3] or same(got, ref))
+
+        # mode 1: optimistic when the previous decode's table would have served that decode too
         plan.set_optimistic(1)
         first = _decode(plan, coded)            # nothing known yet: the ordinary path
-        second = _decode(plan, coded)           # the projection pass recovers, the locator confirms, the recovery skips
-        third = _decode(plan, attacked)         # it recovers again, but nodes are corrupt: the recovery kernel overwrites
-        fourth = _decode(plan, attacked)        # the last decode was not clean: the ordinary path
-        fifth = _decode(plan, coded)            # still the ordinary path (the last decode was not clean), but clean again
-        sixth = _decode(plan, coded)            # optimistic again
-        assert [x[3] for x in (first, second, third, fourth, fifth, sixth)] == [False, True, False, False, False, True]
-        for got in (first, second, fifth, sixth):
-            assert same(got, ref_clean)
-        for got in (third, fourth):
-            assert same(got, ref_attacked)
-        # mode 2: always
+        second = _decode(plan, coded)           # recovers from the table of `first`, the locator confirms, the recovery skips
+        assert not first[3] and second[3]
+        assert same(first, ref_clean) and same(second, ref_clean)
+        # attackers arrive and stay: from the third decode on the table of the decode before avoids them
+        runs = [_decode(plan, attacked) for _ in range(4)]
+        assert all(agrees(got, ref_attacked) for got in runs)
+        assert runs[2][3] and runs[3][3] and same(runs[2], ref_attacked) and same(runs[3], ref_attacked)
+        # they move onto a row of that table: the speculation fails, the recovery kernel runs as usual
+        moved = _decode(plan, attacked_b)
+        assert not moved[3] and same(moved, ref_moved)
+        after = _decode(plan, attacked_b)       # the previous table would not have served: the ordinary path
+        assert not after[3] and same(after, ref_moved)
+        settled = [_decode(plan, attacked_b) for _ in range(2)]
+        assert settled[1][3] and all(same(got, ref_moved) for got in settled)
+        # mode 2: always (from whatever table the last decode left)
         plan.set_optimistic(2)
         a = _decode(plan, attacked)
         b = _decode(plan, coded)
-        c = _decode(plan, attacked)
-        assert [x[3] for x in (a, b, c)] == [False, True, False]
-        assert same(a, ref_attacked) and same(b, ref_clean) and same(c, ref_attacked)
+        c = _decode(plan, coded)
+        assert agrees(a, ref_attacked) and agrees(b, ref_clean) and b[3] and c[3] and same(c, ref_clean)
+        # a decode that fails (more liars than s in a group) leaves nothing behind that the next one trips over
+        too_many = list(range(wl.s + 1))
+        broken = coded.clone()
+        broken[too_many] = synth.byzantine_rows(dataclasses.replace(wl, attack="gaussian", n_byz=wl.s + 1), coded, too_many)
+        failed = _decode(plan, broken)
+        assert failed[0] != 0 and not failed[3]
+        d1 = _decode(plan, coded)
+        d2 = _decode(plan, coded)
+        assert agrees(d1, ref_clean) and d2[3] and same(d2, ref_clean)
         # and the oracle's own decode of the clean matrix
         u, o_mask, o_status = so.decode(coded.cpu().numpy(), wl.d, wl.m, wl.s, so.group_sizes(wl.P, wl.r),
                                         so.node_scalars(so.group_sizes(wl.P, wl.r)), plan.projection_vectors(), tau=1e-5)
