@@ -285,16 +285,17 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
 // itself (routing them through shared memory into 128-bit stores, as the recovery kernel does, made this kernel 20 %
 // slower: its consumer warps are bound by instruction issue).
 constexpr int kOptChunks = 4;
-template <int M>
+// NP: pairs of chunks per lane and pass held in registers (ch <= 2 NP)
+template <int M, int NP>
 __device__ __forceinline__ void opt_recover_slice(const float* base, const int* s_off, const f32x2* s_coeff2, int n_def,
                                                   int cols, int ch, int64_t c0, float* __restrict__ agg, int64_t d, int warp, int lane) {
-  // ch (1..4): chunks per lane and pass; the slice width is a multiple of 256 ch, so that every pass but the one at the
-  // ragged end of a range keeps all lanes busy
+  // ch (1..4): chunks per lane and pass; the slice width is a multiple of 256 ch where that costs little, so that every
+  // pass but the one at the ragged end of a range keeps all lanes busy
   for (int cb = warp * 32; cb < cols; cb += ch * kPipeConsumers) {
     const int c = cb + lane;
-    f32x2 acc[kOptChunks / 2][M];
+    f32x2 acc[NP][M];
 #pragma unroll
-    for (int h = 0; h < kOptChunks / 2; ++h)
+    for (int h = 0; h < NP; ++h)
 #pragma unroll
       for (int l = 0; l < M; ++l) acc[h][l] = 0ULL;          // (+0.0f, +0.0f)
     for (int j = 0; j < n_def; ++j) {
@@ -306,11 +307,11 @@ __device__ __forceinline__ void opt_recover_slice(const float* base, const int* 
         w[2 * t] = ww.x;
         w[2 * t + 1] = ww.y;
       }
-      float v[kOptChunks];
+      float v[2 * NP];
 #pragma unroll
-      for (int i = 0; i < kOptChunks; ++i) v[i] = (i < ch && c + i * kPipeConsumers < cols) ? row[c + i * kPipeConsumers] : 0.0f;
+      for (int i = 0; i < 2 * NP; ++i) v[i] = (i < ch && c + i * kPipeConsumers < cols) ? row[c + i * kPipeConsumers] : 0.0f;
 #pragma unroll
-      for (int h = 0; h < kOptChunks / 2; ++h) {
+      for (int h = 0; h < NP; ++h) {
         if (2 * h < ch) {
           const f32x2 vv = pack2(v[2 * h], v[2 * h + 1]);
 #pragma unroll
@@ -319,7 +320,7 @@ __device__ __forceinline__ void opt_recover_slice(const float* base, const int* 
       }
     }
 #pragma unroll
-    for (int i = 0; i < kOptChunks; ++i) {
+    for (int i = 0; i < 2 * NP; ++i) {
       const int ci = cb + i * kPipeConsumers + lane;
       if (i < ch && ci < cols) {
         const int64_t o = (c0 + ci) * M;
@@ -332,6 +333,14 @@ __device__ __forceinline__ void opt_recover_slice(const float* base, const int* 
       }
     }
   }
+}
+
+template <int M>
+__device__ __forceinline__ void opt_recover_slice_m(const float* base, const int* s_off, const f32x2* s_coeff2, int n_def,
+                                                    int cols, int ch, int64_t c0, float* __restrict__ agg, int64_t d, int warp, int lane) {
+  // fewer accumulators in registers when the passes are narrow (the kernel is at its register limit)
+  if (ch <= 2) opt_recover_slice<M, 1>(base, s_off, s_coeff2, n_def, cols, ch, c0, agg, d, warp, lane);
+  else opt_recover_slice<M, 2>(base, s_off, s_coeff2, n_def, cols, ch, c0, agg, d, warp, lane);
 }
 
 // One slice for the NR rows of this warp: rows[j] point at column 0 of the slice in the warp's j-th row.
@@ -639,12 +648,12 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
             if (opt && b0 == 0) {
               const float* rows0 = reinterpret_cast<const float*>(base);
               switch (pp.m) {
-                case 1: opt_recover_slice<1>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 2: opt_recover_slice<2>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 3: opt_recover_slice<3>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 4: opt_recover_slice<4>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 5: opt_recover_slice<5>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                default: opt_recover_slice<6>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 1: opt_recover_slice_m<1>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 2: opt_recover_slice_m<2>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 3: opt_recover_slice_m<3>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 4: opt_recover_slice_m<4>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 5: opt_recover_slice_m<5>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                default: opt_recover_slice_m<6>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
               }
             }
           }
@@ -728,11 +737,26 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   int64_t range_len = (plan->d_c + grid - 1) / grid;
   range_len = (range_len + 3) / 4 * 4;
   if (range_len < slice) slice = (int)((range_len + 31) / 32 * 32);
-  // the optimistic recovery hands a slice out in passes of 256 opt_ch columns: a width that is a multiple of that
+  // the optimistic recovery hands a slice out in passes of 256 opt_ch columns (opt_ch chunks per consumer thread): a
+  // width that is a multiple of that keeps every lane busy; when that would cost more than an eighth of the slice (more
+  // stages, each with its overhead) the width stays and opt_ch is the one that pads the last pass least
   pp.opt_ch = kOptChunks;
   if (pp.opt_rows > 0 && slice >= kPipeConsumers) {
-    pp.opt_ch = slice / kPipeConsumers < kOptChunks ? slice / kPipeConsumers : kOptChunks;
-    slice = slice / (kPipeConsumers * pp.opt_ch) * (kPipeConsumers * pp.opt_ch);
+    int best_ch = 0, best_slice = 0;
+    for (int ch = 1; ch <= kOptChunks; ++ch) {
+      const int rounded = slice / (kPipeConsumers * ch) * (kPipeConsumers * ch);
+      if (rounded >= best_slice && rounded > 0) { best_slice = rounded; best_ch = ch; }
+    }
+    if (best_slice * 8 >= slice * 7) {
+      slice = best_slice;
+      pp.opt_ch = best_ch;
+    } else {
+      int best_work = 1 << 30;
+      for (int ch = 1; ch <= kOptChunks; ++ch) {
+        const int work = (slice + kPipeConsumers * ch - 1) / (kPipeConsumers * ch) * ch;
+        if (work <= best_work) { best_work = work; pp.opt_ch = ch; }
+      }
+    }
   }
   pp.slice_cols = slice;
   pp.slot_floats = slice + 8;
