@@ -157,15 +157,21 @@ int solon_plan_set_tolerance(solon_plan* plan, double tau);
  * takes its ordinary path afterwards (outcome 3 of solon_plan_get_early_outcome; results unchanged). */
 int solon_plan_set_early_locator(solon_plan* plan, int mode);
 
-/* Optimistic decode (Algorithm 1 with the block decoder's work done ahead of the locator's verdict).  When no node is
- * corrupt the recovery reads a fixed set of rows, m per group.  The projection kernel, which has every row on chip
- * anyway, can apply the inverse for those rows to each column slice as it passes and write the aggregate itself; if the
- * locator then finds every group free of corrupt nodes, the recovery kernel returns at once and the decode has read the
- * received matrix once instead of 1 + q m / P times.  If a node is corrupt the recovery kernel runs as usual and
- * overwrites the aggregate: results never depend on the mode (the optimistic aggregate is computed in the recovery
- * kernel's arithmetic and order, bit for bit).  mode 0: never; 1 (default): for the decode after one that found every
- * node honest (decided on the device, no host round trip); 2: always.  Eligible plans: float32, s > 0, m <= 6 and
- * q m rows fitting in the projection kernel's first batch of rows (at most 32); other plans ignore the mode. */
+/* Optimistic decode (Algorithm 1 with the block decoder's work done ahead of the locator's verdict).  For m <= 6 the
+ * recovery reads m trusted rows per group and applies the inverse of their Vandermonde block (Section 4.2's block
+ * decoder); any m trusted rows give the same sum.  The projection kernel, which has every row on chip anyway, can apply
+ * the inverse for the rows the PREVIOUS decode's recovery read (the locator's last table; before the first decode the
+ * table for no corrupt node) to each column slice as it passes and write the aggregate itself.  If the locator then
+ * finds all of those rows trusted in THIS decode, the recovery kernel returns at once and the decode has read the
+ * received matrix once instead of 1 + q m / P times: with no attackers, or with attackers that stay where they were,
+ * every decode from the second or third on.  If one of those rows is corrupt now, the recovery kernel runs as usual and
+ * overwrites the aggregate.  The mask never depends on the mode.  The aggregate is computed in the recovery kernel's
+ * arithmetic and order: bit for bit what mode 0 gives whenever the previous table is also this decode's table (same
+ * corrupt set), and the same sum up to float32 rounding when it came from other trusted rows - so with mode 1 or 2 the
+ * last bits of an aggregate can depend on the decode before it; mode 0 gives history-independent bits.
+ * mode 0: never; 1 (default): when the previous decode's table would have served that decode too (its rows were all
+ * trusted; decided on the device, no host round trip); 2: always.  Eligible plans: float32, s > 0, m <= 6 and q m rows
+ * fitting in the projection kernel's first batch of rows (at most 32); other plans ignore the mode. */
 int solon_plan_set_optimistic(solon_plan* plan, int mode);
 /* *skipped = 1 if the recovery kernel of the most recent solon_decode had nothing to do.  Synchronises. */
 int solon_plan_get_optimistic_outcome(solon_plan* plan, int* skipped);

@@ -239,8 +239,9 @@ class Plan:
         _check(lib().solon_plan_set_early_locator(self._h, mode), "solon_plan_set_early_locator")
 
     def set_optimistic(self, mode: int) -> None:
-        """0: the projection pass never recovers the aggregate itself; 1 (default): after a decode that found every node
-        honest; 2: always.  The recovery kernel is skipped when the locator confirms that no node is corrupt."""
+        """0: the projection pass never recovers the aggregate itself; 1 (default): it does so, from the rows of the previous
+        decode's recovery table, when that table would have served the previous decode too; 2: always.  The recovery
+        kernel is skipped when the locator finds those rows trusted in this decode."""
         _check(lib().solon_plan_set_optimistic(self._h, mode), "solon_plan_set_optimistic")
 
     def optimistic_outcome(self) -> bool:
