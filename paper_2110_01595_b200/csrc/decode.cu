@@ -18,7 +18,7 @@ static int decode_t(solon_plan* plan, const T* received, T* agg_grad, uint8_t* b
     return SOLON_OK;
   };
   auto project = [&]() -> int {
-    if constexpr (sizeof(T) == 8) return launch_project_f64(plan, received);
+    if constexpr (sizeof(T) == 8) return launch_project_f64(plan, received, nullptr, nullptr, agg_grad);
     else return launch_project(plan, received, nullptr, nullptr, agg_grad);
   };
   auto recover = [&]() -> int {

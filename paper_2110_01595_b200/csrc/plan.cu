@@ -282,7 +282,7 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
         std::vector<int> opt_src;
         const int n_batches = (P + 31) / 32;
         const int batch_rows = (P + n_batches - 1) / n_batches;
-        bool eligible = dtype == SOLON_F32 && s > 0 && m <= SOLON_SUBSET_MAX_M && q * m <= batch_rows;
+        bool eligible = s > 0 && m <= SOLON_SUBSET_MAX_M && q * m <= batch_rows;
         std::vector<int> rows_g((size_t)max_group);
         std::vector<double> coeff_g((size_t)max_group * m);
         for (int g = 0; g < q && eligible; ++g) {

@@ -248,7 +248,7 @@ struct ProjPipe {
   const double* rec_coeff;            // P x m: its weights
   const int* n_rec;                   // q: rows in use per group (m after a decode that succeeded)
   int* opt_flags;                     // [1] this pass recovered (written here), [4] mode, [8 + g] see the locator kernel
-  float* agg;                         // d: the aggregate (written only when this pass recovers)
+  void* agg;                          // d elements of the plan's type: the aggregate (written only when this pass recovers)
   int m;
   int64_t d;
 };
@@ -341,6 +341,49 @@ __device__ __forceinline__ void opt_recover_slice_m(const float* base, const int
   // fewer accumulators in registers when the passes are narrow (the kernel is at its register limit)
   if (ch <= 2) opt_recover_slice<M, 1>(base, s_off, s_coeff2, n_def, cols, ch, c0, agg, d, warp, lane);
   else opt_recover_slice<M, 2>(base, s_off, s_coeff2, n_def, cols, ch, c0, agg, d, warp, lane);
+}
+
+// The same for float64 plans: float64 weights and sums as in the float64 recovery kernel, one or two chunks per lane and pass.
+template <int M>
+__device__ __forceinline__ void opt_recover_slice_m(const double* base, const int* s_off, const f32x2* s_coeff2, int n_def,
+                                                    int cols, int ch, int64_t c0, double* __restrict__ agg, int64_t d, int warp, int lane) {
+  const double* s_coeff = reinterpret_cast<const double*>(s_coeff2);     // eight weights per row
+  for (int cb = warp * 32; cb < cols; cb += ch * kPipeConsumers) {
+    const int c = cb + lane;
+    double acc[2][M];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int l = 0; l < M; ++l) acc[i][l] = 0.0;
+    for (int j = 0; j < n_def; ++j) {
+      const double* row = base + s_off[j];
+      double w[(M + 1) / 2 * 2];
+#pragma unroll
+      for (int t = 0; t < (M + 1) / 2; ++t) {
+        const double2 ww = *reinterpret_cast<const double2*>(s_coeff + j * 8 + 2 * t);
+        w[2 * t] = ww.x;
+        w[2 * t + 1] = ww.y;
+      }
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (i < ch) {
+          const double v = c + i * kPipeConsumers < cols ? row[c + i * kPipeConsumers] : 0.0;
+#pragma unroll
+          for (int l = 0; l < M; ++l) acc[i][l] = fma(w[l], v, acc[i][l]);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int ci = cb + i * kPipeConsumers + lane;
+      if (i < ch && ci < cols) {
+        const int64_t o = (c0 + ci) * M;
+#pragma unroll
+        for (int l = 0; l < M; ++l)
+          if (o + l < d) __stcs(agg + o + l, acc[i][l]);
+      }
+    }
+  }
 }
 
 // One slice for the NR rows of this warp: rows[j] point at column 0 of the slice in the warp's j-th row.
@@ -491,7 +534,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
     *abort_flag = 0;
     pipe::fence_barrier_init();
   }
-  // Optimistic decode (float32 plans): does this pass also recover the aggregate, from the rows of the last recovery table?
+  // Optimistic decode: does this pass also recover the aggregate, from the rows of the last recovery table?
   // Mode 2, or mode 1 and every flag of the previous decode set; and only if that table is whole (m rows in every group,
   // ascending node indices).  Flags, rows and weights are fetched here - one load per thread - and looked at only when the
   // first stage's projection work is done (see below), so that their round trip to device memory hides behind it; with
@@ -500,7 +543,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
   int opt_mode = 0, opt_flag = 1, spec_row = 0;      // raw values: nothing is computed from them before they are needed
   bool spec_whole = false;
   double spec_coeff = 0.0;
-  if constexpr (sizeof(T) == 4) {
+  {
     if (pp.opt_rows > 0) {
       if (tid < 32) {
         opt_mode = pp.opt_flags[4];
@@ -521,7 +564,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
         spec_coeff = pp.rec_coeff[(size_t)pp.spec_src[tid >> 3] * pp.m + (tid & 7)];
     }
   }
-  if (tid == 0 && !(sizeof(T) == 4 && pp.opt_rows > 0 && pp.multi_batch)) s_n_first = 0;
+  if (tid == 0 && !(pp.opt_rows > 0 && pp.multi_batch)) s_n_first = 0;
   if (blockIdx.x == 0 && tid == 0) pp.opt_flags[1] = 0;
   __syncthreads();
   const int n_first = s_n_first;
@@ -620,7 +663,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
           else if (nr == 3) pipe_consume<K, 3>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 2) pipe_consume<K, 2>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
           else if (nr == 1) pipe_consume<K, 1>(rows, fs, pp.slot_floats, cols, lane, rho, nu);
-          if constexpr (sizeof(T) == 4) {
+          {
             if (pp.opt_rows > 0 && b0 == 0 && !opt_resolved) {
               // first stage of this CTA: flags, rows and weights have long arrived; all consumer warps pass here together
               if (tid < 32) {
@@ -637,23 +680,27 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
                 if (tid < pp.opt_rows && spec_whole) {
                   // slot of the row in a stage of the first batch: its position in the kernel's order
                   const int slot = pp.multi_batch ? tid : spec_row;
-                  s_opt_off[tid] = slot * pp.slot_floats + (int)((((int64_t)spec_row & 3) * (d_c & 3)) & 3);
+                  s_opt_off[tid] = slot * pp.slot_floats + (int)((((int64_t)spec_row & (kVec - 1)) * (d_c & (kVec - 1))) & (kVec - 1));
                 }
               }
-              if (tid < pp.opt_rows * 8) s_opt_coeff[tid] = pack2((float)spec_coeff, (float)spec_coeff);   // rounded as the recovery kernel rounds it
+              if (tid < pp.opt_rows * 8) {     // rounded as the recovery kernel of the plan's type rounds it
+                if constexpr (sizeof(T) == 4) s_opt_coeff[tid] = pack2((float)spec_coeff, (float)spec_coeff);
+                else s_opt_coeff[tid] = (f32x2)__double_as_longlong(spec_coeff);
+              }
               pipe::named_barrier_sync(1, kPipeConsumers);
               opt = s_opt_on != 0;
               opt_resolved = true;
             }
             if (opt && b0 == 0) {
-              const float* rows0 = reinterpret_cast<const float*>(base);
+              const T* rows0 = reinterpret_cast<const T*>(base);
+              T* agg_t = reinterpret_cast<T*>(pp.agg);
               switch (pp.m) {
-                case 1: opt_recover_slice_m<1>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 2: opt_recover_slice_m<2>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 3: opt_recover_slice_m<3>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 4: opt_recover_slice_m<4>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                case 5: opt_recover_slice_m<5>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
-                default: opt_recover_slice_m<6>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, pp.agg, pp.d, warp, lane); break;
+                case 1: opt_recover_slice_m<1>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, agg_t, pp.d, warp, lane); break;
+                case 2: opt_recover_slice_m<2>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, agg_t, pp.d, warp, lane); break;
+                case 3: opt_recover_slice_m<3>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, agg_t, pp.d, warp, lane); break;
+                case 4: opt_recover_slice_m<4>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, agg_t, pp.d, warp, lane); break;
+                case 5: opt_recover_slice_m<5>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, agg_t, pp.d, warp, lane); break;
+                default: opt_recover_slice_m<6>(rows0, s_opt_off, s_opt_coeff, pp.opt_rows, cols, pp.opt_ch, c0, agg_t, pp.d, warp, lane); break;
               }
             }
           }
@@ -710,14 +757,14 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   pp.status = plan->d_status;
   pp.progress = plan->d_proj_progress;
   // optimistic decode: only in the whole decode (the aggregate's buffer is known) of a float32 plan that is eligible
-  pp.opt_rows = (!final_reduce && agg && sizeof(T) == 4 && plan->optimistic != 0) ? plan->opt_rows : 0;
+  pp.opt_rows = (!final_reduce && agg && plan->optimistic != 0) ? plan->opt_rows : 0;
   for (int j = 0; j < kPipeRows; ++j) pp.spec_src[j] = j < pp.opt_rows ? (uint16_t)plan->opt_src_host[(size_t)j] : 0;
   pp.q = plan->q;
   pp.rec_rows = plan->d_rec_rows;
   pp.rec_coeff = plan->d_coeff;
   pp.n_rec = plan->d_n_rec;
   pp.opt_flags = plan->d_opt;
-  pp.agg = reinterpret_cast<float*>(agg);
+  pp.agg = agg;
   pp.m = plan->m;
   pp.d = plan->d;
   // two CTAs per SM: the widest slice (multiple of 32 columns) whose ring fits in half of the shared memory
@@ -740,10 +787,11 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   // the optimistic recovery hands a slice out in passes of 256 opt_ch columns (opt_ch chunks per consumer thread): a
   // width that is a multiple of that keeps every lane busy; when that would cost more than an eighth of the slice (more
   // stages, each with its overhead) the width stays and opt_ch is the one that pads the last pass least
-  pp.opt_ch = kOptChunks;
+  const int max_ch = sizeof(T) == 8 ? 2 : kOptChunks;     // float64: two chunks per lane at most (registers)
+  pp.opt_ch = max_ch;
   if (pp.opt_rows > 0 && slice >= kPipeConsumers) {
     int best_ch = 0, best_slice = 0;
-    for (int ch = 1; ch <= kOptChunks; ++ch) {
+    for (int ch = 1; ch <= max_ch; ++ch) {
       const int rounded = slice / (kPipeConsumers * ch) * (kPipeConsumers * ch);
       if (rounded >= best_slice && rounded > 0) { best_slice = rounded; best_ch = ch; }
     }
@@ -752,7 +800,7 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
       pp.opt_ch = best_ch;
     } else {
       int best_work = 1 << 30;
-      for (int ch = 1; ch <= kOptChunks; ++ch) {
+      for (int ch = 1; ch <= max_ch; ++ch) {
         const int work = (slice + kPipeConsumers * ch - 1) / (kPipeConsumers * ch) * ch;
         if (work <= best_work) { best_work = work; pp.opt_ch = ch; }
       }
@@ -804,8 +852,8 @@ static int launch_project_t(solon_plan* plan, const T* received, double* rho_out
 int launch_project(solon_plan* plan, const float* received, double* rho_out, double* nu_out, float* agg) {
   return launch_project_t<float>(plan, received, rho_out, nu_out, agg);
 }
-int launch_project_f64(solon_plan* plan, const double* received, double* rho_out, double* nu_out) {
-  return launch_project_t<double>(plan, received, rho_out, nu_out, nullptr);
+int launch_project_f64(solon_plan* plan, const double* received, double* rho_out, double* nu_out, double* agg) {
+  return launch_project_t<double>(plan, received, rho_out, nu_out, agg);
 }
 
 // ---- projections without any allocation ------------------------------------------------------------

@@ -206,7 +206,7 @@ int launch_encode_f64(solon_plan* plan, const double* grads, double* coded);
 // rho_out / nu_out (and rho / nu below): device buffers, or nullptr for the plan's own
 // agg: where the optimistic decode may write the aggregate (the whole decode only; nullptr: never)
 int launch_project(solon_plan* plan, const float* received, double* rho_out = nullptr, double* nu_out = nullptr, float* agg = nullptr);
-int launch_project_f64(solon_plan* plan, const double* received, double* rho_out = nullptr, double* nu_out = nullptr);
+int launch_project_f64(solon_plan* plan, const double* received, double* rho_out = nullptr, double* nu_out = nullptr, double* agg = nullptr);
 int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho = nullptr, const double* nu = nullptr);
 int launch_recover(solon_plan* plan, const float* received, float* agg);
 int launch_recover_f64(solon_plan* plan, const double* received, double* agg);

@@ -135,8 +135,48 @@ def test_edge_shapes(P, s, m, r, d):
         assert np.abs(agg.cpu().numpy() - want).max() <= AGG_TOL * max(np.abs(want).max(), 1e-30)
 
 
+@pytest.mark.parametrize("P,s,m,r,d", [
+    (15, 2, 5, 9, 150_003),     # one batch of rows, d_c odd: rows off 16-byte boundaries
+    (45, 3, 5, 11, 283_321),    # two batches of rows: the speculated rows are taken first
+    (30, 2, 6, 10, 60_005),
+    (16, 1, 1, 3, 4099),
+])
+def test_float64_plans(P, s, m, r, d):
+    """The same decode for float64 elements: float64 weights and sums as in the float64 recovery kernel."""
+    wl = synth.Workload("opt_f64", P, s, m, d, "normal", 1.0, "gaussian", s, 17 + P)
+    G = synth.make_grads(wl, "cuda").double()
+    want = so.plain_sum(G.cpu().numpy())
+    scale = np.abs(want).max()
+    with binding.Plan(P, s, m, r, d, seed=3, dtype="f64") as plan:
+        coded = plan.encode(G)
+        attacked, nodes = synth.apply_attack(wl, coded)
+        plan.set_optimistic(0)
+        ref_clean = _decode(plan, coded)
+        ref_attacked = _decode(plan, attacked)
+        assert ref_clean[0] == 0 and ref_attacked[0] == 0 and not ref_clean[3] and not ref_attacked[3]
+        assert ref_attacked[2].nonzero().flatten().tolist() == nodes
+        assert np.abs(ref_attacked[1].cpu().numpy() - want).max() <= 1e-9 * scale
+
+        def same(got, ref):
+            return got[0] == ref[0] and torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
+
+        plan.set_optimistic(1)
+        runs = [_decode(plan, attacked) for _ in range(4)]
+        for got in runs:
+            assert got[0] == 0 and torch.equal(got[2], ref_attacked[2])
+            assert np.abs(got[1].cpu().numpy() - want).max() <= 1e-9 * scale
+            assert got[3] or same(got, ref_attacked)
+        assert not runs[0][3] and runs[2][3] and runs[3][3]
+        assert same(runs[2], ref_attacked) and same(runs[3], ref_attacked)
+        plan.set_optimistic(2)
+        a = _decode(plan, coded)
+        b = _decode(plan, coded)
+        assert a[3] and b[3] and same(b, ref_clean)
+        assert np.abs(a[1].cpu().numpy() - want).max() <= 1e-9 * scale
+
+
 def test_plans_that_are_not_eligible_ignore_the_mode():
-    for P, s, m, dtype in ((15, 1, 10, "f32"), (105, 1, 1, "f32"), (15, 2, 5, "f64")):
+    for P, s, m, dtype in ((15, 1, 10, "f32"), (105, 1, 1, "f32"), (15, 1, 8, "f64")):
         wl = synth.Workload("inel", P, s, m, 30_000, "normal", 1.0, "none", 0, 5)
         G = synth.make_grads(wl, "cuda")
         if dtype == "f64":
