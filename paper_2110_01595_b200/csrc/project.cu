@@ -756,7 +756,7 @@ static int launch_project_pipe_k(solon_plan* plan, const T* received, double* rh
   ProjPipe pp;
   pp.status = plan->d_status;
   pp.progress = plan->d_proj_progress;
-  // optimistic decode: only in the whole decode (the aggregate's buffer is known) of a float32 plan that is eligible
+  // optimistic decode: only in the whole decode (the aggregate's buffer is known) of a plan that is eligible
   pp.opt_rows = (!final_reduce && agg && plan->optimistic != 0) ? plan->opt_rows : 0;
   for (int j = 0; j < kPipeRows; ++j) pp.spec_src[j] = j < pp.opt_rows ? (uint16_t)plan->opt_src_host[(size_t)j] : 0;
   pp.q = plan->q;
