@@ -289,9 +289,6 @@ def run_ours(args, wl):
     if status != 0 or mask.nonzero().flatten().tolist() != nodes:
         raise RuntimeError(f"warm-up decode failed: status {status}")
     n_rec, _, _, _ = plan.recovery()
-    # optimistic decode: when the recovery kernel had nothing to do, the decode read the received matrix once
-    skipped = bool(plan.optimistic_outcome()) if sp is None else False
-    enc_b, proj_b, rec_b = algorithmic_bytes(wl, 0 if skipped else int(n_rec.sum()), eb)
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -326,6 +323,10 @@ def run_ours(args, wl):
     status = plan.decode_status()
     if status != 0 or mask.nonzero().flatten().tolist() != nodes:
         raise RuntimeError(f"timed decode failed: status {status}")
+    # optimistic decode: when the recovery kernel had nothing to do (asked after the last timed decode: a steady state
+    # reached during the warm-up holds from then on), the decode read the received matrix once
+    skipped = bool(plan.optimistic_outcome()) if sp is None else False
+    enc_b, proj_b, rec_b = algorithmic_bytes(wl, 0 if skipped else int(n_rec.sum()), eb)
 
     # the same decode with projection vectors drawn anew for every decode (solon_plan_set_fresh_projections; Algorithm 1
     # draws its random vector inside the decoder) instead of reused
@@ -490,7 +491,7 @@ def run_sweep(args):
                 if ev:
                     ev[3].record()
 
-            for _ in range(3):
+            for _ in range(4):      # the single-pass decode, where a plan has one, is the steady state from the fourth decode on
                 step()
             torch.cuda.synchronize()
             n_steps = max(3, min(args.steps, 10))

@@ -164,13 +164,13 @@ int solon_plan_set_early_locator(solon_plan* plan, int mode);
  * table for no corrupt node) to each column slice as it passes and write the aggregate itself.  If the locator then
  * finds all of those rows trusted in THIS decode, the recovery kernel returns at once and the decode has read the
  * received matrix once instead of 1 + q m / P times: with no attackers, or with attackers that stay where they were,
- * every decode from the second or third on.  If one of those rows is corrupt now, the recovery kernel runs as usual and
+ * every decode from the third or fourth on.  If one of those rows is corrupt now, the recovery kernel runs as usual and
  * overwrites the aggregate.  The mask never depends on the mode.  The aggregate is computed in the recovery kernel's
  * arithmetic and order: bit for bit what mode 0 gives whenever the previous table is also this decode's table (same
  * corrupt set), and the same sum up to the rounding of the plan's element type when it came from other trusted rows - so with mode 1 or 2 the
  * last bits of an aggregate can depend on the decode before it; mode 0 gives history-independent bits.
- * mode 0: never; 1 (default): when the previous decode's table would have served that decode too (its rows were all
- * trusted; decided on the device, no host round trip); 2: always.  Eligible plans (either element type): s > 0, m <= 6
+ * mode 0: never; 1 (default): when in each of the last two decodes the table of the decode before would have served (its
+ * rows were all trusted: the attackers, if any, stay where they are; decided on the device, no host round trip); 2: always.  Eligible plans (either element type): s > 0, m <= 6
  * and q m rows fitting in the projection kernel's first batch of rows (at most 32); other plans ignore the mode. */
 int solon_plan_set_optimistic(solon_plan* plan, int mode);
 /* *skipped = 1 if the recovery kernel of the most recent solon_decode had nothing to do.  Synchronises. */

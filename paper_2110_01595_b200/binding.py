@@ -240,7 +240,7 @@ class Plan:
 
     def set_optimistic(self, mode: int) -> None:
         """0: the projection pass never recovers the aggregate itself; 1 (default): it does so, from the rows of the previous
-        decode's recovery table, when that table would have served the previous decode too; 2: always.  The recovery
+        decode's recovery table, when in each of the last two decodes the table of the decode before would have served; 2: always.  The recovery
         kernel is skipped when the locator finds those rows trusted in this decode."""
         _check(lib().solon_plan_set_optimistic(self._h, mode), "solon_plan_set_optimistic")
 

@@ -53,7 +53,8 @@ struct LocateParams {
   int* rec_rows;         // P
   double* coeff;         // P x m
   int* status;
-  int* opt;              // optimistic decode: opt[8 + g] receives whether the rows of group g's previous recovery table are trusted now
+  int* opt;              // optimistic decode: opt[8 + g] counts (up to 2) the decodes in a row in which the rows of group g's previous
+                         // recovery table were all trusted (0: not in this decode)
   int opt_track;         // the plan can decode optimistically (m <= 6): keep opt[8 + g] (else it is written as 0)
   DrawParams draw;       // the vectors f of the next decode, written by the CTAs beyond the q locator CTAs (n_draw_ctas of them)
   int n_draw_ctas;
@@ -162,10 +163,13 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
   __shared__ int s_n_rec, s_t_acc;
   // Optimistic decode: the rows of this group's recovery table as the previous decode left it - the rows the projection
   // kernel of THIS decode may have recovered from - are read before anything here overwrites them.
-  __shared__ int s_old_row[SOLON_SUBSET_MAX_M], s_old_n;
+  __shared__ int s_old_row[SOLON_SUBSET_MAX_M], s_old_n, s_old_streak;
   if (prm.opt_track) {
     if (tid < prm.m) s_old_row[tid] = prm.rec_rows[row0 + tid];
-    if (tid == 0) s_old_n = prm.n_rec[g];
+    if (tid == 0) {
+      s_old_n = prm.n_rec[g];
+      s_old_streak = prm.opt[8 + g];
+    }
   }
   GroupTables tb;
   tb.Qb = prm.qb + prm.qb_off[g];
@@ -316,7 +320,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
           prm.n_rec[g] = n_rec;
           prm.t_acc[g] = s_t_acc;
           prm.early[g] = 1;
-          prm.opt[8 + g] = old_rows_trusted(prm, s_old_row, s_old_n, s_t_acc, sc.mask_l, row0, n);
+          prm.opt[8 + g] = old_rows_trusted(prm, s_old_row, s_old_n, s_t_acc, sc.mask_l, row0, n) ? min(s_old_streak + 1, 2) : 0;
         }
         return;
       }
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
       prm.n_rec[g] = n_rec;
       prm.t_acc[g] = s_t_acc;
       prm.early[g] = !prm.spec ? 0 : (s_ready > 0 ? 2 : (s_ready == 0 ? 3 : 4));
-      prm.opt[8 + g] = old_rows_trusted(prm, s_old_row, s_old_n, s_t_acc, sc.mask_l, row0, n);
+      prm.opt[8 + g] = old_rows_trusted(prm, s_old_row, s_old_n, s_t_acc, sc.mask_l, row0, n) ? min(s_old_streak + 1, 2) : 0;
       (void)ok;      // an undecodable group is reported through t_acc[g] = -1
     }
   }

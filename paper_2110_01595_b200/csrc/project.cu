@@ -234,7 +234,7 @@ struct ProjPipe {
   int* status;
   // Optimistic decode.  The rows of the locator's last recovery table (m per group: what the previous decode's recovery
   // read; opt_rows of them over all groups, ascending) are the ones this decode speculates on.  When the device flags say
-  // so (mode 2, or mode 1 and the previous decode's flags all set) the consumers also recover the aggregate of every
+  // so (mode 2, or mode 1 and every group's count at 2: the last two decodes' previous tables both held) the consumers also recover the aggregate of every
   // column slice from them, exactly as the recovery kernel would with that table.  They must all lie in one stage of the
   // ring: with a single batch of rows the order stays the natural one and nothing has to come from device memory before
   // the first loads are issued; with several batches they are taken first (the other rows follow in ascending order),
@@ -535,12 +535,12 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
     pipe::fence_barrier_init();
   }
   // Optimistic decode: does this pass also recover the aggregate, from the rows of the last recovery table?
-  // Mode 2, or mode 1 and every flag of the previous decode set; and only if that table is whole (m rows in every group,
+  // Mode 2, or mode 1 and every group's count at 2 (two decodes in a row whose previous table held); and only if that table is whole (m rows in every group,
   // ascending node indices).  Flags, rows and weights are fetched here - one load per thread - and looked at only when the
   // first stage's projection work is done (see below), so that their round trip to device memory hides behind it; with
   // several batches of rows the row order depends on the list, and the kernel waits for it here.  CTA 0 records the
   // answer for this decode's recovery kernel (0 until it is known).
-  int opt_mode = 0, opt_flag = 1, spec_row = 0;      // raw values: nothing is computed from them before they are needed
+  int opt_mode = 0, opt_flag = 2, spec_row = 0;      // raw values: nothing is computed from them before they are needed
   bool spec_whole = false;
   double spec_coeff = 0.0;
   {
@@ -672,7 +672,7 @@ __global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) project_pipe_ker
                   const bool lane_ok = spec_whole && (tid >= pp.opt_rows || (spec_row >= 0 && spec_row < P && (tid == 0 || spec_row > below)));
                   spec_whole = __all_sync(0xffffffffu, lane_ok);
                 }
-                const bool all_clean = __all_sync(0xffffffffu, opt_flag != 0);
+                const bool all_clean = __all_sync(0xffffffffu, opt_flag >= 2);     // two decodes in a row whose previous table held
                 if (tid == 0) {
                   s_opt_on = (spec_whole && (opt_mode == 2 || (opt_mode == 1 && all_clean))) ? 1 : 0;
                   if (blockIdx.x == 0) pp.opt_flags[1] = s_opt_on;

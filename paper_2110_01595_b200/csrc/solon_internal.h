@@ -75,11 +75,11 @@ struct solon_plan {
   // optimistic decode (solon_plan_set_optimistic): the projection pass also writes the aggregate, recovered from the rows
   // of the locator's last recovery table (d_rec_rows, d_coeff: what the previous decode's recovery read; before the first
   // decode the table for no corrupt node), and the recovery kernel is skipped when the locator finds all of them trusted
-  int optimistic;          // 0 never, 1 when the previous decode's table would have served that decode too (default), 2 always
+  int optimistic;          // 0 never, 1 when in each of the last two decodes the table of the decode before would have served (default), 2 always
   int opt_rows;            // rows speculated on over all groups: q m (0: the plan is not eligible)
   std::vector<int> opt_src_host;   // their positions in d_rec_rows (and rows of d_coeff): group_start[g] + j, j < m
   int* d_opt;              // [1] the projection pass of this decode recovered too, [4] mode (copied from `optimistic`),
-                           // [8 + g] the rows of group g that the last decode could have speculated on were all trusted in it
+                           // [8 + g] decodes in a row (up to 2) in which the rows group g could have speculated on were all trusted
   int draw_parity;         // which buffer holds the current draw of f (0, 1), or -1: only the device knows (decodes draw anew)
   float* d_f;              // K x f_pitch projection vectors: the draws with an even index
   float* d_f2;             // the draws with an odd index

@@ -57,16 +57,16 @@ def test_full_size(name):
         # a property that holds at any size: the whole aggregate against a float64 device-side sum
         ref = G.sum(dim=0, dtype=torch.float64)
         assert float((agg.double() - ref).abs().max()) <= AGG_TOL * scale
-        # the benchmark's steady state: attackers that stay where they are, so the third decode recovers the aggregate inside
-        # the projection pass from the rows the second one trusted (single-pass decode) - same checks on its outputs
-        for _ in range(2):
+        # the benchmark's steady state: attackers that stay where they are, so the fourth decode recovers the aggregate inside
+        # the projection pass from the rows the third one trusted (single-pass decode) - same checks on its outputs
+        for _ in range(3):
             agg2, mask2 = plan.decode(received)
         assert plan.decode_status() == 0 and plan.optimistic_outcome()
         assert torch.equal(mask2, mask)
         got_s2 = agg2[torch.from_numpy(cols[in_range]).cuda()].cpu().numpy().astype(np.float64)
         assert np.abs(got_s2 - want_s).max() <= AGG_TOL * scale
         assert float((agg2.double() - ref).abs().max()) <= AGG_TOL * scale
-        assert torch.equal(agg2, agg)          # the second decode's table is the first one's: the same bits
+        assert torch.equal(agg2, agg)          # the third decode's table is the first one's: the same bits
         if name == "resnet18":
             # projections of the full received matrix against the oracle's matrix product
             f = plan.projection_vectors()

@@ -66,23 +66,23 @@ def test_modes_agree_with_and_without_attackers(name, d, early):
             ok = got[0] == ref[0] and torch.equal(got[2], ref[2]) and np.abs(got[1].cpu().numpy() - want).max() <= AGG_TOL * scale
             return ok and (got[3] or same(got, ref))
 
-        # mode 1: optimistic when the previous decode's table would have served that decode too
+        # mode 1: optimistic when in each of the last two decodes the table of the decode before would have served
         plan.set_optimistic(1)
-        first = _decode(plan, coded)            # nothing known yet: the ordinary path
-        second = _decode(plan, coded)           # recovers from the table of `first`, the locator confirms, the recovery skips
-        assert not first[3] and second[3]
-        assert same(first, ref_clean) and same(second, ref_clean)
-        # attackers arrive and stay: from the third decode on the table of the decode before avoids them
-        runs = [_decode(plan, attacked) for _ in range(4)]
+        clean = [_decode(plan, coded) for _ in range(4)]
+        # nothing known at first; the third recovers from the table of the second, the locator confirms, the recovery skips
+        assert [x[3] for x in clean] == [False, False, True, True]
+        assert all(same(x, ref_clean) for x in clean)
+        # attackers arrive and stay: from the fourth decode on at the latest the table of the decode before avoids them
+        runs = [_decode(plan, attacked) for _ in range(5)]
         assert all(agrees(got, ref_attacked) for got in runs)
-        assert runs[2][3] and runs[3][3] and same(runs[2], ref_attacked) and same(runs[3], ref_attacked)
+        assert runs[3][3] and runs[4][3] and same(runs[3], ref_attacked) and same(runs[4], ref_attacked)
         # they move onto a row of that table: the speculation fails, the recovery kernel runs as usual
         moved = _decode(plan, attacked_b)
         assert not moved[3] and same(moved, ref_moved)
-        after = _decode(plan, attacked_b)       # the previous table would not have served: the ordinary path
-        assert not after[3] and same(after, ref_moved)
+        after = [_decode(plan, attacked_b) for _ in range(2)]       # no speculation until two tables in a row have held
+        assert not after[0][3] and not after[1][3] and all(same(got, ref_moved) for got in after)
         settled = [_decode(plan, attacked_b) for _ in range(2)]
-        assert settled[1][3] and all(same(got, ref_moved) for got in settled)
+        assert settled[0][3] and settled[1][3] and all(same(got, ref_moved) for got in settled)
         # mode 2: always (from whatever table the last decode left)
         plan.set_optimistic(2)
         a = _decode(plan, attacked)
@@ -161,13 +161,13 @@ def test_float64_plans(P, s, m, r, d):
             return got[0] == ref[0] and torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
 
         plan.set_optimistic(1)
-        runs = [_decode(plan, attacked) for _ in range(4)]
+        runs = [_decode(plan, attacked) for _ in range(5)]
         for got in runs:
             assert got[0] == 0 and torch.equal(got[2], ref_attacked[2])
             assert np.abs(got[1].cpu().numpy() - want).max() <= 1e-9 * scale
             assert got[3] or same(got, ref_attacked)
-        assert not runs[0][3] and runs[2][3] and runs[3][3]
-        assert same(runs[2], ref_attacked) and same(runs[3], ref_attacked)
+        assert not runs[0][3] and not runs[1][3] and runs[3][3] and runs[4][3]
+        assert same(runs[3], ref_attacked) and same(runs[4], ref_attacked)
         plan.set_optimistic(2)
         a = _decode(plan, coded)
         b = _decode(plan, coded)
