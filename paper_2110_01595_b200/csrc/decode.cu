@@ -125,6 +125,68 @@ __global__ void __launch_bounds__(256) overwrite_rows_kernel(T* __restrict__ mat
   }
 }
 
+// The same when rows do not start on 16-byte boundaries (d_c not a multiple of 16 bytes): 16-byte stores at the destination
+// row's own boundaries, each taking its values from the two 16-byte words of the source row that hold them (the offset
+// between the two rows' boundaries is the same along the whole row); the elements before the first and after the last
+// whole word, and the first and last word themselves, go one by one.
+template <typename T>
+__global__ void __launch_bounds__(256) overwrite_rows_shifted_kernel(T* __restrict__ matrix, const T* __restrict__ rows,
+                                                                     const int* __restrict__ nodes, int P, int64_t d_c, int stream_hints) {
+  constexpr int kVec = 16 / sizeof(T);     // elements per 16 bytes
+  union Word {
+    float4 v;
+    T e[kVec];
+  };
+  const int node = nodes[blockIdx.y];
+  if (node < 0 || node >= P) return;
+  T* dst = matrix + (int64_t)node * d_c;
+  const T* src = rows + (int64_t)blockIdx.y * d_c;
+  int64_t head = (int64_t)((kVec - (((uintptr_t)dst / sizeof(T)) & (kVec - 1))) & (kVec - 1));    // elements before dst's first boundary
+  if (head > d_c) head = d_c;
+  const int64_t n_words = (d_c - head) / kVec;
+  const int64_t body_end = head + n_words * kVec;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  if (blockIdx.x == 0) {
+    const int64_t first_end = n_words > 0 ? head + kVec : head;
+    const int64_t last_begin = n_words > 1 ? body_end - kVec : body_end;
+    for (int64_t i = threadIdx.x; i < first_end; i += blockDim.x) dst[i] = src[i];
+    for (int64_t i = last_begin + threadIdx.x; i < d_c; i += blockDim.x) dst[i] = src[i];
+  }
+  if (n_words < 3) return;
+  const T* s0 = src + head;                                                      // source of dst's first whole word
+  const int delta = (int)(((uintptr_t)s0 / sizeof(T)) & (kVec - 1));           // its offset from a 16-byte boundary of its own
+  const float4* sw = reinterpret_cast<const float4*>(s0 - delta);              // word i of dst comes from sw[i] and sw[i + 1]
+  float4* dw = reinterpret_cast<float4*>(dst + head);
+  // words 1 .. n_words - 2: both source words lie inside the row; four words (eight loads) in flight per thread
+  for (int64_t i = 1 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words - 1; i += 4 * stride) {
+    Word a[4], b[4], o[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t w = i + u * stride;
+      if (w < n_words - 1) {
+        a[u].v = __ldcs(sw + w);
+        if (delta) b[u].v = __ldcs(sw + w + 1);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t w = i + u * stride;
+      if (w < n_words - 1) {
+#pragma unroll
+        for (int k = 0; k < kVec; ++k) {
+          T val = a[u].e[k];                                   // delta == 0
+#pragma unroll
+          for (int dlt = 1; dlt < kVec; ++dlt)
+            if (delta == dlt) val = dlt + k < kVec ? a[u].e[(dlt + k) % kVec] : b[u].e[(dlt + k) % kVec];
+          o[u].e[k] = val;
+        }
+        if (stream_hints) __stcs(dw + w, o[u].v);
+        else dw[w] = o[u].v;
+      }
+    }
+  }
+}
+
 template <typename T>
 static int overwrite_rows_t(solon_plan* plan, T* matrix, int n_rows, const int* nodes, const T* rows) {
   if (!plan || n_rows < 0 || n_rows > plan->P) return SOLON_ERR_INVALID_ARG;
@@ -134,12 +196,17 @@ static int overwrite_rows_t(solon_plan* plan, T* matrix, int n_rows, const int* 
   constexpr int kVec = 16 / sizeof(T);
   const int vec = (plan->d_c % kVec == 0 && !((uintptr_t)matrix & 15) && !((uintptr_t)rows & 15)) ? 1 : 0;
   // one wave of CTAs (eight per SM) shared by the rows; every thread then has several batches of eight accesses
-  int64_t per_row = (plan->d_c / (vec ? kVec : 1) + 256 * 8 - 1) / (256 * 8);
+  const bool shifted = !vec && plan->d_c >= 64;      // rows off 16-byte boundaries: realign (element pointers are element-aligned)
+  int64_t per_row = (plan->d_c / ((vec || shifted) ? kVec : 1) + 256 * 8 - 1) / (256 * 8);
   int64_t cap = ((int64_t)plan->num_sms * 8 + n_rows - 1) / n_rows;
   if (per_row > cap) per_row = cap;
   if (per_row < 1) per_row = 1;
-  overwrite_rows_kernel<T><<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec,
-                                                                                               plan->stream_hints);
+  if (shifted)
+    overwrite_rows_shifted_kernel<T><<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c,
+                                                                                                         plan->stream_hints);
+  else
+    overwrite_rows_kernel<T><<<dim3((unsigned)per_row, (unsigned)n_rows), 256, 0, plan->stream>>>(matrix, rows, nodes, plan->P, plan->d_c, vec,
+                                                                                                 plan->stream_hints);
   SOLON_CUDA_TRY(cudaGetLastError());
   plan->launches += 1;
   return SOLON_OK;

@@ -475,18 +475,22 @@ def test_step_host_matches_device_path():
         assert np.abs(agg_h.numpy() - want).max() <= AGG_TOL * np.abs(want).max()
 
 
-@pytest.mark.parametrize("d", [40_000, 40_003])
-def test_overwrite_rows(d):
-    with binding.Plan(15, 2, 1, 5, d) as plan:      # m = 1: d_c = d, a multiple of 4 or not
+@pytest.mark.parametrize("dtype", ["f32", "f64"])
+@pytest.mark.parametrize("d", [40_000, 40_001, 40_002, 40_003, 77, 70, 66, 5])
+def test_overwrite_rows(d, dtype):
+    """Rows that start on 16-byte boundaries or not: every offset between a source row's and a destination row's boundaries
+    occurs among the rows below for the odd widths (the copy realigns), and short rows go element by element."""
+    tdtype = torch.float32 if dtype == "f32" else torch.float64
+    with binding.Plan(15, 2, 1, 5, d, dtype=dtype) as plan:      # m = 1: d_c = d
         g = torch.Generator(device="cuda").manual_seed(3)
-        matrix = torch.randn(15, d, device="cuda", generator=g)
+        matrix = torch.randn(15, d, device="cuda", generator=g, dtype=tdtype)
         before = matrix.clone()
-        rows = torch.randn(4, d, device="cuda", generator=g)
-        nodes = torch.tensor([14, 0, 99, 7], dtype=torch.int32, device="cuda")      # 99: out of range, skipped
+        rows = torch.randn(6, d, device="cuda", generator=g, dtype=tdtype)
+        nodes = torch.tensor([14, 0, 99, 7, 9, 2], dtype=torch.int32, device="cuda")      # 99: out of range, skipped
         plan.overwrite_rows(matrix, nodes, rows)
         torch.cuda.synchronize()
         want = before.clone()
-        want[14], want[0], want[7] = rows[0], rows[1], rows[3]
+        want[14], want[0], want[7], want[9], want[2] = rows[0], rows[1], rows[3], rows[4], rows[5]
         assert torch.equal(matrix, want)
         plan.overwrite_rows(matrix, nodes[:0], rows[:0])                             # nothing to do
         assert torch.equal(matrix, want)
