@@ -56,6 +56,8 @@ struct LocateParams {
   int* opt;              // optimistic decode: opt[8 + g] counts (up to 2) the decodes in a row in which the rows of group g's previous
                          // recovery table were all trusted (0: not in this decode)
   int opt_track;         // the plan can decode optimistically (m <= 6): keep opt[8 + g] (else it is written as 0)
+  int opt_given_projections;      // this decode's projections did not come from the plan's own projection kernel just before (given by the
+                         // caller): no aggregate was recovered ahead, whatever opt[1] still says from an earlier decode
   DrawParams draw;       // the vectors f of the next decode, written by the CTAs beyond the q locator CTAs (n_draw_ctas of them)
   int n_draw_ctas;
 };
@@ -156,6 +158,7 @@ __global__ void __launch_bounds__(32 * (SOLON_MAX_S + 1)) locate_kernel(LocatePa
     draw_projection_vectors(prm.draw, 1, g - ((int)gridDim.x - prm.n_draw_ctas), prm.n_draw_ctas, tid, n_threads);
     return;
   }
+  if (g == 0 && tid == 0 && prm.opt_given_projections) prm.opt[1] = 0;     // (the recovery kernel reads it after this grid)
   const int row0 = prm.group_start[g];
   const int n = prm.group_start[g + 1] - row0;
   double* ws = prm.use_smem ? smem_ws : prm.ws_global + (size_t)g * prm.ws_stride;
@@ -546,6 +549,7 @@ int launch_locate(solon_plan* plan, uint8_t* byz_mask, const double* rho, const 
     SOLON_CUDA_TRY(cudaFuncSetAttribute(locate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prm.opt = plan->d_opt;
   prm.opt_track = plan->opt_rows > 0 ? 1 : 0;
+  prm.opt_given_projections = (rho || nu) ? 1 : 0;
   // CTAs that draw the next decode's vectors beside the locator's: a few per SM, a thread per several quads
   prm.draw = draw_params(plan);
   prm.n_draw_ctas = 0;

@@ -175,6 +175,27 @@ def test_float64_plans(P, s, m, r, d):
         assert np.abs(a[1].cpu().numpy() - want).max() <= 1e-9 * scale
 
 
+def test_finish_with_given_projections_after_a_single_pass_decode():
+    """solon_decode_finish with projections that did not come from this plan's own projection kernel just before: the
+    recovery kernel must run, whatever the last whole decode of the plan did."""
+    wl = synth.small_variant(synth.WORKLOADS["resnet18"], 120_007)
+    G_a = synth.make_grads(wl, "cuda")
+    G_b = synth.make_grads(dataclasses.replace(wl, seed=wl.seed + 1), "cuda")
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=9) as plan, binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=9) as other:
+        coded_a, coded_b = plan.encode(G_a), plan.encode(G_b)
+        for _ in range(4):
+            agg_a, _ = plan.decode(coded_a)
+        assert plan.optimistic_outcome()                     # the plan's last decode was a single-pass one
+        rho = torch.empty(plan.K, wl.P, dtype=torch.float64, device="cuda")
+        nu = torch.empty(wl.P, dtype=torch.float64, device="cuda")
+        other.decode_project(coded_b, rho, nu)               # same seed: the same vectors f
+        agg_b = torch.full((wl.d,), float("nan"), dtype=torch.float32, device="cuda")
+        _, mask = plan.decode_finish(rho, nu, coded_b, agg_b)
+        assert plan.decode_status() == 0 and int(mask.sum()) == 0 and not plan.optimistic_outcome()
+        ref = G_b.sum(dim=0, dtype=torch.float64)
+        assert float((agg_b.double() - ref).abs().max()) <= AGG_TOL * float(ref.abs().max())
+
+
 def test_plans_that_are_not_eligible_ignore_the_mode():
     for P, s, m, dtype in ((15, 1, 10, "f32"), (105, 1, 1, "f32"), (15, 1, 8, "f64")):
         wl = synth.Workload("inel", P, s, m, 30_000, "normal", 1.0, "none", 0, 5)
