@@ -45,14 +45,16 @@ __device__ __forceinline__ void load_tables(const Prm& prm, Acc* coeff_s, int* r
 // weights at coeff_c[i * STRIDE .. + M) (STRIDE: M rounded up so that every row of weights starts on a 16-byte
 // boundary and can be fetched with 128-bit loads).  Returns the number of rows in use.
 // coeff_s (P x M), rows_s, slots_s (P each), start_s (q + 1), n_rec_s (q): staging.
+// nothing_to_do: this thread's view of "the aggregate is already there" (optimistic decode); when every thread of the CTA
+// says so the routine returns -1 at its first barrier, before it packs anything.
 template <typename Acc, int M, int STRIDE, int VEC, typename Prm>
 __device__ __forceinline__ int pack_tables(const Prm& prm, int* rows_s, Acc* coeff_s, int* slots_s, int* start_s,
-                                           int* n_rec_s, int* count_s, Acc* coeff_c, int* rowsh_c) {
+                                           int* n_rec_s, int* count_s, Acc* coeff_c, int* rowsh_c, int nothing_to_do) {
   for (int i = threadIdx.x; i < prm.P * M; i += blockDim.x) coeff_s[i] = (Acc)prm.coeff[i];
   for (int i = threadIdx.x; i < prm.P; i += blockDim.x) rows_s[i] = prm.rec_rows[i];
   for (int i = threadIdx.x; i <= prm.q; i += blockDim.x) start_s[i] = prm.group_start[i];
   for (int i = threadIdx.x; i < prm.q; i += blockDim.x) n_rec_s[i] = prm.n_rec[i];
-  __syncthreads();
+  if (__syncthreads_and(nothing_to_do)) return -1;
   for (int g = threadIdx.x; g < prm.q; g += blockDim.x) {
     int base = 0;
     for (int o = 0; o < g; ++o) base += min(max(n_rec_s[o], 0), start_s[o + 1] - start_s[o]);
@@ -162,8 +164,8 @@ __global__ void __launch_bounds__(NC + 32, kCtasPerSm) recover_kernel(RecoverPar
   // (no branch on the first word before the other loads: they all go out together with the table loads below)
   int clean = prm.opt[1] != 0 ? 1 : 0;
   for (int g = tid; g < prm.q; g += blockDim.x) clean &= prm.opt[8 + g] != 0 ? 1 : 0;
-  const int n_rows = pack_tables<Acc, M, kStride, (int)kVec>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c);
-  if (__syncthreads_and(clean)) return;   // every group's default rows were confirmed and the projection pass recovered from them
+  const int n_rows = pack_tables<Acc, M, kStride, (int)kVec>(prm, rows_p, coeff_p, slots_p, start_s, n_rec_s, count_s, coeff_c, rowsh_c, clean);
+  if (n_rows < 0) return;   // the rows the projection pass recovered from were all confirmed: the aggregate stands
   const int64_t n_tiles = (prm.d_c + kTileChunks - 1) / kTileChunks;
   const int64_t total_floats = (int64_t)prm.P * prm.d_c;
 
