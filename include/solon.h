@@ -171,7 +171,9 @@ int solon_plan_set_early_locator(solon_plan* plan, int mode);
  * last bits of an aggregate can depend on the decode before it; mode 0 gives history-independent bits.
  * mode 0: never; 1 (default): when in each of the last two decodes the table of the decode before would have served (its
  * rows were all trusted: the attackers, if any, stay where they are; decided on the device, no host round trip); 2: always.  Eligible plans (either element type): s > 0, m <= 6
- * and q m rows fitting in the projection kernel's first batch of rows (at most 32); other plans ignore the mode. */
+ * and q m rows fitting in the projection kernel's first batch of rows (at most 32); other plans ignore the mode.
+ * A decode captured in a CUDA graph keeps deciding on the device at every replay; only a graph captured in mode 0
+ * never speculates, whatever the mode set later (its projection kernel was launched without the rows to recover from). */
 int solon_plan_set_optimistic(solon_plan* plan, int mode);
 /* *skipped = 1 if the recovery kernel of the most recent solon_decode had nothing to do.  Synchronises. */
 int solon_plan_get_optimistic_outcome(solon_plan* plan, int* skipped);

@@ -175,6 +175,55 @@ def test_float64_plans(P, s, m, r, d):
         assert np.abs(a[1].cpu().numpy() - want).max() <= 1e-9 * scale
 
 
+def test_replayed_graph_goes_over_to_the_single_pass_decode():
+    """The decision lives on the device: a decode captured in a CUDA graph before anything was known speculates in later
+    replays once two tables in a row have held, and falls back when the attackers move (the received matrix is rewritten
+    in place between replays)."""
+    wl = synth.small_variant(synth.WORKLOADS["vgg13"], 400_003)
+    G = synth.make_grads(wl, "cuda")
+    want = so.plain_sum(G.cpu().numpy())
+    scale = np.abs(want).max()
+    with binding.Plan(wl.P, wl.s, wl.m, wl.r, wl.d, seed=11) as plan:
+        coded = plan.encode(G)
+        attacked, nodes = synth.apply_attack(dataclasses.replace(wl, attack="gaussian", n_byz=wl.s), coded)
+        plan.set_optimistic(0)
+        ref_clean = _decode(plan, coded)
+        ref_attacked = _decode(plan, attacked)
+        received = coded.clone()
+        agg = torch.empty(wl.d, dtype=torch.float32, device="cuda")
+        mask = torch.empty(wl.P, dtype=torch.uint8, device="cuda")
+        plan.set_optimistic(1)                        # the mode in force at capture decides whether the captured kernel can speculate at all
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            plan.set_stream(side)
+            plan.decode(received, agg, mask)          # warm-up on the capture stream, as graph capture wants
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            plan.set_stream(torch.cuda.current_stream())
+            plan.decode(received, agg, mask)
+        plan.set_stream(torch.cuda.current_stream())
+        plan.set_optimistic(1)                        # again: the flags start from nothing
+
+        def replay():
+            graph.replay()
+            torch.cuda.synchronize()
+            return plan.decode_status(), agg.clone(), mask.clone(), plan.optimistic_outcome()
+
+        clean = [replay() for _ in range(4)]
+        assert [x[3] for x in clean] == [False, False, True, True]
+        assert all(x[0] == 0 and torch.equal(x[1], ref_clean[1]) and torch.equal(x[2], ref_clean[2]) for x in clean)
+        received.copy_(attacked)                      # attackers arrive and stay
+        runs = [replay() for _ in range(5)]
+        for x in runs:
+            assert x[0] == 0 and torch.equal(x[2], ref_attacked[2])
+            assert np.abs(x[1].cpu().numpy() - want).max() <= AGG_TOL * scale
+        assert runs[3][3] and runs[4][3] and torch.equal(runs[4][1], ref_attacked[1])
+        assert mask.nonzero().flatten().tolist() == nodes
+
+
 def test_finish_with_given_projections_after_a_single_pass_decode():
     """solon_decode_finish with projections that did not come from this plan's own projection kernel just before: the
     recovery kernel must run, whatever the last whole decode of the plan did."""
