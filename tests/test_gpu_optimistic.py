@@ -175,6 +175,49 @@ def test_float64_plans(P, s, m, r, d):
         assert np.abs(a[1].cpu().numpy() - want).max() <= 1e-9 * scale
 
 
+def test_random_plans_with_attackers_that_stay_and_move():
+    """Random (P, s, m, r, d), a random walk of Byzantine sets (stay for a few decodes, then move; sometimes none): every
+    decode, speculated or not, gives the exact mask and the aggregate within the tolerance; single-pass decodes do occur."""
+    rng = np.random.default_rng(2024)
+    seen_single_pass = 0
+    for trial in range(24):
+        m = int(rng.choice([1, 2, 3, 4, 5, 6]))
+        s = int(rng.integers(1, 4))
+        r = 2 * s + m + int(rng.integers(0, 3))
+        q = int(rng.integers(1, 5))
+        P = q * r + int(rng.integers(0, r))
+        d = int(rng.integers(3_000, 60_000))
+        dtype = "f64" if trial % 4 == 3 else "f32"
+        wl = synth.Workload("opt_rand", P, s, m, d, "normal", 1.0, "gaussian", 0, 100 + trial)
+        G = synth.make_grads(wl, "cuda")
+        if dtype == "f64":
+            G = G.double()
+        ref = G.sum(dim=0, dtype=torch.float64)
+        scale = float(ref.abs().max())
+        tol = (1e-9 if dtype == "f64" else AGG_TOL) * scale
+        sizes = so.group_sizes(P, r)
+        starts = np.concatenate([[0], np.cumsum(sizes)])
+        with binding.Plan(P, s, m, r, d, seed=trial, dtype=dtype) as plan:
+            coded = plan.encode(G)
+            nodes = []
+            for step in range(14):
+                if step % 4 == 0:          # the Byzantine set moves: up to s nodes in each group, or nobody
+                    nodes = []
+                    if rng.random() < 0.8:
+                        for g in range(len(sizes)):
+                            k = int(rng.integers(0, s + 1))
+                            nodes += sorted((starts[g] + rng.choice(sizes[g], size=k, replace=False)).tolist())
+                received = coded.clone()
+                if nodes:
+                    received[nodes] = synth.byzantine_rows(dataclasses.replace(wl, n_byz=len(nodes)), coded, nodes)
+                agg, mask = plan.decode(received)
+                assert plan.decode_status() == 0, (trial, step)
+                assert mask.nonzero().flatten().tolist() == sorted(nodes), (trial, step)
+                assert float((agg.double() - ref).abs().max()) <= tol, (trial, step)
+                seen_single_pass += int(plan.optimistic_outcome())
+    assert seen_single_pass >= 24
+
+
 def test_replayed_graph_goes_over_to_the_single_pass_decode():
     """The decision lives on the device: a decode captured in a CUDA graph before anything was known speculates in later
     replays once two tables in a row have held, and falls back when the attackers move (the received matrix is rewritten
