@@ -288,6 +288,22 @@ def test_finish_with_given_projections_after_a_single_pass_decode():
         assert float((agg_b.double() - ref).abs().max()) <= AGG_TOL * float(ref.abs().max())
 
 
+def test_mode_argument_is_checked():
+    with binding.Plan(8, 1, 2, 4, 4096) as plan:
+        lib = binding.lib()
+        for bad in (-1, 3, 17):
+            assert lib.solon_plan_set_optimistic(plan._h, bad) == binding.ERR_INVALID_ARG
+        assert lib.solon_plan_set_optimistic(None, 1) == binding.ERR_INVALID_ARG
+        assert plan.status() == 0
+        G = torch.randn(8, 4096, device="cuda")
+        coded = plan.encode(G)
+        for _ in range(4):                       # the default mode is still in force
+            agg, mask = plan.decode(coded)
+        assert plan.decode_status() == 0 and plan.optimistic_outcome() and int(mask.sum()) == 0
+        ref = G.sum(dim=0, dtype=torch.float64)
+        assert float((agg.double() - ref).abs().max()) <= AGG_TOL * float(ref.abs().max())
+
+
 def test_plans_that_are_not_eligible_ignore_the_mode():
     for P, s, m, dtype in ((15, 1, 10, "f32"), (105, 1, 1, "f32"), (15, 1, 8, "f64")):
         wl = synth.Workload("inel", P, s, m, 30_000, "normal", 1.0, "none", 0, 5)
