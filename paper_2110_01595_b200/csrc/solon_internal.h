@@ -197,10 +197,19 @@ inline bool early_locator_starved(const solon_plan* plan) { return plan->early_l
 // m = 1 on 15 nodes x 10 M), and the coded matrix no longer lingers in L2 for the projection pass of a decode that
 // follows an encode.  Measured per case (same box, switch in the environment): worth it where the locator is long
 // and the streams are short - m > 6 (all-rows recovery tables, 89 -> 67 us per decode on 15 nodes x 10 M at m = 10) -
-// and a wash or a loss for m <= 6.  How much may stream before the code is gone whatever the marks: at 1.8 GB of
-// gradients per step (45 nodes x 10 M, m = 10) the decode still gains 14 - 22 us and the encode loses 2 - 8; at 4.2 GB
-// (105 nodes) the decode gains nothing and the encode loses 20.  So: m > 6 and at most 2 GB of gradients per step.
-inline bool keeps_l2_for_code(int P, int m, int64_t d) { return m > 6 && (double)P * (double)d * 4.0 <= 2.0e9; }
+// and for m = 4 .. 6 when the decode's own pass is short: at 600 - 670 MB of gradients on 15 nodes (m = 5, a projection
+// pass over 120 - 134 MB) the decode gains 4 - 9 us in the single-pass form and 0 - 6 us in the two-pass form while the encode
+// loses 0 - 2, and at 180 MB on 45 nodes the decode gains 12 - 15; with m = 1, 2 at the same sizes (a projection pass over 300
+// - 600 MB, which evicts the code whatever the marks) the locator gains nothing, and when everything fits in L2 anyway
+// (60 MB of gradients) the marks only cost the encode.  How much may stream before the code is gone whatever the marks: at
+// 1.8 GB of gradients per step (45 nodes x 10 M, m = 10) the decode still gains 14 - 22 us and the encode loses 2 - 8; at
+// 4.2 GB (105 nodes) the decode gains nothing and the encode loses 20.  So: m > 6 and at most 2 GB of gradients per step, or
+// m = 4 .. 6 with 150 MB .. 1 GB of gradients and at most 160 MB of coded vectors.
+inline bool keeps_l2_for_code(int P, int m, int64_t d) {
+  const double grads = (double)P * (double)d * 4.0;
+  if (m > 6) return grads <= 2.0e9;
+  return m >= 4 && grads >= 150e6 && grads <= 1.0e9 && grads / m <= 160e6;
+}
 
 int launch_fill_projection(solon_plan* plan, int advance);   // advance = 1: the next draw (device-side count), 0: redo the current one
 int launch_encode(solon_plan* plan, const float* grads, float* coded);
