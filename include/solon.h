@@ -151,7 +151,7 @@ int solon_plan_set_tolerance(solon_plan* plan, double tau);
  * projections, that the set it found is exactly the set of nodes that do not fit; if that check
  * fails (an attacker who spared those columns) the whole locator runs as it would have anyway.
  * Results do not depend on the mode.  mode 0: never; 1 (default): when the projection pass is long
- * enough to hide the early run (P * d_c * 4 bytes >= 350 MB) and the solver is small (groups of at
+ * enough to hide the early run (P * d_c * 4 bytes >= 350 MB; 250 MB when s = 1) and the solver is small (groups of at
  * most 64 nodes, s <= 5); 2: whenever the solver is small; 3: diagnostic - as 2, but the projection
  * kernel announces no partial sums, so the locator's bounded wait for them (2 ms) runs out and it
  * takes its ordinary path afterwards (outcome 3 of solon_plan_get_early_outcome; results unchanged). */

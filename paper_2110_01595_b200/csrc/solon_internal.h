@@ -182,7 +182,9 @@ struct TraceRange {
 // a streaming kernel (the projection kernel moves about 6 GB per ms).
 inline bool uses_early_locator(const solon_plan* plan) {
   const bool small_solver = plan->s > 0 && plan->max_group <= 64 && plan->s <= 5;
-  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= 350e6;
+  // (a locator with a single error count to try is through sooner: 300 MB suffice at s = 1 - 101 -> 89 us per decode on 15
+  // nodes x 10 M at m = 2 - where s = 3 and s = 5 lose 2 and 8 us)
+  const bool long_pass = (double)plan->P * (double)plan->d_c * 4.0 >= (plan->s <= 1 ? 250e6 : 350e6);
   return small_solver && (plan->early_locator >= 2 || (plan->early_locator == 1 && long_pass));
 }
 // Mode 3 (diagnostic): the locator works ahead as in mode 2 but the projection kernel announces no partial sums,
