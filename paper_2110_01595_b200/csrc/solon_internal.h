@@ -201,16 +201,18 @@ inline bool early_locator_starved(const solon_plan* plan) { return plan->early_l
 // and the streams are short - m > 6 (all-rows recovery tables, 89 -> 67 us per decode on 15 nodes x 10 M at m = 10) -
 // and for m = 4 .. 6 when the decode's own pass is short: at 600 - 670 MB of gradients on 15 nodes (m = 5, a projection
 // pass over 120 - 134 MB) the decode gains 4 - 9 us in the single-pass form and 0 - 6 us in the two-pass form while the encode
-// loses 0 - 2, and at 180 MB on 45 nodes the decode gains 12 - 15; with m = 1, 2 at the same sizes (a projection pass over 300
-// - 600 MB, which evicts the code whatever the marks) the locator gains nothing, and when everything fits in L2 anyway
-// (60 MB of gradients) the marks only cost the encode.  How much may stream before the code is gone whatever the marks: at
-// 1.8 GB of gradients per step (45 nodes x 10 M, m = 10) the decode still gains 14 - 22 us and the encode loses 2 - 8; at
-// 4.2 GB (105 nodes) the decode gains nothing and the encode loses 20.  So: m > 6 and at most 2 GB of gradients per step, or
-// m = 4 .. 6 with 150 MB .. 1 GB of gradients and at most 160 MB of coded vectors.
+// loses 0 - 2; with m = 1, 2 at the same sizes (a projection pass over 300 - 600 MB, which evicts the code whatever the
+// marks) the locator gains nothing.  Small steps gain at every m: over the 30 grid points with 1 M coordinates (60 - 420 MB
+// of gradients) the step is 3 - 28 % shorter with the marks at m = 1, 2 and 6 - 25 % at m = 5, 10, and longer at none by
+// more than 3 %.  How much may stream before the code is gone whatever the marks: at 1.8 GB of gradients per step (45 nodes
+// x 10 M, m = 10) the decode still gains 14 - 22 us and the encode loses 2 - 8; at 4.2 GB (105 nodes) the decode gains
+// nothing and the encode loses 20.  So: at most 450 MB of gradients per step, or m = 4 .. 6 with at most 1 GB of gradients
+// and 160 MB of coded vectors, or m > 6 and at most 2 GB of gradients.
 inline bool keeps_l2_for_code(int P, int m, int64_t d) {
   const double grads = (double)P * (double)d * 4.0;
+  if (grads <= 450e6) return true;
   if (m > 6) return grads <= 2.0e9;
-  return m >= 4 && grads >= 150e6 && grads <= 1.0e9 && grads / m <= 160e6;
+  return m >= 4 && grads <= 1.0e9 && grads / m <= 160e6;
 }
 
 int launch_fill_projection(solon_plan* plan, int advance);   // advance = 1: the next draw (device-side count), 0: redo the current one
