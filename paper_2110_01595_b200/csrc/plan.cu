@@ -214,6 +214,9 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
   p->num_sms = prop.multiProcessorCount;
   p->proj_grid = p->num_sms * 4;
   p->early_locator = 1;
+  if (const char* env = getenv("SOLON_EARLY_LOCATOR")) {     // for measurements, like SOLON_STREAM_HINTS below
+    if (env[0] >= '0' && env[0] <= '2') p->early_locator = env[0] - '0';
+  }
   p->fresh_f = 0;
   p->draw_parity = 0;
   p->stream_hints = keeps_l2_for_code(P, m, dtype == SOLON_F64 ? 2 * d : d) ? 1 : 0;
@@ -305,6 +308,9 @@ int solon_plan_create_ex(int P, int s, int m, int r, int64_t d, uint64_t seed, i
         p->opt_rows = (int)opt_src.size();
         p->opt_src_host = opt_src;
         p->optimistic = 1;
+        if (const char* env = getenv("SOLON_OPTIMISTIC")) {     // for measurements
+          if (env[0] >= '0' && env[0] <= '2') p->optimistic = env[0] - '0';
+        }
         if ((rc = dev_alloc(&p->d_opt, (size_t)8 + q))) break;
         std::vector<int> opt_init((size_t)8 + q, 0);
         opt_init[4] = p->optimistic;
